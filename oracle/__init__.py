@@ -1,0 +1,240 @@
+"""ctypes binding of the CPU oracle (oracle/natcomp_oracle.cpp).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
+benchmark's CPU-baseline leg; never by the package.  Arrays are numpy, host side.
+"""
+import ctypes as C
+
+import numpy as np
+
+from . import build as _build
+
+_lib = C.CDLL(_build.build())
+
+_u8p = C.POINTER(C.c_uint8)
+_u32p = C.POINTER(C.c_uint32)
+_i32p = C.POINTER(C.c_int32)
+_u64p = C.POINTER(C.c_uint64)
+_f32p = C.POINTER(C.c_float)
+_f64p = C.POINTER(C.c_double)
+
+P_INF = 0  # encoding of p = infinity
+
+
+def _sig(name, restype, *argtypes):
+    fn = getattr(_lib, name)
+    fn.restype = restype
+    fn.argtypes = list(argtypes)
+    return fn
+
+
+_set_threads = _sig("orc_set_threads", None, C.c_int)
+_max_threads = _sig("orc_max_threads", C.c_int)
+_philox = _sig("orc_philox4x32_10", None, _u32p, _u32p, _u32p)
+_stream_words = _sig("orc_stream_words", None, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64,
+                     C.c_uint64, _u32p)
+_cnat_values = _sig("orc_cnat_values", None, _f32p, _u32p, C.c_uint64, _f64p)
+_cnat_codes = _sig("orc_cnat_codes", None, _f32p, _u32p, C.c_uint64, _u8p, _u8p)
+_cnat_decode = _sig("orc_cnat_decode", None, _u8p, _u8p, C.c_uint64, _f32p)
+_nc_compress = _sig("orc_nc_compress", None, _f32p, C.c_uint64, C.c_uint64, C.c_uint64,
+                    C.c_uint32, _u8p, _u32p)
+_nc_decode_accumulate = _sig("orc_nc_decode_accumulate", None, _u8p, _u32p, C.c_uint64, _f32p)
+_nc_aggregate = _sig("orc_nc_aggregate", None, C.POINTER(_u8p), C.POINTER(_u32p), C.c_int,
+                     C.c_uint64, _f32p)
+_sum_fp32 = _sig("orc_sum_fp32", None, C.POINTER(_f32p), C.c_int, C.c_uint64, _f32p)
+_norms = _sig("orc_norms", None, _f32p, _u64p, C.c_int, C.c_int, _f32p)
+_nd_level_codes = _sig("orc_nd_level_codes", None, _f64p, _u32p, C.c_uint64, C.c_int, _i32p)
+_nd_compress = _sig("orc_nd_compress", None, _f32p, C.c_uint64, C.c_uint64, _u64p, C.c_int,
+                    C.c_int, C.c_int, C.c_uint64, C.c_uint32, C.c_uint32, C.c_int, _f32p, _u8p,
+                    _u32p)
+_nd_decode_accumulate = _sig("orc_nd_decode_accumulate", None, _f32p, _u8p, _u32p, C.c_uint64,
+                             _u64p, C.c_int, C.c_int, _f32p)
+_nd_aggregate = _sig("orc_nd_aggregate", None, C.POINTER(_f32p), C.POINTER(_u8p),
+                     C.POINTER(_u32p), C.c_int, C.c_uint64, _u64p, C.c_int, C.c_int, _f32p)
+_sparse_compress = _sig("orc_sparse_compress", C.c_uint64, _f32p, C.c_uint64, C.c_uint64,
+                        C.c_float, C.c_int, C.c_int, C.c_uint64, C.c_uint32, _u32p, _u8p,
+                        C.c_uint64, _f32p)
+_sparse_decode_accumulate = _sig("orc_sparse_decode_accumulate", None, _u32p, _u8p, C.c_uint64,
+                                 C.c_float, C.c_int, _f32p)
+
+
+def _arr(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def _p(a, ptype):
+    return a.ctypes.data_as(ptype)
+
+
+def _ptr_array(arrays, ptype):
+    return (ptype * len(arrays))(*[_p(a, ptype) for a in arrays])
+
+
+def set_threads(t: int) -> None:
+    _set_threads(int(t))
+
+
+def max_threads() -> int:
+    return int(_max_threads())
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    ctr = _arr(ctr, np.uint32)
+    key = _arr(key, np.uint32)
+    assert ctr.shape == (4,) and key.shape == (2,)
+    out = np.empty(4, np.uint32)
+    _philox(_p(ctr, _u32p), _p(key, _u32p), _p(out, _u32p))
+    return out
+
+
+def stream_words(seed: int, worker: int, domain: int, j0: int, count: int) -> np.ndarray:
+    out = np.empty(count, np.uint32)
+    _stream_words(seed, worker, domain, j0, count, _p(out, _u32p))
+    return out
+
+
+def cnat_values(t, r23) -> np.ndarray:
+    t = _arr(t, np.float32)
+    r23 = _arr(r23, np.uint32)
+    assert t.shape == r23.shape
+    out = np.empty(t.shape, np.float64)
+    _cnat_values(_p(t, _f32p), _p(r23, _u32p), t.size, _p(out, _f64p))
+    return out
+
+
+def cnat_codes(t, r23):
+    t = _arr(t, np.float32)
+    r23 = _arr(r23, np.uint32)
+    assert t.shape == r23.shape
+    e = np.empty(t.shape, np.uint8)
+    s = np.empty(t.shape, np.uint8)
+    _cnat_codes(_p(t, _f32p), _p(r23, _u32p), t.size, _p(e, _u8p), _p(s, _u8p))
+    return e, s
+
+
+def cnat_decode(exp_bytes, sign_bits) -> np.ndarray:
+    e = _arr(exp_bytes, np.uint8)
+    s = _arr(sign_bits, np.uint8)
+    out = np.empty(e.shape, np.float32)
+    _cnat_decode(_p(e, _u8p), _p(s, _u8p), e.size, _p(out, _f32p))
+    return out
+
+
+def nc_compress(x, seed: int, worker: int, j0: int = 0):
+    """C_nat of one worker's vector (or of the slice starting at element j0)."""
+    x = _arr(x, np.float32)
+    assert j0 % 32 == 0
+    d = x.size
+    e = np.zeros(d, np.uint8)
+    s = np.zeros((d + 31) // 32, np.uint32)
+    _nc_compress(_p(x, _f32p), d, j0, seed, worker, _p(e, _u8p), _p(s, _u32p))
+    return e, s
+
+
+def nc_decode_accumulate(exp, sign, acc) -> None:
+    exp = _arr(exp, np.uint8)
+    sign = _arr(sign, np.uint32)
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    _nc_decode_accumulate(_p(exp, _u8p), _p(sign, _u32p), acc.size, _p(acc, _f32p))
+
+
+def nc_aggregate(exps, signs, d: int) -> np.ndarray:
+    exps = [_arr(a, np.uint8) for a in exps]
+    signs = [_arr(a, np.uint32) for a in signs]
+    out = np.empty(d, np.float32)
+    _nc_aggregate(_ptr_array(exps, _u8p), _ptr_array(signs, _u32p), len(exps), d, _p(out, _f32p))
+    return out
+
+
+def sum_fp32(xs) -> np.ndarray:
+    xs = [_arr(a, np.float32) for a in xs]
+    d = xs[0].size
+    out = np.empty(d, np.float32)
+    _sum_fp32(_ptr_array(xs, _f32p), len(xs), d, _p(out, _f32p))
+    return out
+
+
+def norms(x, bucket_off, p: int) -> np.ndarray:
+    x = _arr(x, np.float32)
+    off = _arr(bucket_off, np.uint64)
+    out = np.empty(off.size - 1, np.float32)
+    _norms(_p(x, _f32p), _p(off, _u64p), off.size - 1, p, _p(out, _f32p))
+    return out
+
+
+def nd_level_codes(y, r23, s: int) -> np.ndarray:
+    y = _arr(y, np.float64)
+    r23 = _arr(r23, np.uint32)
+    assert y.shape == r23.shape
+    out = np.empty(y.shape, np.int32)
+    _nd_level_codes(_p(y, _f64p), _p(r23, _u32p), y.size, s, _p(out, _i32p))
+    return out
+
+
+def nd_compress(x, bucket_off, p: int, s: int, seed: int, worker: int, *, given_norms=None,
+                domain: int = 1, j0: int = 0):
+    """D_nat^{p,s}; definition mode unless given_norms is passed (given-norm mode)."""
+    x = _arr(x, np.float32)
+    off = _arr(bucket_off, np.uint64)
+    assert j0 % 32 == 0 and 1 <= s <= 15
+    d = x.size
+    B = off.size - 1
+    if given_norms is None:
+        nrm = np.zeros(B, np.float32)
+        mode = 0
+    else:
+        nrm = np.array(given_norms, dtype=np.float32, copy=True)
+        assert nrm.size == B
+        mode = 1
+    level = np.zeros((d + 1) // 2, np.uint8)
+    sign = np.zeros((d + 31) // 32, np.uint32)
+    _nd_compress(_p(x, _f32p), d, j0, _p(off, _u64p), B, p, s, seed, worker, domain, mode,
+                 _p(nrm, _f32p), _p(level, _u8p), _p(sign, _u32p))
+    return nrm, level, sign
+
+
+def nd_decode_accumulate(nrm, level, sign, bucket_off, s: int, acc) -> None:
+    nrm = _arr(nrm, np.float32)
+    level = _arr(level, np.uint8)
+    sign = _arr(sign, np.uint32)
+    off = _arr(bucket_off, np.uint64)
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    _nd_decode_accumulate(_p(nrm, _f32p), _p(level, _u8p), _p(sign, _u32p), acc.size,
+                          _p(off, _u64p), off.size - 1, s, _p(acc, _f32p))
+
+
+def nd_aggregate(nrms, levels, signs, bucket_off, s: int, d: int) -> np.ndarray:
+    nrms = [_arr(a, np.float32) for a in nrms]
+    levels = [_arr(a, np.uint8) for a in levels]
+    signs = [_arr(a, np.uint32) for a in signs]
+    off = _arr(bucket_off, np.uint64)
+    out = np.zeros(d, np.float32)
+    _nd_aggregate(_ptr_array(nrms, _f32p), _ptr_array(levels, _u8p), _ptr_array(signs, _u32p),
+                  len(nrms), d, _p(off, _u64p), off.size - 1, s, _p(out, _f32p))
+    return out
+
+
+def sparse_compress(x, keep_threshold: int, scale: float, p: int, s: int, seed: int, worker: int,
+                    cap=None):
+    """S (Bernoulli keep, threshold / 2^32) then D_nat^{p,s}; returns idx, codes, count, norm."""
+    x = _arr(x, np.float32)
+    assert 1 <= s <= 7
+    d = x.size
+    if cap is None:
+        cap = d
+    idx = np.zeros(cap, np.uint32)
+    codes = np.zeros((cap + 1) // 2, np.uint8)
+    nrm = C.c_float(0.0)
+    count = _sparse_compress(_p(x, _f32p), d, keep_threshold, scale, p, s, seed, worker,
+                             _p(idx, _u32p), _p(codes, _u8p), cap, C.byref(nrm))
+    stored = min(int(count), cap)
+    return idx[:stored], codes[:(stored + 1) // 2], int(count), np.float32(nrm.value)
+
+
+def sparse_decode_accumulate(idx, codes, count: int, nrm, s: int, acc) -> None:
+    idx = _arr(idx, np.uint32)
+    codes = _arr(codes, np.uint8)
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    _sparse_decode_accumulate(_p(idx, _u32p), _p(codes, _u8p), count, float(nrm), s,
+                              _p(acc, _f32p))

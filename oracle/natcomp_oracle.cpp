@@ -1,0 +1,424 @@
+// CPU oracle for the natural-compression hot path.  TEST INFRASTRUCTURE ONLY.
+//
+// A plain, slow, scalar restatement of what the operators compute, written from
+// the paper's definitions (arXiv 1905.10988).  It exists so that the CUDA library
+// can be checked against something that is obviously the definition; it is never
+// part of the product path, shares no code with the CUDA sources, and nothing in
+// the package imports it.  Floating point is done in double unless a step is
+// pinned to binary32 (the decoded values, the fixed-order fp32 sum, and the
+// "given-norm" dithering mode).  Build: g++ -O2 -ffp-contract=off (no fast-math,
+// no flush-to-zero), optional OpenMP over independent elements.
+//
+// Every function below is pinned by tests/test_oracle_*.py against values the
+// paper prints, closed forms, exhaustive enumeration of the 2^23 random
+// thresholds, or library routines (numpy); there is no "parity unpinned" function.
+//
+// Random numbers.  The paper only says that the rounding is randomised; this
+// library fixes the random stream as Philox4x32-10 (Salmon, Moraes, Dror, Shaw,
+// "Parallel random numbers: as easy as 1, 2, 3", SC'11):
+//   key     = (low 32 bits of seed, high 32 bits of seed)
+//   counter = (low 32 bits of q, high 32 bits of q, worker, domain),  q = j / 4
+//   element j of a worker's vector uses output word (j mod 4), and of that word
+//   the low 23 bits r23.
+// domain: 0 = natural compression, 1 = natural-dithering rounding, 2 = sparsifier.
+//
+// Edge policy for binary32 inputs the paper does not discuss (Sec. 2 assumes a
+// normal number with an implicit leading one):
+//   +-0            -> +-0 (sign kept), Def. 1 "C_nat(0) = 0"
+//   subnormal t    -> +-0 or +-2^-126, up-probability |t| / 2^-126 (unbiased; the
+//                     9/8 second-moment bound of Thm. 1 does not hold here)
+//   2^127<|t|<inf  -> never rounded up: +-2^127 (saturation, biased)
+//   +-inf, NaN     -> +-inf (exponent byte 255, sign bit kept)
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <cstddef>
+#include <limits>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+// ---------------------------------------------------------------- Philox4x32-10
+// One round: two 32x32->64 multiplies; the high halves are mixed with the other
+// two counter words and the round key, the low halves pass through (SC'11, Sec. 4).
+void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) {            // Weyl key schedule between rounds
+            k0 += 0x9E3779B9u;
+            k1 += 0xBB67AE85u;
+        }
+        const uint64_t prod0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        const uint64_t prod1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        const uint32_t n0 = (uint32_t)(prod1 >> 32) ^ c1 ^ k0;
+        const uint32_t n1 = (uint32_t)prod1;
+        const uint32_t n2 = (uint32_t)(prod0 >> 32) ^ c3 ^ k1;
+        const uint32_t n3 = (uint32_t)prod0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+uint32_t stream_word(uint64_t seed, uint32_t worker, uint32_t domain, uint64_t j) {
+    const uint64_t q = j / 4;
+    const uint32_t ctr[4] = {(uint32_t)(q & 0xFFFFFFFFu), (uint32_t)(q >> 32), worker, domain};
+    const uint32_t key[2] = {(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)};
+    uint32_t out[4];
+    philox4x32_10(ctr, key, out);
+    return out[j % 4];
+}
+
+const double TWO23 = 8388608.0;
+
+// ------------------------------------------------------- natural compression
+// Def. 1: t != 0 is rounded to sign(t) 2^floor(log2|t|) with probability p(t) and
+// to sign(t) 2^ceil(log2|t|) with probability 1 - p(t),
+// p(t) = (2^ceil - |t|) / 2^floor.  The draw: "up" iff r23 < (1 - p(t)) * 2^23.
+// For a binary32 t the product is the integer mantissa field (Sec. 2:
+// p(t) = 1 - m), so the rule is exact, not an approximation.
+double cnat_value(float t, uint32_t r23) {
+    if (t == 0.0f) return (double)t;                                  // keeps -0
+    if (std::isnan(t) || std::isinf(t))
+        return std::copysign(std::numeric_limits<double>::infinity(), (double)t);
+    const double a = std::fabs((double)t);
+    double lo, hi;
+    if (a < 0x1p-126) {               // subnormal: bracket [0, 2^-126]
+        lo = 0.0;
+        hi = 0x1p-126;
+    } else {
+        const int fl = std::ilogb(a);              // floor(log2 |t|)
+        lo = std::ldexp(1.0, fl);
+        hi = std::ldexp(1.0, fl + 1);
+        if (fl >= 127) return std::copysign(lo, (double)t);           // saturate
+    }
+    const double p_floor = (hi - a) / (hi - lo);   // p(t) of Def. 1 (hi - lo = 2^floor)
+    const double p_up = 1.0 - p_floor;
+    const bool up = (double)r23 < p_up * TWO23;
+    return std::copysign(up ? hi : lo, (double)t);
+}
+
+// 9-bit code of a value of the form +-0, +-2^k, +-inf: biased exponent + sign bit.
+void cnat_code(double value, uint8_t* exp_byte, uint32_t* sign_bit) {
+    *sign_bit = std::signbit(value) ? 1u : 0u;
+    const double a = std::fabs(value);
+    if (a == 0.0) *exp_byte = 0;
+    else if (std::isinf(a)) *exp_byte = 255;
+    else *exp_byte = (uint8_t)(std::ilogb(a) + 127);
+}
+
+float cnat_decode(uint8_t exp_byte, uint32_t sign_bit) {
+    double a;
+    if (exp_byte == 0) a = 0.0;
+    else if (exp_byte == 255) a = std::numeric_limits<double>::infinity();
+    else a = std::ldexp(1.0, (int)exp_byte - 127);
+    return (float)(sign_bit ? -a : a);
+}
+
+// ------------------------------------------------------------------- norms
+// ||x||_p of Def. 3 for p in {1, 2, inf (encoded 0)}; double accumulation in index
+// order, rounded once to binary32.  A NaN entry makes every norm NaN.
+float norm_p(const float* x, uint64_t len, int p) {
+    double acc = 0.0;
+    bool saw_nan = false;
+    for (uint64_t i = 0; i < len; ++i) {
+        const double a = std::fabs((double)x[i]);
+        if (std::isnan(a)) saw_nan = true;
+        if (p == 1) acc += a;
+        else if (p == 2) acc += a * a;
+        else if (a > acc) acc = a;
+    }
+    if (saw_nan) return std::numeric_limits<float>::quiet_NaN();
+    if (p == 2) acc = std::sqrt(acc);
+    return (float)acc;
+}
+
+bool norm_degenerate(float norm) {
+    // x = 0 gives D(x) = 0 (Def. 3).  A norm that is subnormal or not finite is
+    // treated the same way: every level code is 0, the norm itself is still stored.
+    return !(norm >= 0x1p-126f) || std::isinf(norm);
+}
+
+// ------------------------------------------------------- natural dithering
+// Def. 3 with the natural levels l_u = 2^-u (u = 0..s-1), l_s = 0.  For
+// l_{u+1} <= y <= l_u, xi(y) = l_u with probability (y - l_{u+1}) / (l_u - l_{u+1}).
+// Returns the level code c in 0..s:  c = 0 <-> 0,  c = k <-> 2^(k-s).
+// The draw: "up" iff r23 < floor(probability * 2^23).
+int nd_level_code(double y, int s, uint32_t r23) {
+    if (y >= 1.0) return s;                       // y = l_0 (or a rounding excess)
+    for (int u = 0; u < s; ++u) {
+        const double upper = std::ldexp(1.0, -u);
+        const double lower = (u + 1 == s) ? 0.0 : std::ldexp(1.0, -(u + 1));
+        if (y >= lower) {
+            const double p_up = (y - lower) / (upper - lower);
+            const double thr = std::floor(p_up * TWO23);
+            const bool up = (double)r23 < thr;
+            return up ? (s - u) : (s - u - 1);
+        }
+    }
+    return 0;   // not reached for y >= 0
+}
+
+// decoded magnitude of level code c under norm: norm * 2^(c-s) as one binary32
+// multiply by an exact power of two; c = 0 decodes to 0 whatever the norm is.
+float nd_decode_value(int c, int s, float norm, uint32_t sign_bit) {
+    float mag;
+    if (c == 0) mag = 0.0f;
+    else mag = norm * (float)std::ldexp(1.0, c - s);
+    return sign_bit ? -mag : mag;
+}
+
+}  // namespace
+
+extern "C" {
+
+void orc_set_threads(int t) {
+#ifdef _OPENMP
+    if (t > 0) omp_set_num_threads(t);
+#else
+    (void)t;
+#endif
+}
+
+int orc_max_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void orc_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) {
+    philox4x32_10(ctr, key, out);
+}
+
+// out[i] = the 32-bit stream word of element j0 + i
+void orc_stream_words(uint64_t seed, uint32_t worker, uint32_t domain, uint64_t j0,
+                      uint64_t count, uint32_t* out) {
+    for (uint64_t i = 0; i < count; ++i) out[i] = stream_word(seed, worker, domain, j0 + i);
+}
+
+// Scalar C_nat with explicit random thresholds: out[i] = C_nat(t[i]; r23[i]).
+void orc_cnat_values(const float* t, const uint32_t* r23, uint64_t count, double* out) {
+    for (uint64_t i = 0; i < count; ++i) out[i] = cnat_value(t[i], r23[i] & 0x7FFFFFu);
+}
+
+// 9-bit codes with explicit random thresholds (exhaustive bit-pattern parity).
+void orc_cnat_codes(const float* t, const uint32_t* r23, uint64_t count, uint8_t* exp_bytes,
+                    uint8_t* sign_bits) {
+    for (uint64_t i = 0; i < count; ++i) {
+        uint32_t sb;
+        cnat_code(cnat_value(t[i], r23[i] & 0x7FFFFFu), &exp_bytes[i], &sb);
+        sign_bits[i] = (uint8_t)sb;
+    }
+}
+
+void orc_cnat_decode(const uint8_t* exp_bytes, const uint8_t* sign_bits, uint64_t count, float* out) {
+    for (uint64_t i = 0; i < count; ++i) out[i] = cnat_decode(exp_bytes[i], sign_bits[i]);
+}
+
+// Worker-side C_nat of x[0..d) whose first entry is element j0 of the worker's
+// vector (j0 a multiple of 32).  exp: d bytes; sign: ceil(d/32) words, bit (j mod 32)
+// of word (j / 32), unused high bits of the last word zero.
+void orc_nc_compress(const float* x, uint64_t d, uint64_t j0, uint64_t seed, uint32_t worker,
+                     uint8_t* exp, uint32_t* sign) {
+    const int64_t words = (int64_t)((d + 31) / 32);
+#pragma omp parallel for schedule(static)
+    for (int64_t w = 0; w < words; ++w) {
+        uint32_t bits = 0;
+        const uint64_t end = ((uint64_t)w * 32 + 32 < d) ? (uint64_t)w * 32 + 32 : d;
+        for (uint64_t i = (uint64_t)w * 32; i < end; ++i) {
+            const uint32_t r23 = stream_word(seed, worker, 0u, j0 + i) & 0x7FFFFFu;
+            uint32_t sb;
+            cnat_code(cnat_value(x[i], r23), &exp[i], &sb);
+            bits |= sb << (i % 32);
+        }
+        sign[w] = bits;
+    }
+}
+
+// Master side, one worker: acc[j] = acc[j] + decode(code_j) in binary32.
+void orc_nc_decode_accumulate(const uint8_t* exp, const uint32_t* sign, uint64_t d, float* acc) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)d; ++i) {
+        const float v = cnat_decode(exp[i], (sign[i / 32] >> (i % 32)) & 1u);
+        acc[i] = acc[i] + v;
+    }
+}
+
+// Master side (Algorithm 1, "aggregate"): out[j] = sum over workers i = 0..n-1 of
+// decode(code_{i,j}), accumulated left to right in binary32 starting from +0.
+void orc_nc_aggregate(const uint8_t* const* exp, const uint32_t* const* sign, int n, uint64_t d,
+                      float* out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < (int64_t)d; ++j) {
+        float acc = 0.0f;
+        for (int i = 0; i < n; ++i) {
+            const float v = cnat_decode(exp[i][j], (sign[i][j / 32] >> (j % 32)) & 1u);
+            acc = acc + v;
+        }
+        out[j] = acc;
+    }
+}
+
+// The uncompressed reference point: out[j] = ((+0 + x_0[j]) + x_1[j]) + ... in binary32.
+void orc_sum_fp32(const float* const* xs, int n, uint64_t d, float* out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < (int64_t)d; ++j) {
+        float acc = 0.0f;
+        for (int i = 0; i < n; ++i) acc = acc + xs[i][j];
+        out[j] = acc;
+    }
+}
+
+// Per-bucket norms; bucket_off has B+1 entries relative to x, bucket b = [off[b], off[b+1]).
+void orc_norms(const float* x, const uint64_t* bucket_off, int B, int p, float* norms) {
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b)
+        norms[b] = norm_p(x + bucket_off[b], bucket_off[b + 1] - bucket_off[b], p);
+}
+
+// Level codes for explicit y and thresholds (enumeration pins).
+void orc_nd_level_codes(const double* y, const uint32_t* r23, uint64_t count, int s, int32_t* codes) {
+    for (uint64_t i = 0; i < count; ++i) codes[i] = nd_level_code(y[i], s, r23[i] & 0x7FFFFFu);
+}
+
+// Natural dithering D_nat^{p,s} of x[0..d) split into B buckets, one norm each.
+//   mode 0 (definition): norms are computed here (double accumulation); y = |x| / norm in double.
+//   mode 1 (given norm): norms[] is an input; y = fl32(|x| * fl32(1 / norm)), all in binary32.
+// domain selects the random stream (1 for the product; 0 lets a test compare with C_nat).
+// level: one 4-bit code per entry, entry j in bits 4*(j mod 2).. of byte j/2 (s <= 15);
+// sign: as for C_nat (sign bit of x).  x[0] is element j0 of the worker's vector
+// (j0 a multiple of 32); ceil(d/2) level bytes and ceil(d/32) sign words are written.
+void orc_nd_compress(const float* x, uint64_t d, uint64_t j0, const uint64_t* bucket_off, int B,
+                     int p, int s, uint64_t seed, uint32_t worker, uint32_t domain, int mode,
+                     float* norms, uint8_t* level, uint32_t* sign) {
+    if (mode == 0) orc_norms(x, bucket_off, B, p, norms);
+    std::memset(level, 0, (size_t)((d + 1) / 2));
+    std::memset(sign, 0, (size_t)((d + 31) / 32) * 4);
+    // bucket starts need not be even or multiples of 32, so buckets are walked serially
+    for (int b = 0; b < B; ++b) {
+        const float norm = norms[b];
+        const bool degenerate = norm_degenerate(norm);
+        const float rinv = degenerate ? 0.0f : 1.0f / norm;
+        for (uint64_t i = bucket_off[b]; i < bucket_off[b + 1]; ++i) {
+            const float t = x[i];
+            const uint32_t sb = std::signbit(t) ? 1u : 0u;
+            int c = 0;
+            if (!degenerate) {
+                double y;
+                if (mode == 0) {
+                    y = std::fabs((double)t) / (double)norm;
+                } else {
+                    const float yf = std::fabs(t) * rinv;
+                    y = (double)yf;
+                }
+                const uint32_t r23 = stream_word(seed, worker, domain, j0 + i) & 0x7FFFFFu;
+                c = nd_level_code(y, s, r23);
+            }
+            level[i / 2] |= (uint8_t)(c << (4 * (i % 2)));
+            sign[i / 32] |= sb << (i % 32);
+        }
+    }
+}
+
+void orc_nd_decode_accumulate(const float* norms, const uint8_t* level, const uint32_t* sign,
+                              uint64_t d, const uint64_t* bucket_off, int B, int s, float* acc) {
+    (void)d;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        for (uint64_t i = bucket_off[b]; i < bucket_off[b + 1]; ++i) {
+            const int c = (level[i / 2] >> (4 * (i % 2))) & 0xF;
+            const float v = nd_decode_value(c, s, norms[b], (sign[i / 32] >> (i % 32)) & 1u);
+            acc[i] = acc[i] + v;
+        }
+    }
+}
+
+void orc_nd_aggregate(const float* const* norms, const uint8_t* const* level,
+                      const uint32_t* const* sign, int n, uint64_t d, const uint64_t* bucket_off,
+                      int B, int s, float* out) {
+    (void)d;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        for (uint64_t j = bucket_off[b]; j < bucket_off[b + 1]; ++j) {
+            float acc = 0.0f;
+            for (int i = 0; i < n; ++i) {
+                const int c = (level[i][j / 2] >> (4 * (j % 2))) & 0xF;
+                const float v =
+                    nd_decode_value(c, s, norms[i][b], (sign[i][j / 32] >> (j % 32)) & 1u);
+                acc = acc + v;
+            }
+            out[j] = acc;
+        }
+    }
+}
+
+// Random sparsification followed by natural dithering, on one bucket (the whole vector).
+// Coordinate j is kept iff its domain-2 stream word is below keep_threshold
+// (independent Bernoulli selection with probability keep_threshold / 2^32; the special
+// value keep_threshold = 2^32 keeps everything), and a kept entry becomes
+// x'_j = fl32(scale * x_j).  Then D_nat^{p,s} of the kept entries with norm
+// ||x'||_p over the kept entries, given-norm arithmetic (mode 1 above) and the
+// domain-1 stream at the dense index j.
+// Output: ascending indices, one byte-packed 4-bit code per kept entry
+// (bit 3 = sign, bits 0..2 = level 0..s, s <= 7; entry k in bits 4*(k mod 2).. of byte k/2),
+// the count and the norm.  Returns the count; entries beyond cap are counted but not stored.
+uint64_t orc_sparse_compress(const float* x, uint64_t d, uint64_t keep_threshold, float scale,
+                             int p, int s, uint64_t seed, uint32_t worker, uint32_t* idx,
+                             uint8_t* codes, uint64_t cap, float* norm_out) {
+    // pass 1: selection and the norm of the kept, scaled entries (double accumulation)
+    double acc = 0.0;
+    bool saw_nan = false;
+    uint64_t count = 0;
+    for (uint64_t j = 0; j < d; ++j) {
+        if ((uint64_t)stream_word(seed, worker, 2u, j) >= keep_threshold) continue;
+        const float xs = scale * x[j];
+        const double a = std::fabs((double)xs);
+        if (std::isnan(a)) saw_nan = true;
+        if (p == 1) acc += a;
+        else if (p == 2) acc += a * a;
+        else if (a > acc) acc = a;
+        ++count;
+    }
+    if (p == 2) acc = std::sqrt(acc);
+    const float norm = saw_nan ? std::numeric_limits<float>::quiet_NaN() : (float)acc;
+    *norm_out = norm;
+    const bool degenerate = norm_degenerate(norm);
+    const float rinv = degenerate ? 0.0f : 1.0f / norm;
+    // pass 2: level codes of the kept entries, in ascending index order
+    uint64_t k = 0;
+    const uint64_t stored = count < cap ? count : cap;
+    std::memset(codes, 0, (size_t)((stored + 1) / 2));
+    for (uint64_t j = 0; j < d && k < stored; ++j) {
+        if ((uint64_t)stream_word(seed, worker, 2u, j) >= keep_threshold) continue;
+        const float xs = scale * x[j];
+        int c = 0;
+        if (!degenerate) {
+            const float yf = std::fabs(xs) * rinv;
+            const uint32_t r23 = stream_word(seed, worker, 1u, j) & 0x7FFFFFu;
+            c = nd_level_code((double)yf, s, r23);
+        }
+        const uint32_t sb = std::signbit(xs) ? 1u : 0u;
+        idx[k] = (uint32_t)j;
+        codes[k / 2] |= (uint8_t)(((sb << 3) | (uint32_t)c) << (4 * (k % 2)));
+        ++k;
+    }
+    return count;
+}
+
+// acc[idx[k]] = acc[idx[k]] + sign * norm * 2^(c-s) for the listed entries.
+void orc_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes, uint64_t count,
+                                  float norm, int s, float* acc) {
+    for (uint64_t k = 0; k < count; ++k) {
+        const uint32_t code = (codes[k / 2] >> (4 * (k % 2))) & 0xFu;
+        const float v = nd_decode_value((int)(code & 7u), s, norm, code >> 3);
+        acc[idx[k]] = acc[idx[k]] + v;
+    }
+}
+
+}  // extern "C"
