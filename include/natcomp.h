@@ -1,0 +1,172 @@
+/* natcomp.h -- C ABI of the natural-compression hot path for NVIDIA B200 (sm_100a).
+ *
+ * The operators are those of "Natural Compression for Distributed Deep Learning"
+ * (arXiv 1905.10988): the per-entry compressor C_nat (Def. 1, Sec. 2), natural
+ * dithering D_nat^{p,s} (Def. 3), random sparsification composed with dithering
+ * (appendix "Sparsification - Formal Definition", Thm. 3) and the master-side
+ * aggregation  Delta = sum_i C(g_i)  of Algorithm 1.
+ *
+ * Conventions shared by every call
+ *   - Pointers are DEVICE pointers unless a parameter is documented as a host array.
+ *     "host array of device pointers" arguments hold at most NC_MAX_WORKERS entries
+ *     and are copied into the kernel's parameters before the call returns.
+ *   - The caller owns every buffer; the library allocates and frees nothing.  Scratch
+ *     memory is passed in as `workspace`; its size is queried with the
+ *     *_workspace_bytes helpers.
+ *   - fp32 vectors (x, acc, out) must be 32-byte aligned; exp, sign, level, idx, codes and
+ *     workspace 16-byte aligned; bucket_off 8-byte, norms and count 4-byte aligned
+ *     (NC_ERR_ALIGN otherwise).
+ *   - Calls are asynchronous on `stream`, never synchronise, and return after the
+ *     launch.  The return value covers argument validation and the launch status.
+ *   - d == 0 returns NC_OK and launches nothing.
+ *   - Packed planes are written including their zero padding up to the size the
+ *     *_bytes helpers return; padding is ignored on decode.
+ *
+ * Random stream (the paper fixes none): Philox4x32-10 with
+ *   key = (low32(seed), high32(seed)), counter = (low32(q), high32(q), worker, domain),
+ *   q = j / 4; element j of a worker's vector uses output word j mod 4, low 23 bits.
+ *   domain 0: C_nat, 1: D_nat rounding, 2: sparsifier selection.
+ * The stream depends on (seed, worker, j) only, so outputs are reproducible and
+ * independent of launch geometry.
+ *
+ * Packed formats
+ *   C_nat, 9 bits per entry (Sec. 2, "From 32 to 9 bits"):
+ *     exp[j]        biased binary32 exponent of C_nat(x_j)   (uint8; 0 encodes +-0, 255 +-inf)
+ *     sign[j / 32]  bit (j mod 32) = sign bit of x_j          (uint32 words)
+ *   D_nat^{p,s}, s <= 15: per bucket one fp32 norm; per entry a level code c in 0..s
+ *     (c = 0 <-> 0, c = k <-> 2^(k-s)) in bits 4*(j mod 2).. of level[j / 2], plus the
+ *     same sign plane.
+ *   Sparse D_nat, s <= 7: ascending uint32 indices; codes[k / 2] bits 4*(k mod 2)..:
+ *     bit 3 = sign, bits 0..2 = level code of the k-th kept entry.
+ *
+ * Inputs the paper does not discuss: +-0 keeps its sign and encodes as exponent 0;
+ * a subnormal x is rounded to +-0 or +-2^-126 with up-probability |x| / 2^-126;
+ * 2^127 < |x| < inf is never rounded up; +-inf and NaN encode as +-inf.
+ */
+#ifndef NATCOMP_H_
+#define NATCOMP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#ifndef __DRIVER_TYPES_H__
+typedef struct CUstream_st* cudaStream_t;
+#endif
+
+typedef enum {
+    NC_OK = 0,
+    NC_ERR_INVALID = -1,     /* null pointer, n or s or p out of range, inconsistent sizes */
+    NC_ERR_ALIGN = -2,       /* a pointer is not aligned as required */
+    NC_ERR_UNSUPPORTED = -3, /* p other than 1, 2, NC_P_INF */
+    NC_ERR_WORKSPACE = -4,   /* workspace_bytes smaller than the query helper's answer */
+    NC_ERR_CUDA = -5         /* the CUDA runtime reported an error at launch */
+} nc_status;
+
+#define NC_MAX_WORKERS 64
+#define NC_P_INF 0 /* value of `p` that selects the max-norm */
+
+/* Human-readable name of a status code (static string). */
+const char* nc_status_string(int status);
+
+/* ---- sizes (host-only arithmetic, no CUDA calls) -------------------------------- */
+size_t nc_exp_bytes(size_t d);   /* d rounded up to a multiple of 16 */
+size_t nc_sign_bytes(size_t d);  /* 4 * ceil(d / 32) rounded up to a multiple of 16 */
+size_t nd_level_bytes(size_t d); /* ceil(d / 2) rounded up to a multiple of 16 */
+size_t nd_workspace_bytes(size_t d, int num_buckets);
+size_t nd_sparse_workspace_bytes(size_t d, size_t cap);
+
+/* ---- C_nat (Def. 1; binary32 form in Sec. 2) ----------------------------------- */
+
+/* Worker side: exp/sign <- code of C_nat(x_j), j = 0..d-1, with the stream (seed, worker, j).
+ * x: fp32[d].  exp: nc_exp_bytes(d).  sign: nc_sign_bytes(d).  Bit-exact w.r.t. Def. 1. */
+nc_status nc_compress(const float* x, size_t d, uint64_t seed, uint32_t worker, uint8_t* exp,
+                      uint32_t* sign, cudaStream_t stream);
+
+/* The same for n workers' vectors of equal length d in one launch.  xs, exps, signs are host
+ * arrays of n device pointers, workers a host array of n worker ids (1 <= n <= NC_MAX_WORKERS). */
+nc_status nc_compress_batch(const float* const* xs, size_t d, uint64_t seed,
+                            const uint32_t* workers, uint8_t* const* exps,
+                            uint32_t* const* signs, int n, cudaStream_t stream);
+
+/* Master side, one worker (Algorithm 1, aggregation step): acc[j] <- acc[j] + decode(code_j),
+ * one binary32 addition per entry.  acc: fp32[d], read and written. */
+nc_status nc_decode_accumulate(const uint8_t* exp, const uint32_t* sign, size_t d, float* acc,
+                               cudaStream_t stream);
+
+/* Master side, n workers (Algorithm 1: Delta = sum_i Delta_i):
+ * out[j] <- (((+0 + v_0j) + v_1j) + ... + v_{n-1,j}) in binary32, v_ij = decode(code of worker i).
+ * exps, signs: host arrays of n device pointers.  out: fp32[d], overwritten.
+ * Identical to zero-filling out and calling nc_decode_accumulate for i = 0..n-1. */
+nc_status nc_aggregate(const uint8_t* const* exps, const uint32_t* const* signs, int n, size_t d,
+                       float* out, cudaStream_t stream);
+
+/* Reference point (the "no compression" baseline of Table 1): out[j] <- ((+0 + x_0j) + x_1j) + ...
+ * xs: host array of n device pointers to fp32[d]. */
+nc_status nc_sum_fp32(const float* const* xs, int n, size_t d, float* out, cudaStream_t stream);
+
+/* ---- D_nat^{p,s} (Def. 3 with levels 2^-u) -------------------------------------- */
+
+/* Worker side.  bucket_off: device array of B+1 ascending element offsets, off[0] = 0, off[B] = d;
+ * bucket b = [off[b], off[b+1]) has its own norm ||x_b||_p, p in {1, 2, NC_P_INF}, 1 <= s <= 15.
+ * norms: fp32[B] out.  level: nd_level_bytes(d).  sign: nc_sign_bytes(d).
+ * workspace: nd_workspace_bytes(d, B) bytes of scratch (contents undefined afterwards).
+ * Arithmetic: norm accumulated in binary64 from per-thread binary32 partial sums, rounded once;
+ * y = fl32(|x| * fl32(1 / norm)); above 2^(1-s) the up-probability is the mantissa fraction of y
+ * (as in C_nat), below it is y * 2^(s-1), both at 2^-23 resolution.  A bucket whose norm is 0,
+ * subnormal or not finite gets level code 0 everywhere (its norm is still stored).
+ * Given the stored norms the codes are bit-exact w.r.t. Def. 3 in that arithmetic. */
+nc_status nd_compress(const float* x, size_t d, const uint64_t* bucket_off, int B, int p, int s,
+                      uint64_t seed, uint32_t worker, float* norms, uint8_t* level,
+                      uint32_t* sign, void* workspace, size_t workspace_bytes,
+                      cudaStream_t stream);
+
+/* Master side, one worker: acc[j] <- acc[j] + sign_j * fl32(norm_b * 2^(c_j - s)); c = 0 adds +-0. */
+nc_status nd_decode_accumulate(const float* norms, const uint8_t* level, const uint32_t* sign,
+                               size_t d, const uint64_t* bucket_off, int B, int s, float* acc,
+                               cudaStream_t stream);
+
+/* Master side, n workers, fixed order 0..n-1 starting from +0 (see nc_aggregate).
+ * norms, levels, signs: host arrays of n device pointers. */
+nc_status nd_aggregate(const float* const* norms, const uint8_t* const* levels,
+                       const uint32_t* const* signs, int n, size_t d, const uint64_t* bucket_off,
+                       int B, int s, float* out, cudaStream_t stream);
+
+/* ---- random sparsification composed with D_nat (Thm. 3; one bucket = the whole vector) ----- */
+
+/* Keep coordinate j iff its domain-2 stream word < keep_threshold (probability
+ * keep_threshold / 2^32; keep_threshold = 2^32 keeps all), x'_j = fl32(scale * x_j), then
+ * D_nat^{p,s} of the kept entries (norm over kept entries; 1 <= s <= 7).
+ * idx: uint32[cap], ascending.  codes: ceil(cap / 2) bytes rounded up to 16.
+ * count: device uint32, number of kept entries (may exceed cap; only cap are stored).
+ * norm: device fp32.  workspace: nd_sparse_workspace_bytes(d, cap).  d < 2^32. */
+nc_status nd_sparse_compress(const float* x, size_t d, uint64_t keep_threshold, float scale,
+                             int p, int s, uint64_t seed, uint32_t worker, uint32_t* idx,
+                             uint8_t* codes, uint32_t* count, float* norm, size_t cap,
+                             void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/* acc[idx[k]] <- acc[idx[k]] + decoded value, k < min(*count, cap).  Indices are unique within
+ * one worker's list, so one call needs no atomics; calls for different workers are applied in
+ * the order they are enqueued on the stream. */
+nc_status nd_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes,
+                                      const uint32_t* count, const float* norm, int s, size_t d,
+                                      size_t cap, float* acc, cudaStream_t stream);
+
+/* ---- host-buffer plumbing (no counterpart in the paper, where workers and master exchange
+ * these buffers over a network) ------------------------------------------------------------- */
+
+/* Asynchronous copies on `stream` between host memory (pinned for real overlap) and device
+ * memory, so that a caller holding gradients on the host can drive the whole path through this
+ * ABI.  bytes == 0 is NC_OK. */
+nc_status nc_copy_to_device(void* dst_device, const void* src_host, size_t bytes,
+                            cudaStream_t stream);
+nc_status nc_copy_to_host(void* dst_host, const void* src_device, size_t bytes,
+                          cudaStream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NATCOMP_H_ */

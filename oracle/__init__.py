@@ -53,7 +53,7 @@ _nd_aggregate = _sig("orc_nd_aggregate", None, C.POINTER(_f32p), C.POINTER(_u8p)
                      C.POINTER(_u32p), C.c_int, C.c_uint64, _u64p, C.c_int, C.c_int, _f32p)
 _sparse_compress = _sig("orc_sparse_compress", C.c_uint64, _f32p, C.c_uint64, C.c_uint64,
                         C.c_float, C.c_int, C.c_int, C.c_uint64, C.c_uint32, _u32p, _u8p,
-                        C.c_uint64, _f32p)
+                        C.c_uint64, _f32p, _f32p)
 _sparse_decode_accumulate = _sig("orc_sparse_decode_accumulate", None, _u32p, _u8p, C.c_uint64,
                                  C.c_float, C.c_int, _f32p)
 
@@ -216,8 +216,9 @@ def nd_aggregate(nrms, levels, signs, bucket_off, s: int, d: int) -> np.ndarray:
 
 
 def sparse_compress(x, keep_threshold: int, scale: float, p: int, s: int, seed: int, worker: int,
-                    cap=None):
-    """S (Bernoulli keep, threshold / 2^32) then D_nat^{p,s}; returns idx, codes, count, norm."""
+                    cap=None, given_norm=None):
+    """S (Bernoulli keep, threshold / 2^32) then D_nat^{p,s}; returns idx, codes, count, norm.
+    given_norm replaces the oracle's own norm of the kept entries (given-norm mode)."""
     x = _arr(x, np.float32)
     assert 1 <= s <= 7
     d = x.size
@@ -226,8 +227,10 @@ def sparse_compress(x, keep_threshold: int, scale: float, p: int, s: int, seed: 
     idx = np.zeros(cap, np.uint32)
     codes = np.zeros((cap + 1) // 2, np.uint8)
     nrm = C.c_float(0.0)
+    gn = None if given_norm is None else C.byref(C.c_float(float(given_norm)))
     count = _sparse_compress(_p(x, _f32p), d, keep_threshold, scale, p, s, seed, worker,
-                             _p(idx, _u32p), _p(codes, _u8p), cap, C.byref(nrm))
+                             _p(idx, _u32p), _p(codes, _u8p), cap, C.byref(nrm),
+                             C.cast(gn, _f32p) if gn is not None else None)
     stored = min(int(count), cap)
     return idx[:stored], codes[:(stored + 1) // 2], int(count), np.float32(nrm.value)
 

@@ -164,10 +164,11 @@ int nd_level_code(double y, int s, uint32_t r23) {
 }
 
 // decoded magnitude of level code c under norm: norm * 2^(c-s) as one binary32
-// multiply by an exact power of two; c = 0 decodes to 0 whatever the norm is.
+// multiply by an exact power of two; c = 0 decodes to 0 whatever the norm is, and so does
+// every code under a norm that is not finite (such a bucket was compressed to all-zero codes).
 float nd_decode_value(int c, int s, float norm, uint32_t sign_bit) {
     float mag;
-    if (c == 0) mag = 0.0f;
+    if (c == 0 || std::isnan(norm) || std::isinf(norm)) mag = 0.0f;
     else mag = norm * (float)std::ldexp(1.0, c - s);
     return sign_bit ? -mag : mag;
 }
@@ -370,7 +371,8 @@ void orc_nd_aggregate(const float* const* norms, const uint8_t* const* level,
 // the count and the norm.  Returns the count; entries beyond cap are counted but not stored.
 uint64_t orc_sparse_compress(const float* x, uint64_t d, uint64_t keep_threshold, float scale,
                              int p, int s, uint64_t seed, uint32_t worker, uint32_t* idx,
-                             uint8_t* codes, uint64_t cap, float* norm_out) {
+                             uint8_t* codes, uint64_t cap, float* norm_out,
+                             const float* given_norm) {
     // pass 1: selection and the norm of the kept, scaled entries (double accumulation)
     double acc = 0.0;
     bool saw_nan = false;
@@ -386,7 +388,8 @@ uint64_t orc_sparse_compress(const float* x, uint64_t d, uint64_t keep_threshold
         ++count;
     }
     if (p == 2) acc = std::sqrt(acc);
-    const float norm = saw_nan ? std::numeric_limits<float>::quiet_NaN() : (float)acc;
+    float norm = saw_nan ? std::numeric_limits<float>::quiet_NaN() : (float)acc;
+    if (given_norm) norm = *given_norm;      // pins the rounding independently of the summation
     *norm_out = norm;
     const bool degenerate = norm_degenerate(norm);
     const float rinv = degenerate ? 0.0f : 1.0f / norm;

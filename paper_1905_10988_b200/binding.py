@@ -1,0 +1,203 @@
+"""Thin ctypes binding of libnatcomp.so: argument marshalling only.
+
+Every function has the name and the argument order of its C entry point
+(include/natcomp.h).  Tensors are torch CUDA tensors used as device memory; the
+binding passes their pointers and the current CUDA stream and raises NatcompError
+on a non-zero status.  There is no CPU fallback: without the built library the
+import fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnatcomp.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "libnatcomp.so is not built; run `python -m paper_1905_10988_b200.build` "
+        "(needs nvcc; targets sm_100a).  There is no CPU fallback.")
+
+lib = C.CDLL(LIB_PATH)
+
+NC_MAX_WORKERS = 64
+P_INF = 0
+
+EXPORTS = (
+    "nc_status_string", "nc_exp_bytes", "nc_sign_bytes", "nd_level_bytes", "nd_workspace_bytes",
+    "nd_sparse_workspace_bytes", "nc_compress", "nc_compress_batch", "nc_decode_accumulate",
+    "nc_aggregate", "nc_sum_fp32", "nd_compress", "nd_decode_accumulate", "nd_aggregate",
+    "nd_sparse_compress", "nd_sparse_decode_accumulate", "nc_copy_to_device", "nc_copy_to_host",
+)
+
+
+class NatcompError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        super().__init__("%s failed: %s (%d)" % (fn, status_string(status), status))
+        self.status = status
+
+
+_vp = C.c_void_p
+_sz = C.c_size_t
+
+
+def _sig(name, restype, *argtypes):
+    fn = getattr(lib, name)
+    fn.restype = restype
+    fn.argtypes = list(argtypes)
+    return fn
+
+
+_status_string = _sig("nc_status_string", C.c_char_p, C.c_int)
+_nc_exp_bytes = _sig("nc_exp_bytes", _sz, _sz)
+_nc_sign_bytes = _sig("nc_sign_bytes", _sz, _sz)
+_nd_level_bytes = _sig("nd_level_bytes", _sz, _sz)
+_nd_workspace_bytes = _sig("nd_workspace_bytes", _sz, _sz, C.c_int)
+_nd_sparse_workspace_bytes = _sig("nd_sparse_workspace_bytes", _sz, _sz, _sz)
+_nc_compress = _sig("nc_compress", C.c_int, _vp, _sz, C.c_uint64, C.c_uint32, _vp, _vp, _vp)
+_nc_compress_batch = _sig("nc_compress_batch", C.c_int, C.POINTER(_vp), _sz, C.c_uint64,
+                          C.POINTER(C.c_uint32), C.POINTER(_vp), C.POINTER(_vp), C.c_int, _vp)
+_nc_decode_accumulate = _sig("nc_decode_accumulate", C.c_int, _vp, _vp, _sz, _vp, _vp)
+_nc_aggregate = _sig("nc_aggregate", C.c_int, C.POINTER(_vp), C.POINTER(_vp), C.c_int, _sz, _vp,
+                     _vp)
+_nc_sum_fp32 = _sig("nc_sum_fp32", C.c_int, C.POINTER(_vp), C.c_int, _sz, _vp, _vp)
+_nd_compress = _sig("nd_compress", C.c_int, _vp, _sz, _vp, C.c_int, C.c_int, C.c_int, C.c_uint64,
+                    C.c_uint32, _vp, _vp, _vp, _vp, _sz, _vp)
+_nd_decode_accumulate = _sig("nd_decode_accumulate", C.c_int, _vp, _vp, _vp, _sz, _vp, C.c_int,
+                             C.c_int, _vp, _vp)
+_nd_aggregate = _sig("nd_aggregate", C.c_int, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp),
+                     C.c_int, _sz, _vp, C.c_int, C.c_int, _vp, _vp)
+_nd_sparse_compress = _sig("nd_sparse_compress", C.c_int, _vp, _sz, C.c_uint64, C.c_float,
+                           C.c_int, C.c_int, C.c_uint64, C.c_uint32, _vp, _vp, _vp, _vp, _sz,
+                           _vp, _sz, _vp)
+_nd_sparse_decode_accumulate = _sig("nd_sparse_decode_accumulate", C.c_int, _vp, _vp, _vp, _vp,
+                                    C.c_int, _sz, _sz, _vp, _vp)
+
+
+_nc_copy_to_device = _sig("nc_copy_to_device", C.c_int, _vp, _vp, _sz, _vp)
+_nc_copy_to_host = _sig("nc_copy_to_host", C.c_int, _vp, _vp, _sz, _vp)
+
+
+def nc_copy_to_device(dst_device, src_host, nbytes, stream=None) -> None:
+    _check("nc_copy_to_device", _nc_copy_to_device(_ptr(dst_device), _ptr(src_host), nbytes,
+                                                   _stream(stream)))
+
+
+def nc_copy_to_host(dst_host, src_device, nbytes, stream=None) -> None:
+    _check("nc_copy_to_host", _nc_copy_to_host(_ptr(dst_host), _ptr(src_device), nbytes,
+                                               _stream(stream)))
+
+
+def status_string(status: int) -> str:
+    return _status_string(int(status)).decode()
+
+
+def _ptr(t) -> int:
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _ptrs(ts: Sequence):
+    return (_vp * len(ts))(*[_ptr(t) for t in ts])
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(fn: str, status: int) -> None:
+    if status != 0:
+        raise NatcompError(fn, status)
+
+
+# ---- sizes ---------------------------------------------------------------------------
+def nc_exp_bytes(d: int) -> int:
+    return int(_nc_exp_bytes(d))
+
+
+def nc_sign_bytes(d: int) -> int:
+    return int(_nc_sign_bytes(d))
+
+
+def nd_level_bytes(d: int) -> int:
+    return int(_nd_level_bytes(d))
+
+
+def nd_workspace_bytes(d: int, num_buckets: int) -> int:
+    return int(_nd_workspace_bytes(d, num_buckets))
+
+
+def nd_sparse_workspace_bytes(d: int, cap: int) -> int:
+    return int(_nd_sparse_workspace_bytes(d, cap))
+
+
+# ---- C_nat ---------------------------------------------------------------------------
+def nc_compress(x, d, seed, worker, exp, sign, stream=None) -> None:
+    _check("nc_compress", _nc_compress(_ptr(x), d, seed, worker, _ptr(exp), _ptr(sign),
+                                       _stream(stream)))
+
+
+def nc_compress_batch(xs, d, seed, workers, exps, signs, n, stream=None) -> None:
+    w = (C.c_uint32 * n)(*[int(v) for v in workers])
+    _check("nc_compress_batch", _nc_compress_batch(_ptrs(xs), d, seed, w, _ptrs(exps),
+                                                   _ptrs(signs), n, _stream(stream)))
+
+
+def nc_decode_accumulate(exp, sign, d, acc, stream=None) -> None:
+    _check("nc_decode_accumulate", _nc_decode_accumulate(_ptr(exp), _ptr(sign), d, _ptr(acc),
+                                                         _stream(stream)))
+
+
+def nc_aggregate(exps, signs, n, d, out, stream=None) -> None:
+    _check("nc_aggregate", _nc_aggregate(_ptrs(exps), _ptrs(signs), n, d, _ptr(out),
+                                         _stream(stream)))
+
+
+def nc_sum_fp32(xs, n, d, out, stream=None) -> None:
+    _check("nc_sum_fp32", _nc_sum_fp32(_ptrs(xs), n, d, _ptr(out), _stream(stream)))
+
+
+# ---- D_nat ---------------------------------------------------------------------------
+def nd_compress(x, d, bucket_off, B, p, s, seed, worker, norms, level, sign, workspace,
+                workspace_bytes, stream=None) -> None:
+    _check("nd_compress", _nd_compress(_ptr(x), d, _ptr(bucket_off), B, p, s, seed, worker,
+                                       _ptr(norms), _ptr(level), _ptr(sign), _ptr(workspace),
+                                       workspace_bytes, _stream(stream)))
+
+
+def nd_decode_accumulate(norms, level, sign, d, bucket_off, B, s, acc, stream=None) -> None:
+    _check("nd_decode_accumulate", _nd_decode_accumulate(_ptr(norms), _ptr(level), _ptr(sign), d,
+                                                         _ptr(bucket_off), B, s, _ptr(acc),
+                                                         _stream(stream)))
+
+
+def nd_aggregate(norms, levels, signs, n, d, bucket_off, B, s, out, stream=None) -> None:
+    _check("nd_aggregate", _nd_aggregate(_ptrs(norms), _ptrs(levels), _ptrs(signs), n, d,
+                                         _ptr(bucket_off), B, s, _ptr(out), _stream(stream)))
+
+
+# ---- sparsifier composed with D_nat ----------------------------------------------------
+def nd_sparse_compress(x, d, keep_threshold, scale, p, s, seed, worker, idx, codes, count, norm,
+                       cap, workspace, workspace_bytes, stream=None) -> None:
+    _check("nd_sparse_compress", _nd_sparse_compress(_ptr(x), d, keep_threshold, scale, p, s,
+                                                     seed, worker, _ptr(idx), _ptr(codes),
+                                                     _ptr(count), _ptr(norm), cap,
+                                                     _ptr(workspace), workspace_bytes,
+                                                     _stream(stream)))
+
+
+def nd_sparse_decode_accumulate(idx, codes, count, norm, s, d, cap, acc, stream=None) -> None:
+    _check("nd_sparse_decode_accumulate",
+           _nd_sparse_decode_accumulate(_ptr(idx), _ptr(codes), _ptr(count), _ptr(norm), s, d,
+                                        cap, _ptr(acc), _stream(stream)))

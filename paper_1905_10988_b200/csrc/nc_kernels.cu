@@ -1,0 +1,287 @@
+// Natural compression C_nat (Def. 1 / Sec. 2 of arXiv 1905.10988) and the master-side
+// aggregation of Algorithm 1, hand-written for sm_100a.
+//
+// Work decomposition: one warp owns a tile of 1024 consecutive elements.  Lane l loads the
+// float4 groups k*32 + l (k = 0..7) of the tile, so every warp-wide access is one contiguous
+// 512-byte (loads, fp32 stores) or 128-byte (exponent bytes, sign words) segment.  A float4
+// group is exactly one Philox4x32-10 block, so no random word is computed twice.
+//
+// C_nat on the binary32 fields is integer-only: with v = bits & 0x7FFFFFFF and r23 the low 23
+// random bits, v + (~r23 & 0x7FFFFF) carries into the exponent field iff r23 < mantissa, i.e.
+// with probability m (Sec. 2: round up with probability m).  The add is suppressed for biased
+// exponents 254 and 255 (saturation / inf / NaN policy).
+#include "common.cuh"
+#include "philox.cuh"
+
+namespace natcomp {
+
+struct CompressBatch {
+    const float* x[NC_MAX_WORKERS];
+    uint8_t* exp[NC_MAX_WORKERS];
+    uint32_t* sign[NC_MAX_WORKERS];
+    uint32_t worker[NC_MAX_WORKERS];
+};
+
+struct PackedPlanes {
+    const uint8_t* exp[NC_MAX_WORKERS];
+    const uint32_t* sign[NC_MAX_WORKERS];
+};
+
+struct DensePlanes {
+    const float* x[NC_MAX_WORKERS];
+};
+
+// exponent byte of C_nat(bits) given the element's random word
+__device__ __forceinline__ uint32_t cnat_exp_byte(uint32_t bits, uint32_t rnd) {
+    uint32_t v = bits & 0x7FFFFFFFu;
+    const uint32_t rr = ~rnd & 0x7FFFFFu;
+    if (v < 0x7F000000u) v += rr;
+    return v >> 23;
+}
+
+// grid: (ceil(tiles / warps per block), n workers)
+__global__ void __launch_bounds__(kBlockThreads)
+nc_compress_kernel(const __grid_constant__ CompressBatch batch, const uint64_t d,
+                   const __grid_constant__ PhiloxKeys keys) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+    const int w = blockIdx.y;
+    const float* __restrict__ x = batch.x[w];
+    uint8_t* __restrict__ exp = batch.exp[w];
+    uint32_t* __restrict__ sign = batch.sign[w];
+    const uint32_t worker = batch.worker[w];
+
+    if (base + kTile <= d) {
+        // ---- full tile ------------------------------------------------------------
+        const uint4* xv = reinterpret_cast<const uint4*>(x + base);
+        uint4 u[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) u[k] = ld_stream_u4(xv + k * 32 + lane);
+
+        uint32_t* ev = reinterpret_cast<uint32_t*>(exp + base);
+        uint32_t nib = 0;   // sign bits of this lane's 32 elements: bit 4k+c <-> group k, element c
+#pragma unroll
+        for (int k = 7; k >= 0; --k) {
+            uint32_t rnd[4];
+            stream_words4((base >> 2) + (uint64_t)(k * 32 + lane), worker, kDomainCnat, keys, rnd);
+            const uint32_t b0 = u[k].x, b1 = u[k].y, b2 = u[k].z, b3 = u[k].w;
+            uint32_t e = cnat_exp_byte(b3, rnd[3]);
+            e = (e << 8) | cnat_exp_byte(b2, rnd[2]);
+            e = (e << 8) | cnat_exp_byte(b1, rnd[1]);
+            e = (e << 8) | cnat_exp_byte(b0, rnd[0]);
+            st_stream_u32(ev + k * 32 + lane, e);
+            nib = __funnelshift_l(b3, nib, 1);
+            nib = __funnelshift_l(b2, nib, 1);
+            nib = __funnelshift_l(b1, nib, 1);
+            nib = __funnelshift_l(b0, nib, 1);
+        }
+        // lane 8g+i holds nibble k of sign word (k, g); after the transpose lane 8g+k holds the
+        // whole word covering elements k*128 + g*32 .. +31 of the tile.
+        const uint32_t word = transpose_nibbles_8x8(nib, lane);
+        st_stream_u32(sign + (base >> 5) + (lane & 7) * 4 + (lane >> 3), word);
+        return;
+    }
+
+    // ---- ragged last tile: one element per lane per step, ballot gives the sign word ----
+    const uint64_t exp_end = round_up16(d);                 // bytes incl. zero padding
+    const uint64_t sign_words = (d + 31) / 32;
+    const uint64_t sign_words_padded = (sign_words + 3) & ~(uint64_t)3;
+    for (uint64_t j0 = base; j0 < exp_end; j0 += 32) {
+        const uint64_t j = j0 + lane;
+        uint32_t bits = 0, e = 0;
+        if (j < d) {
+            bits = __float_as_uint(x[j]);
+            uint32_t rnd[4];
+            stream_words4(j >> 2, worker, kDomainCnat, keys, rnd);
+            const uint32_t r = (j & 3) == 0 ? rnd[0] : (j & 3) == 1 ? rnd[1]
+                             : (j & 3) == 2 ? rnd[2] : rnd[3];
+            e = cnat_exp_byte(bits, r);
+        }
+        if (j < exp_end) exp[j] = (uint8_t)e;
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, (bits >> 31) != 0);
+        if (lane == 0 && (j0 >> 5) < sign_words) sign[j0 >> 5] = word;
+    }
+    if (lane < (int)(sign_words_padded - sign_words)) sign[sign_words + lane] = 0;
+}
+
+// value of a 9-bit code: exponent byte in byte `BYTE` of `e4`, sign in bit 0 of `s`
+template <int BYTE>
+__device__ __forceinline__ float decode9(uint32_t e4, uint32_t s) {
+    const uint32_t hi = __byte_perm(e4, 0u, 0x0444 | (BYTE << 12));   // exponent -> bits 24..31
+    return __uint_as_float(__funnelshift_r(hi, s, 1));                // (hi >> 1) | (s << 31)
+}
+
+// out[j] = (init + v_0j) + v_1j + ... ; init = +0 (aggregate) or acc[j] (decode-accumulate).
+// grid: ceil(tiles / warps per block)
+template <bool kFromAcc>
+__global__ void __launch_bounds__(kBlockThreads)
+nc_aggregate_kernel(const __grid_constant__ PackedPlanes planes, const int n, const uint64_t d,
+                    float* __restrict__ out) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+
+    if (base + kTile <= d) {
+        float4 acc[8];
+        float4* ov = reinterpret_cast<float4*>(out + base);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (kFromAcc) acc[k] = __ldcs(ov + k * 32 + lane);
+            else acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        const int sh = 4 * (lane & 7);
+        for (int i = 0; i < n; ++i) {
+            const uint32_t* ev = reinterpret_cast<const uint32_t*>(planes.exp[i] + base);
+            const uint32_t sw = ld_stream_u32(planes.sign[i] + (base >> 5) + lane);
+            uint32_t e[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) e[k] = ld_stream_u32(ev + k * 32 + lane);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                // sign word (k, g) lives in lane 4k+g; this lane needs group g = lane / 8
+                const uint32_t s = __shfl_sync(0xFFFFFFFFu, sw, k * 4 + (lane >> 3)) >> sh;
+                acc[k].x += decode9<0>(e[k], s);
+                acc[k].y += decode9<1>(e[k], s >> 1);
+                acc[k].z += decode9<2>(e[k], s >> 2);
+                acc[k].w += decode9<3>(e[k], s >> 3);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) __stcs(ov + k * 32 + lane, acc[k]);
+        return;
+    }
+
+    // ragged last tile: scalar
+    for (uint64_t j = base + lane; j < d; j += 32) {
+        float a = kFromAcc ? out[j] : 0.f;
+        for (int i = 0; i < n; ++i) {
+            const uint32_t e = planes.exp[i][j];
+            const uint32_t s = (planes.sign[i][j >> 5] >> (j & 31)) & 1u;
+            a += __uint_as_float((e << 23) | (s << 31));
+        }
+        out[j] = a;
+    }
+}
+
+// uncompressed reference point: n-way fp32 sum in worker order
+__global__ void __launch_bounds__(kBlockThreads)
+nc_sum_fp32_kernel(const __grid_constant__ DensePlanes planes, const int n, const uint64_t d,
+                   float* __restrict__ out) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+    if (base + kTile <= d) {
+        float4 acc[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = 0; i < n; ++i) {
+            const float4* xv = reinterpret_cast<const float4*>(planes.x[i] + base);
+            float4 v[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v[k] = __ldcs(xv + k * 32 + lane);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                acc[k].x += v[k].x; acc[k].y += v[k].y; acc[k].z += v[k].z; acc[k].w += v[k].w;
+            }
+        }
+        float4* ov = reinterpret_cast<float4*>(out + base);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) __stcs(ov + k * 32 + lane, acc[k]);
+        return;
+    }
+    for (uint64_t j = base + lane; j < d; j += 32) {
+        float a = 0.f;
+        for (int i = 0; i < n; ++i) a += planes.x[i][j];
+        out[j] = a;
+    }
+}
+
+inline unsigned tile_blocks(uint64_t d) {
+    const uint64_t tiles = (d + kTile - 1) / kTile;
+    return (unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock);
+}
+
+}  // namespace natcomp
+
+using namespace natcomp;
+
+extern "C" {
+
+nc_status nc_compress_batch(const float* const* xs, size_t d, uint64_t seed,
+                            const uint32_t* workers, uint8_t* const* exps,
+                            uint32_t* const* signs, int n, cudaStream_t stream) {
+    if (!xs || !workers || !exps || !signs || n < 1 || n > NC_MAX_WORKERS) return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    CompressBatch batch;
+    for (int i = 0; i < n; ++i) {
+        if (!xs[i] || !exps[i] || !signs[i]) return NC_ERR_INVALID;
+        if (!aligned32(xs[i]) || !aligned16(exps[i]) || !aligned16(signs[i])) return NC_ERR_ALIGN;
+        batch.x[i] = xs[i];
+        batch.exp[i] = exps[i];
+        batch.sign[i] = signs[i];
+        batch.worker[i] = workers[i];
+    }
+    const PhiloxKeys keys = make_philox_keys(seed);
+    dim3 grid(tile_blocks(d), (unsigned)n);
+    nc_compress_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, (uint64_t)d, keys);
+    return launch_status();
+}
+
+nc_status nc_compress(const float* x, size_t d, uint64_t seed, uint32_t worker, uint8_t* exp,
+                      uint32_t* sign, cudaStream_t stream) {
+    return nc_compress_batch(&x, d, seed, &worker, &exp, &sign, 1, stream);
+}
+
+nc_status nc_aggregate(const uint8_t* const* exps, const uint32_t* const* signs, int n, size_t d,
+                       float* out, cudaStream_t stream) {
+    if (!exps || !signs || !out || n < 1 || n > NC_MAX_WORKERS) return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    if (!aligned32(out)) return NC_ERR_ALIGN;
+    PackedPlanes planes;
+    for (int i = 0; i < n; ++i) {
+        if (!exps[i] || !signs[i]) return NC_ERR_INVALID;
+        if (!aligned16(exps[i]) || !aligned16(signs[i])) return NC_ERR_ALIGN;
+        planes.exp[i] = exps[i];
+        planes.sign[i] = signs[i];
+    }
+    nc_aggregate_kernel<false><<<tile_blocks(d), kBlockThreads, 0, stream>>>(planes, n,
+                                                                             (uint64_t)d, out);
+    return launch_status();
+}
+
+nc_status nc_decode_accumulate(const uint8_t* exp, const uint32_t* sign, size_t d, float* acc,
+                               cudaStream_t stream) {
+    if (!exp || !sign || !acc) return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    if (!aligned16(exp) || !aligned16(sign) || !aligned32(acc)) return NC_ERR_ALIGN;
+    PackedPlanes planes;
+    planes.exp[0] = exp;
+    planes.sign[0] = sign;
+    nc_aggregate_kernel<true><<<tile_blocks(d), kBlockThreads, 0, stream>>>(planes, 1,
+                                                                            (uint64_t)d, acc);
+    return launch_status();
+}
+
+nc_status nc_sum_fp32(const float* const* xs, int n, size_t d, float* out, cudaStream_t stream) {
+    if (!xs || !out || n < 1 || n > NC_MAX_WORKERS) return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    if (!aligned32(out)) return NC_ERR_ALIGN;
+    DensePlanes planes;
+    for (int i = 0; i < n; ++i) {
+        if (!xs[i]) return NC_ERR_INVALID;
+        if (!aligned32(xs[i])) return NC_ERR_ALIGN;
+        planes.x[i] = xs[i];
+    }
+    nc_sum_fp32_kernel<<<tile_blocks(d), kBlockThreads, 0, stream>>>(planes, n, (uint64_t)d, out);
+    return launch_status();
+}
+
+}  // extern "C"

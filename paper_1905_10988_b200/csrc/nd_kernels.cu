@@ -1,0 +1,522 @@
+// Natural dithering D_nat^{p,s} (Def. 3 of arXiv 1905.10988 with the levels 2^-u) for
+// sm_100a: per-bucket p-norm, level rounding + packing, and the master-side decode / n-way sum.
+//
+// Work decomposition: one warp owns a tile of 1024 consecutive elements in four steps of 256;
+// in a step lane l owns the 8 consecutive elements 8l..8l+7 (one 256-bit load, two Philox
+// blocks, one 32-bit word of level nibbles, one byte of sign bits).
+//
+// Norms are deterministic: every (tile, bucket) overlap writes one partial into its own slot
+// (slot = tile index + bucket index, strictly increasing along the vector), and one warp per
+// bucket adds the bucket's slots in a fixed order.  No atomics, no zero-filling.
+//
+// Level rounding (given the bucket norm): y = fl32(|x| * fl32(1/norm)), z = y * 2^s (exact).
+// For z >= 2 the level below is 2^(E_z - 127 - s) and the up-probability is the mantissa
+// fraction of z, exactly as in C_nat; for z < 2 (y below the smallest level 2^(1-s)) the
+// up-probability is y * 2^(s-1), obtained as the mantissa of 1 + z/2 rounded toward zero.
+// In both cases  code = min(((bits(w) + (~r23 & 0x7FFFFF)) >> 23) - 127, s).
+#include "common.cuh"
+#include "philox.cuh"
+
+namespace natcomp {
+
+struct DitherPlanes {
+    const float* norms[NC_MAX_WORKERS];
+    const uint8_t* level[NC_MAX_WORKERS];
+    const uint32_t* sign[NC_MAX_WORKERS];
+};
+
+struct V8 {
+    uint32_t v[8];
+};
+
+__device__ __forceinline__ V8 ld_stream_v8(const void* p) {
+    V8 r;
+    asm volatile("ld.global.cs.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]), "=r"(r.v[4]),
+                   "=r"(r.v[5]), "=r"(r.v[6]), "=r"(r.v[7])
+                 : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ void st_stream_v8(void* p, const V8& r) {
+    asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(r.v[0]),
+                 "r"(r.v[1]), "r"(r.v[2]), "r"(r.v[3]), "r"(r.v[4]), "r"(r.v[5]), "r"(r.v[6]),
+                 "r"(r.v[7])
+                 : "memory");
+}
+
+// 4x4 transpose of bytes across each aligned group of 4 lanes: lane i holds bytes b[i][t]
+// (t = 0..3) -> lane t holds bytes b[i][t] (i = 0..3, byte i).
+__device__ __forceinline__ uint32_t transpose_bytes_4x4(uint32_t v, int lane) {
+    uint32_t t = __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+    v = __byte_perm(v, t, (lane & 2) ? 0x3276 : 0x5410);
+    t = __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+    v = __byte_perm(v, t, (lane & 1) ? 0x3715 : 0x6240);
+    return v;
+}
+
+// largest b in [0, B-1] with off[b] <= pos (pos < off[B]); skips empty buckets by construction
+__device__ __forceinline__ int find_bucket(const uint64_t* __restrict__ off, int B, uint64_t pos) {
+    int lo = 0, hi = B;   // invariant: off[lo] <= pos < off[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(off + mid) <= pos) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ uint32_t warp_max(uint32_t v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+
+// One partial per (tile, bucket) overlap.  p = 1: sum |x|, p = 2: sum x^2 (binary32 products,
+// chains of at most 8 terms in binary32, everything above that in binary64), p = inf: the
+// largest |x| as a bit pattern (NaN patterns compare above inf, so a NaN survives).
+template <int P>
+struct NormAcc {
+    float f[4];
+    double q[4];
+    double dsum;
+    uint32_t m;
+    __device__ __forceinline__ void init() {
+        f[0] = f[1] = f[2] = f[3] = 0.f;
+        q[0] = q[1] = q[2] = q[3] = 0.0;
+        dsum = 0.0;
+        m = 0;
+    }
+    __device__ __forceinline__ void add(uint32_t bits, int chain) {
+        const uint32_t a = bits & 0x7FFFFFFFu;
+        if (P == NC_P_INF) m = max(m, a);
+        else if (P == 1) f[chain] += __uint_as_float(a);
+        else {
+            // squares in binary64: a binary32 square underflows for |x| < 2^-63
+            const double v = (double)__uint_as_float(a);
+            q[chain] = fma(v, v, q[chain]);
+        }
+    }
+    __device__ __forceinline__ void flush() {
+        if (P == 1) {
+            dsum += ((double)f[0] + (double)f[1]) + ((double)f[2] + (double)f[3]);
+            f[0] = f[1] = f[2] = f[3] = 0.f;
+        } else if (P == 2) {
+            dsum += (q[0] + q[1]) + (q[2] + q[3]);
+            q[0] = q[1] = q[2] = q[3] = 0.0;
+        }
+    }
+    // warp-wide result as 64 bits for the slot
+    __device__ __forceinline__ uint64_t reduce() {
+        if (P == NC_P_INF) return (uint64_t)warp_max(m);
+        flush();
+        return (uint64_t)__double_as_longlong(warp_sum(dsum));
+    }
+};
+
+// grid: ceil(tiles / warps per block)
+template <int P>
+__global__ void __launch_bounds__(kBlockThreads)
+nd_norm_partials_kernel(const float* __restrict__ x, const uint64_t d,
+                        const uint64_t* __restrict__ off, const int B,
+                        uint64_t* __restrict__ slots, uint32_t* __restrict__ tile_bucket) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+    const uint64_t end = (base + kTile <= d) ? base + kTile : d;
+    const bool full = (base + kTile <= d);
+
+    V8 u[4];
+    if (full) {
+#pragma unroll
+        for (int it = 0; it < 4; ++it) u[it] = ld_stream_v8(x + base + it * 256 + lane * 8);
+    }
+    int b = find_bucket(off, B, base);
+    if (lane == 0) tile_bucket[tile] = (uint32_t)b;
+
+    NormAcc<P> acc;
+    if (full && __ldg(off + b + 1) >= end) {
+        acc.init();
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) acc.add(u[it].v[c], c & 3);
+        }
+        const uint64_t r = acc.reduce();
+        if (lane == 0) slots[tile + (uint64_t)b] = r;
+        return;
+    }
+    // the tile spans several buckets or is ragged: one segment at a time, lane-strided
+    uint64_t pos = base;
+    while (pos < end) {
+        uint64_t seg_end = __ldg(off + b + 1);
+        if (seg_end > end) seg_end = end;
+        acc.init();
+        int cnt = 0;
+        for (uint64_t j = pos + lane; j < seg_end; j += 32) {
+            acc.add(__float_as_uint(x[j]), 0);
+            if (++cnt == 8) { acc.flush(); cnt = 0; }
+        }
+        const uint64_t r = acc.reduce();
+        if (lane == 0) slots[tile + (uint64_t)b] = r;
+        pos = seg_end;
+        if (pos < end) {
+            ++b;
+            while (__ldg(off + b + 1) <= pos) ++b;   // skip empty buckets
+        }
+    }
+}
+
+// one warp per bucket: fixed-order sum (or max) of the bucket's slots -> norms[b]
+template <int P>
+__global__ void __launch_bounds__(kBlockThreads)
+nd_norm_finalize_kernel(const uint64_t* __restrict__ off, const int B,
+                        const uint64_t* __restrict__ slots, float* __restrict__ norms) {
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    if (b >= B) return;
+    const uint64_t lo = off[b], hi = off[b + 1];
+    float result = 0.f;
+    if (hi > lo) {
+        const uint64_t t_first = lo / kTile, t_last = (hi - 1) / kTile;
+        if (P == NC_P_INF) {
+            uint32_t m = 0;
+            for (uint64_t t = t_first + lane; t <= t_last; t += 32)
+                m = max(m, (uint32_t)slots[t + (uint64_t)b]);
+            result = __uint_as_float(warp_max(m));
+        } else {
+            double s = 0.0;
+            for (uint64_t t = t_first + lane; t <= t_last; t += 32)
+                s += __longlong_as_double((long long)slots[t + (uint64_t)b]);
+            s = warp_sum(s);
+            if (P == 2) s = sqrt(s);
+            result = (float)s;
+        }
+    }
+    if (lane == 0) norms[b] = result;
+}
+
+struct BucketScale {
+    float rinv;      // fl32(1 / norm), or 0 for a degenerate bucket
+    uint32_t smax;   // s, or 0 for a degenerate bucket (forces every code to 0)
+};
+
+__device__ __forceinline__ BucketScale bucket_scale(float norm, int s) {
+    BucketScale r;
+    const bool ok = (norm >= 1.17549435e-38f) && (norm <= 3.40282347e38f);
+    r.rinv = ok ? __fdiv_rn(1.0f, norm) : 0.f;
+    r.smax = ok ? (uint32_t)s : 0u;
+    return r;
+}
+
+// level code of one entry; pow2s = 2^s as a float
+__device__ __forceinline__ uint32_t level_code(uint32_t bits, uint32_t rnd, const BucketScale sc,
+                                               float pow2s) {
+    const float ax = __uint_as_float(bits & 0x7FFFFFFFu);
+    const float y = __fmul_rn(ax, sc.rinv);
+    const float z = __fmul_rn(y, pow2s);
+    float w = z;
+    if (z < 2.0f) w = __fmaf_rz(z, 0.5f, 1.0f);
+    const uint32_t t = __float_as_uint(w) + (~rnd & 0x7FFFFFu) - 0x3F800000u;
+    return min(t >> 23, sc.smax);
+}
+
+// grid: ceil(tiles / warps per block)
+__global__ void __launch_bounds__(kBlockThreads)
+nd_round_pack_kernel(const float* __restrict__ x, const uint64_t d,
+                     const uint64_t* __restrict__ off, const int B, const int s,
+                     const uint32_t worker, const __grid_constant__ PhiloxKeys keys,
+                     const float* __restrict__ norms, const uint32_t* __restrict__ tile_bucket,
+                     uint8_t* __restrict__ level, uint32_t* __restrict__ sign) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+    const bool full = (base + kTile <= d);
+    const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
+
+    V8 u[4];
+    if (full) {
+#pragma unroll
+        for (int it = 0; it < 4; ++it) u[it] = ld_stream_v8(x + base + it * 256 + lane * 8);
+    }
+    int b = (int)tile_bucket[tile];
+
+    if (full && __ldg(off + b + 1) >= base + kTile) {
+        const BucketScale sc = bucket_scale(norms[b], s);
+        uint32_t* lv = reinterpret_cast<uint32_t*>(level + (base >> 1));
+        uint32_t sbytes = 0;     // byte `it` = sign bits of this lane's 8 elements in step it
+#pragma unroll
+        for (int it = 3; it >= 0; --it) {
+            uint32_t rnd[8];
+            const uint64_t q = (base >> 2) + (uint64_t)(it * 64 + lane * 2);
+            {
+                uint32_t r4[4];
+                stream_words4(q, worker, kDomainDnat, keys, r4);
+                rnd[0] = r4[0]; rnd[1] = r4[1]; rnd[2] = r4[2]; rnd[3] = r4[3];
+                stream_words4(q + 1, worker, kDomainDnat, keys, r4);
+                rnd[4] = r4[0]; rnd[5] = r4[1]; rnd[6] = r4[2]; rnd[7] = r4[3];
+            }
+            uint32_t nib = 0;
+#pragma unroll
+            for (int c = 7; c >= 0; --c) {
+                nib = (nib << 4) | level_code(u[it].v[c], rnd[c], sc, pow2s);
+                sbytes = __funnelshift_l(u[it].v[c], sbytes, 1);
+            }
+            st_stream_u32(lv + it * 32 + lane, nib);
+        }
+        // lane 4g+i holds byte i of sign word (it, g) = word it*8 + g of the tile
+        const uint32_t word = transpose_bytes_4x4(sbytes, lane);
+        st_stream_u32(sign + (base >> 5) + (lane & 3) * 8 + (lane >> 2), word);
+        return;
+    }
+
+    // tile spans several buckets or is the ragged end: one element per lane per step
+    const uint64_t lvl_end = round_up16((d + 1) / 2) * 2;   // elements covered by level bytes
+    const uint64_t sign_words = (d + 31) / 32;
+    const uint64_t sign_words_padded = (sign_words + 3) & ~(uint64_t)3;
+    uint64_t tile_end = base + kTile;
+    if (!full) tile_end = lvl_end > base ? lvl_end : base;
+    if (tile_end > base + kTile) tile_end = base + kTile;
+    int bl = b;                    // per-lane bucket cursor
+    uint64_t bend = __ldg(off + bl + 1);
+    BucketScale sc = bucket_scale(norms[bl], s);
+    for (uint64_t j0 = base; j0 < tile_end; j0 += 32) {
+        const uint64_t j = j0 + lane;
+        uint32_t bits = 0, code = 0;
+        if (j < d) {
+            if (j >= bend) {
+                do { ++bl; bend = __ldg(off + bl + 1); } while (j >= bend);
+                sc = bucket_scale(norms[bl], s);
+            }
+            bits = __float_as_uint(x[j]);
+            uint32_t r4[4];
+            stream_words4(j >> 2, worker, kDomainDnat, keys, r4);
+            const uint32_t r = (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1]
+                             : (j & 3) == 2 ? r4[2] : r4[3];
+            code = level_code(bits, r, sc, pow2s);
+        }
+        const uint32_t next = __shfl_down_sync(0xFFFFFFFFu, code, 1);
+        if ((lane & 1) == 0 && j < lvl_end) level[j >> 1] = (uint8_t)(code | (next << 4));
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, (bits >> 31) != 0);
+        if (lane == 0 && (j0 >> 5) < sign_words) sign[j0 >> 5] = word;
+    }
+    if (!full && lane < (int)(sign_words_padded - sign_words)) sign[sign_words + lane] = 0;
+}
+
+// ---- master side ------------------------------------------------------------------------
+
+// 8 level nibbles -> exponent bytes of 2^(c-s) (0 for c = 0), four per register
+__device__ __forceinline__ void level_exp_bytes(uint32_t nib8, uint32_t kexp, uint32_t& lo4,
+                                                uint32_t& hi4) {
+    // spread nibbles to bytes: lo4 = nibbles 0..3, hi4 = nibbles 4..7
+    uint32_t a = nib8 & 0xFFFFu, b = nib8 >> 16;
+    a = (a | (a << 8)) & 0x00FF00FFu;
+    a = (a | (a << 4)) & 0x0F0F0F0Fu;
+    b = (b | (b << 8)) & 0x00FF00FFu;
+    b = (b | (b << 4)) & 0x0F0F0F0Fu;
+    // add (127 - s) to every non-zero byte: (x + 0x7F) has bit 7 set iff x >= 1
+    const uint32_t ma = ((a + 0x7F7F7F7Fu) & 0x80808080u) >> 7;
+    const uint32_t mb = ((b + 0x7F7F7F7Fu) & 0x80808080u) >> 7;
+    lo4 = a + ma * kexp;
+    hi4 = b + mb * kexp;
+}
+
+template <int BYTE>
+__device__ __forceinline__ float pow2_signed(uint32_t e4, uint32_t s) {
+    const uint32_t hi = __byte_perm(e4, 0u, 0x0444 | (BYTE << 12));
+    return __uint_as_float(__funnelshift_r(hi, s, 1));
+}
+
+// fl32(norm * p) followed by a separate binary32 add (p = +-2^(c-s) or +-0)
+__device__ __forceinline__ float add_scaled(float acc, float norm, float p) {
+    return __fadd_rn(acc, __fmul_rn(norm, p));
+}
+
+// grid: ceil(tiles / warps per block)
+template <bool kFromAcc>
+__global__ void __launch_bounds__(kBlockThreads)
+nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, const uint64_t d,
+                    const uint64_t* __restrict__ off, const int B, const int s,
+                    float* __restrict__ out) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+    const bool full = (base + kTile <= d);
+    int b = find_bucket(off, B, base);
+
+    if (full && __ldg(off + b + 1) >= base + kTile) {
+        V8 acc[4];
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            if (kFromAcc) acc[it] = ld_stream_v8(out + base + it * 256 + lane * 8);
+            else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) acc[it].v[c] = 0u;
+            }
+        }
+        const uint32_t kexp = (uint32_t)(127 - s);
+        const int sh = 8 * (lane & 3);
+        for (int i = 0; i < n; ++i) {
+            float norm = __ldg(planes.norms[i] + b);
+            if (!(fabsf(norm) <= 3.40282347e38f)) norm = 0.f;   // codes of such a bucket are 0
+            const uint32_t* lv = reinterpret_cast<const uint32_t*>(planes.level[i] + (base >> 1));
+            const uint32_t sw = ld_stream_u32(planes.sign[i] + (base >> 5) + lane);
+            uint32_t nb[4];
+#pragma unroll
+            for (int it = 0; it < 4; ++it) nb[it] = ld_stream_u32(lv + it * 32 + lane);
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+                const uint32_t sg = __shfl_sync(0xFFFFFFFFu, sw, it * 8 + (lane >> 2)) >> sh;
+                uint32_t lo4, hi4;
+                level_exp_bytes(nb[it], kexp, lo4, hi4);
+                float* a = reinterpret_cast<float*>(acc[it].v);
+                a[0] = add_scaled(a[0], norm, pow2_signed<0>(lo4, sg));
+                a[1] = add_scaled(a[1], norm, pow2_signed<1>(lo4, sg >> 1));
+                a[2] = add_scaled(a[2], norm, pow2_signed<2>(lo4, sg >> 2));
+                a[3] = add_scaled(a[3], norm, pow2_signed<3>(lo4, sg >> 3));
+                a[4] = add_scaled(a[4], norm, pow2_signed<0>(hi4, sg >> 4));
+                a[5] = add_scaled(a[5], norm, pow2_signed<1>(hi4, sg >> 5));
+                a[6] = add_scaled(a[6], norm, pow2_signed<2>(hi4, sg >> 6));
+                a[7] = add_scaled(a[7], norm, pow2_signed<3>(hi4, sg >> 7));
+            }
+        }
+#pragma unroll
+        for (int it = 0; it < 4; ++it) st_stream_v8(out + base + it * 256 + lane * 8, acc[it]);
+        return;
+    }
+
+    // tile spans several buckets or is ragged: scalar, per-lane bucket cursor
+    const uint64_t end = full ? base + kTile : d;
+    uint64_t bend = __ldg(off + b + 1);
+    for (uint64_t j = base + lane; j < end; j += 32) {
+        while (j >= bend) { ++b; bend = __ldg(off + b + 1); }
+        float a = kFromAcc ? out[j] : 0.f;
+        for (int i = 0; i < n; ++i) {
+            float norm = __ldg(planes.norms[i] + b);
+            if (!(fabsf(norm) <= 3.40282347e38f)) norm = 0.f;
+            const uint32_t c = (planes.level[i][j >> 1] >> (4 * (j & 1))) & 0xFu;
+            const uint32_t sg = (planes.sign[i][j >> 5] >> (j & 31)) & 1u;
+            const uint32_t pb = (c ? ((c + 127u - (uint32_t)s) << 23) : 0u) | (sg << 31);
+            a = add_scaled(a, norm, __uint_as_float(pb));
+        }
+        out[j] = a;
+    }
+}
+
+inline unsigned nd_tile_blocks(uint64_t d) {
+    const uint64_t tiles = (d + kTile - 1) / kTile;
+    return (unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock);
+}
+
+inline uint64_t nd_tiles(uint64_t d) { return (d + kTile - 1) / kTile; }
+
+}  // namespace natcomp
+
+using namespace natcomp;
+
+extern "C" {
+
+size_t nd_workspace_bytes(size_t d, int num_buckets) {
+    if (num_buckets < 0) num_buckets = 0;
+    const uint64_t tiles = nd_tiles(d);
+    // slots: one 64-bit partial per (tile, bucket) overlap; then the tile -> bucket map
+    return round_up16((tiles + (uint64_t)num_buckets + 1) * 8) + round_up16(tiles * 4);
+}
+
+nc_status nd_compress(const float* x, size_t d, const uint64_t* bucket_off, int B, int p, int s,
+                      uint64_t seed, uint32_t worker, float* norms, uint8_t* level,
+                      uint32_t* sign, void* workspace, size_t workspace_bytes,
+                      cudaStream_t stream) {
+    if (!x || !bucket_off || !norms || !level || !sign || B < 1 || s < 1 || s > 15)
+        return NC_ERR_INVALID;
+    if (p != 1 && p != 2 && p != NC_P_INF) return NC_ERR_UNSUPPORTED;
+    if (d == 0) return NC_OK;
+    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    if (!workspace) return NC_ERR_INVALID;
+    if (!aligned32(x) || !aligned16(level) || !aligned16(sign) || !aligned16(workspace) ||
+        !aligned4(norms) || ((uintptr_t)bucket_off & 7u))
+        return NC_ERR_ALIGN;
+    if (workspace_bytes < nd_workspace_bytes(d, B)) return NC_ERR_WORKSPACE;
+    const uint64_t tiles = nd_tiles(d);
+    uint64_t* slots = reinterpret_cast<uint64_t*>(workspace);
+    uint32_t* tile_bucket = reinterpret_cast<uint32_t*>(
+        reinterpret_cast<char*>(workspace) + round_up16((tiles + (uint64_t)B + 1) * 8));
+    const unsigned grid = nd_tile_blocks(d);
+    const unsigned fgrid = (unsigned)((B + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    if (p == 1) {
+        nd_norm_partials_kernel<1><<<grid, kBlockThreads, 0, stream>>>(x, d, bucket_off, B, slots,
+                                                                       tile_bucket);
+        nd_norm_finalize_kernel<1><<<fgrid, kBlockThreads, 0, stream>>>(bucket_off, B, slots,
+                                                                        norms);
+    } else if (p == 2) {
+        nd_norm_partials_kernel<2><<<grid, kBlockThreads, 0, stream>>>(x, d, bucket_off, B, slots,
+                                                                       tile_bucket);
+        nd_norm_finalize_kernel<2><<<fgrid, kBlockThreads, 0, stream>>>(bucket_off, B, slots,
+                                                                        norms);
+    } else {
+        nd_norm_partials_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
+            x, d, bucket_off, B, slots, tile_bucket);
+        nd_norm_finalize_kernel<NC_P_INF><<<fgrid, kBlockThreads, 0, stream>>>(bucket_off, B,
+                                                                               slots, norms);
+    }
+    const PhiloxKeys keys = make_philox_keys(seed);
+    nd_round_pack_kernel<<<grid, kBlockThreads, 0, stream>>>(x, d, bucket_off, B, s, worker, keys,
+                                                             norms, tile_bucket, level, sign);
+    return launch_status();
+}
+
+static nc_status nd_check_planes(const float* const* norms, const uint8_t* const* levels,
+                                 const uint32_t* const* signs, int n, DitherPlanes* planes) {
+    for (int i = 0; i < n; ++i) {
+        if (!norms[i] || !levels[i] || !signs[i]) return NC_ERR_INVALID;
+        if (!aligned4(norms[i]) || !aligned16(levels[i]) || !aligned16(signs[i]))
+            return NC_ERR_ALIGN;
+        planes->norms[i] = norms[i];
+        planes->level[i] = levels[i];
+        planes->sign[i] = signs[i];
+    }
+    return NC_OK;
+}
+
+nc_status nd_aggregate(const float* const* norms, const uint8_t* const* levels,
+                       const uint32_t* const* signs, int n, size_t d, const uint64_t* bucket_off,
+                       int B, int s, float* out, cudaStream_t stream) {
+    if (!norms || !levels || !signs || !bucket_off || !out || n < 1 || n > NC_MAX_WORKERS ||
+        B < 1 || s < 1 || s > 15)
+        return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    if (!aligned32(out) || ((uintptr_t)bucket_off & 7u)) return NC_ERR_ALIGN;
+    DitherPlanes planes;
+    const nc_status st = nd_check_planes(norms, levels, signs, n, &planes);
+    if (st != NC_OK) return st;
+    nd_aggregate_kernel<false><<<nd_tile_blocks(d), kBlockThreads, 0, stream>>>(
+        planes, n, (uint64_t)d, bucket_off, B, s, out);
+    return launch_status();
+}
+
+nc_status nd_decode_accumulate(const float* norms, const uint8_t* level, const uint32_t* sign,
+                               size_t d, const uint64_t* bucket_off, int B, int s, float* acc,
+                               cudaStream_t stream) {
+    if (!norms || !level || !sign || !bucket_off || !acc || B < 1 || s < 1 || s > 15)
+        return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    if (!aligned32(acc) || ((uintptr_t)bucket_off & 7u)) return NC_ERR_ALIGN;
+    DitherPlanes planes;
+    const nc_status st = nd_check_planes(&norms, &level, &sign, 1, &planes);
+    if (st != NC_OK) return st;
+    nd_aggregate_kernel<true><<<nd_tile_blocks(d), kBlockThreads, 0, stream>>>(
+        planes, 1, (uint64_t)d, bucket_off, B, s, acc);
+    return launch_status();
+}
+
+}  // extern "C"

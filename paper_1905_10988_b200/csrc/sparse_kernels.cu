@@ -1,0 +1,336 @@
+// Random sparsification composed with natural dithering (the sparsifier S of the paper's
+// appendix with independent per-coordinate selection, then D_nat^{p,s} of Def. 3 on the kept
+// entries), and the sparse master-side accumulate, for sm_100a.
+//
+// Selection is a Philox word per coordinate compared with a threshold, so the cost of this
+// path is integer ALU work, not memory: x is read only where a coordinate is kept.
+//
+// Order-preserving compaction without any inter-block waiting:
+//   select : per 1024-element tile, selection bitmask (canonical bit order), kept count and
+//            a norm partial of the kept, scaled entries
+//   scan   : one block turns the tile counts into exclusive offsets and the partials into the norm
+//   emit   : per tile, rank of every kept entry = tile offset + prefix popcount; writes the
+//            index list and one code byte per entry
+//   pack   : two code bytes -> one byte of 4-bit codes
+#include "common.cuh"
+#include "philox.cuh"
+
+namespace natcomp {
+
+constexpr int kScanThreads = 1024;
+
+struct SparseWorkspace {
+    uint32_t* bitmask;      // tiles * 32 words
+    uint32_t* tile_count;   // tiles (becomes the exclusive offset after the scan)
+    uint64_t* tile_partial; // tiles
+    uint8_t* tmp_codes;     // cap bytes
+};
+
+__host__ __device__ inline uint64_t sparse_tiles(uint64_t d) { return (d + kTile - 1) / kTile; }
+
+inline size_t sparse_ws_bytes(uint64_t d, uint64_t cap) {
+    const uint64_t t = sparse_tiles(d);
+    return round_up16(t * 128) + round_up16(t * 4) + round_up16(t * 8) + round_up16(cap);
+}
+
+inline SparseWorkspace sparse_ws_carve(void* ws, uint64_t d) {
+    const uint64_t t = sparse_tiles(d);
+    char* p = reinterpret_cast<char*>(ws);
+    SparseWorkspace w;
+    w.bitmask = reinterpret_cast<uint32_t*>(p);      p += round_up16(t * 128);
+    w.tile_count = reinterpret_cast<uint32_t*>(p);   p += round_up16(t * 4);
+    w.tile_partial = reinterpret_cast<uint64_t*>(p); p += round_up16(t * 8);
+    w.tmp_codes = reinterpret_cast<uint8_t*>(p);
+    return w;
+}
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+__device__ __forceinline__ uint32_t warp_max_u(uint32_t v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ uint32_t warp_sum_u(uint32_t v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// grid: ceil(tiles / warps per block)
+template <int P>
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_select_kernel(const float* __restrict__ x, const uint64_t d, const uint32_t thr32,
+                     const bool keep_all, const float scale, const uint32_t worker,
+                     const __grid_constant__ PhiloxKeys keys, uint32_t* __restrict__ bitmask,
+                     uint32_t* __restrict__ tile_count, uint64_t* __restrict__ tile_partial) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+
+    uint32_t nib = 0;        // bit 4k+c <-> element base + k*128 + 4*lane + c
+    double dsum = 0.0;
+    uint32_t vmax = 0;
+#pragma unroll 1
+    for (int k = 7; k >= 0; --k) {
+        const uint64_t j4 = base + (uint64_t)(k * 128 + lane * 4);
+        uint32_t rnd[4];
+        stream_words4(j4 >> 2, worker, kDomainSelect, keys, rnd);
+#pragma unroll
+        for (int c = 3; c >= 0; --c) {
+            const bool keep = (keep_all || rnd[c] < thr32) && (j4 + c < d);
+            nib = (nib << 1) | (keep ? 1u : 0u);
+            if (keep) {
+                const float xs = __fmul_rn(scale, x[j4 + c]);
+                const uint32_t a = __float_as_uint(xs) & 0x7FFFFFFFu;
+                if (P == NC_P_INF) vmax = max(vmax, a);
+                else if (P == 1) dsum += (double)__uint_as_float(a);
+                else dsum = fma((double)xs, (double)xs, dsum);
+            }
+        }
+    }
+    const uint32_t word = transpose_nibbles_8x8(nib, lane);
+    bitmask[tile * 32 + (lane & 7) * 4 + (lane >> 3)] = word;
+    const uint32_t cnt = warp_sum_u(__popc(nib));
+    uint64_t part;
+    if (P == NC_P_INF) part = (uint64_t)warp_max_u(vmax);
+    else part = (uint64_t)__double_as_longlong(warp_sum_d(dsum));
+    if (lane == 0) {
+        tile_count[tile] = cnt;
+        tile_partial[tile] = part;
+    }
+}
+
+// one block: exclusive scan of the tile counts (in place), total count, norm
+template <int P>
+__global__ void __launch_bounds__(kScanThreads)
+sparse_scan_kernel(const uint64_t tiles, uint32_t* __restrict__ tile_count,
+                   const uint64_t* __restrict__ tile_partial, uint32_t* __restrict__ count,
+                   float* __restrict__ norm) {
+    __shared__ uint32_t s_cnt[kScanThreads];
+    __shared__ double s_sum[kScanThreads];
+    __shared__ uint32_t s_max[kScanThreads];
+    const int t = threadIdx.x;
+    const uint64_t per = (tiles + kScanThreads - 1) / kScanThreads;
+    const uint64_t t0 = (uint64_t)t * per;
+    const uint64_t t1 = (t0 + per < tiles) ? t0 + per : tiles;
+    uint32_t c = 0, m = 0;
+    double s = 0.0;
+    for (uint64_t i = t0; i < t1; ++i) {
+        c += tile_count[i];
+        if (P == NC_P_INF) m = max(m, (uint32_t)tile_partial[i]);
+        else s += __longlong_as_double((long long)tile_partial[i]);
+    }
+    s_cnt[t] = c;
+    s_sum[t] = s;
+    s_max[t] = m;
+    __syncthreads();
+    // inclusive Hillis-Steele scan of the per-thread counts
+    for (int o = 1; o < kScanThreads; o <<= 1) {
+        const uint32_t v = (t >= o) ? s_cnt[t - o] : 0u;
+        __syncthreads();
+        s_cnt[t] += v;
+        __syncthreads();
+    }
+    // fixed-shape tree for the norm partials
+    for (int o = kScanThreads / 2; o > 0; o >>= 1) {
+        if (t < o) {
+            s_sum[t] += s_sum[t + o];
+            s_max[t] = max(s_max[t], s_max[t + o]);
+        }
+        __syncthreads();
+    }
+    uint32_t run = s_cnt[t] - c;     // exclusive prefix of this thread's chunk
+    for (uint64_t i = t0; i < t1; ++i) {
+        const uint32_t v = tile_count[i];
+        tile_count[i] = run;
+        run += v;
+    }
+    if (t == 0) {
+        *count = s_cnt[kScanThreads - 1];
+        float r;
+        if (P == NC_P_INF) r = __uint_as_float(s_max[0]);
+        else if (P == 1) r = (float)s_sum[0];
+        else r = (float)sqrt(s_sum[0]);
+        *norm = r;
+    }
+}
+
+struct Scale {
+    float rinv;
+    uint32_t smax;
+};
+
+__device__ __forceinline__ Scale make_scale(float norm, int s) {
+    Scale r;
+    const bool ok = (norm >= 1.17549435e-38f) && (norm <= 3.40282347e38f);
+    r.rinv = ok ? __fdiv_rn(1.0f, norm) : 0.f;
+    r.smax = ok ? (uint32_t)s : 0u;
+    return r;
+}
+
+// same rounding rule as the dense dithering kernel (Def. 3, natural levels)
+__device__ __forceinline__ uint32_t sparse_level_code(uint32_t bits, uint32_t rnd, const Scale sc,
+                                                      float pow2s) {
+    const float ax = __uint_as_float(bits & 0x7FFFFFFFu);
+    const float y = __fmul_rn(ax, sc.rinv);
+    const float z = __fmul_rn(y, pow2s);
+    float w = z;
+    if (z < 2.0f) w = __fmaf_rz(z, 0.5f, 1.0f);
+    const uint32_t t = __float_as_uint(w) + (~rnd & 0x7FFFFFu) - 0x3F800000u;
+    return min(t >> 23, sc.smax);
+}
+
+// grid: ceil(tiles / warps per block)
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_emit_kernel(const float* __restrict__ x, const uint64_t d, const float scale, const int s,
+                   const uint32_t worker, const __grid_constant__ PhiloxKeys keys,
+                   const uint32_t* __restrict__ bitmask, const uint32_t* __restrict__ tile_offset,
+                   const float* __restrict__ norm, const uint64_t cap, uint32_t* __restrict__ idx,
+                   uint8_t* __restrict__ tmp_codes) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+    uint32_t word = bitmask[tile * 32 + lane];
+    const uint32_t cnt = __popc(word);
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    uint64_t k = (uint64_t)tile_offset[tile] + (incl - cnt);
+    if (word == 0) return;
+    const Scale sc = make_scale(*norm, s);
+    const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
+    while (word) {
+        const int bit = __ffs(word) - 1;
+        word &= word - 1;
+        const uint64_t j = base + (uint64_t)(lane * 32 + bit);
+        if (k < cap) {
+            const float xs = __fmul_rn(scale, x[j]);
+            const uint32_t bits = __float_as_uint(xs);
+            uint32_t r4[4];
+            stream_words4(j >> 2, worker, kDomainDnat, keys, r4);
+            const uint32_t r = (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1]
+                             : (j & 3) == 2 ? r4[2] : r4[3];
+            const uint32_t code = sparse_level_code(bits, r, sc, pow2s);
+            idx[k] = (uint32_t)j;
+            tmp_codes[k] = (uint8_t)(((bits >> 31) << 3) | code);
+        }
+        ++k;
+    }
+}
+
+// thread t -> output byte t; zero padding up to the next multiple of 16 bytes
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_pack_kernel(const uint8_t* __restrict__ tmp_codes, const uint32_t* __restrict__ count,
+                   const uint64_t cap, uint8_t* __restrict__ codes) {
+    const uint64_t t = (uint64_t)blockIdx.x * kBlockThreads + threadIdx.x;
+    const uint64_t total = min((uint64_t)*count, cap);
+    const uint64_t nbytes = (total + 1) / 2;
+    const uint64_t padded = min(round_up16(nbytes), round_up16((cap + 1) / 2));
+    if (t >= padded) return;
+    uint32_t b = 0;
+    if (t < nbytes) {
+        b = tmp_codes[2 * t];
+        if (2 * t + 1 < total) b |= (uint32_t)tmp_codes[2 * t + 1] << 4;
+    }
+    codes[t] = (uint8_t)b;
+}
+
+// grid: ceil(cap / threads)
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_decode_accumulate_kernel(const uint32_t* __restrict__ idx, const uint8_t* __restrict__ codes,
+                                const uint32_t* __restrict__ count, const float* __restrict__ norm,
+                                const int s, const uint64_t d, const uint64_t cap,
+                                float* __restrict__ acc) {
+    const uint64_t k = (uint64_t)blockIdx.x * kBlockThreads + threadIdx.x;
+    const uint64_t total = min((uint64_t)*count, cap);
+    if (k >= total) return;
+    float nv = *norm;
+    if (!(fabsf(nv) <= 3.40282347e38f)) nv = 0.f;
+    const uint32_t j = idx[k];
+    if (j >= d) return;
+    const uint32_t code = (codes[k >> 1] >> (4 * (k & 1))) & 0xFu;
+    const uint32_t c = code & 7u;
+    const uint32_t pb = (c ? ((c + 127u - (uint32_t)s) << 23) : 0u) | ((code >> 3) << 31);
+    acc[j] = __fadd_rn(acc[j], __fmul_rn(nv, __uint_as_float(pb)));
+}
+
+}  // namespace natcomp
+
+using namespace natcomp;
+
+extern "C" {
+
+size_t nd_sparse_workspace_bytes(size_t d, size_t cap) { return sparse_ws_bytes(d, cap); }
+
+nc_status nd_sparse_compress(const float* x, size_t d, uint64_t keep_threshold, float scale,
+                             int p, int s, uint64_t seed, uint32_t worker, uint32_t* idx,
+                             uint8_t* codes, uint32_t* count, float* norm, size_t cap,
+                             void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (!x || !idx || !codes || !count || !norm || s < 1 || s > 7 || cap < 1 ||
+        keep_threshold > ((uint64_t)1 << 32))
+        return NC_ERR_INVALID;
+    if (p != 1 && p != 2 && p != NC_P_INF) return NC_ERR_UNSUPPORTED;
+    if (d == 0) return NC_OK;
+    if (d > 0xFFFFFFFFull) return NC_ERR_INVALID;
+    if (!workspace) return NC_ERR_INVALID;
+    if (!aligned32(x) || !aligned16(idx) || !aligned16(codes) || !aligned16(workspace) ||
+        !aligned4(count) || !aligned4(norm))
+        return NC_ERR_ALIGN;
+    if (workspace_bytes < sparse_ws_bytes(d, cap)) return NC_ERR_WORKSPACE;
+    const SparseWorkspace ws = sparse_ws_carve(workspace, d);
+    const uint64_t tiles = sparse_tiles(d);
+    const unsigned grid = (unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    const PhiloxKeys keys = make_philox_keys(seed);
+    const bool keep_all = keep_threshold >= ((uint64_t)1 << 32);
+    const uint32_t thr32 = keep_all ? 0xFFFFFFFFu : (uint32_t)keep_threshold;
+    if (p == 1) {
+        sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(
+            x, d, thr32, keep_all, scale, worker, keys, ws.bitmask, ws.tile_count, ws.tile_partial);
+        sparse_scan_kernel<1><<<1, kScanThreads, 0, stream>>>(tiles, ws.tile_count,
+                                                              ws.tile_partial, count, norm);
+    } else if (p == 2) {
+        sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(
+            x, d, thr32, keep_all, scale, worker, keys, ws.bitmask, ws.tile_count, ws.tile_partial);
+        sparse_scan_kernel<2><<<1, kScanThreads, 0, stream>>>(tiles, ws.tile_count,
+                                                              ws.tile_partial, count, norm);
+    } else {
+        sparse_select_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
+            x, d, thr32, keep_all, scale, worker, keys, ws.bitmask, ws.tile_count, ws.tile_partial);
+        sparse_scan_kernel<NC_P_INF><<<1, kScanThreads, 0, stream>>>(tiles, ws.tile_count,
+                                                                     ws.tile_partial, count, norm);
+    }
+    sparse_emit_kernel<<<grid, kBlockThreads, 0, stream>>>(x, d, scale, s, worker, keys, ws.bitmask,
+                                                           ws.tile_count, norm, cap, idx,
+                                                           ws.tmp_codes);
+    const uint64_t pack_threads = round_up16((cap + 1) / 2);
+    const unsigned pgrid = (unsigned)((pack_threads + kBlockThreads - 1) / kBlockThreads);
+    sparse_pack_kernel<<<pgrid, kBlockThreads, 0, stream>>>(ws.tmp_codes, count, cap, codes);
+    return launch_status();
+}
+
+nc_status nd_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes,
+                                      const uint32_t* count, const float* norm, int s, size_t d,
+                                      size_t cap, float* acc, cudaStream_t stream) {
+    if (!idx || !codes || !count || !norm || !acc || s < 1 || s > 7 || cap < 1)
+        return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > 0xFFFFFFFFull) return NC_ERR_INVALID;
+    if (!aligned16(idx) || !aligned16(codes) || !aligned32(acc) || !aligned4(count) ||
+        !aligned4(norm))
+        return NC_ERR_ALIGN;
+    const unsigned grid = (unsigned)((cap + kBlockThreads - 1) / kBlockThreads);
+    sparse_decode_accumulate_kernel<<<grid, kBlockThreads, 0, stream>>>(idx, codes, count, norm, s,
+                                                                        d, cap, acc);
+    return launch_status();
+}
+
+}  // extern "C"

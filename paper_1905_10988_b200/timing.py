@@ -1,0 +1,59 @@
+"""Benchmark plumbing shared by bench.py and its tests: rank reduction of timings and the
+end-to-end (host buffers) variant of a step.  None of the method's arithmetic lives here."""
+from __future__ import annotations
+
+import torch
+
+
+def max_over_ranks(value: float, dist=None, device="cpu") -> float:
+    """The slowest rank's value (multi-GPU numbers are reported as the max over ranks)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(value: float, dist=None, device="cpu") -> float:
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def replica_worker_ids(rank: int, n_workers: int):
+    """Replicas are independent: rank r simulates workers r*n .. r*n + n - 1."""
+    return [rank * n_workers + w for w in range(n_workers)]
+
+
+def e2e_host_steps(nc, hp, steps: int) -> dict:
+    """Runs `steps` steps with the inputs in pinned host memory: every step copies the n
+    gradient vectors host -> device through the C ABI, runs the whole path, and copies the
+    three aggregates back to pinned host memory.  Returns ms per step and bytes moved."""
+    n, d = hp.n, hp.d
+    host_x = [torch.empty(d, dtype=torch.float32, pin_memory=True) for _ in range(n)]
+    for w in range(n):
+        host_x[w].copy_(hp.x[w])
+    host_out = [torch.empty(d, dtype=torch.float32, pin_memory=True) for _ in range(3)]
+    torch.cuda.synchronize()
+
+    def one_step():
+        for w in range(n):
+            nc.nc_copy_to_device(hp.x[w], host_x[w], 4 * d)
+        hp.step()
+        for dst, src in zip(host_out, (hp.out_nc, hp.out_nd, hp.out_sp)):
+            nc.nc_copy_to_host(dst, src, 4 * d)
+
+    one_step()                                   # warm-up
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one_step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return {"ms_per_step": ms, "h2d_bytes_per_step": 4 * d * n, "d2h_bytes_per_step": 4 * d * 3,
+            "steps": steps}

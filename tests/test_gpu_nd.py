@@ -1,0 +1,227 @@
+"""GPU parity, natural dithering: norms within 1e-6 relative (max-norm exact); level codes
+bit-exact against the oracle run on the GPU's own norms (given-norm mode) and within
+1e-5 adjacent-only differences against the oracle's definition mode; signs, padding and the
+decode / n-way sum bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1905_10988_b200 as nc
+from paper_1905_10988_b200 import workloads
+from gpu_util import Guarded, dev, unpack_nibbles
+
+pytestmark = pytest.mark.gpu
+
+NORM_RTOL = 1e-6
+CODE_MISMATCH = 1e-5
+
+
+def gpu_nd_compress(x_dev, off, p, s, seed, worker):
+    d = x_dev.numel()
+    B = len(off) - 1
+    off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
+    norms = Guarded(4 * B)
+    level = Guarded(nc.nd_level_bytes(d))
+    sign = Guarded(nc.nc_sign_bytes(d))
+    ws_bytes = nc.nd_workspace_bytes(d, B)
+    ws = Guarded(ws_bytes)
+    nc.nd_compress(x_dev, d, off_dev, B, p, s, seed, worker, norms.buf, level.buf, sign.buf,
+                   ws.buf, ws_bytes)
+    torch.cuda.synchronize()
+    for g in (norms, level, sign, ws):
+        g.check()
+    return norms, level, sign
+
+
+def check_against_oracle(x, off, p, s, seed, worker, norms, level, sign, *, slack=0):
+    d = x.size
+    gn = norms.numpy(np.float32)
+    lv = level.numpy(np.uint8)
+    sg = sign.numpy(np.uint32)
+    # definition mode: the oracle's own norms
+    n0, l0, s0 = oracle.nd_compress(x, off, p, s, seed, worker)
+    finite = np.isfinite(n0)
+    assert np.array_equal(np.isnan(gn), np.isnan(n0))
+    assert np.array_equal(np.isinf(gn), np.isinf(n0))
+    if p == nc.P_INF:
+        assert np.array_equal(gn[finite], n0[finite])
+    else:
+        assert np.all(np.abs(gn[finite] - n0[finite]) <= NORM_RTOL * np.abs(n0[finite]))
+    nw = (d + 31) // 32
+    assert np.array_equal(sg[:nw], s0) and np.all(sg[nw:] == 0)
+    assert np.all(lv[(d + 1) // 2:] == 0)
+    cg = unpack_nibbles(lv, d).astype(np.int64)
+    # given-norm mode: same norms as the GPU -> codes must be identical
+    _, l1, _ = oracle.nd_compress(x, off, p, s, seed, worker, given_norms=gn)
+    assert np.array_equal(lv[:(d + 1) // 2], l1), "level plane differs from given-norm oracle"
+    # definition mode: few, adjacent differences only
+    c0 = unpack_nibbles(l0, d).astype(np.int64)
+    diff = cg != c0
+    assert diff.sum() <= CODE_MISMATCH * d + slack
+    assert np.all(np.abs(cg - c0)[diff] == 1)
+    return gn
+
+
+@pytest.mark.parametrize("p", [1, 2, 0])
+@pytest.mark.parametrize("d,s", [(1, 4), (33, 1), (1000, 8), (1024, 8), (5000, 15), (70001, 8),
+                                 ((1 << 18) + 40, 4)])
+def test_compress_ragged_bucket_tables(d, s, p):
+    rng = np.random.default_rng(d * 31 + s)
+    off = workloads.small_bucket_table(d, seed=d + s)
+    sig = 10.0 ** rng.uniform(-5, -2, len(off) - 1)
+    x = (rng.standard_normal(d) * np.repeat(sig, np.diff(off))).astype(np.float32)
+    norms, level, sign = gpu_nd_compress(dev(x), off, p, s, seed=d, worker=s)
+    check_against_oracle(x, off, p, s, d, s, norms, level, sign, slack=2)
+
+
+def test_compress_single_bucket_and_aligned_buckets():
+    rng = np.random.default_rng(5)
+    d = 1 << 17
+    x = (rng.standard_normal(d) * 2e-3).astype(np.float32)
+    for off in ([0, d], list(range(0, d + 1, 4096)), [0, 1024, 1024, 2048, d]):
+        norms, level, sign = gpu_nd_compress(dev(x), off, 2, 8, seed=1, worker=0)
+        check_against_oracle(x, off, 2, 8, 1, 0, norms, level, sign, slack=2)
+
+
+def test_compress_degenerate_buckets():
+    rng = np.random.default_rng(6)
+    d = 6000
+    x = (rng.standard_normal(d) * 1e-2).astype(np.float32)
+    off = [0, 100, 1500, 1500, 2600, 4000, 5000, d]
+    x[100:1500] = 0.0                  # x = 0 -> D(x) = 0
+    x[100:1500:2] = -0.0
+    x[2600:4000] = (rng.standard_normal(1400) * 1e-42).astype(np.float32)   # subnormal norm
+    x[4100] = np.inf                   # non-finite norm
+    x[5100] = np.nan
+    for p in (1, 2, 0):
+        norms, level, sign = gpu_nd_compress(dev(x), off, p, 8, seed=2, worker=1)
+        gn = check_against_oracle(x, off, p, 8, 2, 1, norms, level, sign, slack=2)
+        c = unpack_nibbles(level.numpy(np.uint8), d)
+        assert gn[1] == 0 and gn[2] == 0 and 0 < gn[4] < 2.0 ** -126
+        assert np.isinf(gn[5]) and np.isnan(gn[6])
+        for b in (1, 4, 5, 6):
+            assert np.all(c[off[b]:off[b + 1]] == 0)
+        assert np.any(c[off[3]:off[4]] > 0)
+        assert np.any(c[:100] > 0)
+
+
+def _random_planes(rng, n, d, B, s):
+    norms = [(10.0 ** rng.uniform(-6, 1, B)).astype(np.float32) for _ in range(n)]
+    levels, signs = [], []
+    for _ in range(n):
+        c = rng.integers(0, s + 1, nc.nd_level_bytes(d) * 2).astype(np.uint8)
+        levels.append((c[0::2] | (c[1::2] << 4)).astype(np.uint8))
+        signs.append(rng.integers(0, 1 << 32, nc.nc_sign_bytes(d) // 4, dtype=np.uint64)
+                     .astype(np.uint32))
+    return norms, levels, signs
+
+
+@pytest.mark.parametrize("n,d,s", [(1, 999, 8), (3, 4096, 4), (8, 70001, 8), (16, 5000, 15),
+                                   (64, 2100, 1)])
+def test_aggregate_and_decode_accumulate_are_bit_exact(n, d, s):
+    rng = np.random.default_rng(n * 7 + d)
+    off = workloads.small_bucket_table(d, seed=n + d)
+    B = len(off) - 1
+    norms, levels, signs = _random_planes(rng, n, d, B, s)
+    norms[0][0] = 2.0 ** -130                  # subnormal products
+    if B > 2:
+        norms[-1][1] = np.inf                  # a non-finite norm decodes as zero
+        norms[0][2] = 0.0
+    off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
+    nd_ = [dev(a) for a in norms]
+    ld = [dev(a) for a in levels]
+    sd = [dev(a) for a in signs]
+    out = Guarded(4 * d)
+    nc.nd_aggregate(nd_, ld, sd, n, d, off_dev, B, s, out.buf)
+    torch.cuda.synchronize()
+    out.check()
+    want = oracle.nd_aggregate(norms, [l[:(d + 1) // 2] for l in levels], signs, off, s, d)
+    assert np.array_equal(out.numpy(np.uint32), want.view(np.uint32))
+    acc = Guarded(4 * d)
+    start = rng.standard_normal(d).astype(np.float32)
+    acc.buf.copy_(dev(start).view(torch.uint8))
+    ref = start.copy()
+    for i in range(n):
+        nc.nd_decode_accumulate(nd_[i], ld[i], sd[i], d, off_dev, B, s, acc.buf)
+        oracle.nd_decode_accumulate(norms[i], levels[i][:(d + 1) // 2], signs[i], off, s, ref)
+    torch.cuda.synchronize()
+    acc.check()
+    assert np.array_equal(acc.numpy(np.uint32), ref.view(np.uint32))
+
+
+def test_config3_full_size():
+    # D_nat^{2,8} on the ResNet-50-shaped buckets, n = 8; two workers checked in full against the
+    # oracle, the aggregate on sampled buckets
+    n, p, s = 8, 2, 8
+    sizes = workloads.resnet50_tensor_sizes()
+    off = workloads.offsets_from_sizes(sizes)
+    d, B = off[-1], len(sizes)
+    off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
+    xd = [workloads.config2_vector(w, "cuda", sizes) for w in range(n)]
+    ws_bytes = nc.nd_workspace_bytes(d, B)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    norms = [torch.empty(B, dtype=torch.float32, device="cuda") for _ in range(n)]
+    levels = [torch.empty(nc.nd_level_bytes(d), dtype=torch.uint8, device="cuda")
+              for _ in range(n)]
+    signs = [torch.empty(nc.nc_sign_bytes(d), dtype=torch.uint8, device="cuda") for _ in range(n)]
+    for w in range(n):
+        nc.nd_compress(xd[w], d, off_dev, B, p, s, 0, w, norms[w], levels[w], signs[w], ws,
+                       ws_bytes)
+    out = torch.empty(d, dtype=torch.float32, device="cuda")
+    nc.nd_aggregate(norms, levels, signs, n, d, off_dev, B, s, out)
+    torch.cuda.synchronize()
+    for w in (0, n - 1):
+        x = xd[w].cpu().numpy()
+        gn = norms[w].cpu().numpy()
+        n0, l0, s0 = oracle.nd_compress(x, off, p, s, 0, w)
+        assert np.all(np.abs(gn - n0) <= NORM_RTOL * n0)
+        assert np.array_equal(signs[w].cpu().numpy().view(np.uint32)[:(d + 31) // 32], s0)
+        _, l1, _ = oracle.nd_compress(x, off, p, s, 0, w, given_norms=gn)
+        lv = levels[w].cpu().numpy()[:(d + 1) // 2]
+        assert np.array_equal(lv, l1)
+        cg = unpack_nibbles(lv, d).astype(np.int64)
+        c0 = unpack_nibbles(l0, d).astype(np.int64)
+        diff = cg != c0
+        assert diff.sum() <= CODE_MISMATCH * d
+        assert np.all(np.abs(cg - c0)[diff] == 1)
+    # aggregate: sampled buckets (small, medium, the largest, the last)
+    order = np.argsort(sizes)
+    picks = sorted(set([0, 1, 2, int(order[0]), int(order[len(order) // 2]), int(order[-1]),
+                        B - 2, B - 1]))
+    for b in picks:
+        lo, hi = off[b], off[b + 1]
+        assert lo % 32 == 0
+        sub_off = [0, hi - lo]
+        nr = [norms[w][b:b + 1].cpu().numpy() for w in range(n)]
+        lv = [levels[w][lo // 2:(hi + 1) // 2].cpu().numpy() for w in range(n)]
+        sg = [signs[w].view(torch.int32)[lo // 32:(hi + 31) // 32].cpu().numpy().view(np.uint32)
+              for w in range(n)]
+        want = oracle.nd_aggregate(nr, lv, sg, sub_off, s, hi - lo)
+        assert np.array_equal(out[lo:hi].cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+def test_unbiasedness_of_the_gpu_path_over_seeds():
+    # E D(x) = x (Def. 3): average the decoded GPU output over many seeds
+    rng = np.random.default_rng(9)
+    d, s, trials = 2048, 4, 400
+    x = (rng.standard_normal(d) * 1e-3).astype(np.float32)
+    off = [0, 700, d]
+    off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
+    xdev = dev(x)
+    ws_bytes = nc.nd_workspace_bytes(d, 2)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    norms = torch.empty(2, dtype=torch.float32, device="cuda")
+    level = torch.empty(nc.nd_level_bytes(d), dtype=torch.uint8, device="cuda")
+    sign = torch.empty(nc.nc_sign_bytes(d), dtype=torch.uint8, device="cuda")
+    acc = torch.zeros(d, dtype=torch.float32, device="cuda")
+    for t in range(trials):
+        nc.nd_compress(xdev, d, off_dev, 2, 2, s, t, 0, norms, level, sign, ws, ws_bytes)
+        nc.nd_decode_accumulate(norms, level, sign, d, off_dev, 2, s, acc)
+    torch.cuda.synchronize()
+    mean = acc.cpu().numpy().astype(np.float64) / trials
+    nrm = norms.cpu().numpy().astype(np.float64)
+    per = np.repeat(nrm, np.diff(off))
+    # per-entry variance <= max(y (2^(1-s)) , y^2 / 8) * norm^2 <= norm^2 * 2^(1-s) * max(y, ...)
+    sigma = per * np.sqrt(np.maximum(np.abs(x) / per * 2.0 ** (1 - s), (x / per) ** 2 / 8))
+    assert np.all(np.abs(mean - x) <= 6 * sigma / np.sqrt(trials) + 1e-12)

@@ -1,0 +1,137 @@
+"""GPU parity, random sparsification composed with natural dithering, and the sparse
+accumulate: index lists, codes, counts and the max-norm are compared bit-exactly."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1905_10988_b200 as nc
+from paper_1905_10988_b200 import workloads
+from gpu_util import Guarded, dev
+
+pytestmark = pytest.mark.gpu
+
+
+def gpu_sparse_compress(x_dev, thr, scale, p, s, seed, worker, cap):
+    d = x_dev.numel()
+    idx = Guarded(4 * cap)
+    codes = Guarded(((cap + 1) // 2 + 15) // 16 * 16)
+    count = Guarded(4)
+    norm = Guarded(4)
+    ws_bytes = nc.nd_sparse_workspace_bytes(d, cap)
+    ws = Guarded(ws_bytes)
+    nc.nd_sparse_compress(x_dev, d, thr, scale, p, s, seed, worker, idx.buf, codes.buf,
+                          count.buf, norm.buf, cap, ws.buf, ws_bytes)
+    torch.cuda.synchronize()
+    for g in (idx, codes, count, norm, ws):
+        g.check()
+    return idx, codes, int(count.numpy(np.uint32)[0]), norm.numpy(np.float32)[0]
+
+
+def check_sparse(x, thr, scale, p, s, seed, worker, cap, got):
+    idx, codes, count, norm = got
+    given = None if p == nc.P_INF else norm
+    i_ref, c_ref, count_ref, n_ref = oracle.sparse_compress(x, thr, scale, p, s, seed, worker,
+                                                            cap=cap, given_norm=given)
+    assert count == count_ref
+    stored = min(count, cap)
+    if p == nc.P_INF:
+        assert norm == n_ref or (np.isnan(norm) and np.isnan(n_ref))
+    else:
+        own = oracle.sparse_compress(x, thr, scale, p, s, seed, worker, cap=1)[3]
+        assert abs(float(norm) - float(own)) <= 1e-6 * abs(float(own))
+    assert np.array_equal(idx.numpy(np.uint32)[:stored], i_ref)
+    cg = codes.numpy(np.uint8)
+    nb = (stored + 1) // 2
+    assert np.array_equal(cg[:nb], c_ref)
+    pad_end = min((nb + 15) // 16 * 16, cg.size)
+    assert np.all(cg[nb:pad_end] == 0)
+
+
+@pytest.mark.parametrize("d", [1, 31, 1000, 1024, 4097, 200_003, (1 << 20) + 9])
+@pytest.mark.parametrize("thr,scale", [(42_949_673, 100.0), (1 << 30, 4.0), (1 << 32, 1.0)])
+def test_sparse_compress_matches_oracle(d, thr, scale):
+    rng = np.random.default_rng(d)
+    x = rng.standard_normal(d).astype(np.float32)
+    cap = d
+    got = gpu_sparse_compress(dev(x), thr, scale, nc.P_INF, 4, seed=d, worker=3, cap=cap)
+    check_sparse(x, thr, scale, nc.P_INF, 4, d, 3, cap, got)
+
+
+@pytest.mark.parametrize("p,s", [(1, 7), (2, 4), (0, 1)])
+def test_sparse_other_norms_levels_and_cap(p, s):
+    rng = np.random.default_rng(70 + p)
+    d = 150_000
+    x = (rng.standard_normal(d) * 3e-2).astype(np.float32)
+    thr, scale = 1 << 28, 16.0
+    cap = 5000                                    # fewer than the ~9400 kept entries
+    got = gpu_sparse_compress(dev(x), thr, scale, p, s, seed=8, worker=0, cap=cap)
+    assert got[2] > cap
+    check_sparse(x, thr, scale, p, s, 8, 0, cap, got)
+
+
+def test_sparse_all_zero_and_nonfinite_inputs():
+    d = 5000
+    for fillv in (0.0, np.inf):
+        x = np.zeros(d, np.float32)
+        x[10:20] = fillv
+        got = gpu_sparse_compress(dev(x), 1 << 31, 2.0, nc.P_INF, 4, seed=1, worker=1, cap=d)
+        check_sparse(x, 1 << 31, 2.0, nc.P_INF, 4, 1, 1, d, got)
+        codes = got[1].numpy(np.uint8)
+        assert np.all((codes & 0x77) == 0)        # degenerate norm: every level code is 0
+
+
+def test_sparse_decode_accumulate_workers_in_order():
+    rng = np.random.default_rng(21)
+    d, n, s = 300_000, 5, 4
+    thr, scale = workloads.KEEP_1PCT_THRESHOLD * 8, 12.5
+    cap = 40_000
+    acc = Guarded(4 * d)
+    start = rng.standard_normal(d).astype(np.float32)
+    acc.buf.copy_(dev(start).view(torch.uint8))
+    ref = start.copy()
+    keep = []
+    for w in range(n):
+        x = rng.standard_normal(d).astype(np.float32)
+        idx, codes, count, norm = gpu_sparse_compress(dev(x), thr, scale, nc.P_INF, s, 3, w, cap)
+        keep.append((idx, codes))
+        cnt = dev(np.uint32([count]).view(np.int32))
+        nrm = dev(np.float32([norm]))
+        nc.nd_sparse_decode_accumulate(idx.buf, codes.buf, cnt, nrm, s, d, cap, acc.buf)
+        i_ref, c_ref, count_ref, n_ref = oracle.sparse_compress(x, thr, scale, nc.P_INF, s, 3, w)
+        oracle.sparse_decode_accumulate(i_ref, c_ref, count_ref, n_ref, s, ref)
+    torch.cuda.synchronize()
+    acc.check()
+    assert np.array_equal(acc.numpy(np.uint32), ref.view(np.uint32))
+
+
+def test_config5_full_size_one_worker():
+    # d = 2^28, keep 1 %, D_nat^{inf,4}: one worker in full against the oracle
+    d, s = 1 << 28, 4
+    thr, scale = workloads.KEEP_1PCT_THRESHOLD, workloads.KEEP_1PCT_SCALE
+    cap = int(d * 0.0125)
+    x = workloads.config5_vector(0, d, "cuda")
+    idx = torch.empty(cap, dtype=torch.int32, device="cuda")
+    codes = torch.empty((cap + 1) // 2 + 16, dtype=torch.uint8, device="cuda")
+    count = torch.zeros(1, dtype=torch.int32, device="cuda")
+    norm = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ws_bytes = nc.nd_sparse_workspace_bytes(d, cap)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    nc.nd_sparse_compress(x, d, thr, scale, nc.P_INF, s, 0, 0, idx, codes, count, norm, cap, ws,
+                          ws_bytes)
+    acc = torch.zeros(d, dtype=torch.float32, device="cuda")
+    nc.nd_sparse_decode_accumulate(idx, codes, count, norm, s, d, cap, acc)
+    torch.cuda.synchronize()
+    cnt = int(count.cpu().numpy().view(np.uint32)[0])
+    assert abs(cnt - 0.01 * d) <= 5 * np.sqrt(d * 0.01 * 0.99)
+    full = oracle.max_threads()
+    i_ref, c_ref, count_ref, n_ref = oracle.sparse_compress(x.cpu().numpy(), thr, scale,
+                                                            nc.P_INF, s, 0, 0, cap=cap)
+    oracle.set_threads(full)
+    assert cnt == count_ref and float(norm.cpu()[0]) == float(n_ref)
+    assert np.array_equal(idx[:cnt].cpu().numpy().view(np.uint32), i_ref)
+    assert np.array_equal(codes[:(cnt + 1) // 2].cpu().numpy(), c_ref)
+    ref = np.zeros(d, np.float32)
+    oracle.sparse_decode_accumulate(i_ref, c_ref, count_ref, n_ref, s, ref)
+    got = acc.cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
