@@ -120,17 +120,19 @@ class HotPath:
     GROUPS = ("nc_compress", "nc_aggregate", "nd_compress", "nd_aggregate", "sparse_compress",
               "sparse_accumulate", "sum_fp32")
 
-    def __init__(self, nc, rank, device):
+    def __init__(self, nc, rank, device, n_workers=N_WORKERS, only=None):
         from paper_1905_10988_b200 import workloads
         self.nc = nc
-        self.n = N_WORKERS
+        self.n = n_workers
+        self.only = only
         sizes = workloads.resnet50_tensor_sizes()
         off = workloads.offsets_from_sizes(sizes)
         self.d, self.B = off[-1], len(sizes)
         n, d, B = self.n, self.d, self.B
         u8 = dict(dtype=torch.uint8, device=device)
         f32 = dict(dtype=torch.float32, device=device)
-        self.workers = [rank * n + w for w in range(n)]
+        from paper_1905_10988_b200 import timing
+        self.workers = timing.replica_worker_ids(rank, n)
         self.x = [workloads.config2_vector(w, device, sizes) for w in self.workers]
         self.off = torch.tensor(off, dtype=torch.int64, device=device)
         self.exp = [torch.empty(nc.nc_exp_bytes(d), **u8) for _ in range(n)]
@@ -139,7 +141,7 @@ class HotPath:
         self.norms = [torch.empty(B, **f32) for _ in range(n)]
         self.level = [torch.empty(nc.nd_level_bytes(d), **u8) for _ in range(n)]
         self.sign_nd = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
-        self.ws_bytes = nc.nd_workspace_bytes(d, B)
+        self.ws_bytes = nc.nd_batch_workspace_bytes(d, B, n)
         self.ws = torch.empty(self.ws_bytes, **u8)
         self.out_nd = torch.empty(d, **f32)
         self.cap = int(d * SPARSE_CAP_FRACTION)
@@ -147,11 +149,13 @@ class HotPath:
         self.codes = [torch.empty((self.cap + 1) // 2 + 16, **u8) for _ in range(n)]
         self.count = [torch.zeros(1, dtype=torch.int32, device=device) for _ in range(n)]
         self.snorm = [torch.zeros(1, **f32) for _ in range(n)]
-        self.sws_bytes = nc.nd_sparse_workspace_bytes(d, self.cap)
+        self.sws_bytes = nc.nd_sparse_batch_workspace_bytes(d, self.cap, n)
         self.sws = torch.empty(self.sws_bytes, **u8)
         self.out_sp = torch.empty(d, **f32)
         self.out_sum = torch.empty(d, **f32)
-        self.launches_per_step = 1 + 1 + 3 * n + 1 + 4 * n + n + 1
+        # nc_compress_batch 1, nc_aggregate 1, nd_compress_batch 3, nd_aggregate 1,
+        # nd_sparse_compress_batch 4, nd_sparse_decode_accumulate n, nc_sum_fp32 1
+        self.launches_per_step = 1 + 1 + 3 + 1 + 4 + n + 1
         self.seed = 0
 
     def step(self, marks=None):
@@ -164,31 +168,39 @@ class HotPath:
                 ev.record()
                 marks.append((name, ev))
 
+        def want(name):
+            return self.only is None or self.only == name
+
         mark("start")
-        nc.nc_compress_batch(self.x, d, self.seed, self.workers, self.exp, self.sign, n)
+        if want("nc_compress"):
+            nc.nc_compress_batch(self.x, d, self.seed, self.workers, self.exp, self.sign, n)
         mark("nc_compress")
-        nc.nc_aggregate(self.exp, self.sign, n, d, self.out_nc)
+        if want("nc_aggregate"):
+            nc.nc_aggregate(self.exp, self.sign, n, d, self.out_nc)
         mark("nc_aggregate")
-        for w in range(n):
-            nc.nd_compress(self.x[w], d, self.off, B, P_DITHER, S_DITHER, self.seed,
-                           self.workers[w], self.norms[w], self.level[w], self.sign_nd[w],
-                           self.ws, self.ws_bytes)
+        if want("nd_compress"):
+            nc.nd_compress_batch(self.x, d, self.off, B, P_DITHER, S_DITHER, self.seed,
+                                 self.workers, self.norms, self.level, self.sign_nd, n, self.ws,
+                                 self.ws_bytes)
         mark("nd_compress")
-        nc.nd_aggregate(self.norms, self.level, self.sign_nd, n, d, self.off, B, S_DITHER,
-                        self.out_nd)
+        if want("nd_aggregate"):
+            nc.nd_aggregate(self.norms, self.level, self.sign_nd, n, d, self.off, B, S_DITHER,
+                            self.out_nd)
         mark("nd_aggregate")
-        for w in range(n):
-            nc.nd_sparse_compress(self.x[w], d, workloads.KEEP_1PCT_THRESHOLD,
-                                  workloads.KEEP_1PCT_SCALE, nc.P_INF, S_SPARSE, self.seed,
-                                  self.workers[w], self.idx[w], self.codes[w], self.count[w],
-                                  self.snorm[w], self.cap, self.sws, self.sws_bytes)
+        if want("sparse_compress"):
+            nc.nd_sparse_compress_batch(self.x, d, workloads.KEEP_1PCT_THRESHOLD,
+                                        workloads.KEEP_1PCT_SCALE, nc.P_INF, S_SPARSE, self.seed,
+                                        self.workers, self.idx, self.codes, self.count,
+                                        self.snorm, self.cap, n, self.sws, self.sws_bytes)
         mark("sparse_compress")
-        self.out_sp.zero_()
-        for w in range(n):
-            nc.nd_sparse_decode_accumulate(self.idx[w], self.codes[w], self.count[w],
-                                           self.snorm[w], S_SPARSE, d, self.cap, self.out_sp)
+        if want("sparse_accumulate"):
+            self.out_sp.zero_()
+            for w in range(n):
+                nc.nd_sparse_decode_accumulate(self.idx[w], self.codes[w], self.count[w],
+                                               self.snorm[w], S_SPARSE, d, self.cap, self.out_sp)
         mark("sparse_accumulate")
-        nc.nc_sum_fp32(self.x, n, d, self.out_sum)
+        if want("sum_fp32"):
+            nc.nc_sum_fp32(self.x, n, d, self.out_sum)
         mark("sum_fp32")
 
     def algorithmic_bytes(self):
@@ -272,11 +284,15 @@ def run_reference(args, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--only", default=None, choices=list(HotPath.GROUPS),
+                    help="profiling aid: time one call group alone")
+    ap.add_argument("--workers", type=int, default=N_WORKERS,
+                    help="number of simulated workers with --only")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -299,6 +315,27 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
+
+    if args.only:
+        # profiling aid: one call group alone, on a smaller case (still larger than L2)
+        hp = HotPath(nc, rank, device, n_workers=args.workers)
+        hp.step()                               # produces the planes the master-side calls read
+        hp.only = args.only
+        for _ in range(args.warmup):
+            hp.step()
+        torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            hp.step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        gb = hp.algorithmic_bytes()[args.only]
+        print(json.dumps({"only": args.only, "workers": hp.n, "d": hp.d, "ms": ms,
+                          "algorithmic_GBps": gb / ms / 1e6}))
+        return
 
     hp = HotPath(nc, rank, device)
     for _ in range(args.warmup):
@@ -364,7 +401,7 @@ def main():
 
     # end to end: host buffers -> device -> whole path -> aggregates back on the host
     e2e = None
-    if rank == 0 or world > 1:
+    if args.e2e_steps > 0:
         e2e = timing.e2e_host_steps(nc, hp, args.e2e_steps)
         e2e_ms = timing.max_over_ranks(e2e["ms_per_step"], dist, device)
         e2e["value"] = world * units_per_step / (e2e_ms * 1e-3) / 1e9

@@ -124,6 +124,15 @@ nc_status nd_compress(const float* x, size_t d, const uint64_t* bucket_off, int 
                       uint32_t* sign, void* workspace, size_t workspace_bytes,
                       cudaStream_t stream);
 
+/* The same for n workers' vectors of equal length d and one shared bucket table, in three launches
+ * in total.  xs, norms, levels, signs: host arrays of n device pointers; workers: host array of n
+ * worker ids.  workspace: nd_batch_workspace_bytes(d, B, n). */
+size_t nd_batch_workspace_bytes(size_t d, int num_buckets, int n);
+nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B,
+                            int p, int s, uint64_t seed, const uint32_t* workers,
+                            float* const* norms, uint8_t* const* levels, uint32_t* const* signs,
+                            int n, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
 /* Master side, one worker: acc[j] <- acc[j] + sign_j * fl32(norm_b * 2^(c_j - s)); c = 0 adds +-0. */
 nc_status nd_decode_accumulate(const float* norms, const uint8_t* level, const uint32_t* sign,
                                size_t d, const uint64_t* bucket_off, int B, int s, float* acc,
@@ -147,6 +156,17 @@ nc_status nd_sparse_compress(const float* x, size_t d, uint64_t keep_threshold, 
                              int p, int s, uint64_t seed, uint32_t worker, uint32_t* idx,
                              uint8_t* codes, uint32_t* count, float* norm, size_t cap,
                              void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/* The same for n workers' vectors of equal length d in four launches in total.  xs, idxs, codes,
+ * counts, norms: host arrays of n device pointers (each worker has its own list of `cap` entries);
+ * workspace: nd_sparse_batch_workspace_bytes(d, cap, n). */
+size_t nd_sparse_batch_workspace_bytes(size_t d, size_t cap, int n);
+nc_status nd_sparse_compress_batch(const float* const* xs, size_t d, uint64_t keep_threshold,
+                                   float scale, int p, int s, uint64_t seed,
+                                   const uint32_t* workers, uint32_t* const* idxs,
+                                   uint8_t* const* codes, uint32_t* const* counts,
+                                   float* const* norms, size_t cap, int n, void* workspace,
+                                   size_t workspace_bytes, cudaStream_t stream);
 
 /* acc[idx[k]] <- acc[idx[k]] + decoded value, k < min(*count, cap).  Indices are unique within
  * one worker's list, so one call needs no atomics; calls for different workers are applied in

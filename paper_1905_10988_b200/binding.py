@@ -32,6 +32,8 @@ EXPORTS = (
     "nd_sparse_workspace_bytes", "nc_compress", "nc_compress_batch", "nc_decode_accumulate",
     "nc_aggregate", "nc_sum_fp32", "nd_compress", "nd_decode_accumulate", "nd_aggregate",
     "nd_sparse_compress", "nd_sparse_decode_accumulate", "nc_copy_to_device", "nc_copy_to_host",
+    "nd_batch_workspace_bytes", "nd_compress_batch", "nd_sparse_batch_workspace_bytes",
+    "nd_sparse_compress_batch",
 )
 
 
@@ -76,6 +78,44 @@ _nd_sparse_compress = _sig("nd_sparse_compress", C.c_int, _vp, _sz, C.c_uint64, 
                            _vp, _sz, _vp)
 _nd_sparse_decode_accumulate = _sig("nd_sparse_decode_accumulate", C.c_int, _vp, _vp, _vp, _vp,
                                     C.c_int, _sz, _sz, _vp, _vp)
+
+
+_nd_batch_workspace_bytes = _sig("nd_batch_workspace_bytes", _sz, _sz, C.c_int, C.c_int)
+_nd_compress_batch = _sig("nd_compress_batch", C.c_int, C.POINTER(_vp), _sz, _vp, C.c_int, C.c_int,
+                          C.c_int, C.c_uint64, C.POINTER(C.c_uint32), C.POINTER(_vp),
+                          C.POINTER(_vp), C.POINTER(_vp), C.c_int, _vp, _sz, _vp)
+_nd_sparse_batch_workspace_bytes = _sig("nd_sparse_batch_workspace_bytes", _sz, _sz, _sz, C.c_int)
+_nd_sparse_compress_batch = _sig("nd_sparse_compress_batch", C.c_int, C.POINTER(_vp), _sz,
+                                 C.c_uint64, C.c_float, C.c_int, C.c_int, C.c_uint64,
+                                 C.POINTER(C.c_uint32), C.POINTER(_vp), C.POINTER(_vp),
+                                 C.POINTER(_vp), C.POINTER(_vp), _sz, C.c_int, _vp, _sz, _vp)
+
+
+def nd_batch_workspace_bytes(d: int, num_buckets: int, n: int) -> int:
+    return int(_nd_batch_workspace_bytes(d, num_buckets, n))
+
+
+def nd_compress_batch(xs, d, bucket_off, B, p, s, seed, workers, norms, levels, signs, n,
+                      workspace, workspace_bytes, stream=None) -> None:
+    w = (C.c_uint32 * n)(*[int(v) for v in workers])
+    _check("nd_compress_batch", _nd_compress_batch(_ptrs(xs), d, _ptr(bucket_off), B, p, s, seed,
+                                                   w, _ptrs(norms), _ptrs(levels), _ptrs(signs),
+                                                   n, _ptr(workspace), workspace_bytes,
+                                                   _stream(stream)))
+
+
+def nd_sparse_batch_workspace_bytes(d: int, cap: int, n: int) -> int:
+    return int(_nd_sparse_batch_workspace_bytes(d, cap, n))
+
+
+def nd_sparse_compress_batch(xs, d, keep_threshold, scale, p, s, seed, workers, idxs, codes,
+                             counts, norms, cap, n, workspace, workspace_bytes,
+                             stream=None) -> None:
+    w = (C.c_uint32 * n)(*[int(v) for v in workers])
+    _check("nd_sparse_compress_batch",
+           _nd_sparse_compress_batch(_ptrs(xs), d, keep_threshold, scale, p, s, seed, w,
+                                     _ptrs(idxs), _ptrs(codes), _ptrs(counts), _ptrs(norms), cap,
+                                     n, _ptr(workspace), workspace_bytes, _stream(stream)))
 
 
 _nc_copy_to_device = _sig("nc_copy_to_device", C.c_int, _vp, _vp, _sz, _vp)

@@ -61,21 +61,53 @@ nc_compress_kernel(const __grid_constant__ CompressBatch batch, const uint64_t d
         for (int k = 0; k < 8; ++k) u[k] = ld_stream_u4(xv + k * 32 + lane);
 
         uint32_t* ev = reinterpret_cast<uint32_t*>(exp + base);
-        uint32_t nib = 0;   // sign bits of this lane's 32 elements: bit 4k+c <-> group k, element c
+        const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainCnat, keys);
+        const uint32_t q_lo = (uint32_t)(base >> 2) + lane;   // + k*32 stays below 2^32: no carry
+
+        // Biased exponents 254 / 255 must not be rounded up.  If every element of the tile has
+        // (bits & 0x7F000000) != 0x7F000000 the guard can be dropped; the OR over the lane's
+        // elements is a cheap conservative test (false positives only cost the guarded path).
+        uint32_t any = 0;
 #pragma unroll
-        for (int k = 7; k >= 0; --k) {
-            uint32_t rnd[4];
-            stream_words4((base >> 2) + (uint64_t)(k * 32 + lane), worker, kDomainCnat, keys, rnd);
-            const uint32_t b0 = u[k].x, b1 = u[k].y, b2 = u[k].z, b3 = u[k].w;
-            uint32_t e = cnat_exp_byte(b3, rnd[3]);
-            e = (e << 8) | cnat_exp_byte(b2, rnd[2]);
-            e = (e << 8) | cnat_exp_byte(b1, rnd[1]);
-            e = (e << 8) | cnat_exp_byte(b0, rnd[0]);
-            st_stream_u32(ev + k * 32 + lane, e);
-            nib = __funnelshift_l(b3, nib, 1);
-            nib = __funnelshift_l(b2, nib, 1);
-            nib = __funnelshift_l(b1, nib, 1);
-            nib = __funnelshift_l(b0, nib, 1);
+        for (int k = 0; k < 8; ++k) any |= u[k].x | u[k].y | u[k].z | u[k].w;
+        const bool guarded = __any_sync(0xFFFFFFFFu, (any & 0x7F000000u) == 0x7F000000u);
+
+        uint32_t nib = 0;   // sign bits of this lane's 32 elements: bit 4k+c <-> group k, element c
+        if (!guarded) {
+#pragma unroll
+            for (int k = 7; k >= 0; --k) {
+                uint32_t rnd[4];
+                stream_words4_tile(q_lo + k * 32, pt, keys, rnd);
+                const uint32_t b0 = u[k].x, b1 = u[k].y, b2 = u[k].z, b3 = u[k].w;
+                // (bits + (~r23 & 0x7FFFFF)) << 1: sign shifted out, rounded exponent in byte 3
+                const uint32_t t0 = (b0 + (~rnd[0] & 0x7FFFFFu)) << 1;
+                const uint32_t t1 = (b1 + (~rnd[1] & 0x7FFFFFu)) << 1;
+                const uint32_t t2 = (b2 + (~rnd[2] & 0x7FFFFFu)) << 1;
+                const uint32_t t3 = (b3 + (~rnd[3] & 0x7FFFFFu)) << 1;
+                const uint32_t e = __byte_perm(__byte_perm(t0, t1, 0x0073),
+                                               __byte_perm(t2, t3, 0x0073), 0x5410);
+                st_stream_u32(ev + k * 32 + lane, e);
+                nib = __funnelshift_l(b3, nib, 1);
+                nib = __funnelshift_l(b2, nib, 1);
+                nib = __funnelshift_l(b1, nib, 1);
+                nib = __funnelshift_l(b0, nib, 1);
+            }
+        } else {
+#pragma unroll
+            for (int k = 7; k >= 0; --k) {
+                uint32_t rnd[4];
+                stream_words4_tile(q_lo + k * 32, pt, keys, rnd);
+                const uint32_t b0 = u[k].x, b1 = u[k].y, b2 = u[k].z, b3 = u[k].w;
+                uint32_t e = cnat_exp_byte(b3, rnd[3]);
+                e = (e << 8) | cnat_exp_byte(b2, rnd[2]);
+                e = (e << 8) | cnat_exp_byte(b1, rnd[1]);
+                e = (e << 8) | cnat_exp_byte(b0, rnd[0]);
+                st_stream_u32(ev + k * 32 + lane, e);
+                nib = __funnelshift_l(b3, nib, 1);
+                nib = __funnelshift_l(b2, nib, 1);
+                nib = __funnelshift_l(b1, nib, 1);
+                nib = __funnelshift_l(b0, nib, 1);
+            }
         }
         // lane 8g+i holds nibble k of sign word (k, g); after the transpose lane 8g+k holds the
         // whole word covering elements k*128 + g*32 .. +31 of the tile.

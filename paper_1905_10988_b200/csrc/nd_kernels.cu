@@ -25,6 +25,14 @@ struct DitherPlanes {
     const uint32_t* sign[NC_MAX_WORKERS];
 };
 
+struct DitherBatch {
+    const float* x[NC_MAX_WORKERS];
+    float* norms[NC_MAX_WORKERS];
+    uint8_t* level[NC_MAX_WORKERS];
+    uint32_t* sign[NC_MAX_WORKERS];
+    uint32_t worker[NC_MAX_WORKERS];
+};
+
 struct V8 {
     uint32_t v[8];
 };
@@ -119,16 +127,19 @@ struct NormAcc {
     }
 };
 
-// grid: ceil(tiles / warps per block)
+// grid: (ceil(tiles / warps per block), n workers); worker w uses slots + w * slot_stride
 template <int P>
 __global__ void __launch_bounds__(kBlockThreads)
-nd_norm_partials_kernel(const float* __restrict__ x, const uint64_t d,
+nd_norm_partials_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d,
                         const uint64_t* __restrict__ off, const int B,
-                        uint64_t* __restrict__ slots, uint32_t* __restrict__ tile_bucket) {
+                        uint64_t* __restrict__ slots_all, const uint64_t slot_stride,
+                        uint32_t* __restrict__ tile_bucket) {
     const int lane = threadIdx.x & 31;
     const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint64_t base = tile * kTile;
     if (base >= d) return;
+    const float* __restrict__ x = batch.x[blockIdx.y];
+    uint64_t* __restrict__ slots = slots_all + (uint64_t)blockIdx.y * slot_stride;
     const uint64_t end = (base + kTile <= d) ? base + kTile : d;
     const bool full = (base + kTile <= d);
 
@@ -173,33 +184,51 @@ nd_norm_partials_kernel(const float* __restrict__ x, const uint64_t d,
     }
 }
 
-// one warp per bucket: fixed-order sum (or max) of the bucket's slots -> norms[b]
+// one block per (bucket, worker): fixed-order sum (or max) of the bucket's slots -> norms[b]
 template <int P>
 __global__ void __launch_bounds__(kBlockThreads)
-nd_norm_finalize_kernel(const uint64_t* __restrict__ off, const int B,
-                        const uint64_t* __restrict__ slots, float* __restrict__ norms) {
+nd_norm_finalize_kernel(const __grid_constant__ DitherBatch batch,
+                        const uint64_t* __restrict__ off, const int B,
+                        const uint64_t* __restrict__ slots_all, const uint64_t slot_stride) {
     const int lane = threadIdx.x & 31;
-    const int b = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    if (b >= B) return;
+    const int b = blockIdx.x;
+    const uint64_t* __restrict__ slots = slots_all + (uint64_t)blockIdx.y * slot_stride;
+    float* __restrict__ norms = batch.norms[blockIdx.y];
+    __shared__ double s_sum[kWarpsPerBlock];
+    __shared__ uint32_t s_max[kWarpsPerBlock];
     const uint64_t lo = off[b], hi = off[b + 1];
-    float result = 0.f;
-    if (hi > lo) {
-        const uint64_t t_first = lo / kTile, t_last = (hi - 1) / kTile;
-        if (P == NC_P_INF) {
-            uint32_t m = 0;
-            for (uint64_t t = t_first + lane; t <= t_last; t += 32)
-                m = max(m, (uint32_t)slots[t + (uint64_t)b]);
-            result = __uint_as_float(warp_max(m));
-        } else {
-            double s = 0.0;
-            for (uint64_t t = t_first + lane; t <= t_last; t += 32)
-                s += __longlong_as_double((long long)slots[t + (uint64_t)b]);
-            s = warp_sum(s);
-            if (P == 2) s = sqrt(s);
-            result = (float)s;
-        }
+    if (hi <= lo) {                      // empty bucket (uniform over the block)
+        if (threadIdx.x == 0) norms[b] = 0.f;
+        return;
     }
-    if (lane == 0) norms[b] = result;
+    const uint64_t t_first = lo / kTile, t_last = (hi - 1) / kTile;
+    uint32_t m = 0;
+    double s = 0.0;
+    for (uint64_t t = t_first + threadIdx.x; t <= t_last; t += kBlockThreads) {
+        const uint64_t v = slots[t + (uint64_t)b];
+        if (P == NC_P_INF) m = max(m, (uint32_t)v);
+        else s += __longlong_as_double((long long)v);
+    }
+    if (P == NC_P_INF) m = warp_max(m);
+    else s = warp_sum(s);
+    if (lane == 0) {
+        s_sum[threadIdx.x >> 5] = s;
+        s_max[threadIdx.x >> 5] = m;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float result;
+        if (P == NC_P_INF) {
+            for (int w = 1; w < kWarpsPerBlock; ++w) m = max(m, s_max[w]);
+            result = __uint_as_float(m);
+        } else {
+            double tot = 0.0;
+            for (int w = 0; w < kWarpsPerBlock; ++w) tot += s_sum[w];     // fixed order
+            if (P == 2) tot = sqrt(tot);
+            result = (float)tot;
+        }
+        norms[b] = result;
+    }
 }
 
 struct BucketScale {
@@ -218,8 +247,7 @@ __device__ __forceinline__ BucketScale bucket_scale(float norm, int s) {
 // level code of one entry; pow2s = 2^s as a float
 __device__ __forceinline__ uint32_t level_code(uint32_t bits, uint32_t rnd, const BucketScale sc,
                                                float pow2s) {
-    const float ax = __uint_as_float(bits & 0x7FFFFFFFu);
-    const float y = __fmul_rn(ax, sc.rinv);
+    const float y = __fmul_rn(fabsf(__uint_as_float(bits)), sc.rinv);   // |x| is an operand modifier
     const float z = __fmul_rn(y, pow2s);
     float w = z;
     if (z < 2.0f) w = __fmaf_rz(z, 0.5f, 1.0f);
@@ -229,15 +257,19 @@ __device__ __forceinline__ uint32_t level_code(uint32_t bits, uint32_t rnd, cons
 
 // grid: ceil(tiles / warps per block)
 __global__ void __launch_bounds__(kBlockThreads)
-nd_round_pack_kernel(const float* __restrict__ x, const uint64_t d,
+nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d,
                      const uint64_t* __restrict__ off, const int B, const int s,
-                     const uint32_t worker, const __grid_constant__ PhiloxKeys keys,
-                     const float* __restrict__ norms, const uint32_t* __restrict__ tile_bucket,
-                     uint8_t* __restrict__ level, uint32_t* __restrict__ sign) {
+                     const __grid_constant__ PhiloxKeys keys,
+                     const uint32_t* __restrict__ tile_bucket) {
     const int lane = threadIdx.x & 31;
     const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint64_t base = tile * kTile;
     if (base >= d) return;
+    const float* __restrict__ x = batch.x[blockIdx.y];
+    const float* __restrict__ norms = batch.norms[blockIdx.y];
+    uint8_t* __restrict__ level = batch.level[blockIdx.y];
+    uint32_t* __restrict__ sign = batch.sign[blockIdx.y];
+    const uint32_t worker = batch.worker[blockIdx.y];
     const bool full = (base + kTile <= d);
     const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
 
@@ -251,16 +283,18 @@ nd_round_pack_kernel(const float* __restrict__ x, const uint64_t d,
     if (full && __ldg(off + b + 1) >= base + kTile) {
         const BucketScale sc = bucket_scale(norms[b], s);
         uint32_t* lv = reinterpret_cast<uint32_t*>(level + (base >> 1));
+        const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainDnat, keys);
+        const uint32_t q_lo = (uint32_t)(base >> 2) + (uint32_t)(lane * 2);
         uint32_t sbytes = 0;     // byte `it` = sign bits of this lane's 8 elements in step it
 #pragma unroll
         for (int it = 3; it >= 0; --it) {
             uint32_t rnd[8];
-            const uint64_t q = (base >> 2) + (uint64_t)(it * 64 + lane * 2);
+            const uint32_t q = q_lo + (uint32_t)(it * 64);   // stays below 2^32: no carry
             {
                 uint32_t r4[4];
-                stream_words4(q, worker, kDomainDnat, keys, r4);
+                stream_words4_tile(q, pt, keys, r4);
                 rnd[0] = r4[0]; rnd[1] = r4[1]; rnd[2] = r4[2]; rnd[3] = r4[3];
-                stream_words4(q + 1, worker, kDomainDnat, keys, r4);
+                stream_words4_tile(q + 1, pt, keys, r4);
                 rnd[4] = r4[0]; rnd[5] = r4[1]; rnd[6] = r4[2]; rnd[7] = r4[3];
             }
             uint32_t nib = 0;
@@ -364,19 +398,47 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
         }
         const uint32_t kexp = (uint32_t)(127 - s);
         const int sh = 8 * (lane & 3);
-        for (int i = 0; i < n; ++i) {
-            float norm = __ldg(planes.norms[i] + b);
-            if (!(fabsf(norm) <= 3.40282347e38f)) norm = 0.f;   // codes of such a bucket are 0
-            const uint32_t* lv = reinterpret_cast<const uint32_t*>(planes.level[i] + (base >> 1));
-            const uint32_t sw = ld_stream_u32(planes.sign[i] + (base >> 5) + lane);
-            uint32_t nb[4];
+        // exponent bytes of 2^(c-s) for c = 0..7 (0 for c = 0): a byte-permute with the four level
+        // nibbles as selector looks four of them up at once; codes 8..15 take the arithmetic path
+        uint32_t tbl_lo = 0, tbl_hi = 0;
+#pragma unroll
+        for (int c = 1; c < 8; ++c) {
+            const uint32_t e = (uint32_t)c + kexp;
+            if (c < 4) tbl_lo |= e << (8 * c); else tbl_hi |= e << (8 * (c - 4));
+        }
+        // software pipeline over the workers: the planes of worker i+1 are in flight while
+        // worker i is decoded
+        uint32_t nb[4], sw;
+        float norm;
+        {
+            const uint32_t* lv = reinterpret_cast<const uint32_t*>(planes.level[0] + (base >> 1));
+            norm = __ldg(planes.norms[0] + b);
+            sw = ld_stream_u32(planes.sign[0] + (base >> 5) + lane);
 #pragma unroll
             for (int it = 0; it < 4; ++it) nb[it] = ld_stream_u32(lv + it * 32 + lane);
+        }
+        for (int i = 0; i < n; ++i) {
+            uint32_t nb_n[4] = {0u, 0u, 0u, 0u}, sw_n = 0u;
+            float norm_n = 0.f;
+            if (i + 1 < n) {
+                const uint32_t* lv =
+                    reinterpret_cast<const uint32_t*>(planes.level[i + 1] + (base >> 1));
+                norm_n = __ldg(planes.norms[i + 1] + b);
+                sw_n = ld_stream_u32(planes.sign[i + 1] + (base >> 5) + lane);
+#pragma unroll
+                for (int it = 0; it < 4; ++it) nb_n[it] = ld_stream_u32(lv + it * 32 + lane);
+            }
+            if (!(fabsf(norm) <= 3.40282347e38f)) norm = 0.f;   // codes of such a bucket are 0
 #pragma unroll
             for (int it = 0; it < 4; ++it) {
                 const uint32_t sg = __shfl_sync(0xFFFFFFFFu, sw, it * 8 + (lane >> 2)) >> sh;
                 uint32_t lo4, hi4;
-                level_exp_bytes(nb[it], kexp, lo4, hi4);
+                if ((nb[it] & 0x88888888u) == 0u) {
+                    lo4 = __byte_perm(tbl_lo, tbl_hi, nb[it] & 0xFFFFu);
+                    hi4 = __byte_perm(tbl_lo, tbl_hi, nb[it] >> 16);
+                } else {
+                    level_exp_bytes(nb[it], kexp, lo4, hi4);
+                }
                 float* a = reinterpret_cast<float*>(acc[it].v);
                 a[0] = add_scaled(a[0], norm, pow2_signed<0>(lo4, sg));
                 a[1] = add_scaled(a[1], norm, pow2_signed<1>(lo4, sg >> 1));
@@ -387,6 +449,10 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
                 a[6] = add_scaled(a[6], norm, pow2_signed<2>(hi4, sg >> 6));
                 a[7] = add_scaled(a[7], norm, pow2_signed<3>(hi4, sg >> 7));
             }
+#pragma unroll
+            for (int it = 0; it < 4; ++it) nb[it] = nb_n[it];
+            sw = sw_n;
+            norm = norm_n;
         }
 #pragma unroll
         for (int it = 0; it < 4; ++it) st_stream_v8(out + base + it * 256 + lane * 8, acc[it]);
@@ -424,53 +490,78 @@ using namespace natcomp;
 
 extern "C" {
 
-size_t nd_workspace_bytes(size_t d, int num_buckets) {
+size_t nd_batch_workspace_bytes(size_t d, int num_buckets, int n) {
     if (num_buckets < 0) num_buckets = 0;
+    if (n < 1) n = 1;
     const uint64_t tiles = nd_tiles(d);
-    // slots: one 64-bit partial per (tile, bucket) overlap; then the tile -> bucket map
-    return round_up16((tiles + (uint64_t)num_buckets + 1) * 8) + round_up16(tiles * 4);
+    // per worker: one 64-bit partial per (tile, bucket) overlap; shared: the tile -> bucket map
+    return (size_t)n * round_up16((tiles + (uint64_t)num_buckets + 1) * 8) + round_up16(tiles * 4);
+}
+
+size_t nd_workspace_bytes(size_t d, int num_buckets) {
+    return nd_batch_workspace_bytes(d, num_buckets, 1);
+}
+
+nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B,
+                            int p, int s, uint64_t seed, const uint32_t* workers,
+                            float* const* norms, uint8_t* const* levels, uint32_t* const* signs,
+                            int n, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (!xs || !bucket_off || !workers || !norms || !levels || !signs || n < 1 ||
+        n > NC_MAX_WORKERS || B < 1 || s < 1 || s > 15)
+        return NC_ERR_INVALID;
+    if (p != 1 && p != 2 && p != NC_P_INF) return NC_ERR_UNSUPPORTED;
+    if (d == 0) return NC_OK;
+    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    if (!workspace) return NC_ERR_INVALID;
+    if (!aligned16(workspace) || ((uintptr_t)bucket_off & 7u)) return NC_ERR_ALIGN;
+    DitherBatch batch;
+    for (int i = 0; i < n; ++i) {
+        if (!xs[i] || !norms[i] || !levels[i] || !signs[i]) return NC_ERR_INVALID;
+        if (!aligned32(xs[i]) || !aligned16(levels[i]) || !aligned16(signs[i]) ||
+            !aligned4(norms[i]))
+            return NC_ERR_ALIGN;
+        batch.x[i] = xs[i];
+        batch.norms[i] = norms[i];
+        batch.level[i] = levels[i];
+        batch.sign[i] = signs[i];
+        batch.worker[i] = workers[i];
+    }
+    if (workspace_bytes < nd_batch_workspace_bytes(d, B, n)) return NC_ERR_WORKSPACE;
+    const uint64_t tiles = nd_tiles(d);
+    const uint64_t slot_stride = round_up16((tiles + (uint64_t)B + 1) * 8) / 8;
+    uint64_t* slots = reinterpret_cast<uint64_t*>(workspace);
+    uint32_t* tile_bucket = reinterpret_cast<uint32_t*>(slots + (uint64_t)n * slot_stride);
+    const dim3 grid(nd_tile_blocks(d), (unsigned)n);
+    const dim3 fgrid((unsigned)B, (unsigned)n);
+    if (p == 1) {
+        nd_norm_partials_kernel<1><<<grid, kBlockThreads, 0, stream>>>(
+            batch, d, bucket_off, B, slots, slot_stride, tile_bucket);
+        nd_norm_finalize_kernel<1><<<fgrid, kBlockThreads, 0, stream>>>(batch, bucket_off, B,
+                                                                        slots, slot_stride);
+    } else if (p == 2) {
+        nd_norm_partials_kernel<2><<<grid, kBlockThreads, 0, stream>>>(
+            batch, d, bucket_off, B, slots, slot_stride, tile_bucket);
+        nd_norm_finalize_kernel<2><<<fgrid, kBlockThreads, 0, stream>>>(batch, bucket_off, B,
+                                                                        slots, slot_stride);
+    } else {
+        nd_norm_partials_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
+            batch, d, bucket_off, B, slots, slot_stride, tile_bucket);
+        nd_norm_finalize_kernel<NC_P_INF><<<fgrid, kBlockThreads, 0, stream>>>(
+            batch, bucket_off, B, slots, slot_stride);
+    }
+    const PhiloxKeys keys = make_philox_keys(seed);
+    nd_round_pack_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, bucket_off, B, s, keys,
+                                                             tile_bucket);
+    return launch_status();
 }
 
 nc_status nd_compress(const float* x, size_t d, const uint64_t* bucket_off, int B, int p, int s,
                       uint64_t seed, uint32_t worker, float* norms, uint8_t* level,
                       uint32_t* sign, void* workspace, size_t workspace_bytes,
                       cudaStream_t stream) {
-    if (!x || !bucket_off || !norms || !level || !sign || B < 1 || s < 1 || s > 15)
-        return NC_ERR_INVALID;
-    if (p != 1 && p != 2 && p != NC_P_INF) return NC_ERR_UNSUPPORTED;
-    if (d == 0) return NC_OK;
-    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
-    if (!workspace) return NC_ERR_INVALID;
-    if (!aligned32(x) || !aligned16(level) || !aligned16(sign) || !aligned16(workspace) ||
-        !aligned4(norms) || ((uintptr_t)bucket_off & 7u))
-        return NC_ERR_ALIGN;
-    if (workspace_bytes < nd_workspace_bytes(d, B)) return NC_ERR_WORKSPACE;
-    const uint64_t tiles = nd_tiles(d);
-    uint64_t* slots = reinterpret_cast<uint64_t*>(workspace);
-    uint32_t* tile_bucket = reinterpret_cast<uint32_t*>(
-        reinterpret_cast<char*>(workspace) + round_up16((tiles + (uint64_t)B + 1) * 8));
-    const unsigned grid = nd_tile_blocks(d);
-    const unsigned fgrid = (unsigned)((B + kWarpsPerBlock - 1) / kWarpsPerBlock);
-    if (p == 1) {
-        nd_norm_partials_kernel<1><<<grid, kBlockThreads, 0, stream>>>(x, d, bucket_off, B, slots,
-                                                                       tile_bucket);
-        nd_norm_finalize_kernel<1><<<fgrid, kBlockThreads, 0, stream>>>(bucket_off, B, slots,
-                                                                        norms);
-    } else if (p == 2) {
-        nd_norm_partials_kernel<2><<<grid, kBlockThreads, 0, stream>>>(x, d, bucket_off, B, slots,
-                                                                       tile_bucket);
-        nd_norm_finalize_kernel<2><<<fgrid, kBlockThreads, 0, stream>>>(bucket_off, B, slots,
-                                                                        norms);
-    } else {
-        nd_norm_partials_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
-            x, d, bucket_off, B, slots, tile_bucket);
-        nd_norm_finalize_kernel<NC_P_INF><<<fgrid, kBlockThreads, 0, stream>>>(bucket_off, B,
-                                                                               slots, norms);
-    }
-    const PhiloxKeys keys = make_philox_keys(seed);
-    nd_round_pack_kernel<<<grid, kBlockThreads, 0, stream>>>(x, d, bucket_off, B, s, worker, keys,
-                                                             norms, tile_bucket, level, sign);
-    return launch_status();
+    if (!x || !norms || !level || !sign) return NC_ERR_INVALID;
+    return nd_compress_batch(&x, d, bucket_off, B, p, s, seed, &worker, &norms, &level, &sign, 1,
+                             workspace, workspace_bytes, stream);
 }
 
 static nc_status nd_check_planes(const float* const* norms, const uint8_t* const* levels,

@@ -6,11 +6,12 @@
 // path is integer ALU work, not memory: x is read only where a coordinate is kept.
 //
 // Order-preserving compaction without any inter-block waiting:
-//   select : per 1024-element tile, selection bitmask (canonical bit order), kept count and
-//            a norm partial of the kept, scaled entries
-//   scan   : one block turns the tile counts into exclusive offsets and the partials into the norm
-//   emit   : per tile, rank of every kept entry = tile offset + prefix popcount; writes the
-//            index list and one code byte per entry
+//   select : per 1024-element tile a selection bitmask (canonical bit order); per block of 8
+//            tiles the kept count and a norm partial of the kept, scaled entries
+//   scan   : one block turns the block counts into exclusive offsets and the partials into the norm
+//   emit   : rank of every kept entry = block offset + popcounts of the earlier tiles of the
+//            block + prefix popcount inside the tile; writes the index list and one code byte
+//            per entry
 //   pack   : two code bytes -> one byte of 4-bit codes
 #include "common.cuh"
 #include "philox.cuh"
@@ -19,10 +20,19 @@ namespace natcomp {
 
 constexpr int kScanThreads = 1024;
 
+struct SparseBatch {
+    const float* x[NC_MAX_WORKERS];
+    uint32_t* idx[NC_MAX_WORKERS];
+    uint8_t* codes[NC_MAX_WORKERS];
+    uint32_t* count[NC_MAX_WORKERS];
+    float* norm[NC_MAX_WORKERS];
+    uint32_t worker[NC_MAX_WORKERS];
+};
+
 struct SparseWorkspace {
     uint32_t* bitmask;      // tiles * 32 words
-    uint32_t* tile_count;   // tiles (becomes the exclusive offset after the scan)
-    uint64_t* tile_partial; // tiles
+    uint32_t* block_count;   // one per block of 8 tiles (the exclusive offset after the scan)
+    uint64_t* block_partial; // one per block of 8 tiles
     uint8_t* tmp_codes;     // cap bytes
 };
 
@@ -33,13 +43,13 @@ inline size_t sparse_ws_bytes(uint64_t d, uint64_t cap) {
     return round_up16(t * 128) + round_up16(t * 4) + round_up16(t * 8) + round_up16(cap);
 }
 
-inline SparseWorkspace sparse_ws_carve(void* ws, uint64_t d) {
+__host__ __device__ inline SparseWorkspace sparse_ws_carve(void* ws, uint64_t d) {
     const uint64_t t = sparse_tiles(d);
     char* p = reinterpret_cast<char*>(ws);
     SparseWorkspace w;
     w.bitmask = reinterpret_cast<uint32_t*>(p);      p += round_up16(t * 128);
-    w.tile_count = reinterpret_cast<uint32_t*>(p);   p += round_up16(t * 4);
-    w.tile_partial = reinterpret_cast<uint64_t*>(p); p += round_up16(t * 8);
+    w.block_count = reinterpret_cast<uint32_t*>(p);   p += round_up16(t * 4);
+    w.block_partial = reinterpret_cast<uint64_t*>(p); p += round_up16(t * 8);
     w.tmp_codes = reinterpret_cast<uint8_t*>(p);
     return w;
 }
@@ -63,23 +73,30 @@ __device__ __forceinline__ uint32_t warp_sum_u(uint32_t v) {
 // grid: ceil(tiles / warps per block)
 template <int P>
 __global__ void __launch_bounds__(kBlockThreads)
-sparse_select_kernel(const float* __restrict__ x, const uint64_t d, const uint32_t thr32,
-                     const bool keep_all, const float scale, const uint32_t worker,
-                     const __grid_constant__ PhiloxKeys keys, uint32_t* __restrict__ bitmask,
-                     uint32_t* __restrict__ tile_count, uint64_t* __restrict__ tile_partial) {
+sparse_select_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
+                     const uint32_t thr32, const bool keep_all, const float scale,
+                     const __grid_constant__ PhiloxKeys keys, char* __restrict__ ws_all,
+                     const uint64_t ws_stride) {
     const int lane = threadIdx.x & 31;
     const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint64_t base = tile * kTile;
-    if (base >= d) return;
+    const bool active = base < d;        // whole warps; inactive ones only join the block sum
+    const float* __restrict__ x = batch.x[blockIdx.y];
+    const uint32_t worker = batch.worker[blockIdx.y];
+    const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
+    uint32_t* __restrict__ bitmask = ws.bitmask;
+    __shared__ uint32_t s_cnt[kWarpsPerBlock];
+    __shared__ uint64_t s_part[kWarpsPerBlock];
 
     uint32_t nib = 0;        // bit 4k+c <-> element base + k*128 + 4*lane + c
     double dsum = 0.0;
     uint32_t vmax = 0;
-#pragma unroll 1
-    for (int k = 7; k >= 0; --k) {
+    const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainSelect, keys);
+#pragma unroll 2
+    for (int k = active ? 7 : -1; k >= 0; --k) {
         const uint64_t j4 = base + (uint64_t)(k * 128 + lane * 4);
         uint32_t rnd[4];
-        stream_words4(j4 >> 2, worker, kDomainSelect, keys, rnd);
+        stream_words4_tile((uint32_t)(j4 >> 2), pt, keys, rnd);
 #pragma unroll
         for (int c = 3; c >= 0; --c) {
             const bool keep = (keep_all || rnd[c] < thr32) && (j4 + c < d);
@@ -94,23 +111,41 @@ sparse_select_kernel(const float* __restrict__ x, const uint64_t d, const uint32
         }
     }
     const uint32_t word = transpose_nibbles_8x8(nib, lane);
-    bitmask[tile * 32 + (lane & 7) * 4 + (lane >> 3)] = word;
+    if (active) bitmask[tile * 32 + (lane & 7) * 4 + (lane >> 3)] = word;
     const uint32_t cnt = warp_sum_u(__popc(nib));
     uint64_t part;
     if (P == NC_P_INF) part = (uint64_t)warp_max_u(vmax);
     else part = (uint64_t)__double_as_longlong(warp_sum_d(dsum));
     if (lane == 0) {
-        tile_count[tile] = cnt;
-        tile_partial[tile] = part;
+        s_cnt[threadIdx.x >> 5] = cnt;
+        s_part[threadIdx.x >> 5] = part;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t c = 0, m = 0;
+        double sum = 0.0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) {     // fixed order
+            c += s_cnt[w];
+            if (P == NC_P_INF) m = max(m, (uint32_t)s_part[w]);
+            else sum += __longlong_as_double((long long)s_part[w]);
+        }
+        ws.block_count[blockIdx.x] = c;
+        ws.block_partial[blockIdx.x] =
+            (P == NC_P_INF) ? (uint64_t)m : (uint64_t)__double_as_longlong(sum);
     }
 }
 
-// one block: exclusive scan of the tile counts (in place), total count, norm
+// one block: exclusive scan of the per-block counts (in place), total count, norm
 template <int P>
 __global__ void __launch_bounds__(kScanThreads)
-sparse_scan_kernel(const uint64_t tiles, uint32_t* __restrict__ tile_count,
-                   const uint64_t* __restrict__ tile_partial, uint32_t* __restrict__ count,
-                   float* __restrict__ norm) {
+sparse_scan_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
+                   char* __restrict__ ws_all, const uint64_t ws_stride) {
+    const uint64_t tiles = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;   // blocks
+    const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
+    uint32_t* __restrict__ tile_count = ws.block_count;
+    const uint64_t* __restrict__ tile_partial = ws.block_partial;
+    uint32_t* __restrict__ count = batch.count[blockIdx.y];
+    float* __restrict__ norm = batch.norm[blockIdx.y];
     __shared__ uint32_t s_cnt[kScanThreads];
     __shared__ double s_sum[kScanThreads];
     __shared__ uint32_t s_max[kScanThreads];
@@ -187,16 +222,22 @@ __device__ __forceinline__ uint32_t sparse_level_code(uint32_t bits, uint32_t rn
 
 // grid: ceil(tiles / warps per block)
 __global__ void __launch_bounds__(kBlockThreads)
-sparse_emit_kernel(const float* __restrict__ x, const uint64_t d, const float scale, const int s,
-                   const uint32_t worker, const __grid_constant__ PhiloxKeys keys,
-                   const uint32_t* __restrict__ bitmask, const uint32_t* __restrict__ tile_offset,
-                   const float* __restrict__ norm, const uint64_t cap, uint32_t* __restrict__ idx,
-                   uint8_t* __restrict__ tmp_codes) {
+sparse_emit_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d, const float scale,
+                   const int s, const __grid_constant__ PhiloxKeys keys, const uint64_t cap,
+                   char* __restrict__ ws_all, const uint64_t ws_stride) {
     const int lane = threadIdx.x & 31;
     const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint64_t base = tile * kTile;
-    if (base >= d) return;
-    uint32_t word = bitmask[tile * 32 + lane];
+    const bool active = base < d;
+    const float* __restrict__ x = batch.x[blockIdx.y];
+    const uint32_t worker = batch.worker[blockIdx.y];
+    const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
+    const uint32_t* __restrict__ bitmask = ws.bitmask;
+    const float* __restrict__ norm = batch.norm[blockIdx.y];
+    uint32_t* __restrict__ idx = batch.idx[blockIdx.y];
+    uint8_t* __restrict__ tmp_codes = ws.tmp_codes;
+    __shared__ uint32_t s_tile[kWarpsPerBlock];
+    uint32_t word = active ? bitmask[tile * 32 + lane] : 0u;
     const uint32_t cnt = __popc(word);
     uint32_t incl = cnt;
 #pragma unroll
@@ -204,7 +245,10 @@ sparse_emit_kernel(const float* __restrict__ x, const uint64_t d, const float sc
         const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
         if (lane >= o) incl += v;
     }
-    uint64_t k = (uint64_t)tile_offset[tile] + (incl - cnt);
+    if (lane == 31) s_tile[threadIdx.x >> 5] = incl;      // kept entries of this tile
+    __syncthreads();
+    uint64_t k = (uint64_t)ws.block_count[blockIdx.x] + (incl - cnt);
+    for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) k += s_tile[w];
     if (word == 0) return;
     const Scale sc = make_scale(*norm, s);
     const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
@@ -229,8 +273,12 @@ sparse_emit_kernel(const float* __restrict__ x, const uint64_t d, const float sc
 
 // thread t -> output byte t; zero padding up to the next multiple of 16 bytes
 __global__ void __launch_bounds__(kBlockThreads)
-sparse_pack_kernel(const uint8_t* __restrict__ tmp_codes, const uint32_t* __restrict__ count,
-                   const uint64_t cap, uint8_t* __restrict__ codes) {
+sparse_pack_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d, const uint64_t cap,
+                   char* __restrict__ ws_all, const uint64_t ws_stride) {
+    const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
+    const uint8_t* __restrict__ tmp_codes = ws.tmp_codes;
+    const uint32_t* __restrict__ count = batch.count[blockIdx.y];
+    uint8_t* __restrict__ codes = batch.codes[blockIdx.y];
     const uint64_t t = (uint64_t)blockIdx.x * kBlockThreads + threadIdx.x;
     const uint64_t total = min((uint64_t)*count, cap);
     const uint64_t nbytes = (total + 1) / 2;
@@ -271,50 +319,75 @@ extern "C" {
 
 size_t nd_sparse_workspace_bytes(size_t d, size_t cap) { return sparse_ws_bytes(d, cap); }
 
-nc_status nd_sparse_compress(const float* x, size_t d, uint64_t keep_threshold, float scale,
-                             int p, int s, uint64_t seed, uint32_t worker, uint32_t* idx,
-                             uint8_t* codes, uint32_t* count, float* norm, size_t cap,
-                             void* workspace, size_t workspace_bytes, cudaStream_t stream) {
-    if (!x || !idx || !codes || !count || !norm || s < 1 || s > 7 || cap < 1 ||
-        keep_threshold > ((uint64_t)1 << 32))
+size_t nd_sparse_batch_workspace_bytes(size_t d, size_t cap, int n) {
+    return (size_t)(n < 1 ? 1 : n) * sparse_ws_bytes(d, cap);
+}
+
+nc_status nd_sparse_compress_batch(const float* const* xs, size_t d, uint64_t keep_threshold,
+                                   float scale, int p, int s, uint64_t seed,
+                                   const uint32_t* workers, uint32_t* const* idxs,
+                                   uint8_t* const* codes, uint32_t* const* counts,
+                                   float* const* norms, size_t cap, int n, void* workspace,
+                                   size_t workspace_bytes, cudaStream_t stream) {
+    if (!xs || !workers || !idxs || !codes || !counts || !norms || n < 1 || n > NC_MAX_WORKERS ||
+        s < 1 || s > 7 || cap < 1 || keep_threshold > ((uint64_t)1 << 32))
         return NC_ERR_INVALID;
     if (p != 1 && p != 2 && p != NC_P_INF) return NC_ERR_UNSUPPORTED;
     if (d == 0) return NC_OK;
     if (d > 0xFFFFFFFFull) return NC_ERR_INVALID;
     if (!workspace) return NC_ERR_INVALID;
-    if (!aligned32(x) || !aligned16(idx) || !aligned16(codes) || !aligned16(workspace) ||
-        !aligned4(count) || !aligned4(norm))
-        return NC_ERR_ALIGN;
-    if (workspace_bytes < sparse_ws_bytes(d, cap)) return NC_ERR_WORKSPACE;
-    const SparseWorkspace ws = sparse_ws_carve(workspace, d);
+    if (!aligned16(workspace)) return NC_ERR_ALIGN;
+    SparseBatch batch;
+    for (int i = 0; i < n; ++i) {
+        if (!xs[i] || !idxs[i] || !codes[i] || !counts[i] || !norms[i]) return NC_ERR_INVALID;
+        if (!aligned32(xs[i]) || !aligned16(idxs[i]) || !aligned16(codes[i]) ||
+            !aligned4(counts[i]) || !aligned4(norms[i]))
+            return NC_ERR_ALIGN;
+        batch.x[i] = xs[i];
+        batch.idx[i] = idxs[i];
+        batch.codes[i] = codes[i];
+        batch.count[i] = counts[i];
+        batch.norm[i] = norms[i];
+        batch.worker[i] = workers[i];
+    }
+    const uint64_t ws_stride = sparse_ws_bytes(d, cap);
+    if (workspace_bytes < (size_t)n * ws_stride) return NC_ERR_WORKSPACE;
+    char* ws = reinterpret_cast<char*>(workspace);
     const uint64_t tiles = sparse_tiles(d);
-    const unsigned grid = (unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    const dim3 grid((unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
     const PhiloxKeys keys = make_philox_keys(seed);
     const bool keep_all = keep_threshold >= ((uint64_t)1 << 32);
     const uint32_t thr32 = keep_all ? 0xFFFFFFFFu : (uint32_t)keep_threshold;
+    const dim3 sgrid(1, (unsigned)n);
     if (p == 1) {
-        sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(
-            x, d, thr32, keep_all, scale, worker, keys, ws.bitmask, ws.tile_count, ws.tile_partial);
-        sparse_scan_kernel<1><<<1, kScanThreads, 0, stream>>>(tiles, ws.tile_count,
-                                                              ws.tile_partial, count, norm);
+        sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(batch, d, thr32, keep_all,
+                                                                    scale, keys, ws, ws_stride);
+        sparse_scan_kernel<1><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
     } else if (p == 2) {
-        sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(
-            x, d, thr32, keep_all, scale, worker, keys, ws.bitmask, ws.tile_count, ws.tile_partial);
-        sparse_scan_kernel<2><<<1, kScanThreads, 0, stream>>>(tiles, ws.tile_count,
-                                                              ws.tile_partial, count, norm);
+        sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(batch, d, thr32, keep_all,
+                                                                    scale, keys, ws, ws_stride);
+        sparse_scan_kernel<2><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
     } else {
         sparse_select_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
-            x, d, thr32, keep_all, scale, worker, keys, ws.bitmask, ws.tile_count, ws.tile_partial);
-        sparse_scan_kernel<NC_P_INF><<<1, kScanThreads, 0, stream>>>(tiles, ws.tile_count,
-                                                                     ws.tile_partial, count, norm);
+            batch, d, thr32, keep_all, scale, keys, ws, ws_stride);
+        sparse_scan_kernel<NC_P_INF><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
     }
-    sparse_emit_kernel<<<grid, kBlockThreads, 0, stream>>>(x, d, scale, s, worker, keys, ws.bitmask,
-                                                           ws.tile_count, norm, cap, idx,
-                                                           ws.tmp_codes);
+    sparse_emit_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap, ws,
+                                                           ws_stride);
     const uint64_t pack_threads = round_up16((cap + 1) / 2);
-    const unsigned pgrid = (unsigned)((pack_threads + kBlockThreads - 1) / kBlockThreads);
-    sparse_pack_kernel<<<pgrid, kBlockThreads, 0, stream>>>(ws.tmp_codes, count, cap, codes);
+    const dim3 pgrid((unsigned)((pack_threads + kBlockThreads - 1) / kBlockThreads), (unsigned)n);
+    sparse_pack_kernel<<<pgrid, kBlockThreads, 0, stream>>>(batch, d, cap, ws, ws_stride);
     return launch_status();
+}
+
+nc_status nd_sparse_compress(const float* x, size_t d, uint64_t keep_threshold, float scale,
+                             int p, int s, uint64_t seed, uint32_t worker, uint32_t* idx,
+                             uint8_t* codes, uint32_t* count, float* norm, size_t cap,
+                             void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (!x || !idx || !codes || !count || !norm) return NC_ERR_INVALID;
+    return nd_sparse_compress_batch(&x, d, keep_threshold, scale, p, s, seed, &worker, &idx,
+                                    &codes, &count, &norm, cap, 1, workspace, workspace_bytes,
+                                    stream);
 }
 
 nc_status nd_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes,

@@ -225,3 +225,32 @@ def test_unbiasedness_of_the_gpu_path_over_seeds():
     # per-entry variance <= max(y (2^(1-s)) , y^2 / 8) * norm^2 <= norm^2 * 2^(1-s) * max(y, ...)
     sigma = per * np.sqrt(np.maximum(np.abs(x) / per * 2.0 ** (1 - s), (x / per) ** 2 / 8))
     assert np.all(np.abs(mean - x) <= 6 * sigma / np.sqrt(trials) + 1e-12)
+
+
+def test_batch_launch_equals_single_launches():
+    rng = np.random.default_rng(33)
+    n, d, p, s = 5, 70001 + 96, 2, 8
+    off = workloads.small_bucket_table(d, seed=3)
+    B = len(off) - 1
+    off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
+    xs = [(rng.standard_normal(d) * 10.0 ** rng.uniform(-4, -1)).astype(np.float32)
+          for _ in range(n)]
+    xd = [dev(x) for x in xs]
+    workers = [7, 3, 0, 12, 5]
+    norms = [Guarded(4 * B) for _ in range(n)]
+    levels = [Guarded(nc.nd_level_bytes(d)) for _ in range(n)]
+    signs = [Guarded(nc.nc_sign_bytes(d)) for _ in range(n)]
+    ws_bytes = nc.nd_batch_workspace_bytes(d, B, n)
+    ws = Guarded(ws_bytes)
+    nc.nd_compress_batch(xd, d, off_dev, B, p, s, 11, workers, [g.buf for g in norms],
+                         [g.buf for g in levels], [g.buf for g in signs], n, ws.buf, ws_bytes)
+    torch.cuda.synchronize()
+    for g in norms + levels + signs + [ws]:
+        g.check()
+    for i in range(n):
+        n1, l1, s1 = gpu_nd_compress(xd[i], off, p, s, 11, workers[i])
+        assert np.array_equal(norms[i].numpy(np.uint32), n1.numpy(np.uint32))
+        assert np.array_equal(levels[i].numpy(np.uint8), l1.numpy(np.uint8))
+        assert np.array_equal(signs[i].numpy(np.uint32), s1.numpy(np.uint32))
+        check_against_oracle(xs[i], off, p, s, 11, workers[i], norms[i], levels[i], signs[i],
+                             slack=2)

@@ -77,7 +77,8 @@ def test_sparse_all_zero_and_nonfinite_inputs():
         x[10:20] = fillv
         got = gpu_sparse_compress(dev(x), 1 << 31, 2.0, nc.P_INF, 4, seed=1, worker=1, cap=d)
         check_sparse(x, 1 << 31, 2.0, nc.P_INF, 4, 1, 1, d, got)
-        codes = got[1].numpy(np.uint8)
+        codes = got[1].numpy(np.uint8)[:(got[2] + 1) // 2]
+        assert got[2] > 0
         assert np.all((codes & 0x77) == 0)        # degenerate norm: every level code is 0
 
 
@@ -135,3 +136,29 @@ def test_config5_full_size_one_worker():
     oracle.sparse_decode_accumulate(i_ref, c_ref, count_ref, n_ref, s, ref)
     got = acc.cpu().numpy()
     assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+
+
+def test_sparse_batch_launch_equals_single_launches():
+    rng = np.random.default_rng(44)
+    n, d, s = 4, 200_003, 4
+    thr, scale = workloads.KEEP_1PCT_THRESHOLD * 4, 25.0
+    cap = 12_000
+    xs = [rng.standard_normal(d).astype(np.float32) for _ in range(n)]
+    xd = [dev(x) for x in xs]
+    workers = [2, 9, 0, 5]
+    idx = [Guarded(4 * cap) for _ in range(n)]
+    codes = [Guarded(((cap + 1) // 2 + 15) // 16 * 16) for _ in range(n)]
+    count = [Guarded(4) for _ in range(n)]
+    norm = [Guarded(4) for _ in range(n)]
+    ws_bytes = nc.nd_sparse_batch_workspace_bytes(d, cap, n)
+    ws = Guarded(ws_bytes)
+    nc.nd_sparse_compress_batch(xd, d, thr, scale, nc.P_INF, s, 6, workers,
+                                [g.buf for g in idx], [g.buf for g in codes],
+                                [g.buf for g in count], [g.buf for g in norm], cap, n, ws.buf,
+                                ws_bytes)
+    torch.cuda.synchronize()
+    for g in idx + codes + count + norm + [ws]:
+        g.check()
+    for i in range(n):
+        got = (idx[i], codes[i], int(count[i].numpy(np.uint32)[0]), norm[i].numpy(np.float32)[0])
+        check_sparse(xs[i], thr, scale, nc.P_INF, s, 6, workers[i], cap, got)
