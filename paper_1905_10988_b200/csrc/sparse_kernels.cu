@@ -70,11 +70,34 @@ __device__ __forceinline__ uint32_t warp_sum_u(uint32_t v) {
     return v;
 }
 
+// Lists the set bits of a 1024-bit tile mask (lane l holds word l) in ascending order into the
+// warp's shared-memory list as in-tile positions; returns how many there are.  After this the
+// t-th kept entry can be handled by lane t mod 32, so the gathers from x run in parallel
+// instead of one dependent load per set bit of a lane's own word.
+__device__ __forceinline__ uint32_t warp_list_positions(uint32_t word, int lane,
+                                                        uint16_t* __restrict__ list) {
+    const uint32_t cnt = __popc(word);
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    uint32_t at = incl - cnt;
+    while (word) {
+        const int bit = __ffs(word) - 1;
+        word &= word - 1;
+        list[at++] = (uint16_t)(lane * 32 + bit);
+    }
+    __syncwarp();
+    return __shfl_sync(0xFFFFFFFFu, incl, 31);
+}
+
 // grid: ceil(tiles / warps per block)
 template <int P>
 __global__ void __launch_bounds__(kBlockThreads)
 sparse_select_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
-                     const uint32_t thr32, const bool keep_all, const float scale,
+                     const uint32_t neg_thr, const bool keep_none, const float scale,
                      const __grid_constant__ PhiloxKeys keys, char* __restrict__ ws_all,
                      const uint64_t ws_stride) {
     const int lane = threadIdx.x & 31;
@@ -88,31 +111,57 @@ sparse_select_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d
     __shared__ uint32_t s_cnt[kWarpsPerBlock];
     __shared__ uint64_t s_part[kWarpsPerBlock];
 
+    __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
+    uint16_t* list = s_list[threadIdx.x >> 5];
+
+    // phase 1: the 1024 selection bits of the tile, no memory traffic
     uint32_t nib = 0;        // bit 4k+c <-> element base + k*128 + 4*lane + c
-    double dsum = 0.0;
-    uint32_t vmax = 0;
     const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainSelect, keys);
-#pragma unroll 2
-    for (int k = active ? 7 : -1; k >= 0; --k) {
-        const uint64_t j4 = base + (uint64_t)(k * 128 + lane * 4);
-        uint32_t rnd[4];
-        stream_words4_tile((uint32_t)(j4 >> 2), pt, keys, rnd);
+    if (active && !keep_none) {
+        // coordinate j is dropped iff word >= threshold, i.e. iff word + (2^32 - threshold)
+        // carries out of 32 bits.  The drop bits are shifted in straight from that carry: two
+        // integer instructions per coordinate on top of the generator.
+        const uint32_t q_lo = (uint32_t)(base >> 2) + (uint32_t)lane;
+        uint32_t drop = 0;
 #pragma unroll
-        for (int c = 3; c >= 0; --c) {
-            const bool keep = (keep_all || rnd[c] < thr32) && (j4 + c < d);
-            nib = (nib << 1) | (keep ? 1u : 0u);
-            if (keep) {
-                const float xs = __fmul_rn(scale, x[j4 + c]);
-                const uint32_t a = __float_as_uint(xs) & 0x7FFFFFFFu;
-                if (P == NC_P_INF) vmax = max(vmax, a);
-                else if (P == 1) dsum += (double)__uint_as_float(a);
-                else dsum = fma((double)xs, (double)xs, dsum);
+        for (int k = 7; k >= 0; --k) {
+            uint32_t rnd[4];
+            stream_words4_tile(q_lo + (uint32_t)(k * 32), pt, keys, rnd);
+#pragma unroll
+            for (int c = 3; c >= 0; --c) {
+                uint32_t tmp;
+                asm("add.cc.u32 %1, %2, %3;\n\taddc.u32 %0, %0, %0;"
+                    : "+r"(drop), "=r"(tmp)
+                    : "r"(rnd[c]), "r"(neg_thr));
+            }
+        }
+        nib = ~drop;
+        if (base + kTile > d) {          // ragged last tile: clear the bits past the end
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if (base + (uint64_t)(k * 128 + lane * 4 + c) >= d) nib &= ~(1u << (4 * k + c));
+                }
             }
         }
     }
-    const uint32_t word = transpose_nibbles_8x8(nib, lane);
-    if (active) bitmask[tile * 32 + (lane & 7) * 4 + (lane >> 3)] = word;
-    const uint32_t cnt = warp_sum_u(__popc(nib));
+    // canonical order: after the transpose lane 8g+k holds word 4k+g; bring word l to lane l
+    uint32_t word = transpose_nibbles_8x8(nib, lane);
+    word = __shfl_sync(0xFFFFFFFFu, word, 8 * (lane & 3) + (lane >> 2));
+    if (active) bitmask[tile * 32 + lane] = word;
+
+    // phase 2: gather the kept entries, spread evenly over the lanes
+    const uint32_t cnt = warp_list_positions(word, lane, list);
+    double dsum = 0.0;
+    uint32_t vmax = 0;
+    for (uint32_t t = lane; t < cnt; t += 32) {
+        const float xs = __fmul_rn(scale, x[base + list[t]]);
+        const uint32_t a = __float_as_uint(xs) & 0x7FFFFFFFu;
+        if (P == NC_P_INF) vmax = max(vmax, a);
+        else if (P == 1) dsum += (double)__uint_as_float(a);
+        else dsum = fma((double)xs, (double)xs, dsum);
+    }
     uint64_t part;
     if (P == NC_P_INF) part = (uint64_t)warp_max_u(vmax);
     else part = (uint64_t)__double_as_longlong(warp_sum_d(dsum));
@@ -237,37 +286,30 @@ sparse_emit_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d, 
     uint32_t* __restrict__ idx = batch.idx[blockIdx.y];
     uint8_t* __restrict__ tmp_codes = ws.tmp_codes;
     __shared__ uint32_t s_tile[kWarpsPerBlock];
-    uint32_t word = active ? bitmask[tile * 32 + lane] : 0u;
-    const uint32_t cnt = __popc(word);
-    uint32_t incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) s_tile[threadIdx.x >> 5] = incl;      // kept entries of this tile
+    __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
+    uint16_t* list = s_list[threadIdx.x >> 5];
+    const uint32_t word = active ? bitmask[tile * 32 + lane] : 0u;
+    const uint32_t cnt = warp_list_positions(word, lane, list);
+    if (lane == 0) s_tile[threadIdx.x >> 5] = cnt;        // kept entries of this tile
     __syncthreads();
-    uint64_t k = (uint64_t)ws.block_count[blockIdx.x] + (incl - cnt);
-    for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) k += s_tile[w];
-    if (word == 0) return;
+    uint64_t k0 = (uint64_t)ws.block_count[blockIdx.x];
+    for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) k0 += s_tile[w];
+    if (cnt == 0) return;
     const Scale sc = make_scale(*norm, s);
     const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
-    while (word) {
-        const int bit = __ffs(word) - 1;
-        word &= word - 1;
-        const uint64_t j = base + (uint64_t)(lane * 32 + bit);
-        if (k < cap) {
-            const float xs = __fmul_rn(scale, x[j]);
-            const uint32_t bits = __float_as_uint(xs);
-            uint32_t r4[4];
-            stream_words4(j >> 2, worker, kDomainDnat, keys, r4);
-            const uint32_t r = (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1]
-                             : (j & 3) == 2 ? r4[2] : r4[3];
-            const uint32_t code = sparse_level_code(bits, r, sc, pow2s);
-            idx[k] = (uint32_t)j;
-            tmp_codes[k] = (uint8_t)(((bits >> 31) << 3) | code);
-        }
-        ++k;
+    for (uint32_t t = lane; t < cnt; t += 32) {      // the t-th kept entry of the tile
+        const uint64_t k = k0 + t;
+        if (k >= cap) break;
+        const uint64_t j = base + list[t];
+        const float xs = __fmul_rn(scale, x[j]);
+        const uint32_t bits = __float_as_uint(xs);
+        uint32_t r4[4];
+        stream_words4(j >> 2, worker, kDomainDnat, keys, r4);
+        const uint32_t r = (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1]
+                         : (j & 3) == 2 ? r4[2] : r4[3];
+        const uint32_t code = sparse_level_code(bits, r, sc, pow2s);
+        idx[k] = (uint32_t)j;
+        tmp_codes[k] = (uint8_t)(((bits >> 31) << 3) | code);
     }
 }
 
@@ -356,20 +398,20 @@ nc_status nd_sparse_compress_batch(const float* const* xs, size_t d, uint64_t ke
     const uint64_t tiles = sparse_tiles(d);
     const dim3 grid((unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
     const PhiloxKeys keys = make_philox_keys(seed);
-    const bool keep_all = keep_threshold >= ((uint64_t)1 << 32);
-    const uint32_t thr32 = keep_all ? 0xFFFFFFFFu : (uint32_t)keep_threshold;
+    const bool keep_none = keep_threshold == 0;
+    const uint32_t neg_thr = (uint32_t)(0ull - keep_threshold);   // 2^32 - threshold (mod 2^32)
     const dim3 sgrid(1, (unsigned)n);
     if (p == 1) {
-        sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(batch, d, thr32, keep_all,
+        sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
                                                                     scale, keys, ws, ws_stride);
         sparse_scan_kernel<1><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
     } else if (p == 2) {
-        sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(batch, d, thr32, keep_all,
+        sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
                                                                     scale, keys, ws, ws_stride);
         sparse_scan_kernel<2><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
     } else {
         sparse_select_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
-            batch, d, thr32, keep_all, scale, keys, ws, ws_stride);
+            batch, d, neg_thr, keep_none, scale, keys, ws, ws_stride);
         sparse_scan_kernel<NC_P_INF><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
     }
     sparse_emit_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap, ws,
