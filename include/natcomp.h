@@ -63,7 +63,8 @@ typedef enum {
     NC_ERR_ALIGN = -2,       /* a pointer is not aligned as required */
     NC_ERR_UNSUPPORTED = -3, /* p other than 1, 2, NC_P_INF */
     NC_ERR_WORKSPACE = -4,   /* workspace_bytes smaller than the query helper's answer */
-    NC_ERR_CUDA = -5         /* the CUDA runtime reported an error at launch */
+    NC_ERR_CUDA = -5,        /* the CUDA runtime reported an error at launch */
+    NC_ERR_TOO_LARGE = -6    /* the problem does not fit the fixed scratch of a *_static call */
 } nc_status;
 
 #define NC_MAX_WORKERS 64
@@ -132,6 +133,30 @@ nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bu
                             int p, int s, uint64_t seed, const uint32_t* workers,
                             float* const* norms, uint8_t* const* levels, uint32_t* const* signs,
                             int n, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/* nd_compress for callers that have no device memory to hand over as workspace and may not
+ * allocate any.  (The paper has no counterpart; this is a deployment convenience.)  Typical
+ * cases: a gradient hook running while a framework's caching allocator owns all device memory
+ * and communication kernels are in flight, where a cudaMalloc would synchronise the device or
+ * simply fail; or a process whose memory budget was fixed at start-up.  Such callers still pass
+ * the input and every output buffer, but the scratch the kernels need lives in a fixed array
+ * inside the library image: nd_static_scratch_bytes() bytes (1 MiB), present on every GPU that
+ * loads the library for as long as the process runs.
+ *   - Accepted sizes: nd_workspace_bytes(d, B) <= nd_static_scratch_bytes(), i.e. roughly
+ *     d <= 89 million entries for a few hundred buckets; anything larger returns
+ *     NC_ERR_TOO_LARGE and launches nothing.
+ *   - Results are identical to nd_compress with the same arguments.
+ *   - The call allocates and frees nothing.  The first call on each device looks up the device
+ *     address of the array (a CUDA runtime query, made with that device current); make that
+ *     first call before starting any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the previous call left in
+ *     it.  Nothing in it needs to start at zero (every slot is written before it is read), but
+ *     two calls that overlap on the GPU (different streams, or several host threads) race on
+ *     it: serialise them, or use nd_compress with separate workspaces. */
+size_t nd_static_scratch_bytes(void);
+nc_status nd_compress_static(const float* x, size_t d, const uint64_t* bucket_off, int B, int p,
+                             int s, uint64_t seed, uint32_t worker, float* norms, uint8_t* level,
+                             uint32_t* sign, cudaStream_t stream);
 
 /* Master side, one worker: acc[j] <- acc[j] + sign_j * fl32(norm_b * 2^(c_j - s)); c = 0 adds +-0. */
 nc_status nd_decode_accumulate(const float* norms, const uint8_t* level, const uint32_t* sign,

@@ -33,7 +33,7 @@ EXPORTS = (
     "nc_aggregate", "nc_sum_fp32", "nd_compress", "nd_decode_accumulate", "nd_aggregate",
     "nd_sparse_compress", "nd_sparse_decode_accumulate", "nc_copy_to_device", "nc_copy_to_host",
     "nd_batch_workspace_bytes", "nd_compress_batch", "nd_sparse_batch_workspace_bytes",
-    "nd_sparse_compress_batch",
+    "nd_sparse_compress_batch", "nd_static_scratch_bytes", "nd_compress_static",
 )
 
 
@@ -116,6 +116,26 @@ def nd_sparse_compress_batch(xs, d, keep_threshold, scale, p, s, seed, workers, 
            _nd_sparse_compress_batch(_ptrs(xs), d, keep_threshold, scale, p, s, seed, w,
                                      _ptrs(idxs), _ptrs(codes), _ptrs(counts), _ptrs(norms), cap,
                                      n, _ptr(workspace), workspace_bytes, _stream(stream)))
+
+
+_nd_static_scratch_bytes = _sig("nd_static_scratch_bytes", _sz)
+_nd_compress_static = _sig("nd_compress_static", C.c_int, _vp, _sz, _vp, C.c_int, C.c_int,
+                           C.c_int, C.c_uint64, C.c_uint32, _vp, _vp, _vp, _vp)
+
+
+def nd_static_scratch_bytes() -> int:
+    return int(_nd_static_scratch_bytes())
+
+
+def nd_compress_static(x, d, bucket_off, B, p, s, seed, worker, norms, level, sign,
+                       stream=None) -> None:
+    """nd_compress with the library's built-in scratch array instead of a workspace argument:
+    for callers that may not allocate device memory.  Raises NatcompError(NC_ERR_TOO_LARGE) when
+    nd_workspace_bytes(d, B) exceeds nd_static_scratch_bytes().  Calls on one device share the
+    scratch, so they must not overlap on the GPU."""
+    _check("nd_compress_static", _nd_compress_static(_ptr(x), d, _ptr(bucket_off), B, p, s, seed,
+                                                     worker, _ptr(norms), _ptr(level), _ptr(sign),
+                                                     _stream(stream)))
 
 
 _nc_copy_to_device = _sig("nc_copy_to_device", C.c_int, _vp, _vp, _sz, _vp)

@@ -13,6 +13,7 @@ const char* nc_status_string(int status) {
         case NC_ERR_UNSUPPORTED: return "NC_ERR_UNSUPPORTED";
         case NC_ERR_WORKSPACE: return "NC_ERR_WORKSPACE";
         case NC_ERR_CUDA: return "NC_ERR_CUDA";
+        case NC_ERR_TOO_LARGE: return "NC_ERR_TOO_LARGE";
         default: return "NC_ERR_UNKNOWN";
     }
 }

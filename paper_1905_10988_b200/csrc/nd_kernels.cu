@@ -611,3 +611,48 @@ nc_status nd_decode_accumulate(const float* norms, const uint8_t* level, const u
 }
 
 }  // extern "C"
+
+// ---- nd_compress without a caller-provided workspace ------------------------------------
+//
+// Scratch for callers that cannot allocate device memory: a fixed array that lives in the
+// library image on every GPU that loads it.  In host code `g_nd_static_scratch` is only a
+// handle for the runtime; its device address is looked up once per device with
+// cudaGetSymbolAddress and passed to the kernels like any other workspace pointer.
+namespace natcomp {
+
+constexpr size_t kStaticScratchBytes = (size_t)1 << 20;   // 1 MiB
+
+static __device__ __align__(256) unsigned char g_nd_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_static_scratch_addr[kMaxDevices];   // per device ordinal; 0 = not looked up yet
+
+// Device address of the scratch array on the current device (nullptr on failure).
+static void* static_scratch_address() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    void* p = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
+    if (p) return p;
+    if (cudaGetSymbolAddress(&p, g_nd_static_scratch) != cudaSuccess || !p) return nullptr;
+    __atomic_store_n(&g_static_scratch_addr[dev], p, __ATOMIC_RELEASE);
+    return p;
+}
+
+}  // namespace natcomp
+
+extern "C" {
+
+size_t nd_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+nc_status nd_compress_static(const float* x, size_t d, const uint64_t* bucket_off, int B, int p,
+                             int s, uint64_t seed, uint32_t worker, float* norms, uint8_t* level,
+                             uint32_t* sign, cudaStream_t stream) {
+    if (B < 0) return NC_ERR_INVALID;
+    if (nd_workspace_bytes(d, B) > kStaticScratchBytes) return NC_ERR_TOO_LARGE;
+    void* scratch = static_scratch_address();
+    if (!scratch) return NC_ERR_CUDA;
+    return nd_compress(x, d, bucket_off, B, p, s, seed, worker, norms, level, sign, scratch,
+                       kStaticScratchBytes, stream);
+}
+
+}  // extern "C"
