@@ -105,6 +105,15 @@ nc_status nc_decode_accumulate(const uint8_t* exp, const uint32_t* sign, size_t 
 nc_status nc_aggregate(const uint8_t* const* exps, const uint32_t* const* signs, int n, size_t d,
                        float* out, cudaStream_t stream);
 
+/* Master side with compression of the aggregate (Algorithm 1, "compress g = C_M(Delta)", with
+ * C_M = C_nat; the bidirectional-compression models of the speed-up appendix): the 9-bit code of
+ * C_nat(sum_i v_ij), the sum taken as in nc_aggregate and never written to memory.  The rounding
+ * uses the C_nat stream of (seed, worker = master, j).  out_exp: nc_exp_bytes(d), out_sign:
+ * nc_sign_bytes(d).  Identical to nc_aggregate followed by nc_compress(.., seed, master, ..). */
+nc_status nc_aggregate_compress(const uint8_t* const* exps, const uint32_t* const* signs, int n,
+                                size_t d, uint64_t seed, uint32_t master, uint8_t* out_exp,
+                                uint32_t* out_sign, cudaStream_t stream);
+
 /* Reference point (the "no compression" baseline of Table 1): out[j] <- ((+0 + x_0j) + x_1j) + ...
  * xs: host array of n device pointers to fp32[d]. */
 nc_status nc_sum_fp32(const float* const* xs, int n, size_t d, float* out, cudaStream_t stream);

@@ -34,6 +34,7 @@ EXPORTS = (
     "nd_sparse_compress", "nd_sparse_decode_accumulate", "nc_copy_to_device", "nc_copy_to_host",
     "nd_batch_workspace_bytes", "nd_compress_batch", "nd_sparse_batch_workspace_bytes",
     "nd_sparse_compress_batch", "nd_static_scratch_bytes", "nd_compress_static",
+    "nc_aggregate_compress",
 )
 
 
@@ -116,6 +117,16 @@ def nd_sparse_compress_batch(xs, d, keep_threshold, scale, p, s, seed, workers, 
            _nd_sparse_compress_batch(_ptrs(xs), d, keep_threshold, scale, p, s, seed, w,
                                      _ptrs(idxs), _ptrs(codes), _ptrs(counts), _ptrs(norms), cap,
                                      n, _ptr(workspace), workspace_bytes, _stream(stream)))
+
+
+_nc_aggregate_compress = _sig("nc_aggregate_compress", C.c_int, C.POINTER(_vp), C.POINTER(_vp),
+                              C.c_int, _sz, C.c_uint64, C.c_uint32, _vp, _vp, _vp)
+
+
+def nc_aggregate_compress(exps, signs, n, d, seed, master, out_exp, out_sign, stream=None) -> None:
+    _check("nc_aggregate_compress",
+           _nc_aggregate_compress(_ptrs(exps), _ptrs(signs), n, d, seed, master, _ptr(out_exp),
+                                  _ptr(out_sign), _stream(stream)))
 
 
 _nd_static_scratch_bytes = _sig("nd_static_scratch_bytes", _sz)

@@ -39,84 +39,75 @@ __device__ __forceinline__ uint32_t cnat_exp_byte(uint32_t bits, uint32_t rnd) {
     return v >> 23;
 }
 
-// grid: (ceil(tiles / warps per block), n workers)
-__global__ void __launch_bounds__(kBlockThreads)
-nc_compress_kernel(const __grid_constant__ CompressBatch batch, const uint64_t d,
-                   const __grid_constant__ PhiloxKeys keys) {
-    const int lane = threadIdx.x & 31;
-    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    const uint64_t base = tile * kTile;
-    if (base >= d) return;
-    const int w = blockIdx.y;
-    const float* __restrict__ x = batch.x[w];
-    uint8_t* __restrict__ exp = batch.exp[w];
-    uint32_t* __restrict__ sign = batch.sign[w];
-    const uint32_t worker = batch.worker[w];
+// C_nat of one full tile held in registers (lane l: float4 groups k*32 + l, k = 0..7):
+// writes the tile's 1024 exponent bytes and 32 sign words.
+__device__ __forceinline__ void cnat_full_tile(const uint4 (&u)[8], const uint64_t base,
+                                               const uint32_t worker, const PhiloxKeys& keys,
+                                               uint8_t* __restrict__ exp,
+                                               uint32_t* __restrict__ sign, const int lane) {
+    uint32_t* ev = reinterpret_cast<uint32_t*>(exp + base);
+    const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainCnat, keys);
+    const uint32_t q_lo = (uint32_t)(base >> 2) + lane;   // + k*32 stays below 2^32: no carry
 
-    if (base + kTile <= d) {
-        // ---- full tile ------------------------------------------------------------
-        const uint4* xv = reinterpret_cast<const uint4*>(x + base);
-        uint4 u[8];
+    // Biased exponents 254 / 255 must not be rounded up.  If every element of the tile has
+    // (bits & 0x7F000000) != 0x7F000000 the guard can be dropped; the OR over the lane's
+    // elements is a cheap conservative test (false positives only cost the guarded path).
+    uint32_t any = 0;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) u[k] = ld_stream_u4(xv + k * 32 + lane);
+    for (int k = 0; k < 8; ++k) any |= u[k].x | u[k].y | u[k].z | u[k].w;
+    const bool guarded = __any_sync(0xFFFFFFFFu, (any & 0x7F000000u) == 0x7F000000u);
 
-        uint32_t* ev = reinterpret_cast<uint32_t*>(exp + base);
-        const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainCnat, keys);
-        const uint32_t q_lo = (uint32_t)(base >> 2) + lane;   // + k*32 stays below 2^32: no carry
-
-        // Biased exponents 254 / 255 must not be rounded up.  If every element of the tile has
-        // (bits & 0x7F000000) != 0x7F000000 the guard can be dropped; the OR over the lane's
-        // elements is a cheap conservative test (false positives only cost the guarded path).
-        uint32_t any = 0;
+    uint32_t nib = 0;   // sign bits of this lane's 32 elements: bit 4k+c <-> group k, element c
+    if (!guarded) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) any |= u[k].x | u[k].y | u[k].z | u[k].w;
-        const bool guarded = __any_sync(0xFFFFFFFFu, (any & 0x7F000000u) == 0x7F000000u);
-
-        uint32_t nib = 0;   // sign bits of this lane's 32 elements: bit 4k+c <-> group k, element c
-        if (!guarded) {
-#pragma unroll
-            for (int k = 7; k >= 0; --k) {
-                uint32_t rnd[4];
-                stream_words4_tile(q_lo + k * 32, pt, keys, rnd);
-                const uint32_t b0 = u[k].x, b1 = u[k].y, b2 = u[k].z, b3 = u[k].w;
-                // (bits + (~r23 & 0x7FFFFF)) << 1: sign shifted out, rounded exponent in byte 3
-                const uint32_t t0 = (b0 + (~rnd[0] & 0x7FFFFFu)) << 1;
-                const uint32_t t1 = (b1 + (~rnd[1] & 0x7FFFFFu)) << 1;
-                const uint32_t t2 = (b2 + (~rnd[2] & 0x7FFFFFu)) << 1;
-                const uint32_t t3 = (b3 + (~rnd[3] & 0x7FFFFFu)) << 1;
-                const uint32_t e = __byte_perm(__byte_perm(t0, t1, 0x0073),
-                                               __byte_perm(t2, t3, 0x0073), 0x5410);
-                st_stream_u32(ev + k * 32 + lane, e);
-                nib = __funnelshift_l(b3, nib, 1);
-                nib = __funnelshift_l(b2, nib, 1);
-                nib = __funnelshift_l(b1, nib, 1);
-                nib = __funnelshift_l(b0, nib, 1);
-            }
-        } else {
-#pragma unroll
-            for (int k = 7; k >= 0; --k) {
-                uint32_t rnd[4];
-                stream_words4_tile(q_lo + k * 32, pt, keys, rnd);
-                const uint32_t b0 = u[k].x, b1 = u[k].y, b2 = u[k].z, b3 = u[k].w;
-                uint32_t e = cnat_exp_byte(b3, rnd[3]);
-                e = (e << 8) | cnat_exp_byte(b2, rnd[2]);
-                e = (e << 8) | cnat_exp_byte(b1, rnd[1]);
-                e = (e << 8) | cnat_exp_byte(b0, rnd[0]);
-                st_stream_u32(ev + k * 32 + lane, e);
-                nib = __funnelshift_l(b3, nib, 1);
-                nib = __funnelshift_l(b2, nib, 1);
-                nib = __funnelshift_l(b1, nib, 1);
-                nib = __funnelshift_l(b0, nib, 1);
-            }
+        for (int k = 7; k >= 0; --k) {
+            uint32_t rnd[4];
+            stream_words4_tile(q_lo + k * 32, pt, keys, rnd);
+            const uint32_t b0 = u[k].x, b1 = u[k].y, b2 = u[k].z, b3 = u[k].w;
+            // (bits + (~r23 & 0x7FFFFF)) << 1: sign shifted out, rounded exponent in byte 3
+            const uint32_t t0 = (b0 + (~rnd[0] & 0x7FFFFFu)) << 1;
+            const uint32_t t1 = (b1 + (~rnd[1] & 0x7FFFFFu)) << 1;
+            const uint32_t t2 = (b2 + (~rnd[2] & 0x7FFFFFu)) << 1;
+            const uint32_t t3 = (b3 + (~rnd[3] & 0x7FFFFFu)) << 1;
+            const uint32_t e = __byte_perm(__byte_perm(t0, t1, 0x0073),
+                                           __byte_perm(t2, t3, 0x0073), 0x5410);
+            st_stream_u32(ev + k * 32 + lane, e);
+            nib = __funnelshift_l(b3, nib, 1);
+            nib = __funnelshift_l(b2, nib, 1);
+            nib = __funnelshift_l(b1, nib, 1);
+            nib = __funnelshift_l(b0, nib, 1);
         }
-        // lane 8g+i holds nibble k of sign word (k, g); after the transpose lane 8g+k holds the
-        // whole word covering elements k*128 + g*32 .. +31 of the tile.
-        const uint32_t word = transpose_nibbles_8x8(nib, lane);
-        st_stream_u32(sign + (base >> 5) + (lane & 7) * 4 + (lane >> 3), word);
-        return;
+    } else {
+#pragma unroll
+        for (int k = 7; k >= 0; --k) {
+            uint32_t rnd[4];
+            stream_words4_tile(q_lo + k * 32, pt, keys, rnd);
+            const uint32_t b0 = u[k].x, b1 = u[k].y, b2 = u[k].z, b3 = u[k].w;
+            uint32_t e = cnat_exp_byte(b3, rnd[3]);
+            e = (e << 8) | cnat_exp_byte(b2, rnd[2]);
+            e = (e << 8) | cnat_exp_byte(b1, rnd[1]);
+            e = (e << 8) | cnat_exp_byte(b0, rnd[0]);
+            st_stream_u32(ev + k * 32 + lane, e);
+            nib = __funnelshift_l(b3, nib, 1);
+            nib = __funnelshift_l(b2, nib, 1);
+            nib = __funnelshift_l(b1, nib, 1);
+            nib = __funnelshift_l(b0, nib, 1);
+        }
     }
+    // lane 8g+i holds nibble k of sign word (k, g); after the transpose lane 8g+k holds the
+    // whole word covering elements k*128 + g*32 .. +31 of the tile.
+    const uint32_t word = transpose_nibbles_8x8(nib, lane);
+    st_stream_u32(sign + (base >> 5) + (lane & 7) * 4 + (lane >> 3), word);
+}
 
-    // ---- ragged last tile: one element per lane per step, ballot gives the sign word ----
+// C_nat of the ragged last tile, one element per lane per step (a ballot gives the sign word);
+// also writes the zero padding of both planes.  load_bits(j) returns the binary32 pattern of
+// element j.
+template <typename LoadBits>
+__device__ __forceinline__ void cnat_ragged_tile(LoadBits load_bits, const uint64_t base,
+                                                 const uint64_t d, const uint32_t worker,
+                                                 const PhiloxKeys& keys, uint8_t* __restrict__ exp,
+                                                 uint32_t* __restrict__ sign, const int lane) {
     const uint64_t exp_end = round_up16(d);                 // bytes incl. zero padding
     const uint64_t sign_words = (d + 31) / 32;
     const uint64_t sign_words_padded = (sign_words + 3) & ~(uint64_t)3;
@@ -124,7 +115,7 @@ nc_compress_kernel(const __grid_constant__ CompressBatch batch, const uint64_t d
         const uint64_t j = j0 + lane;
         uint32_t bits = 0, e = 0;
         if (j < d) {
-            bits = __float_as_uint(x[j]);
+            bits = load_bits(j);
             uint32_t rnd[4];
             stream_words4(j >> 2, worker, kDomainCnat, keys, rnd);
             const uint32_t r = (j & 3) == 0 ? rnd[0] : (j & 3) == 1 ? rnd[1]
@@ -138,11 +129,67 @@ nc_compress_kernel(const __grid_constant__ CompressBatch batch, const uint64_t d
     if (lane < (int)(sign_words_padded - sign_words)) sign[sign_words + lane] = 0;
 }
 
+// grid: (ceil(tiles / warps per block), n workers)
+__global__ void __launch_bounds__(kBlockThreads)
+nc_compress_kernel(const __grid_constant__ CompressBatch batch, const uint64_t d,
+                   const __grid_constant__ PhiloxKeys keys) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+    const int w = blockIdx.y;
+    const float* __restrict__ x = batch.x[w];
+    if (base + kTile <= d) {
+        const uint4* xv = reinterpret_cast<const uint4*>(x + base);
+        uint4 u[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) u[k] = ld_stream_u4(xv + k * 32 + lane);
+        cnat_full_tile(u, base, batch.worker[w], keys, batch.exp[w], batch.sign[w], lane);
+        return;
+    }
+    cnat_ragged_tile([&](uint64_t j) { return __float_as_uint(x[j]); }, base, d, batch.worker[w],
+                     keys, batch.exp[w], batch.sign[w], lane);
+}
+
 // value of a 9-bit code: exponent byte in byte `BYTE` of `e4`, sign in bit 0 of `s`
 template <int BYTE>
 __device__ __forceinline__ float decode9(uint32_t e4, uint32_t s) {
     const uint32_t hi = __byte_perm(e4, 0u, 0x0444 | (BYTE << 12));   // exponent -> bits 24..31
     return __uint_as_float(__funnelshift_r(hi, s, 1));                // (hi >> 1) | (s << 31)
+}
+
+// acc[k] += decoded values of workers 0..n-1, in that order, for one full tile
+__device__ __forceinline__ void aggregate_full_tile(const PackedPlanes& planes, const int n,
+                                                    const uint64_t base, float4 (&acc)[8],
+                                                    const int lane) {
+    const int sh = 4 * (lane & 7);
+    for (int i = 0; i < n; ++i) {
+        const uint32_t* ev = reinterpret_cast<const uint32_t*>(planes.exp[i] + base);
+        const uint32_t sw = ld_stream_u32(planes.sign[i] + (base >> 5) + lane);
+        uint32_t e[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) e[k] = ld_stream_u32(ev + k * 32 + lane);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            // sign word (k, g) lives in lane 4k+g; this lane needs group g = lane / 8
+            const uint32_t s = __shfl_sync(0xFFFFFFFFu, sw, k * 4 + (lane >> 3)) >> sh;
+            acc[k].x += decode9<0>(e[k], s);
+            acc[k].y += decode9<1>(e[k], s >> 1);
+            acc[k].z += decode9<2>(e[k], s >> 2);
+            acc[k].w += decode9<3>(e[k], s >> 3);
+        }
+    }
+}
+
+// the same sum for one element (ragged tile)
+__device__ __forceinline__ float aggregate_element(const PackedPlanes& planes, const int n,
+                                                   const uint64_t j, float a) {
+    for (int i = 0; i < n; ++i) {
+        const uint32_t e = planes.exp[i][j];
+        const uint32_t s = (planes.sign[i][j >> 5] >> (j & 31)) & 1u;
+        a += __uint_as_float((e << 23) | (s << 31));
+    }
+    return a;
 }
 
 // out[j] = (init + v_0j) + v_1j + ... ; init = +0 (aggregate) or acc[j] (decode-accumulate).
@@ -164,38 +211,43 @@ nc_aggregate_kernel(const __grid_constant__ PackedPlanes planes, const int n, co
             if (kFromAcc) acc[k] = __ldcs(ov + k * 32 + lane);
             else acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        const int sh = 4 * (lane & 7);
-        for (int i = 0; i < n; ++i) {
-            const uint32_t* ev = reinterpret_cast<const uint32_t*>(planes.exp[i] + base);
-            const uint32_t sw = ld_stream_u32(planes.sign[i] + (base >> 5) + lane);
-            uint32_t e[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) e[k] = ld_stream_u32(ev + k * 32 + lane);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                // sign word (k, g) lives in lane 4k+g; this lane needs group g = lane / 8
-                const uint32_t s = __shfl_sync(0xFFFFFFFFu, sw, k * 4 + (lane >> 3)) >> sh;
-                acc[k].x += decode9<0>(e[k], s);
-                acc[k].y += decode9<1>(e[k], s >> 1);
-                acc[k].z += decode9<2>(e[k], s >> 2);
-                acc[k].w += decode9<3>(e[k], s >> 3);
-            }
-        }
+        aggregate_full_tile(planes, n, base, acc, lane);
 #pragma unroll
         for (int k = 0; k < 8; ++k) __stcs(ov + k * 32 + lane, acc[k]);
         return;
     }
+    for (uint64_t j = base + lane; j < d; j += 32)      // ragged last tile: scalar
+        out[j] = aggregate_element(planes, n, j, kFromAcc ? out[j] : 0.f);
+}
 
-    // ragged last tile: scalar
-    for (uint64_t j = base + lane; j < d; j += 32) {
-        float a = kFromAcc ? out[j] : 0.f;
-        for (int i = 0; i < n; ++i) {
-            const uint32_t e = planes.exp[i][j];
-            const uint32_t s = (planes.sign[i][j >> 5] >> (j & 31)) & 1u;
-            a += __uint_as_float((e << 23) | (s << 31));
-        }
-        out[j] = a;
+// Master side with compression of the aggregate (Algorithm 1: g = C_M(sum_i Delta_i) with
+// C_M = C_nat): the fp32 sum never leaves the registers, only its 9-bit code is written.
+// grid: ceil(tiles / warps per block)
+__global__ void __launch_bounds__(kBlockThreads)
+nc_aggregate_compress_kernel(const __grid_constant__ PackedPlanes planes, const int n,
+                             const uint64_t d, const uint32_t master,
+                             const __grid_constant__ PhiloxKeys keys, uint8_t* __restrict__ exp,
+                             uint32_t* __restrict__ sign) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+    if (base + kTile <= d) {
+        float4 acc[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        aggregate_full_tile(planes, n, base, acc, lane);
+        uint4 u[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            u[k] = make_uint4(__float_as_uint(acc[k].x), __float_as_uint(acc[k].y),
+                              __float_as_uint(acc[k].z), __float_as_uint(acc[k].w));
+        cnat_full_tile(u, base, master, keys, exp, sign, lane);
+        return;
     }
+    cnat_ragged_tile(
+        [&](uint64_t j) { return __float_as_uint(aggregate_element(planes, n, j, 0.f)); }, base,
+        d, master, keys, exp, sign, lane);
 }
 
 // uncompressed reference point: n-way fp32 sum in worker order
@@ -284,6 +336,27 @@ nc_status nc_aggregate(const uint8_t* const* exps, const uint32_t* const* signs,
     }
     nc_aggregate_kernel<false><<<tile_blocks(d), kBlockThreads, 0, stream>>>(planes, n,
                                                                              (uint64_t)d, out);
+    return launch_status();
+}
+
+nc_status nc_aggregate_compress(const uint8_t* const* exps, const uint32_t* const* signs, int n,
+                                size_t d, uint64_t seed, uint32_t master, uint8_t* out_exp,
+                                uint32_t* out_sign, cudaStream_t stream) {
+    if (!exps || !signs || !out_exp || !out_sign || n < 1 || n > NC_MAX_WORKERS)
+        return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    if (!aligned16(out_exp) || !aligned16(out_sign)) return NC_ERR_ALIGN;
+    PackedPlanes planes;
+    for (int i = 0; i < n; ++i) {
+        if (!exps[i] || !signs[i]) return NC_ERR_INVALID;
+        if (!aligned16(exps[i]) || !aligned16(signs[i])) return NC_ERR_ALIGN;
+        planes.exp[i] = exps[i];
+        planes.sign[i] = signs[i];
+    }
+    const PhiloxKeys keys = make_philox_keys(seed);
+    nc_aggregate_compress_kernel<<<tile_blocks(d), kBlockThreads, 0, stream>>>(
+        planes, n, (uint64_t)d, master, keys, out_exp, out_sign);
     return launch_status();
 }
 
