@@ -1,0 +1,154 @@
+"""Per-call timings on the five benchmark workloads (one GPU).
+
+    python -m paper_1905_10988_b200.config_bench --config c4 [--iters 20]
+
+For every C-ABI call the workload uses it prints one JSON line with the device time (CUDA
+events, median and best over the iterations, after warm-up), the rate in Gelem/s and the
+algorithmic HBM bytes per second.  bench.py at the repository root is the whole-path step
+benchmark on c2; this tool covers the other shapes: c1 (small, launch-bound), c3 (D_nat on the
+c2 buffers), c4 (n = 16, d = 335 M, beside the uncompressed 16-way sum) and c5 (sparse, d = 2^28).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+
+import torch
+
+from . import binding as nc
+from . import workloads
+
+HBM_PEAK_FALLBACK = 6650.0
+
+
+def _time(fn, iters, warmup=3):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(iters):
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    return statistics.median(times), min(times)
+
+
+def _report(config, call, ms_med, ms_best, elems, nbytes, peak, extra=None):
+    line = {"config": config, "call": call, "ms_median": round(ms_med, 4),
+            "ms_best": round(ms_best, 4), "Gelem_per_s": round(elems / ms_med / 1e6, 1),
+            "algorithmic_GBps": round(nbytes / ms_med / 1e6, 1),
+            "frac_of_hbm_peak": round(nbytes / ms_med / 1e6 / peak, 4)}
+    if extra:
+        line.update(extra)
+    print(json.dumps(line), flush=True)
+
+
+def run_cnat(config, n, d, make_vector, iters, peak, with_sum=True):
+    dev = "cuda"
+    u8 = dict(dtype=torch.uint8, device=dev)
+    xs = [make_vector(w) for w in range(n)]
+    es = [torch.empty(nc.nc_exp_bytes(d), **u8) for _ in range(n)]
+    ss = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
+    out = torch.empty(d, dtype=torch.float32, device=dev)
+    ge = torch.empty(nc.nc_exp_bytes(d), **u8)
+    gs = torch.empty(nc.nc_sign_bytes(d), **u8)
+    workers = list(range(n))
+    m, b = _time(lambda: nc.nc_compress_batch(xs, d, 0, workers, es, ss, n), iters)
+    _report(config, "nc_compress_batch", m, b, n * d, n * d * 5.125, peak, {"n": n, "d": d})
+    m, b = _time(lambda: nc.nc_aggregate(es, ss, n, d, out), iters)
+    _report(config, "nc_aggregate", m, b, d, d * (1.125 * n + 4), peak)
+    m, b = _time(lambda: nc.nc_aggregate_compress(es, ss, n, d, 0, 0xFFFFFFFF, ge, gs), iters)
+    _report(config, "nc_aggregate_compress", m, b, d, d * (1.125 * n + 1.125), peak)
+    if with_sum:
+        m, b = _time(lambda: nc.nc_sum_fp32(xs, n, d, out), iters)
+        _report(config, "nc_sum_fp32 (uncompressed reference point)", m, b, d, d * (4 * n + 4),
+                peak)
+
+
+def run_dnat(config, n, sizes, iters, peak, p=2, s=8):
+    dev = "cuda"
+    u8 = dict(dtype=torch.uint8, device=dev)
+    off = workloads.offsets_from_sizes(sizes)
+    d, B = off[-1], len(sizes)
+    off_dev = torch.tensor(off, dtype=torch.int64, device=dev)
+    xs = [workloads.config2_vector(w, dev, sizes) for w in range(n)]
+    norms = [torch.empty(B, dtype=torch.float32, device=dev) for _ in range(n)]
+    levels = [torch.empty(nc.nd_level_bytes(d), **u8) for _ in range(n)]
+    signs = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
+    ws_bytes = nc.nd_batch_workspace_bytes(d, B, n)
+    ws = torch.empty(ws_bytes, **u8)
+    out = torch.empty(d, dtype=torch.float32, device=dev)
+    workers = list(range(n))
+    m, b = _time(lambda: nc.nd_compress_batch(xs, d, off_dev, B, p, s, 0, workers, norms, levels,
+                                              signs, n, ws, ws_bytes), iters)
+    _report(config, "nd_compress_batch", m, b, n * d, n * d * 8.625, peak,
+            {"n": n, "d": d, "B": B, "note": "bytes count x twice (norm pass + rounding pass)"})
+    m, b = _time(lambda: nc.nd_aggregate(norms, levels, signs, n, d, off_dev, B, s, out), iters)
+    _report(config, "nd_aggregate", m, b, d, d * (0.625 * n + 4), peak)
+
+
+def run_sparse(config, n, d, iters, peak, s=4):
+    dev = "cuda"
+    u8 = dict(dtype=torch.uint8, device=dev)
+    cap = int(d * 0.0125)
+    xs = [workloads.config5_vector(w, d, dev) for w in range(n)]
+    idx = [torch.empty(cap, dtype=torch.int32, device=dev) for _ in range(n)]
+    codes = [torch.empty((cap + 1) // 2 + 16, **u8) for _ in range(n)]
+    count = [torch.zeros(1, dtype=torch.int32, device=dev) for _ in range(n)]
+    norm = [torch.zeros(1, dtype=torch.float32, device=dev) for _ in range(n)]
+    ws_bytes = nc.nd_sparse_batch_workspace_bytes(d, cap, n)
+    ws = torch.empty(ws_bytes, **u8)
+    acc = torch.zeros(d, dtype=torch.float32, device=dev)
+    workers = list(range(n))
+    thr, scale = workloads.KEEP_1PCT_THRESHOLD, workloads.KEEP_1PCT_SCALE
+    m, b = _time(lambda: nc.nd_sparse_compress_batch(xs, d, thr, scale, nc.P_INF, s, 0, workers,
+                                                     idx, codes, count, norm, cap, n, ws,
+                                                     ws_bytes), iters)
+    kept = 0.01 * d
+    _report(config, "nd_sparse_compress_batch", m, b, n * d, n * kept * 68.5, peak,
+            {"n": n, "d": d, "Gcoord_per_s": round(n * d / m / 1e6, 1),
+             "note": "ALU-bound: one Philox block per 4 coordinates; the multiplier-pipe ceiling "
+                     "is about 2070 Gcoord/s at 1965 MHz"})
+
+    def accumulate():
+        for w in range(n):
+            nc.nd_sparse_decode_accumulate(idx[w], codes[w], count[w], norm[w], s, d, cap, acc)
+
+    m, b = _time(accumulate, iters)
+    _report(config, "nd_sparse_decode_accumulate x n", m, b, n * kept, n * kept * 68.5, peak)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", required=True, choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--peak-gbs", type=float, default=HBM_PEAK_FALLBACK,
+                    help="HBM bandwidth the fractions are quoted against")
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("needs a CUDA device")
+    peak = args.peak_gbs
+    if args.config == "c1":
+        d = 1 << 20
+        run_cnat("c1", 4, d, lambda w: workloads.config1_vector(w, d, "cuda"), args.iters, peak)
+    elif args.config == "c2":
+        sizes = workloads.resnet50_tensor_sizes()
+        d = sum(sizes)
+        run_cnat("c2", 8, d, lambda w: workloads.config2_vector(w, "cuda", sizes), args.iters,
+                 peak)
+    elif args.config == "c3":
+        run_dnat("c3", 8, workloads.resnet50_tensor_sizes(), args.iters, peak)
+    elif args.config == "c4":
+        d = sum(workloads.bert_large_bucket_sizes())
+        run_cnat("c4", 16, d, lambda w: workloads.config4_vector(w, d, "cuda"), args.iters, peak)
+    else:
+        run_sparse("c5", 8, 1 << 28, args.iters, peak)
+
+
+if __name__ == "__main__":
+    main()

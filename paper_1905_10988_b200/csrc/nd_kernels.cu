@@ -6,7 +6,7 @@
 // blocks, one 32-bit word of level nibbles, one byte of sign bits).
 //
 // Norms are deterministic: every (tile, bucket) overlap writes one partial into its own slot
-// (slot = tile index + bucket index, strictly increasing along the vector), and one warp per
+// (slot = tile index + bucket index, strictly increasing along the vector), and one block per
 // bucket adds the bucket's slots in a fixed order.  No atomics, no zero-filling.
 //
 // Level rounding (given the bucket norm): y = fl32(|x| * fl32(1/norm)), z = y * 2^s (exact).
@@ -85,9 +85,10 @@ __device__ __forceinline__ uint32_t warp_max(uint32_t v) {
     return v;
 }
 
-// One partial per (tile, bucket) overlap.  p = 1: sum |x|, p = 2: sum x^2 (binary32 products,
-// chains of at most 8 terms in binary32, everything above that in binary64), p = inf: the
-// largest |x| as a bit pattern (NaN patterns compare above inf, so a NaN survives).
+// One partial per (tile, bucket) overlap.  p = 1: sum |x| (chains of at most 8 terms in
+// binary32, everything above that in binary64), p = 2: sum x^2 with squares and sums in
+// binary64, p = inf: the largest |x| as a bit pattern (NaN patterns compare above inf, so a
+// NaN survives).
 template <int P>
 struct NormAcc {
     float f[4];
