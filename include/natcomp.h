@@ -93,6 +93,15 @@ nc_status nc_compress_batch(const float* const* xs, size_t d, uint64_t seed,
                             const uint32_t* workers, uint8_t* const* exps,
                             uint32_t* const* signs, int n, cudaStream_t stream);
 
+/* The paper's deterministic control variant (experimental set-up appendix: "deterministic
+ * rounding to the nearest power of 2", used to expose the cost of sampling): the same 9-bit code,
+ * but every entry goes to the nearer of its two neighbouring powers of two (the midpoint
+ * 1.5 * 2^k goes up), with no random numbers.  Biased.  Edge cases as for nc_compress. */
+nc_status nc_compress_nearest(const float* x, size_t d, uint8_t* exp, uint32_t* sign,
+                              cudaStream_t stream);
+nc_status nc_compress_nearest_batch(const float* const* xs, size_t d, uint8_t* const* exps,
+                                    uint32_t* const* signs, int n, cudaStream_t stream);
+
 /* Master side, one worker (Algorithm 1, aggregation step): acc[j] <- acc[j] + decode(code_j),
  * one binary32 addition per entry.  acc: fp32[d], read and written. */
 nc_status nc_decode_accumulate(const uint8_t* exp, const uint32_t* sign, size_t d, float* acc,

@@ -241,3 +241,39 @@ def sparse_decode_accumulate(idx, codes, count: int, nrm, s: int, acc) -> None:
     assert acc.dtype == np.float32 and acc.flags.c_contiguous
     _sparse_decode_accumulate(_p(idx, _u32p), _p(codes, _u8p), count, float(nrm), s,
                               _p(acc, _f32p))
+
+
+_dsta_level_index = _sig("orc_dsta_level_index", None, _f64p, _u32p, C.c_uint64, C.c_int, _i32p)
+_dsta_apply = _sig("orc_dsta_apply", None, _f32p, C.c_uint64, C.c_int, C.c_int, C.c_uint64,
+                   C.c_uint32, _f64p)
+
+
+def dsta_level_index(y, r23, u: int) -> np.ndarray:
+    """Standard-dithering level index (0..u) of y for explicit thresholds."""
+    y = _arr(y, np.float64)
+    r23 = _arr(r23, np.uint32)
+    assert y.shape == r23.shape
+    out = np.empty(y.shape, np.int32)
+    _dsta_level_index(_p(y, _f64p), _p(r23, _u32p), y.size, u, _p(out, _i32p))
+    return out
+
+
+def dsta_apply(x, p: int, u: int, seed: int, worker: int) -> np.ndarray:
+    """D_sta^{p,u}(x) decoded, one bucket (oracle-side comparison operator)."""
+    x = _arr(x, np.float32)
+    out = np.empty(x.size, np.float64)
+    _dsta_apply(_p(x, _f32p), x.size, p, u, seed, worker, _p(out, _f64p))
+    return out
+
+
+_nc_compress_nearest = _sig("orc_nc_compress_nearest", None, _f32p, C.c_uint64, _u8p, _u32p)
+
+
+def nc_compress_nearest(x):
+    """Codes of x rounded to the nearest power of two (the deterministic control variant)."""
+    x = _arr(x, np.float32)
+    d = x.size
+    e = np.zeros(d, np.uint8)
+    s = np.zeros((d + 31) // 32, np.uint32)
+    _nc_compress_nearest(_p(x, _f32p), d, _p(e, _u8p), _p(s, _u32p))
+    return e, s

@@ -102,6 +102,29 @@ double cnat_value(float t, uint32_t r23) {
     return std::copysign(up ? hi : lo, (double)t);
 }
 
+// The paper's "deterministic" control variant (experimental set-up appendix): t is rounded to
+// the nearest power of two, no randomness (biased).  Nearest in absolute distance, the midpoint
+// 1.5 * 2^floor going up; zeros, subnormals, overflow and non-finite inputs as for C_nat
+// (a subnormal goes to 0 or 2^-126, whichever is nearer).
+double nearest_pow2_value(float t) {
+    if (t == 0.0f) return (double)t;
+    if (std::isnan(t) || std::isinf(t))
+        return std::copysign(std::numeric_limits<double>::infinity(), (double)t);
+    const double a = std::fabs((double)t);
+    double lo, hi;
+    if (a < 0x1p-126) {
+        lo = 0.0;
+        hi = 0x1p-126;
+    } else {
+        const int fl = std::ilogb(a);
+        lo = std::ldexp(1.0, fl);
+        hi = std::ldexp(1.0, fl + 1);
+        if (fl >= 127) return std::copysign(lo, (double)t);
+    }
+    const bool up = (a - lo) >= (hi - a);
+    return std::copysign(up ? hi : lo, (double)t);
+}
+
 // 9-bit code of a value of the form +-0, +-2^k, +-inf: biased exponent + sign bit.
 void cnat_code(double value, uint8_t* exp_byte, uint32_t* sign_bit) {
     *sign_bit = std::signbit(value) ? 1u : 0u;
@@ -242,6 +265,22 @@ void orc_nc_compress(const float* x, uint64_t d, uint64_t j0, uint64_t seed, uin
     }
 }
 
+// Deterministic variant of orc_nc_compress: codes of the nearest power of two.
+void orc_nc_compress_nearest(const float* x, uint64_t d, uint8_t* exp, uint32_t* sign) {
+    const int64_t words = (int64_t)((d + 31) / 32);
+#pragma omp parallel for schedule(static)
+    for (int64_t w = 0; w < words; ++w) {
+        uint32_t bits = 0;
+        const uint64_t end = ((uint64_t)w * 32 + 32 < d) ? (uint64_t)w * 32 + 32 : d;
+        for (uint64_t i = (uint64_t)w * 32; i < end; ++i) {
+            uint32_t sb;
+            cnat_code(nearest_pow2_value(x[i]), &exp[i], &sb);
+            bits |= sb << (i % 32);
+        }
+        sign[w] = bits;
+    }
+}
+
 // Master side, one worker: acc[j] = acc[j] + decode(code_j) in binary32.
 void orc_nc_decode_accumulate(const uint8_t* exp, const uint32_t* sign, uint64_t d, float* acc) {
 #pragma omp parallel for schedule(static)
@@ -286,6 +325,38 @@ void orc_norms(const float* x, const uint64_t* bucket_off, int B, int p, float* 
 // Level codes for explicit y and thresholds (enumeration pins).
 void orc_nd_level_codes(const double* y, const uint32_t* r23, uint64_t count, int s, int32_t* codes) {
     for (uint64_t i = 0; i < count; ++i) codes[i] = nd_level_code(y[i], s, r23[i] & 0x7FFFFFu);
+}
+
+// Standard dithering D_sta^{p,u} (Def. 3 with the linear levels k/u, C = identity), oracle side
+// only: it is the comparison operator of the empirical-variance experiment (Appendix A.2) and of
+// Thm. 5, not part of the CUDA path.  Level index of y in [0, 1]: floor(y u) or that plus one,
+// the upper one with probability y u - floor(y u); the draw is "up iff r23 < floor(p 2^23)".
+void orc_dsta_level_index(const double* y, const uint32_t* r23, uint64_t count, int u,
+                          int32_t* index) {
+    for (uint64_t i = 0; i < count; ++i) {
+        double yy = y[i];
+        if (yy >= 1.0) { index[i] = u; continue; }
+        const double scaled = yy * (double)u;
+        const double k = std::floor(scaled);
+        const double thr = std::floor((scaled - k) * TWO23);
+        index[i] = (int32_t)k + (((double)(r23[i] & 0x7FFFFFu) < thr) ? 1 : 0);
+    }
+}
+
+// out[i] = D_sta^{p,u}(x)_i = ||x||_p sign(x_i) xi(|x_i| / ||x||_p), one bucket, norm and y in
+// double, random thresholds from the domain-1 stream of (seed, worker).
+void orc_dsta_apply(const float* x, uint64_t d, int p, int u, uint64_t seed, uint32_t worker,
+                    double* out) {
+    const float norm_f = norm_p(x, d, p);
+    const double norm = (double)norm_f;
+    for (uint64_t i = 0; i < d; ++i) {
+        if (!(norm > 0.0) || std::isinf(norm)) { out[i] = 0.0; continue; }
+        const double y = std::fabs((double)x[i]) / norm;
+        const uint32_t r = stream_word(seed, worker, 1u, i) & 0x7FFFFFu;
+        int32_t idx;
+        orc_dsta_level_index(&y, &r, 1, u, &idx);
+        out[i] = std::copysign(norm * (double)idx / (double)u, (double)x[i]);
+    }
 }
 
 // Natural dithering D_nat^{p,s} of x[0..d) split into B buckets, one norm each.

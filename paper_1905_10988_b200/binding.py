@@ -34,7 +34,7 @@ EXPORTS = (
     "nd_sparse_compress", "nd_sparse_decode_accumulate", "nc_copy_to_device", "nc_copy_to_host",
     "nd_batch_workspace_bytes", "nd_compress_batch", "nd_sparse_batch_workspace_bytes",
     "nd_sparse_compress_batch", "nd_static_scratch_bytes", "nd_compress_static",
-    "nc_aggregate_compress",
+    "nc_aggregate_compress", "nc_compress_nearest", "nc_compress_nearest_batch",
 )
 
 
@@ -127,6 +127,22 @@ def nc_aggregate_compress(exps, signs, n, d, seed, master, out_exp, out_sign, st
     _check("nc_aggregate_compress",
            _nc_aggregate_compress(_ptrs(exps), _ptrs(signs), n, d, seed, master, _ptr(out_exp),
                                   _ptr(out_sign), _stream(stream)))
+
+
+_nc_compress_nearest = _sig("nc_compress_nearest", C.c_int, _vp, _sz, _vp, _vp, _vp)
+_nc_compress_nearest_batch = _sig("nc_compress_nearest_batch", C.c_int, C.POINTER(_vp), _sz,
+                                  C.POINTER(_vp), C.POINTER(_vp), C.c_int, _vp)
+
+
+def nc_compress_nearest(x, d, exp, sign, stream=None) -> None:
+    _check("nc_compress_nearest", _nc_compress_nearest(_ptr(x), d, _ptr(exp), _ptr(sign),
+                                                       _stream(stream)))
+
+
+def nc_compress_nearest_batch(xs, d, exps, signs, n, stream=None) -> None:
+    _check("nc_compress_nearest_batch",
+           _nc_compress_nearest_batch(_ptrs(xs), d, _ptrs(exps), _ptrs(signs), n,
+                                      _stream(stream)))
 
 
 _nd_static_scratch_bytes = _sig("nd_static_scratch_bytes", _sz)

@@ -60,6 +60,10 @@ def run_cnat(config, n, d, make_vector, iters, peak, with_sum=True):
     workers = list(range(n))
     m, b = _time(lambda: nc.nc_compress_batch(xs, d, 0, workers, es, ss, n), iters)
     _report(config, "nc_compress_batch", m, b, n * d, n * d * 5.125, peak, {"n": n, "d": d})
+    m_det, b = _time(lambda: nc.nc_compress_nearest_batch(xs, d, es, ss, n), iters)
+    _report(config, "nc_compress_nearest_batch (no sampling)", m_det, b, n * d, n * d * 5.125, peak,
+            {"sampling_overhead": round(m / m_det - 1.0, 3)})
+    nc.nc_compress_batch(xs, d, 0, workers, es, ss, n)       # planes of the stochastic operator
     m, b = _time(lambda: nc.nc_aggregate(es, ss, n, d, out), iters)
     _report(config, "nc_aggregate", m, b, d, d * (1.125 * n + 4), peak)
     m, b = _time(lambda: nc.nc_aggregate_compress(es, ss, n, d, 0, 0xFFFFFFFF, ge, gs), iters)

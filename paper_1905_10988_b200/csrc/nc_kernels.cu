@@ -31,6 +31,10 @@ struct DensePlanes {
     const float* x[NC_MAX_WORKERS];
 };
 
+// With this value in place of the random word, "up iff r23 < mantissa" becomes "up iff the
+// mantissa field is at least 2^22", i.e. rounding to the nearest power of two, ties upward.
+constexpr uint32_t kNearestThreshold = 0x3FFFFFu;
+
 // exponent byte of C_nat(bits) given the element's random word
 __device__ __forceinline__ uint32_t cnat_exp_byte(uint32_t bits, uint32_t rnd) {
     uint32_t v = bits & 0x7FFFFFFFu;
@@ -41,6 +45,7 @@ __device__ __forceinline__ uint32_t cnat_exp_byte(uint32_t bits, uint32_t rnd) {
 
 // C_nat of one full tile held in registers (lane l: float4 groups k*32 + l, k = 0..7):
 // writes the tile's 1024 exponent bytes and 32 sign words.
+template <bool kDet>
 __device__ __forceinline__ void cnat_full_tile(const uint4 (&u)[8], const uint64_t base,
                                                const uint32_t worker, const PhiloxKeys& keys,
                                                uint8_t* __restrict__ exp,
@@ -62,7 +67,8 @@ __device__ __forceinline__ void cnat_full_tile(const uint4 (&u)[8], const uint64
 #pragma unroll
         for (int k = 7; k >= 0; --k) {
             uint32_t rnd[4];
-            stream_words4_tile(q_lo + k * 32, pt, keys, rnd);
+            if (kDet) rnd[0] = rnd[1] = rnd[2] = rnd[3] = kNearestThreshold;
+            else stream_words4_tile(q_lo + k * 32, pt, keys, rnd);
             const uint32_t b0 = u[k].x, b1 = u[k].y, b2 = u[k].z, b3 = u[k].w;
             // (bits + (~r23 & 0x7FFFFF)) << 1: sign shifted out, rounded exponent in byte 3
             const uint32_t t0 = (b0 + (~rnd[0] & 0x7FFFFFu)) << 1;
@@ -81,7 +87,8 @@ __device__ __forceinline__ void cnat_full_tile(const uint4 (&u)[8], const uint64
 #pragma unroll
         for (int k = 7; k >= 0; --k) {
             uint32_t rnd[4];
-            stream_words4_tile(q_lo + k * 32, pt, keys, rnd);
+            if (kDet) rnd[0] = rnd[1] = rnd[2] = rnd[3] = kNearestThreshold;
+            else stream_words4_tile(q_lo + k * 32, pt, keys, rnd);
             const uint32_t b0 = u[k].x, b1 = u[k].y, b2 = u[k].z, b3 = u[k].w;
             uint32_t e = cnat_exp_byte(b3, rnd[3]);
             e = (e << 8) | cnat_exp_byte(b2, rnd[2]);
@@ -103,7 +110,7 @@ __device__ __forceinline__ void cnat_full_tile(const uint4 (&u)[8], const uint64
 // C_nat of the ragged last tile, one element per lane per step (a ballot gives the sign word);
 // also writes the zero padding of both planes.  load_bits(j) returns the binary32 pattern of
 // element j.
-template <typename LoadBits>
+template <bool kDet, typename LoadBits>
 __device__ __forceinline__ void cnat_ragged_tile(LoadBits load_bits, const uint64_t base,
                                                  const uint64_t d, const uint32_t worker,
                                                  const PhiloxKeys& keys, uint8_t* __restrict__ exp,
@@ -116,10 +123,12 @@ __device__ __forceinline__ void cnat_ragged_tile(LoadBits load_bits, const uint6
         uint32_t bits = 0, e = 0;
         if (j < d) {
             bits = load_bits(j);
-            uint32_t rnd[4];
-            stream_words4(j >> 2, worker, kDomainCnat, keys, rnd);
-            const uint32_t r = (j & 3) == 0 ? rnd[0] : (j & 3) == 1 ? rnd[1]
-                             : (j & 3) == 2 ? rnd[2] : rnd[3];
+            uint32_t r = kNearestThreshold;
+            if (!kDet) {
+                uint32_t rnd[4];
+                stream_words4(j >> 2, worker, kDomainCnat, keys, rnd);
+                r = (j & 3) == 0 ? rnd[0] : (j & 3) == 1 ? rnd[1] : (j & 3) == 2 ? rnd[2] : rnd[3];
+            }
             e = cnat_exp_byte(bits, r);
         }
         if (j < exp_end) exp[j] = (uint8_t)e;
@@ -129,7 +138,9 @@ __device__ __forceinline__ void cnat_ragged_tile(LoadBits load_bits, const uint6
     if (lane < (int)(sign_words_padded - sign_words)) sign[sign_words + lane] = 0;
 }
 
-// grid: (ceil(tiles / warps per block), n workers)
+// grid: (ceil(tiles / warps per block), n workers).  kDet: round to the nearest power of two
+// instead of drawing (the paper's "deterministic" control variant, no generator).
+template <bool kDet>
 __global__ void __launch_bounds__(kBlockThreads)
 nc_compress_kernel(const __grid_constant__ CompressBatch batch, const uint64_t d,
                    const __grid_constant__ PhiloxKeys keys) {
@@ -144,11 +155,11 @@ nc_compress_kernel(const __grid_constant__ CompressBatch batch, const uint64_t d
         uint4 u[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) u[k] = ld_stream_u4(xv + k * 32 + lane);
-        cnat_full_tile(u, base, batch.worker[w], keys, batch.exp[w], batch.sign[w], lane);
+        cnat_full_tile<kDet>(u, base, batch.worker[w], keys, batch.exp[w], batch.sign[w], lane);
         return;
     }
-    cnat_ragged_tile([&](uint64_t j) { return __float_as_uint(x[j]); }, base, d, batch.worker[w],
-                     keys, batch.exp[w], batch.sign[w], lane);
+    cnat_ragged_tile<kDet>([&](uint64_t j) { return __float_as_uint(x[j]); }, base, d,
+                           batch.worker[w], keys, batch.exp[w], batch.sign[w], lane);
 }
 
 // value of a 9-bit code: exponent byte in byte `BYTE` of `e4`, sign in bit 0 of `s`
@@ -242,10 +253,10 @@ nc_aggregate_compress_kernel(const __grid_constant__ PackedPlanes planes, const 
         for (int k = 0; k < 8; ++k)
             u[k] = make_uint4(__float_as_uint(acc[k].x), __float_as_uint(acc[k].y),
                               __float_as_uint(acc[k].z), __float_as_uint(acc[k].w));
-        cnat_full_tile(u, base, master, keys, exp, sign, lane);
+        cnat_full_tile<false>(u, base, master, keys, exp, sign, lane);
         return;
     }
-    cnat_ragged_tile(
+    cnat_ragged_tile<false>(
         [&](uint64_t j) { return __float_as_uint(aggregate_element(planes, n, j, 0.f)); }, base,
         d, master, keys, exp, sign, lane);
 }
@@ -295,10 +306,12 @@ using namespace natcomp;
 
 extern "C" {
 
-nc_status nc_compress_batch(const float* const* xs, size_t d, uint64_t seed,
-                            const uint32_t* workers, uint8_t* const* exps,
-                            uint32_t* const* signs, int n, cudaStream_t stream) {
-    if (!xs || !workers || !exps || !signs || n < 1 || n > NC_MAX_WORKERS) return NC_ERR_INVALID;
+static nc_status compress_batch_impl(const float* const* xs, size_t d, uint64_t seed,
+                                     const uint32_t* workers, uint8_t* const* exps,
+                                     uint32_t* const* signs, int n, bool deterministic,
+                                     cudaStream_t stream) {
+    if (!xs || !exps || !signs || n < 1 || n > NC_MAX_WORKERS) return NC_ERR_INVALID;
+    if (!workers && !deterministic) return NC_ERR_INVALID;
     if (d == 0) return NC_OK;
     if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
     CompressBatch batch;
@@ -308,12 +321,31 @@ nc_status nc_compress_batch(const float* const* xs, size_t d, uint64_t seed,
         batch.x[i] = xs[i];
         batch.exp[i] = exps[i];
         batch.sign[i] = signs[i];
-        batch.worker[i] = workers[i];
+        batch.worker[i] = workers ? workers[i] : 0u;
     }
     const PhiloxKeys keys = make_philox_keys(seed);
     dim3 grid(tile_blocks(d), (unsigned)n);
-    nc_compress_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, (uint64_t)d, keys);
+    if (deterministic)
+        nc_compress_kernel<true><<<grid, kBlockThreads, 0, stream>>>(batch, (uint64_t)d, keys);
+    else
+        nc_compress_kernel<false><<<grid, kBlockThreads, 0, stream>>>(batch, (uint64_t)d, keys);
     return launch_status();
+}
+
+nc_status nc_compress_batch(const float* const* xs, size_t d, uint64_t seed,
+                            const uint32_t* workers, uint8_t* const* exps,
+                            uint32_t* const* signs, int n, cudaStream_t stream) {
+    return compress_batch_impl(xs, d, seed, workers, exps, signs, n, false, stream);
+}
+
+nc_status nc_compress_nearest_batch(const float* const* xs, size_t d, uint8_t* const* exps,
+                                    uint32_t* const* signs, int n, cudaStream_t stream) {
+    return compress_batch_impl(xs, d, 0, nullptr, exps, signs, n, true, stream);
+}
+
+nc_status nc_compress_nearest(const float* x, size_t d, uint8_t* exp, uint32_t* sign,
+                              cudaStream_t stream) {
+    return compress_batch_impl(&x, d, 0, nullptr, &exp, &sign, 1, true, stream);
 }
 
 nc_status nc_compress(const float* x, size_t d, uint64_t seed, uint32_t worker, uint8_t* exp,
