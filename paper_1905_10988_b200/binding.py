@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libnatcomp.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
-        "libnatcomp.so is not built; run `python -m paper_1905_10988_b200.build` "
+        "libnatcomp.so is not built; run `python paper_1905_10988_b200/build.py` "
         "(needs nvcc; targets sm_100a).  There is no CPU fallback.")
 
 lib = C.CDLL(LIB_PATH)

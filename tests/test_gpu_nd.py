@@ -159,15 +159,15 @@ def test_config3_full_size():
     d, B = off[-1], len(sizes)
     off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
     xd = [workloads.config2_vector(w, "cuda", sizes) for w in range(n)]
-    ws_bytes = nc.nd_workspace_bytes(d, B)
+    ws_bytes = nc.nd_batch_workspace_bytes(d, B, n)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     norms = [torch.empty(B, dtype=torch.float32, device="cuda") for _ in range(n)]
     levels = [torch.empty(nc.nd_level_bytes(d), dtype=torch.uint8, device="cuda")
               for _ in range(n)]
     signs = [torch.empty(nc.nc_sign_bytes(d), dtype=torch.uint8, device="cuda") for _ in range(n)]
-    for w in range(n):
-        nc.nd_compress(xd[w], d, off_dev, B, p, s, 0, w, norms[w], levels[w], signs[w], ws,
-                       ws_bytes)
+    # the launch configuration the benchmark times: one batch call for the 8 workers
+    nc.nd_compress_batch(xd, d, off_dev, B, p, s, 0, list(range(n)), norms, levels, signs, n, ws,
+                         ws_bytes)
     out = torch.empty(d, dtype=torch.float32, device="cuda")
     nc.nd_aggregate(norms, levels, signs, n, d, off_dev, B, s, out)
     torch.cuda.synchronize()
@@ -254,3 +254,22 @@ def test_batch_launch_equals_single_launches():
         assert np.array_equal(signs[i].numpy(np.uint32), s1.numpy(np.uint32))
         check_against_oracle(xs[i], off, p, s, 11, workers[i], norms[i], levels[i], signs[i],
                              slack=2)
+
+
+def test_one_element_buckets_and_many_empty_buckets():
+    # every tile takes the multi-bucket path: B = d one-element buckets, then a table that is
+    # mostly empty buckets
+    rng = np.random.default_rng(55)
+    d = 3000
+    x = (rng.standard_normal(d) * 1e-2).astype(np.float32)
+    x[7] = 0.0
+    off = list(range(d + 1))
+    for p in (2, 0):
+        norms, level, sign = gpu_nd_compress(dev(x), off, p, 8, seed=4, worker=2)
+        gn = check_against_oracle(x, off, p, 8, 4, 2, norms, level, sign, slack=2)
+        assert np.array_equal(gn, np.abs(x))            # a one-element bucket: norm = |x|
+        c = unpack_nibbles(level.numpy(np.uint8), d)
+        assert c[7] == 0 and np.all(c[np.abs(x) >= 2.0 ** -126] == 8)   # y = 1 exactly
+    off2 = sorted([0] + list(rng.integers(0, d, 40)) * 3 + [d])
+    norms, level, sign = gpu_nd_compress(dev(x), off2, 1, 4, seed=5, worker=0)
+    check_against_oracle(x, off2, 1, 4, 5, 0, norms, level, sign, slack=2)

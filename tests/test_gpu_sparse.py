@@ -162,3 +162,36 @@ def test_sparse_batch_launch_equals_single_launches():
     for i in range(n):
         got = (idx[i], codes[i], int(count[i].numpy(np.uint32)[0]), norm[i].numpy(np.float32)[0])
         check_sparse(xs[i], thr, scale, nc.P_INF, s, 6, workers[i], cap, got)
+
+
+def test_sparse_bench_launch_configuration_sampled():
+    # the shape the benchmark times: 8 workers, d = 25,557,032, one batch call, keep 1 %
+    n, s = 8, 4
+    sizes = workloads.resnet50_tensor_sizes()
+    d = sum(sizes)
+    cap = int(d * 0.0125)
+    thr, scale = workloads.KEEP_1PCT_THRESHOLD, workloads.KEEP_1PCT_SCALE
+    xd = [workloads.config2_vector(w, "cuda", sizes) for w in range(n)]
+    idx = [torch.empty(cap, dtype=torch.int32, device="cuda") for _ in range(n)]
+    codes = [torch.empty((cap + 1) // 2 + 16, dtype=torch.uint8, device="cuda") for _ in range(n)]
+    count = [torch.zeros(1, dtype=torch.int32, device="cuda") for _ in range(n)]
+    norm = [torch.zeros(1, dtype=torch.float32, device="cuda") for _ in range(n)]
+    ws_bytes = nc.nd_sparse_batch_workspace_bytes(d, cap, n)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    nc.nd_sparse_compress_batch(xd, d, thr, scale, nc.P_INF, s, 0, list(range(n)), idx, codes,
+                                count, norm, cap, n, ws, ws_bytes)
+    acc = torch.zeros(d, dtype=torch.float32, device="cuda")
+    for w in range(n):
+        nc.nd_sparse_decode_accumulate(idx[w], codes[w], count[w], norm[w], s, d, cap, acc)
+    torch.cuda.synchronize()
+    ref = np.zeros(d, np.float32)
+    for w in range(n):
+        x = xd[w].cpu().numpy()
+        i_ref, c_ref, count_ref, n_ref = oracle.sparse_compress(x, thr, scale, nc.P_INF, s, 0, w,
+                                                                cap=cap)
+        cnt = int(count[w].cpu().numpy().view(np.uint32)[0])
+        assert cnt == count_ref and float(norm[w].cpu()[0]) == float(n_ref)
+        assert np.array_equal(idx[w][:cnt].cpu().numpy().view(np.uint32), i_ref)
+        assert np.array_equal(codes[w][:(cnt + 1) // 2].cpu().numpy(), c_ref)
+        oracle.sparse_decode_accumulate(i_ref, c_ref, count_ref, n_ref, s, ref)
+    assert np.array_equal(acc.cpu().numpy().view(np.uint32), ref.view(np.uint32))
