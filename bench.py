@@ -5,7 +5,8 @@ One step = one pass of the whole path over one batch of synthetic gradients, on 
 ResNet-50-shaped workload (n = 8 workers, d = 25,557,032 fp32 entries in 161 buckets):
   C_nat  : nc_compress_batch (8 workers, one launch) + nc_aggregate
   D_nat  : nd_compress x 8 (p = 2, s = 8, per-bucket norms) + nd_aggregate
-  sparse : nd_sparse_compress x 8 (keep 1 %, p = inf, s = 4) + nd_sparse_decode_accumulate x 8
+  sparse : nd_sparse_compact_compress_batch (keep 1 %, p = inf, s = 4, 3-bit codes)
+           + nd_sparse_compact_decode_accumulate x 8
   ref    : nc_sum_fp32 (uncompressed 8-way sum, the reference point)
 The metric is worker-entries taken through the whole path per second (n * d per step).
 Inputs (818 MB) are larger than the 126 MB L2, so no flush is needed between steps.
@@ -149,7 +150,8 @@ class HotPath:
         self.out_nd = torch.empty(d, **f32)
         self.cap = int(d * SPARSE_CAP_FRACTION)
         self.idx = [torch.empty(self.cap, dtype=torch.int32, device=device) for _ in range(n)]
-        self.codes = [torch.empty((self.cap + 1) // 2 + 16, **u8) for _ in range(n)]
+        self.codes = [torch.empty(nc.nd_sparse_plane_bytes(self.cap, S_SPARSE), **u8)
+                      for _ in range(n)]
         self.count = [torch.zeros(1, dtype=torch.int32, device=device) for _ in range(n)]
         self.snorm = [torch.zeros(1, **f32) for _ in range(n)]
         self.sws_bytes = nc.nd_sparse_batch_workspace_bytes(d, self.cap, n)
@@ -157,8 +159,8 @@ class HotPath:
         self.out_sp = torch.empty(d, **f32)
         self.out_sum = torch.empty(d, **f32)
         # nc_compress_batch 1, nc_aggregate 1, nd_compress_batch 3, nd_aggregate 1,
-        # nd_sparse_compress_batch 4, nd_sparse_decode_accumulate n, nc_sum_fp32 1
-        self.launches_per_step = 1 + 1 + 3 + 1 + 4 + n + 1
+        # nd_sparse_compact_compress_batch 7, nd_sparse_compact_decode_accumulate n, nc_sum_fp32 1
+        self.launches_per_step = 1 + 1 + 3 + 1 + 7 + n + 1
         self.seed = 0
 
     def step(self, marks=None):
@@ -191,16 +193,18 @@ class HotPath:
                             self.out_nd)
         mark("nd_aggregate")
         if want("sparse_compress"):
-            nc.nd_sparse_compress_batch(self.x, d, workloads.KEEP_1PCT_THRESHOLD,
-                                        workloads.KEEP_1PCT_SCALE, nc.P_INF, S_SPARSE, self.seed,
-                                        self.workers, self.idx, self.codes, self.count,
-                                        self.snorm, self.cap, n, self.sws, self.sws_bytes)
+            nc.nd_sparse_compact_compress_batch(self.x, d, workloads.KEEP_1PCT_THRESHOLD,
+                                                workloads.KEEP_1PCT_SCALE, nc.P_INF, S_SPARSE,
+                                                self.seed, self.workers, self.idx, self.codes,
+                                                self.count, self.snorm, self.cap, n, self.sws,
+                                                self.sws_bytes)
         mark("sparse_compress")
         if want("sparse_accumulate"):
             self.out_sp.zero_()
             for w in range(n):
-                nc.nd_sparse_decode_accumulate(self.idx[w], self.codes[w], self.count[w],
-                                               self.snorm[w], S_SPARSE, d, self.cap, self.out_sp)
+                nc.nd_sparse_compact_decode_accumulate(self.idx[w], self.codes[w], self.count[w],
+                                                       self.snorm[w], S_SPARSE, d, self.cap,
+                                                       self.out_sp)
         mark("sparse_accumulate")
         if want("sum_fp32"):
             nc.nc_sum_fp32(self.x, n, d, self.out_sum)
@@ -215,8 +219,10 @@ class HotPath:
             "nc_aggregate": d * (1.125 * n + 4),
             "nd_compress": n * d * (4 + 4 + 0.625),        # x is read by the norm and rounding passes
             "nd_aggregate": d * (0.625 * n + 4),
-            "sparse_compress": n * kept * (32 + 32 + 4 + 0.5),   # two sector reads per kept entry
-            "sparse_accumulate": 4 * d + n * kept * (4.5 + 64),
+            # kept entries are read as 32-byte sectors in three passes (norm, filter, emit);
+            # about half of them survive the level-0 filter and are listed (4 B index + 3 bits)
+            "sparse_compress": n * kept * (3 * 32 + 0.5 * 4.375),
+            "sparse_accumulate": 4 * d + n * kept * 0.5 * (4.375 + 64),
             "sum_fp32": d * (4 * n + 4),
         }
 
@@ -246,10 +252,10 @@ def cpu_baseline_sample(steps=1):
                             S_DITHER, d)
         acc = np.zeros(d, np.float32)
         for w in range(n):
-            idx, codes, count, nrm = oracle.sparse_compress(
+            idx, planes, count, nrm = oracle.sparse_compact_compress(
                 xs[w], workloads.KEEP_1PCT_THRESHOLD, workloads.KEEP_1PCT_SCALE, oracle.P_INF,
                 S_SPARSE, 0, w)
-            oracle.sparse_decode_accumulate(idx, codes, count, nrm, S_SPARSE, acc)
+            oracle.sparse_compact_decode_accumulate(idx, planes, count, nrm, S_SPARSE, acc)
         oracle.sum_fp32(xs)
         times.append(time.perf_counter() - t0)
     sample = ("first %d tensors of the ResNet-50 layout (%d entries) x %d workers, whole path; "

@@ -218,6 +218,35 @@ nc_status nd_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes,
                                       const uint32_t* count, const float* norm, int s, size_t d,
                                       size_t cap, float* acc, cudaStream_t stream);
 
+/* ---- compact sparse format: zero levels dropped, codes as bit planes ------------------------
+ * Same operator as nd_sparse_compress (sparsifier definition + Def. 3, composition of Thm. 3), in
+ * the format "index list + log2(s)+1 bits per listed entry" that the paper's bit counts for
+ * sparsified dithering assume: a kept coordinate whose level rounds to 0 decodes to +-0 and is
+ * left out of the list.  Listed entry k has level 1..s and code (sign << nb) | (level - 1),
+ * nb = ceil(log2 s) (s <= 4: 3-bit codes; s <= 8 supported).  For the g-th group of 32 listed
+ * entries, word planes[g * (nb + 1) + b] holds bit b of the 32 codes (entry k in bit k mod 32).
+ * idx: uint32[cap]; planes: nd_sparse_plane_bytes(cap, s) bytes, written for all ceil(cap/32)
+ * groups (zero beyond the count); count: listed entries (may exceed cap); norm: p-norm over ALL
+ * kept entries, as in nd_sparse_compress; workspace: nd_sparse_batch_workspace_bytes(d, cap, n). */
+size_t nd_sparse_plane_bytes(size_t cap, int s);
+nc_status nd_sparse_compact_compress(const float* x, size_t d, uint64_t keep_threshold,
+                                     float scale, int p, int s, uint64_t seed, uint32_t worker,
+                                     uint32_t* idx, uint32_t* planes, uint32_t* count, float* norm,
+                                     size_t cap, void* workspace, size_t workspace_bytes,
+                                     cudaStream_t stream);
+nc_status nd_sparse_compact_compress_batch(const float* const* xs, size_t d,
+                                           uint64_t keep_threshold, float scale, int p, int s,
+                                           uint64_t seed, const uint32_t* workers,
+                                           uint32_t* const* idxs, uint32_t* const* planes,
+                                           uint32_t* const* counts, float* const* norms,
+                                           size_t cap, int n, void* workspace,
+                                           size_t workspace_bytes, cudaStream_t stream);
+/* acc[idx[k]] <- acc[idx[k]] + sign * fl32(norm * 2^(level - s)) for the listed entries. */
+nc_status nd_sparse_compact_decode_accumulate(const uint32_t* idx, const uint32_t* planes,
+                                              const uint32_t* count, const float* norm, int s,
+                                              size_t d, size_t cap, float* acc,
+                                              cudaStream_t stream);
+
 /* ---- host-buffer plumbing (no counterpart in the paper, where workers and master exchange
  * these buffers over a network) ------------------------------------------------------------- */
 

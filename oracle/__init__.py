@@ -277,3 +277,42 @@ def nc_compress_nearest(x):
     s = np.zeros((d + 31) // 32, np.uint32)
     _nc_compress_nearest(_p(x, _f32p), d, _p(e, _u8p), _p(s, _u32p))
     return e, s
+
+
+_sparse_compact_compress = _sig("orc_sparse_compact_compress", C.c_uint64, _f32p, C.c_uint64,
+                                C.c_uint64, C.c_float, C.c_int, C.c_int, C.c_uint64, C.c_uint32,
+                                _u32p, _u32p, C.c_uint64, _f32p)
+_sparse_compact_decode_accumulate = _sig("orc_sparse_compact_decode_accumulate", None, _u32p,
+                                         _u32p, C.c_uint64, C.c_float, C.c_int, _f32p)
+
+
+def code_bits(s: int) -> int:
+    """Bits per code of the compact sparse format: sign + ceil(log2 s)."""
+    nb = 0
+    while (1 << nb) < s:
+        nb += 1
+    return nb + 1
+
+
+def sparse_compact_compress(x, keep_threshold: int, scale: float, p: int, s: int, seed: int,
+                            worker: int, cap=None):
+    """Sparsifier + D_nat with zero-level entries dropped; returns idx, planes, count, norm."""
+    x = _arr(x, np.float32)
+    d = x.size
+    if cap is None:
+        cap = d
+    idx = np.zeros(cap, np.uint32)
+    planes = np.zeros(((cap + 31) // 32) * code_bits(s), np.uint32)
+    nrm = C.c_float(0.0)
+    count = _sparse_compact_compress(_p(x, _f32p), d, keep_threshold, scale, p, s, seed, worker,
+                                     _p(idx, _u32p), _p(planes, _u32p), cap, C.byref(nrm))
+    stored = min(int(count), cap)
+    return idx[:stored], planes, int(count), np.float32(nrm.value)
+
+
+def sparse_compact_decode_accumulate(idx, planes, count: int, nrm, s: int, acc) -> None:
+    idx = _arr(idx, np.uint32)
+    planes = _arr(planes, np.uint32)
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    _sparse_compact_decode_accumulate(_p(idx, _u32p), _p(planes, _u32p), count, float(nrm), s,
+                                      _p(acc, _f32p))

@@ -495,4 +495,72 @@ void orc_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes, uin
     }
 }
 
+// The compact form of the sparsified + dithered vector: entries whose level rounds to 0 carry no
+// information and are left out of the list.  Same selection, scaling, norm (over all kept
+// entries) and rounding as orc_sparse_compress.  A listed entry has level 1..s and the code
+// (sign << nb) | (level - 1) with nb = bits needed for s - 1 (2 for s <= 4, so 3-bit codes).
+// Codes are stored as bit planes: for the g-th group of 32 listed entries, word
+// planes[g * (nb + 1) + b] holds bit b of the 32 codes (entry k in bit k mod 32).
+// Returns the number of listed entries (those beyond cap are counted, not stored).
+static int bits_for(int s) {
+    int nb = 0;
+    while ((1 << nb) < s) ++nb;
+    return nb;
+}
+
+uint64_t orc_sparse_compact_compress(const float* x, uint64_t d, uint64_t keep_threshold,
+                                     float scale, int p, int s, uint64_t seed, uint32_t worker,
+                                     uint32_t* idx, uint32_t* planes, uint64_t cap,
+                                     float* norm_out) {
+    double acc = 0.0;
+    bool saw_nan = false;
+    for (uint64_t j = 0; j < d; ++j) {
+        if ((uint64_t)stream_word(seed, worker, 2u, j) >= keep_threshold) continue;
+        const float xs = scale * x[j];
+        const double a = std::fabs((double)xs);
+        if (std::isnan(a)) saw_nan = true;
+        if (p == 1) acc += a;
+        else if (p == 2) acc += a * a;
+        else if (a > acc) acc = a;
+    }
+    if (p == 2) acc = std::sqrt(acc);
+    const float norm = saw_nan ? std::numeric_limits<float>::quiet_NaN() : (float)acc;
+    *norm_out = norm;
+    const int nb = bits_for(s);
+    const uint64_t groups = (cap + 31) / 32;
+    std::memset(planes, 0, (size_t)(groups * (uint64_t)(nb + 1)) * 4);
+    if (norm_degenerate(norm)) return 0;            // every level is 0: nothing to list
+    const float rinv = 1.0f / norm;
+    uint64_t k = 0;
+    for (uint64_t j = 0; j < d; ++j) {
+        if ((uint64_t)stream_word(seed, worker, 2u, j) >= keep_threshold) continue;
+        const float xs = scale * x[j];
+        const float yf = std::fabs(xs) * rinv;
+        const uint32_t r23 = stream_word(seed, worker, 1u, j) & 0x7FFFFFu;
+        const int c = nd_level_code((double)yf, s, r23);
+        if (c == 0) continue;
+        if (k < cap) {
+            const uint32_t code = ((std::signbit(xs) ? 1u : 0u) << nb) | (uint32_t)(c - 1);
+            idx[k] = (uint32_t)j;
+            for (int b = 0; b <= nb; ++b)
+                planes[(k / 32) * (uint64_t)(nb + 1) + (uint64_t)b] |= ((code >> b) & 1u) << (k % 32);
+        }
+        ++k;
+    }
+    return k;
+}
+
+void orc_sparse_compact_decode_accumulate(const uint32_t* idx, const uint32_t* planes,
+                                          uint64_t count, float norm, int s, float* acc) {
+    const int nb = bits_for(s);
+    for (uint64_t k = 0; k < count; ++k) {
+        uint32_t code = 0;
+        for (int b = 0; b <= nb; ++b)
+            code |= ((planes[(k / 32) * (uint64_t)(nb + 1) + (uint64_t)b] >> (k % 32)) & 1u) << b;
+        const int level = (int)(code & ((1u << nb) - 1u)) + 1;
+        const float v = nd_decode_value(level, s, norm, code >> nb);
+        acc[idx[k]] = acc[idx[k]] + v;
+    }
+}
+
 }  // extern "C"

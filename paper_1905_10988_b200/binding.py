@@ -35,6 +35,8 @@ EXPORTS = (
     "nd_batch_workspace_bytes", "nd_compress_batch", "nd_sparse_batch_workspace_bytes",
     "nd_sparse_compress_batch", "nd_static_scratch_bytes", "nd_compress_static",
     "nc_aggregate_compress", "nc_compress_nearest", "nc_compress_nearest_batch",
+    "nd_sparse_plane_bytes", "nd_sparse_compact_compress", "nd_sparse_compact_compress_batch",
+    "nd_sparse_compact_decode_accumulate",
 )
 
 
@@ -143,6 +145,49 @@ def nc_compress_nearest_batch(xs, d, exps, signs, n, stream=None) -> None:
     _check("nc_compress_nearest_batch",
            _nc_compress_nearest_batch(_ptrs(xs), d, _ptrs(exps), _ptrs(signs), n,
                                       _stream(stream)))
+
+
+_nd_sparse_plane_bytes = _sig("nd_sparse_plane_bytes", _sz, _sz, C.c_int)
+_nd_sparse_compact_compress = _sig("nd_sparse_compact_compress", C.c_int, _vp, _sz, C.c_uint64,
+                                   C.c_float, C.c_int, C.c_int, C.c_uint64, C.c_uint32, _vp, _vp,
+                                   _vp, _vp, _sz, _vp, _sz, _vp)
+_nd_sparse_compact_compress_batch = _sig("nd_sparse_compact_compress_batch", C.c_int,
+                                         C.POINTER(_vp), _sz, C.c_uint64, C.c_float, C.c_int,
+                                         C.c_int, C.c_uint64, C.POINTER(C.c_uint32),
+                                         C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp),
+                                         C.POINTER(_vp), _sz, C.c_int, _vp, _sz, _vp)
+_nd_sparse_compact_decode_accumulate = _sig("nd_sparse_compact_decode_accumulate", C.c_int, _vp,
+                                            _vp, _vp, _vp, C.c_int, _sz, _sz, _vp, _vp)
+
+
+def nd_sparse_plane_bytes(cap: int, s: int) -> int:
+    return int(_nd_sparse_plane_bytes(cap, s))
+
+
+def nd_sparse_compact_compress(x, d, keep_threshold, scale, p, s, seed, worker, idx, planes, count,
+                               norm, cap, workspace, workspace_bytes, stream=None) -> None:
+    _check("nd_sparse_compact_compress",
+           _nd_sparse_compact_compress(_ptr(x), d, keep_threshold, scale, p, s, seed, worker,
+                                       _ptr(idx), _ptr(planes), _ptr(count), _ptr(norm), cap,
+                                       _ptr(workspace), workspace_bytes, _stream(stream)))
+
+
+def nd_sparse_compact_compress_batch(xs, d, keep_threshold, scale, p, s, seed, workers, idxs,
+                                     planes, counts, norms, cap, n, workspace, workspace_bytes,
+                                     stream=None) -> None:
+    w = (C.c_uint32 * n)(*[int(v) for v in workers])
+    _check("nd_sparse_compact_compress_batch",
+           _nd_sparse_compact_compress_batch(_ptrs(xs), d, keep_threshold, scale, p, s, seed, w,
+                                             _ptrs(idxs), _ptrs(planes), _ptrs(counts),
+                                             _ptrs(norms), cap, n, _ptr(workspace),
+                                             workspace_bytes, _stream(stream)))
+
+
+def nd_sparse_compact_decode_accumulate(idx, planes, count, norm, s, d, cap, acc,
+                                        stream=None) -> None:
+    _check("nd_sparse_compact_decode_accumulate",
+           _nd_sparse_compact_decode_accumulate(_ptr(idx), _ptr(planes), _ptr(count), _ptr(norm),
+                                                s, d, cap, _ptr(acc), _stream(stream)))
 
 
 _nd_static_scratch_bytes = _sig("nd_static_scratch_bytes", _sz)

@@ -126,6 +126,25 @@ def run_sparse(config, n, d, iters, peak, s=4):
     m, b = _time(accumulate, iters)
     _report(config, "nd_sparse_decode_accumulate x n", m, b, n * kept, n * kept * 68.5, peak)
 
+    # the compact format: level-0 entries dropped, 3-bit codes as bit planes
+    planes = [torch.empty(nc.nd_sparse_plane_bytes(cap, s), **u8) for _ in range(n)]
+    m, b = _time(lambda: nc.nd_sparse_compact_compress_batch(xs, d, thr, scale, nc.P_INF, s, 0,
+                                                             workers, idx, planes, count, norm,
+                                                             cap, n, ws, ws_bytes), iters)
+    listed = sum(int(c.cpu().numpy().view("uint32")[0]) for c in count)
+    _report(config, "nd_sparse_compact_compress_batch", m, b, n * d,
+            n * kept * 96 + listed * 4.375, peak,
+            {"Gcoord_per_s": round(n * d / m / 1e6, 1), "listed_fraction_of_kept":
+             round(listed / (n * kept), 3)})
+
+    def accumulate_compact():
+        for w in range(n):
+            nc.nd_sparse_compact_decode_accumulate(idx[w], planes[w], count[w], norm[w], s, d,
+                                                   cap, acc)
+
+    m, b = _time(accumulate_compact, iters)
+    _report(config, "nd_sparse_compact_decode_accumulate x n", m, b, listed, listed * 68.4, peak)
+
 
 def main():
     ap = argparse.ArgumentParser()

@@ -449,3 +449,264 @@ nc_status nd_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes,
 }
 
 }  // extern "C"
+
+// ---- compact list: entries whose level rounds to 0 are dropped, codes as bit planes -----------
+//
+// A kept coordinate whose level code is 0 decodes to +-0, so leaving it out of the index list
+// loses nothing; the remaining codes are (sign << nb) | (level - 1) with nb = ceil(log2 s) bits
+// (s <= 4: 3-bit codes) stored as nb + 1 bit planes per 32 listed entries.
+//   select        : as above (bitmask of kept coordinates, norm partials)
+//   scan          : norm (and the kept count, unused here)
+//   round_filter  : level of every kept entry; clears the mask bit of level-0 entries, recounts
+//   scan          : offsets of the surviving entries, final count
+//   emit_compact  : index list + one code byte per surviving entry
+//   pack_planes   : 32 code bytes -> nb + 1 plane words (warp ballots)
+namespace natcomp {
+
+__host__ __device__ inline int code_value_bits(int s) {
+    int nb = 0;
+    while ((1 << nb) < s) ++nb;
+    return nb;
+}
+
+// grid: (ceil(tiles / warps per block), n workers)
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_round_filter_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
+                           const float scale, const int s,
+                           const __grid_constant__ PhiloxKeys keys, char* __restrict__ ws_all,
+                           const uint64_t ws_stride) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const uint64_t base = tile * kTile;
+    const bool active = base < d;
+    const float* __restrict__ x = batch.x[blockIdx.y];
+    const uint32_t worker = batch.worker[blockIdx.y];
+    const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
+    __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
+    __shared__ uint32_t s_mask[kWarpsPerBlock][32];
+    __shared__ uint32_t s_cnt[kWarpsPerBlock];
+    uint16_t* list = s_list[warp];
+    const uint32_t word = active ? ws.bitmask[tile * 32 + lane] : 0u;
+    s_mask[warp][lane] = word;
+    const uint32_t cnt = warp_list_positions(word, lane, list);     // ends with __syncwarp
+    const Scale sc = make_scale(*batch.norm[blockIdx.y], s);
+    const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
+    for (uint32_t t = lane; t < cnt; t += 32) {
+        const uint32_t pos = list[t];
+        const uint64_t j = base + pos;
+        const float xs = __fmul_rn(scale, x[j]);
+        uint32_t r4[4];
+        stream_words4(j >> 2, worker, kDomainDnat, keys, r4);
+        const uint32_t r = (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1]
+                         : (j & 3) == 2 ? r4[2] : r4[3];
+        if (sparse_level_code(__float_as_uint(xs), r, sc, pow2s) == 0u)
+            atomicAnd(&s_mask[warp][pos >> 5], ~(1u << (pos & 31)));
+    }
+    __syncwarp();
+    const uint32_t kept = s_mask[warp][lane];
+    if (active) ws.bitmask[tile * 32 + lane] = kept;
+    const uint32_t total = warp_sum_u(__popc(kept));
+    if (lane == 0) s_cnt[warp] = total;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t c = 0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) c += s_cnt[w];
+        ws.block_count[blockIdx.x] = c;
+    }
+}
+
+// grid: (ceil(tiles / warps per block), n workers)
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_emit_compact_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
+                           const float scale, const int s,
+                           const __grid_constant__ PhiloxKeys keys, const uint64_t cap,
+                           char* __restrict__ ws_all, const uint64_t ws_stride) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const uint64_t base = tile * kTile;
+    const bool active = base < d;
+    const float* __restrict__ x = batch.x[blockIdx.y];
+    const uint32_t worker = batch.worker[blockIdx.y];
+    const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
+    uint32_t* __restrict__ idx = batch.idx[blockIdx.y];
+    __shared__ uint32_t s_tile[kWarpsPerBlock];
+    __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
+    uint16_t* list = s_list[warp];
+    const uint32_t word = active ? ws.bitmask[tile * 32 + lane] : 0u;
+    const uint32_t cnt = warp_list_positions(word, lane, list);
+    if (lane == 0) s_tile[warp] = cnt;
+    __syncthreads();
+    uint64_t k0 = (uint64_t)ws.block_count[blockIdx.x];
+    for (int w = 0; w < warp; ++w) k0 += s_tile[w];
+    if (cnt == 0) return;
+    const Scale sc = make_scale(*batch.norm[blockIdx.y], s);
+    const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
+    const int nb = code_value_bits(s);
+    for (uint32_t t = lane; t < cnt; t += 32) {
+        const uint64_t k = k0 + t;
+        if (k >= cap) break;
+        const uint64_t j = base + list[t];
+        const float xs = __fmul_rn(scale, x[j]);
+        const uint32_t bits = __float_as_uint(xs);
+        uint32_t r4[4];
+        stream_words4(j >> 2, worker, kDomainDnat, keys, r4);
+        const uint32_t r = (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1]
+                         : (j & 3) == 2 ? r4[2] : r4[3];
+        const uint32_t level = sparse_level_code(bits, r, sc, pow2s);   // >= 1 after the filter
+        idx[k] = (uint32_t)j;
+        ws.tmp_codes[k] = (uint8_t)(((bits >> 31) << nb) | (level - 1u));
+    }
+}
+
+// one warp per 32 listed entries; grid: (ceil(groups / warps per block), n workers)
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_pack_planes_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
+                          const uint64_t cap, const int s, char* __restrict__ ws_all,
+                          const uint64_t ws_stride) {
+    const int lane = threadIdx.x & 31;
+    const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
+    const uint64_t group = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t groups = (cap + 31) / 32;
+    if (group >= groups) return;
+    const uint64_t total = min((uint64_t)*batch.count[blockIdx.y], cap);
+    const uint64_t k = group * 32 + lane;
+    const uint32_t code = (k < total) ? ws.tmp_codes[k] : 0u;
+    const int planes = code_value_bits(s) + 1;
+    uint32_t* out = reinterpret_cast<uint32_t*>(batch.codes[blockIdx.y]) + group * planes;
+    for (int b = 0; b < planes; ++b) {
+        const uint32_t wv = __ballot_sync(0xFFFFFFFFu, (code >> b) & 1u);
+        if (lane == 0) out[b] = wv;
+    }
+}
+
+// grid: ceil(cap / threads)
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_compact_decode_accumulate_kernel(const uint32_t* __restrict__ idx,
+                                        const uint32_t* __restrict__ planes,
+                                        const uint32_t* __restrict__ count,
+                                        const float* __restrict__ norm, const int s,
+                                        const uint64_t d, const uint64_t cap,
+                                        float* __restrict__ acc) {
+    const uint64_t k = (uint64_t)blockIdx.x * kBlockThreads + threadIdx.x;
+    const uint64_t total = min((uint64_t)*count, cap);
+    if (k >= total) return;
+    float nv = *norm;
+    if (!(fabsf(nv) <= 3.40282347e38f)) nv = 0.f;
+    const uint32_t j = idx[k];
+    if (j >= d) return;
+    const int nb = code_value_bits(s);
+    const uint32_t* pw = planes + (k >> 5) * (uint64_t)(nb + 1);
+    uint32_t code = 0;
+    for (int b = 0; b <= nb; ++b) code |= ((pw[b] >> (k & 31)) & 1u) << b;
+    const uint32_t level = (code & ((1u << nb) - 1u)) + 1u;
+    const uint32_t pb = ((level + 127u - (uint32_t)s) << 23) | ((code >> nb) << 31);
+    acc[j] = __fadd_rn(acc[j], __fmul_rn(nv, __uint_as_float(pb)));
+}
+
+}  // namespace natcomp
+
+extern "C" {
+
+size_t nd_sparse_plane_bytes(size_t cap, int s) {
+    if (s < 1) s = 1;
+    return round_up16(((cap + 31) / 32) * (size_t)(code_value_bits(s) + 1) * 4);
+}
+
+nc_status nd_sparse_compact_compress_batch(const float* const* xs, size_t d,
+                                           uint64_t keep_threshold, float scale, int p, int s,
+                                           uint64_t seed, const uint32_t* workers,
+                                           uint32_t* const* idxs, uint32_t* const* planes,
+                                           uint32_t* const* counts, float* const* norms,
+                                           size_t cap, int n, void* workspace,
+                                           size_t workspace_bytes, cudaStream_t stream) {
+    if (!xs || !workers || !idxs || !planes || !counts || !norms || n < 1 ||
+        n > NC_MAX_WORKERS || s < 1 || s > 8 || cap < 1 || keep_threshold > ((uint64_t)1 << 32))
+        return NC_ERR_INVALID;
+    if (p != 1 && p != 2 && p != NC_P_INF) return NC_ERR_UNSUPPORTED;
+    if (d == 0) return NC_OK;
+    if (d > 0xFFFFFFFFull) return NC_ERR_INVALID;
+    if (!workspace) return NC_ERR_INVALID;
+    if (!aligned16(workspace)) return NC_ERR_ALIGN;
+    SparseBatch batch;
+    for (int i = 0; i < n; ++i) {
+        if (!xs[i] || !idxs[i] || !planes[i] || !counts[i] || !norms[i]) return NC_ERR_INVALID;
+        if (!aligned32(xs[i]) || !aligned16(idxs[i]) || !aligned16(planes[i]) ||
+            !aligned4(counts[i]) || !aligned4(norms[i]))
+            return NC_ERR_ALIGN;
+        batch.x[i] = xs[i];
+        batch.idx[i] = idxs[i];
+        batch.codes[i] = reinterpret_cast<uint8_t*>(planes[i]);
+        batch.count[i] = counts[i];
+        batch.norm[i] = norms[i];
+        batch.worker[i] = workers[i];
+    }
+    const uint64_t ws_stride = sparse_ws_bytes(d, cap);
+    if (workspace_bytes < (size_t)n * ws_stride) return NC_ERR_WORKSPACE;
+    char* ws = reinterpret_cast<char*>(workspace);
+    const uint64_t tiles = sparse_tiles(d);
+    const dim3 grid((unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
+    const dim3 sgrid(1, (unsigned)n);
+    const PhiloxKeys keys = make_philox_keys(seed);
+    const bool keep_none = keep_threshold == 0;
+    const uint32_t neg_thr = (uint32_t)(0ull - keep_threshold);
+    if (p == 1) {
+        sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
+                                                                    scale, keys, ws, ws_stride);
+        sparse_scan_kernel<1><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
+    } else if (p == 2) {
+        sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
+                                                                    scale, keys, ws, ws_stride);
+        sparse_scan_kernel<2><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
+    } else {
+        sparse_select_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
+            batch, d, neg_thr, keep_none, scale, keys, ws, ws_stride);
+        sparse_scan_kernel<NC_P_INF><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
+    }
+    sparse_round_filter_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, ws,
+                                                                   ws_stride);
+    // second scan: offsets and count of the surviving entries (the norm partials are unchanged)
+    if (p == 1) sparse_scan_kernel<1><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
+    else if (p == 2)
+        sparse_scan_kernel<2><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
+    else
+        sparse_scan_kernel<NC_P_INF><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
+    sparse_emit_compact_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap,
+                                                                   ws, ws_stride);
+    const uint64_t groups = (cap + 31) / 32;
+    const dim3 pgrid((unsigned)((groups + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
+    sparse_pack_planes_kernel<<<pgrid, kBlockThreads, 0, stream>>>(batch, d, cap, s, ws,
+                                                                   ws_stride);
+    return launch_status();
+}
+
+nc_status nd_sparse_compact_compress(const float* x, size_t d, uint64_t keep_threshold,
+                                     float scale, int p, int s, uint64_t seed, uint32_t worker,
+                                     uint32_t* idx, uint32_t* planes, uint32_t* count, float* norm,
+                                     size_t cap, void* workspace, size_t workspace_bytes,
+                                     cudaStream_t stream) {
+    if (!x || !idx || !planes || !count || !norm) return NC_ERR_INVALID;
+    return nd_sparse_compact_compress_batch(&x, d, keep_threshold, scale, p, s, seed, &worker,
+                                            &idx, &planes, &count, &norm, cap, 1, workspace,
+                                            workspace_bytes, stream);
+}
+
+nc_status nd_sparse_compact_decode_accumulate(const uint32_t* idx, const uint32_t* planes,
+                                              const uint32_t* count, const float* norm, int s,
+                                              size_t d, size_t cap, float* acc,
+                                              cudaStream_t stream) {
+    if (!idx || !planes || !count || !norm || !acc || s < 1 || s > 8 || cap < 1)
+        return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > 0xFFFFFFFFull) return NC_ERR_INVALID;
+    if (!aligned16(idx) || !aligned16(planes) || !aligned32(acc) || !aligned4(count) ||
+        !aligned4(norm))
+        return NC_ERR_ALIGN;
+    const unsigned grid = (unsigned)((cap + kBlockThreads - 1) / kBlockThreads);
+    sparse_compact_decode_accumulate_kernel<<<grid, kBlockThreads, 0, stream>>>(
+        idx, planes, count, norm, s, d, cap, acc);
+    return launch_status();
+}
+
+}  // extern "C"
