@@ -159,8 +159,8 @@ class HotPath:
         self.out_sp = torch.empty(d, **f32)
         self.out_sum = torch.empty(d, **f32)
         # nc_compress_batch 1, nc_aggregate 1, nd_compress_batch 3, nd_aggregate 1,
-        # nd_sparse_compact_compress_batch 7, nd_sparse_compact_decode_accumulate n, nc_sum_fp32 1
-        self.launches_per_step = 1 + 1 + 3 + 1 + 7 + n + 1
+        # nd_sparse_compact_compress_batch 6, nd_sparse_compact_decode_accumulate n, nc_sum_fp32 1
+        self.launches_per_step = 1 + 1 + 3 + 1 + 6 + n + 1
         self.seed = 0
 
     def step(self, marks=None):

@@ -206,7 +206,7 @@ __device__ __forceinline__ float aggregate_element(const PackedPlanes& planes, c
 // out[j] = (init + v_0j) + v_1j + ... ; init = +0 (aggregate) or acc[j] (decode-accumulate).
 // grid: ceil(tiles / warps per block)
 template <bool kFromAcc>
-__global__ void __launch_bounds__(kBlockThreads)
+__global__ void __launch_bounds__(kBlockThreads, 5)
 nc_aggregate_kernel(const __grid_constant__ PackedPlanes planes, const int n, const uint64_t d,
                     float* __restrict__ out) {
     const int lane = threadIdx.x & 31;

@@ -256,8 +256,18 @@ __device__ __forceinline__ uint32_t level_code(uint32_t bits, uint32_t rnd, cons
     return min(t >> 23, sc.smax);
 }
 
+// level code from z = |x| * (rinv * 2^s) directly (see the fast path of the rounding kernel)
+__device__ __forceinline__ uint32_t level_code_scaled(uint32_t bits, uint32_t rnd, float rinv_s,
+                                                      uint32_t smax) {
+    const float z = __fmul_rn(fabsf(__uint_as_float(bits)), rinv_s);
+    float w = z;
+    if (z < 2.0f) w = __fmaf_rz(z, 0.5f, 1.0f);
+    const uint32_t t = __float_as_uint(w) + (~rnd & 0x7FFFFFu) - 0x3F800000u;
+    return min(t >> 23, smax);
+}
+
 // grid: ceil(tiles / warps per block)
-__global__ void __launch_bounds__(kBlockThreads)
+__global__ void __launch_bounds__(kBlockThreads, 5)
 nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d,
                      const uint64_t* __restrict__ off, const int B, const int s,
                      const __grid_constant__ PhiloxKeys keys,
@@ -281,8 +291,14 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
     }
     int b = (int)tile_bucket[tile];
 
-    if (full && __ldg(off + b + 1) >= base + kTile) {
-        const BucketScale sc = bucket_scale(norms[b], s);
+    // Fast path: the tile lies in one bucket.  z = fl32(fl32(|x| * rinv) * 2^s) is computed as
+    // fl32(|x| * (rinv * 2^s)): scaling by 2^s is exact, so the two agree whenever the inner
+    // product is a normal number, and when it is subnormal both give z < 2^-100, threshold 0 and
+    // level code 0.  If rinv * 2^s overflows (norm below 2^(s-126)) the general path is used.
+    const BucketScale sc0 = bucket_scale(norms[b], s);
+    const float rinv_s = __fmul_rn(sc0.rinv, pow2s);
+    if (full && __ldg(off + b + 1) >= base + kTile && rinv_s <= 3.40282347e38f) {
+        const BucketScale sc = sc0;
         uint32_t* lv = reinterpret_cast<uint32_t*>(level + (base >> 1));
         const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainDnat, keys);
         const uint32_t q_lo = (uint32_t)(base >> 2) + (uint32_t)(lane * 2);
@@ -301,7 +317,7 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
             uint32_t nib = 0;
 #pragma unroll
             for (int c = 7; c >= 0; --c) {
-                nib = (nib << 4) | level_code(u[it].v[c], rnd[c], sc, pow2s);
+                nib = (nib << 4) | level_code_scaled(u[it].v[c], rnd[c], rinv_s, sc.smax);
                 sbytes = __funnelshift_l(u[it].v[c], sbytes, 1);
             }
             st_stream_u32(lv + it * 32 + lane, nib);
