@@ -247,6 +247,32 @@ nc_status nd_sparse_compact_decode_accumulate(const uint32_t* idx, const uint32_
                                               size_t d, size_t cap, float* acc,
                                               cudaStream_t stream);
 
+/* ---- the paper's 8-bit wire format and integer aggregation ----------------------------------
+ * Experimental set-up appendix ("1 bit for the sign ... clip the exponents in the range -50~10 ...
+ * the remaining one bit is used to represent zeros", "64-bit integers to store the intermediate
+ * results") and the "fast aggregation" appendix (values restored as integers with one non-zero
+ * bit).  Code byte: bit 7 sign, bit 6 zero flag, bits 0..5 = exponent + 50 of C_nat(x) with the
+ * exponent clipped to [-50, 10] (+-inf and NaN clip to +-2^10).  Planes hold nc_exp_bytes(d) bytes. */
+
+/* Worker side: code[j] <- 8-bit code of C_nat(x_j) with the stream (seed, worker, j). */
+nc_status nc8_compress(const float* x, size_t d, uint64_t seed, uint32_t worker, uint8_t* code,
+                       cudaStream_t stream);
+nc_status nc8_compress_batch(const float* const* xs, size_t d, uint64_t seed,
+                             const uint32_t* workers, uint8_t* const* codes, int n,
+                             cudaStream_t stream);
+
+/* Master side: every code is restored as the 64-bit integer +-2^(exponent + 50) (0 for the zero
+ * flag), the n integers are added, out[j] <- fl32(sum) * 2^-50.  The result does not depend on the
+ * order of the workers.  Exact while |sum| < 2^63 (any n <= 7; any n if no entry is at 2^10). */
+nc_status nc8_aggregate(const uint8_t* const* codes, int n, size_t d, float* out,
+                        cudaStream_t stream);
+
+/* The same sum, compressed again by C_nat into the 8-bit format (Algorithm 1, g = C_M(Delta)):
+ * for the integer S with 2^e <= |S| < 2^(e+1) the code of +-2^(e-50) or +-2^(e+1-50), the upper one
+ * iff r23 < floor((|S| - 2^e) 2^23 / 2^e), r23 from the C_nat stream of (seed, master, j). */
+nc_status nc8_aggregate_compress(const uint8_t* const* codes, int n, size_t d, uint64_t seed,
+                                 uint32_t master, uint8_t* out_code, cudaStream_t stream);
+
 /* ---- host-buffer plumbing (no counterpart in the paper, where workers and master exchange
  * these buffers over a network) ------------------------------------------------------------- */
 

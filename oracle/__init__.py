@@ -316,3 +316,44 @@ def sparse_compact_decode_accumulate(idx, planes, count: int, nrm, s: int, acc) 
     assert acc.dtype == np.float32 and acc.flags.c_contiguous
     _sparse_compact_decode_accumulate(_p(idx, _u32p), _p(planes, _u32p), count, float(nrm), s,
                                       _p(acc, _f32p))
+
+
+_i64p = C.POINTER(C.c_int64)
+_nc8_compress = _sig("orc_nc8_compress", None, _f32p, C.c_uint64, C.c_uint64, C.c_uint64,
+                     C.c_uint32, _u8p)
+_nc8_decode = _sig("orc_nc8_decode", None, _u8p, C.c_uint64, _f32p)
+_nc8_aggregate = _sig("orc_nc8_aggregate", None, C.POINTER(_u8p), C.c_int, C.c_uint64, _f32p,
+                      _i64p)
+_nc8_aggregate_compress = _sig("orc_nc8_aggregate_compress", None, C.POINTER(_u8p), C.c_int,
+                               C.c_uint64, C.c_uint64, C.c_uint32, _u8p)
+
+
+def nc8_compress(x, seed: int, worker: int, j0: int = 0) -> np.ndarray:
+    """C_nat followed by the paper's 8-bit code (sign, zero flag, exponent clipped to -50..10)."""
+    x = _arr(x, np.float32)
+    out = np.zeros(x.size, np.uint8)
+    _nc8_compress(_p(x, _f32p), x.size, j0, seed, worker, _p(out, _u8p))
+    return out
+
+
+def nc8_decode(code) -> np.ndarray:
+    code = _arr(code, np.uint8)
+    out = np.empty(code.size, np.float32)
+    _nc8_decode(_p(code, _u8p), code.size, _p(out, _f32p))
+    return out
+
+
+def nc8_aggregate(codes, d: int):
+    """Integer aggregation; returns (fp32 result, exact int64 sums)."""
+    codes = [_arr(c, np.uint8) for c in codes]
+    out = np.empty(d, np.float32)
+    sums = np.empty(d, np.int64)
+    _nc8_aggregate(_ptr_array(codes, _u8p), len(codes), d, _p(out, _f32p), _p(sums, _i64p))
+    return out, sums
+
+
+def nc8_aggregate_compress(codes, d: int, seed: int, master: int) -> np.ndarray:
+    codes = [_arr(c, np.uint8) for c in codes]
+    out = np.zeros(d, np.uint8)
+    _nc8_aggregate_compress(_ptr_array(codes, _u8p), len(codes), d, seed, master, _p(out, _u8p))
+    return out

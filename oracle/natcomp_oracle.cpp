@@ -563,4 +563,73 @@ void orc_sparse_compact_decode_accumulate(const uint32_t* idx, const uint32_t* p
     }
 }
 
+// ---- the paper's 8-bit wire format and integer aggregation ---------------------------------
+// Experimental set-up appendix: 1 sign bit, exponents clipped to [-50, 10] (6 bits), one bit
+// that flags zeros; the aggregator restores the values as 64-bit integers and adds them.
+// Byte layout chosen here: bit 7 sign, bit 6 zero flag, bits 0..5 exponent + 50.
+static uint8_t code8_of_value(double value) {
+    const uint8_t sign = std::signbit(value) ? 0x80 : 0x00;
+    const double a = std::fabs(value);
+    if (a == 0.0) return (uint8_t)(sign | 0x40);
+    int e = std::isinf(a) ? 1000 : std::ilogb(a);
+    if (e < -50) e = -50;
+    if (e > 10) e = 10;
+    return (uint8_t)(sign | (uint8_t)(e + 50));
+}
+
+static long long restore8_int(uint8_t c) {
+    if (c & 0x40) return 0;
+    const long long v = (long long)1 << (c & 0x3F);
+    return (c & 0x80) ? -v : v;
+}
+
+void orc_nc8_compress(const float* x, uint64_t d, uint64_t j0, uint64_t seed, uint32_t worker,
+                      uint8_t* code) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)d; ++i) {
+        const uint32_t r23 = stream_word(seed, worker, 0u, j0 + (uint64_t)i) & 0x7FFFFFu;
+        code[i] = code8_of_value(cnat_value(x[i], r23));
+    }
+}
+
+// decoded values +-2^(e-50) (0 for the zero flag)
+void orc_nc8_decode(const uint8_t* code, uint64_t d, float* out) {
+    for (uint64_t i = 0; i < d; ++i)
+        out[i] = (float)std::ldexp((double)restore8_int(code[i]), -50);
+}
+
+// exact integer sums (returned as well, for the pins) and their fp32 value fl32(sum) * 2^-50
+void orc_nc8_aggregate(const uint8_t* const* codes, int n, uint64_t d, float* out,
+                       int64_t* sums) {
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < (int64_t)d; ++j) {
+        long long acc = 0;
+        for (int i = 0; i < n; ++i) acc += restore8_int(codes[i][j]);
+        if (sums) sums[j] = acc;
+        out[j] = (float)acc * 0x1p-50f;
+    }
+}
+
+// C_nat of the integer sum S (value S 2^-50), Def. 1 on exact integers: floor power 2^e, ceil
+// power 2^(e+1), up-probability (|S| - 2^e) / 2^e, the draw "up iff r23 < floor(p 2^23)".
+void orc_nc8_aggregate_compress(const uint8_t* const* codes, int n, uint64_t d, uint64_t seed,
+                                uint32_t master, uint8_t* out_code) {
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < (int64_t)d; ++j) {
+        long long acc = 0;
+        for (int i = 0; i < n; ++i) acc += restore8_int(codes[i][j]);
+        if (acc == 0) { out_code[j] = 0x40; continue; }
+        const bool neg = acc < 0;
+        const unsigned __int128 a = neg ? (unsigned __int128)(-(__int128)acc) : (unsigned __int128)acc;
+        int e = 0;
+        while ((a >> (e + 1)) != 0) ++e;
+        const unsigned __int128 lo = (unsigned __int128)1 << e;
+        const uint64_t thr = (uint64_t)(((a - lo) << 23) >> e);       // floor(p_up * 2^23)
+        const uint32_t r23 = stream_word(seed, master, 0u, (uint64_t)j) & 0x7FFFFFu;
+        const int e_out = e + ((uint64_t)r23 < thr ? 1 : 0);
+        const double value = std::ldexp(neg ? -1.0 : 1.0, e_out - 50);
+        out_code[j] = code8_of_value(value);
+    }
+}
+
 }  // extern "C"

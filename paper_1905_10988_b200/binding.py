@@ -36,7 +36,8 @@ EXPORTS = (
     "nd_sparse_compress_batch", "nd_static_scratch_bytes", "nd_compress_static",
     "nc_aggregate_compress", "nc_compress_nearest", "nc_compress_nearest_batch",
     "nd_sparse_plane_bytes", "nd_sparse_compact_compress", "nd_sparse_compact_compress_batch",
-    "nd_sparse_compact_decode_accumulate",
+    "nd_sparse_compact_decode_accumulate", "nc8_compress", "nc8_compress_batch", "nc8_aggregate",
+    "nc8_aggregate_compress",
 )
 
 
@@ -188,6 +189,34 @@ def nd_sparse_compact_decode_accumulate(idx, planes, count, norm, s, d, cap, acc
     _check("nd_sparse_compact_decode_accumulate",
            _nd_sparse_compact_decode_accumulate(_ptr(idx), _ptr(planes), _ptr(count), _ptr(norm),
                                                 s, d, cap, _ptr(acc), _stream(stream)))
+
+
+_nc8_compress = _sig("nc8_compress", C.c_int, _vp, _sz, C.c_uint64, C.c_uint32, _vp, _vp)
+_nc8_compress_batch = _sig("nc8_compress_batch", C.c_int, C.POINTER(_vp), _sz, C.c_uint64,
+                           C.POINTER(C.c_uint32), C.POINTER(_vp), C.c_int, _vp)
+_nc8_aggregate = _sig("nc8_aggregate", C.c_int, C.POINTER(_vp), C.c_int, _sz, _vp, _vp)
+_nc8_aggregate_compress = _sig("nc8_aggregate_compress", C.c_int, C.POINTER(_vp), C.c_int, _sz,
+                               C.c_uint64, C.c_uint32, _vp, _vp)
+
+
+def nc8_compress(x, d, seed, worker, code, stream=None) -> None:
+    _check("nc8_compress", _nc8_compress(_ptr(x), d, seed, worker, _ptr(code), _stream(stream)))
+
+
+def nc8_compress_batch(xs, d, seed, workers, codes, n, stream=None) -> None:
+    w = (C.c_uint32 * n)(*[int(v) for v in workers])
+    _check("nc8_compress_batch", _nc8_compress_batch(_ptrs(xs), d, seed, w, _ptrs(codes), n,
+                                                     _stream(stream)))
+
+
+def nc8_aggregate(codes, n, d, out, stream=None) -> None:
+    _check("nc8_aggregate", _nc8_aggregate(_ptrs(codes), n, d, _ptr(out), _stream(stream)))
+
+
+def nc8_aggregate_compress(codes, n, d, seed, master, out_code, stream=None) -> None:
+    _check("nc8_aggregate_compress",
+           _nc8_aggregate_compress(_ptrs(codes), n, d, seed, master, _ptr(out_code),
+                                   _stream(stream)))
 
 
 _nd_static_scratch_bytes = _sig("nd_static_scratch_bytes", _sz)

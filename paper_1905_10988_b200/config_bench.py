@@ -68,6 +68,11 @@ def run_cnat(config, n, d, make_vector, iters, peak, with_sum=True):
     _report(config, "nc_aggregate", m, b, d, d * (1.125 * n + 4), peak)
     m, b = _time(lambda: nc.nc_aggregate_compress(es, ss, n, d, 0, 0xFFFFFFFF, ge, gs), iters)
     _report(config, "nc_aggregate_compress", m, b, d, d * (1.125 * n + 1.125), peak)
+    # the paper's 8-bit wire format with integer (order-independent) aggregation
+    m, b = _time(lambda: nc.nc8_compress_batch(xs, d, 0, workers, es, n), iters)
+    _report(config, "nc8_compress_batch (8-bit codes)", m, b, n * d, n * d * 5.0, peak)
+    m, b = _time(lambda: nc.nc8_aggregate(es, n, d, out), iters)
+    _report(config, "nc8_aggregate (int64 sums)", m, b, d, d * (1.0 * n + 4), peak)
     if with_sum:
         m, b = _time(lambda: nc.nc_sum_fp32(xs, n, d, out), iters)
         _report(config, "nc_sum_fp32 (uncompressed reference point)", m, b, d, d * (4 * n + 4),
