@@ -93,3 +93,50 @@ def test_bidirectional_round_on_config1():
     # E||C_M(sum C(x_i)) - sum x_i||^2 <= (1/8) E||sum C(x_i)||^2 + (1/8) sum ||x_i||^2
     s2 = float((exact ** 2).sum())
     assert err2 <= (1 / 8) * (s2 + x2 / 8) + x2 / 8 + 0.02 * x2
+
+
+def test_dithering_with_naturally_compressed_norm():
+    # Def. 3 with C = C_nat on the norm (the variant the paper proposes for in-network
+    # aggregation: the norm travels as an 8-bit exponent and decoding is exponent addition).
+    # Recipe with the existing calls: nd_compress, then nc_compress on the vector of norms,
+    # decode it on the master, nd_aggregate with the decoded (power-of-two) norms.
+    rng = np.random.default_rng(3)
+    n, d, p, s = 3, 50_000, 2, 8
+    off = workloads.small_bucket_table(d, seed=2)
+    B = len(off) - 1
+    off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
+    xs = [(rng.standard_normal(d) * 1e-3).astype(np.float32) for _ in range(n)]
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    norms, levels, signs, tx = [], [], [], []
+    ws_bytes = nc.nd_workspace_bytes(d, B)
+    ws = torch.empty(ws_bytes, **u8)
+    ref_norms, ref_levels, ref_signs = [], [], []
+    for w in range(n):
+        nm = torch.empty(B, dtype=torch.float32, device="cuda")
+        lv = torch.empty(nc.nd_level_bytes(d), **u8)
+        sg = torch.empty(nc.nc_sign_bytes(d), **u8)
+        nc.nd_compress(dev(xs[w]), d, off_dev, B, p, s, 1, w, nm, lv, sg, ws, ws_bytes)
+        # the norm vector goes through C_nat with its own worker id (here 1000 + w)
+        ne = torch.empty(nc.nc_exp_bytes(B), **u8)
+        ns = torch.empty(nc.nc_sign_bytes(B), **u8)
+        nc.nc_compress(nm, B, 1, 1000 + w, ne, ns)
+        dec = torch.zeros(B, dtype=torch.float32, device="cuda")
+        nc.nc_decode_accumulate(ne, ns, B, dec)
+        norms.append(nm); levels.append(lv); signs.append(sg); tx.append(dec)
+        # oracle side of the same recipe
+        gn = nm.cpu().numpy()
+        r = oracle.nd_compress(xs[w], off, p, s, 1, w, given_norms=gn)
+        e_ref, s_ref = oracle.nc_compress(gn, 1, 1000 + w)
+        dn = np.zeros(B, np.float32)
+        oracle.nc_decode_accumulate(e_ref, s_ref, dn)
+        ref_norms.append(dn); ref_levels.append(r[1]); ref_signs.append(r[2])
+        assert np.array_equal(dec.cpu().numpy(), dn)
+        # a compressed norm is a power of two within a factor two of the norm
+        ratio = dn / gn
+        assert np.all((ratio > 0.5) & (ratio < 2.0))
+        assert np.all(np.frexp(dn)[0] == 0.5)
+    out = torch.empty(d, dtype=torch.float32, device="cuda")
+    nc.nd_aggregate(tx, levels, signs, n, d, off_dev, B, s, out)
+    torch.cuda.synchronize()
+    want = oracle.nd_aggregate(ref_norms, ref_levels, ref_signs, off, s, d)
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), want.view(np.uint32))
