@@ -357,3 +357,57 @@ def nc8_aggregate_compress(codes, d: int, seed: int, master: int) -> np.ndarray:
     out = np.zeros(d, np.uint8)
     _nc8_aggregate_compress(_ptr_array(codes, _u8p), len(codes), d, seed, master, _p(out, _u8p))
     return out
+
+
+_select_smallest = _sig("orc_select_smallest", None, _u32p, C.c_uint64, C.c_uint64, _u8p)
+_sparse_exact_compress = _sig("orc_sparse_exact_compress", C.c_uint64, _f32p, C.c_uint64,
+                              C.c_uint64, C.c_float, C.c_int, C.c_int, C.c_uint64, C.c_uint32,
+                              _u32p, _u32p, C.c_uint64, _f32p)
+_topk_compress = _sig("orc_topk_compress", None, _f32p, C.c_uint64, C.c_uint64, C.c_uint64,
+                      C.c_uint32, _u32p, _u8p, _u32p)
+_topk_decode_accumulate = _sig("orc_topk_decode_accumulate", None, _u32p, _u8p, _u32p, C.c_uint64,
+                               _f32p)
+
+
+def select_smallest(keys, q: int) -> np.ndarray:
+    """mask of the q smallest keys, ties to the lower index."""
+    keys = _arr(keys, np.uint32)
+    mask = np.zeros(keys.size, np.uint8)
+    _select_smallest(_p(keys, _u32p), keys.size, q, _p(mask, _u8p))
+    return mask
+
+
+def sparse_exact_compress(x, q: int, scale: float, p: int, s: int, seed: int, worker: int,
+                          cap=None):
+    """S^q with exactly q kept coordinates, then D_nat, compact form."""
+    x = _arr(x, np.float32)
+    d = x.size
+    if cap is None:
+        cap = d
+    idx = np.zeros(cap, np.uint32)
+    planes = np.zeros(((cap + 31) // 32) * code_bits(s), np.uint32)
+    nrm = C.c_float(0.0)
+    count = _sparse_exact_compress(_p(x, _f32p), d, q, scale, p, s, seed, worker, _p(idx, _u32p),
+                                   _p(planes, _u32p), cap, C.byref(nrm))
+    return idx[:min(int(count), cap)], planes, int(count), np.float32(nrm.value)
+
+
+def topk_compress(x, K: int, seed: int, worker: int):
+    """TopK by magnitude then C_nat: ascending indices, exponent bytes, sign words."""
+    x = _arr(x, np.float32)
+    listed = min(K, x.size)
+    idx = np.zeros(listed, np.uint32)
+    exp = np.zeros(listed, np.uint8)
+    sign = np.zeros((listed + 31) // 32, np.uint32)
+    _topk_compress(_p(x, _f32p), x.size, K, seed, worker, _p(idx, _u32p), _p(exp, _u8p),
+                   _p(sign, _u32p))
+    return idx, exp, sign
+
+
+def topk_decode_accumulate(idx, exp, sign, acc) -> None:
+    idx = _arr(idx, np.uint32)
+    exp = _arr(exp, np.uint8)
+    sign = _arr(sign, np.uint32)
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    _topk_decode_accumulate(_p(idx, _u32p), _p(exp, _u8p), _p(sign, _u32p), idx.size,
+                            _p(acc, _f32p))

@@ -30,11 +30,13 @@
 //   2^127<|t|<inf  -> never rounded up: +-2^127 (saturation, biased)
 //   +-inf, NaN     -> +-inf (exponent byte 255, sign bit kept)
 
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
 #include <cstddef>
 #include <limits>
+#include <vector>
 
 #ifdef _OPENMP
 #include <omp.h>
@@ -629,6 +631,103 @@ void orc_nc8_aggregate_compress(const uint8_t* const* codes, int n, uint64_t d, 
         const int e_out = e + ((uint64_t)r23 < thr ? 1 : 0);
         const double value = std::ldexp(neg ? -1.0 : 1.0, e_out - 50);
         out_code[j] = code8_of_value(value);
+    }
+}
+
+// ---- selection of exactly q coordinates -----------------------------------------------------
+// mask[j] = 1 for the q coordinates with the smallest keys, ties going to the lower index.
+// With i.i.d. uniform keys this is a uniformly random subset of size q, which is the mask xi of
+// the sparsifier definition (S^q: exactly q non-zeros).  Written as the definition: sort.
+void orc_select_smallest(const uint32_t* keys, uint64_t d, uint64_t q, uint8_t* mask) {
+    std::vector<uint64_t> order(d);
+    for (uint64_t j = 0; j < d; ++j) order[j] = j;
+    std::stable_sort(order.begin(), order.end(),
+                     [&](uint64_t a, uint64_t b) { return keys[a] < keys[b]; });
+    std::memset(mask, 0, (size_t)d);
+    for (uint64_t k = 0; k < q && k < d; ++k) mask[order[k]] = 1;
+}
+
+// S^q with exactly q kept coordinates (keys = the domain-2 stream words), x' = (d / q) x on the
+// kept coordinates (scale passed in as binary32), then D_nat^{p,s} in the compact form of
+// orc_sparse_compact_compress.  Returns the number of listed entries.
+uint64_t orc_sparse_exact_compress(const float* x, uint64_t d, uint64_t q, float scale, int p,
+                                   int s, uint64_t seed, uint32_t worker, uint32_t* idx,
+                                   uint32_t* planes, uint64_t cap, float* norm_out) {
+    std::vector<uint32_t> keys(d);
+    for (uint64_t j = 0; j < d; ++j) keys[j] = stream_word(seed, worker, 2u, j);
+    std::vector<uint8_t> mask(d);
+    orc_select_smallest(keys.data(), d, q, mask.data());
+    double acc = 0.0;
+    bool saw_nan = false;
+    for (uint64_t j = 0; j < d; ++j) {
+        if (!mask[j]) continue;
+        const float xs = scale * x[j];
+        const double a = std::fabs((double)xs);
+        if (std::isnan(a)) saw_nan = true;
+        if (p == 1) acc += a;
+        else if (p == 2) acc += a * a;
+        else if (a > acc) acc = a;
+    }
+    if (p == 2) acc = std::sqrt(acc);
+    const float norm = saw_nan ? std::numeric_limits<float>::quiet_NaN() : (float)acc;
+    *norm_out = norm;
+    const int nb = bits_for(s);
+    std::memset(planes, 0, (size_t)(((cap + 31) / 32) * (uint64_t)(nb + 1)) * 4);
+    if (norm_degenerate(norm)) return 0;
+    const float rinv = 1.0f / norm;
+    uint64_t k = 0;
+    for (uint64_t j = 0; j < d; ++j) {
+        if (!mask[j]) continue;
+        const float xs = scale * x[j];
+        const float yf = std::fabs(xs) * rinv;
+        const uint32_t r23 = stream_word(seed, worker, 1u, j) & 0x7FFFFFu;
+        const int c = nd_level_code((double)yf, s, r23);
+        if (c == 0) continue;
+        if (k < cap) {
+            const uint32_t code = ((std::signbit(xs) ? 1u : 0u) << nb) | (uint32_t)(c - 1);
+            idx[k] = (uint32_t)j;
+            for (int b = 0; b <= nb; ++b)
+                planes[(k / 32) * (uint64_t)(nb + 1) + (uint64_t)b] |= ((code >> b) & 1u) << (k % 32);
+        }
+        ++k;
+    }
+    return k;
+}
+
+// TopK followed by C_nat (the paper's TopK-C_nat of the experiments section): the K entries of
+// largest magnitude (compared as binary32 bit patterns with the sign cleared, so NaN patterns
+// rank above inf; equal magnitudes: lower index first), listed in ascending index order, each
+// with the 9-bit code of C_nat(x_j) drawn from the stream (seed, worker, j).
+// exp: one byte per listed entry; sign: bit (k mod 32) of word k / 32.
+void orc_topk_compress(const float* x, uint64_t d, uint64_t K, uint64_t seed, uint32_t worker,
+                       uint32_t* idx, uint8_t* exp, uint32_t* sign) {
+    std::vector<uint32_t> keys(d);
+    for (uint64_t j = 0; j < d; ++j) {
+        uint32_t bits;
+        std::memcpy(&bits, &x[j], 4);
+        keys[j] = ~(bits & 0x7FFFFFFFu);            // largest magnitude = smallest key
+    }
+    std::vector<uint8_t> mask(d);
+    orc_select_smallest(keys.data(), d, K, mask.data());
+    const uint64_t listed = K < d ? K : d;
+    std::memset(sign, 0, (size_t)((listed + 31) / 32) * 4);
+    uint64_t k = 0;
+    for (uint64_t j = 0; j < d; ++j) {
+        if (!mask[j]) continue;
+        const uint32_t r23 = stream_word(seed, worker, 0u, j) & 0x7FFFFFu;
+        uint32_t sb;
+        cnat_code(cnat_value(x[j], r23), &exp[k], &sb);
+        idx[k] = (uint32_t)j;
+        sign[k / 32] |= sb << (k % 32);
+        ++k;
+    }
+}
+
+void orc_topk_decode_accumulate(const uint32_t* idx, const uint8_t* exp, const uint32_t* sign,
+                                uint64_t count, float* acc) {
+    for (uint64_t k = 0; k < count; ++k) {
+        const float v = cnat_decode(exp[k], (sign[k / 32] >> (k % 32)) & 1u);
+        acc[idx[k]] = acc[idx[k]] + v;
     }
 }
 
