@@ -273,6 +273,39 @@ nc_status nc8_aggregate(const uint8_t* const* codes, int n, size_t d, float* out
 nc_status nc8_aggregate_compress(const uint8_t* const* codes, int n, size_t d, uint64_t seed,
                                  uint32_t master, uint8_t* out_code, cudaStream_t stream);
 
+/* ---- exactly q kept coordinates: S^q then D_nat, and TopK then C_nat -------------------------
+ * The sparsifier definition of the appendix with exactly q non-zeros ("S^q": xi a uniformly random
+ * subset of size q, probabilities q/d), composed with D_nat^{p,s} (Def. 3, Thm. 3), and the
+ * TopK-C_nat composition of the experiments.  The random subset is the q coordinates with the
+ * smallest words of the selection stream (seed, worker, domain 2, j), equal words by ascending j;
+ * TopK takes the K largest |x_j| compared as binary32 bit patterns with the sign cleared (NaN
+ * patterns rank above inf), equal magnitudes by ascending j.  Device pointers; x 32-byte aligned,
+ * the other buffers 16-byte; workspace: nc_select_workspace_bytes(d, cap) (cap = K for TopK). */
+size_t nc_select_workspace_bytes(size_t d, size_t cap);
+
+/* S^q then D_nat^{p,s}: x'_j = scale * x_j on the q selected coordinates (the caller passes
+ * scale = fl32(d / q)), norm = ||x'||_p over the selected entries, levels drawn from the dithering
+ * stream (domain 1) of coordinate j.  Output in the compact format of nd_sparse_compact_compress
+ * (idx, planes, count, norm, cap with the same meaning), decoded by
+ * nd_sparse_compact_decode_accumulate.  q > d is taken as d; q = 0 gives count 0 and norm 0. */
+nc_status nd_sparse_exact_compress(const float* x, size_t d, uint64_t q, float scale, int p, int s,
+                                   uint64_t seed, uint32_t worker, uint32_t* idx,
+                                   uint32_t* planes, uint32_t* count, float* norm, size_t cap,
+                                   void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/* TopK then C_nat (Def. 1): min(K, d) entries listed by ascending coordinate: idx[k] = j,
+ * exp[k] = exponent byte of C_nat(x_j) drawn from the stream (seed, worker, domain 0, j) (the
+ * same draw nc_compress makes for coordinate j), sign: bit k mod 32 of word k / 32.
+ * idx: uint32[K]; exp: K bytes; sign: ceil(K / 32) words.  K = 0 or d = 0 writes nothing. */
+nc_status nc_topk_compress(const float* x, size_t d, uint64_t K, uint64_t seed, uint32_t worker,
+                           uint32_t* idx, uint8_t* exp, uint32_t* sign, void* workspace,
+                           size_t workspace_bytes, cudaStream_t stream);
+
+/* Master side: acc[idx[k]] <- acc[idx[k]] + decoded value, k < count (host integer); indices
+ * >= d are skipped.  Indices of one list are distinct, so no atomics are needed. */
+nc_status nc_topk_decode_accumulate(const uint32_t* idx, const uint8_t* exp, const uint32_t* sign,
+                                    size_t count, size_t d, float* acc, cudaStream_t stream);
+
 /* ---- host-buffer plumbing (no counterpart in the paper, where workers and master exchange
  * these buffers over a network) ------------------------------------------------------------- */
 

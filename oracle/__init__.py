@@ -362,7 +362,7 @@ def nc8_aggregate_compress(codes, d: int, seed: int, master: int) -> np.ndarray:
 _select_smallest = _sig("orc_select_smallest", None, _u32p, C.c_uint64, C.c_uint64, _u8p)
 _sparse_exact_compress = _sig("orc_sparse_exact_compress", C.c_uint64, _f32p, C.c_uint64,
                               C.c_uint64, C.c_float, C.c_int, C.c_int, C.c_uint64, C.c_uint32,
-                              _u32p, _u32p, C.c_uint64, _f32p)
+                              _u32p, _u32p, C.c_uint64, _f32p, _f32p)
 _topk_compress = _sig("orc_topk_compress", None, _f32p, C.c_uint64, C.c_uint64, C.c_uint64,
                       C.c_uint32, _u32p, _u8p, _u32p)
 _topk_decode_accumulate = _sig("orc_topk_decode_accumulate", None, _u32p, _u8p, _u32p, C.c_uint64,
@@ -378,7 +378,7 @@ def select_smallest(keys, q: int) -> np.ndarray:
 
 
 def sparse_exact_compress(x, q: int, scale: float, p: int, s: int, seed: int, worker: int,
-                          cap=None):
+                          cap=None, given_norm=None):
     """S^q with exactly q kept coordinates, then D_nat, compact form."""
     x = _arr(x, np.float32)
     d = x.size
@@ -387,8 +387,9 @@ def sparse_exact_compress(x, q: int, scale: float, p: int, s: int, seed: int, wo
     idx = np.zeros(cap, np.uint32)
     planes = np.zeros(((cap + 31) // 32) * code_bits(s), np.uint32)
     nrm = C.c_float(0.0)
+    gn = None if given_norm is None else C.byref(C.c_float(float(given_norm)))
     count = _sparse_exact_compress(_p(x, _f32p), d, q, scale, p, s, seed, worker, _p(idx, _u32p),
-                                   _p(planes, _u32p), cap, C.byref(nrm))
+                                   _p(planes, _u32p), cap, C.byref(nrm), gn)
     return idx[:min(int(count), cap)], planes, int(count), np.float32(nrm.value)
 
 

@@ -652,7 +652,8 @@ void orc_select_smallest(const uint32_t* keys, uint64_t d, uint64_t q, uint8_t* 
 // orc_sparse_compact_compress.  Returns the number of listed entries.
 uint64_t orc_sparse_exact_compress(const float* x, uint64_t d, uint64_t q, float scale, int p,
                                    int s, uint64_t seed, uint32_t worker, uint32_t* idx,
-                                   uint32_t* planes, uint64_t cap, float* norm_out) {
+                                   uint32_t* planes, uint64_t cap, float* norm_out,
+                                   const float* given_norm) {
     std::vector<uint32_t> keys(d);
     for (uint64_t j = 0; j < d; ++j) keys[j] = stream_word(seed, worker, 2u, j);
     std::vector<uint8_t> mask(d);
@@ -669,7 +670,10 @@ uint64_t orc_sparse_exact_compress(const float* x, uint64_t d, uint64_t q, float
         else if (a > acc) acc = a;
     }
     if (p == 2) acc = std::sqrt(acc);
-    const float norm = saw_nan ? std::numeric_limits<float>::quiet_NaN() : (float)acc;
+    // given_norm: round against a norm computed elsewhere (binary32), for checking the level
+    // codes of an implementation whose norm differs in the last bits by summation order
+    const float norm = given_norm ? *given_norm
+                     : saw_nan ? std::numeric_limits<float>::quiet_NaN() : (float)acc;
     *norm_out = norm;
     const int nb = bits_for(s);
     std::memset(planes, 0, (size_t)(((cap + 31) / 32) * (uint64_t)(nb + 1)) * 4);

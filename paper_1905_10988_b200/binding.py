@@ -37,7 +37,8 @@ EXPORTS = (
     "nc_aggregate_compress", "nc_compress_nearest", "nc_compress_nearest_batch",
     "nd_sparse_plane_bytes", "nd_sparse_compact_compress", "nd_sparse_compact_compress_batch",
     "nd_sparse_compact_decode_accumulate", "nc8_compress", "nc8_compress_batch", "nc8_aggregate",
-    "nc8_aggregate_compress",
+    "nc8_aggregate_compress", "nc_select_workspace_bytes", "nd_sparse_exact_compress",
+    "nc_topk_compress", "nc_topk_decode_accumulate",
 )
 
 
@@ -362,3 +363,39 @@ def nd_sparse_decode_accumulate(idx, codes, count, norm, s, d, cap, acc, stream=
     _check("nd_sparse_decode_accumulate",
            _nd_sparse_decode_accumulate(_ptr(idx), _ptr(codes), _ptr(count), _ptr(norm), s, d,
                                         cap, _ptr(acc), _stream(stream)))
+
+
+# ---- exactly q kept coordinates (S^q then D_nat) and TopK then C_nat ----------------------
+_nc_select_workspace_bytes = _sig("nc_select_workspace_bytes", _sz, _sz, _sz)
+_nd_sparse_exact_compress = _sig("nd_sparse_exact_compress", C.c_int, _vp, _sz, C.c_uint64,
+                                 C.c_float, C.c_int, C.c_int, C.c_uint64, C.c_uint32, _vp, _vp,
+                                 _vp, _vp, _sz, _vp, _sz, _vp)
+_nc_topk_compress = _sig("nc_topk_compress", C.c_int, _vp, _sz, C.c_uint64, C.c_uint64,
+                         C.c_uint32, _vp, _vp, _vp, _vp, _sz, _vp)
+_nc_topk_decode_accumulate = _sig("nc_topk_decode_accumulate", C.c_int, _vp, _vp, _vp, _sz, _sz,
+                                  _vp, _vp)
+
+
+def nc_select_workspace_bytes(d: int, cap: int) -> int:
+    return int(_nc_select_workspace_bytes(d, cap))
+
+
+def nd_sparse_exact_compress(x, d, q, scale, p, s, seed, worker, idx, planes, count, norm, cap,
+                             workspace, workspace_bytes, stream=None) -> None:
+    _check("nd_sparse_exact_compress",
+           _nd_sparse_exact_compress(_ptr(x), d, q, scale, p, s, seed, worker, _ptr(idx),
+                                     _ptr(planes), _ptr(count), _ptr(norm), cap, _ptr(workspace),
+                                     workspace_bytes, _stream(stream)))
+
+
+def nc_topk_compress(x, d, K, seed, worker, idx, exp, sign, workspace, workspace_bytes,
+                     stream=None) -> None:
+    _check("nc_topk_compress",
+           _nc_topk_compress(_ptr(x), d, K, seed, worker, _ptr(idx), _ptr(exp), _ptr(sign),
+                             _ptr(workspace), workspace_bytes, _stream(stream)))
+
+
+def nc_topk_decode_accumulate(idx, exp, sign, count, d, acc, stream=None) -> None:
+    _check("nc_topk_decode_accumulate",
+           _nc_topk_decode_accumulate(_ptr(idx), _ptr(exp), _ptr(sign), count, d, _ptr(acc),
+                                      _stream(stream)))

@@ -150,6 +150,26 @@ def run_sparse(config, n, d, iters, peak, s=4):
     m, b = _time(accumulate_compact, iters)
     _report(config, "nd_sparse_compact_decode_accumulate x n", m, b, listed, listed * 68.4, peak)
 
+    # exactly q = d / 100 kept coordinates (radix select over the selection words), one worker
+    q = d // 100
+    sel_bytes = nc.nc_select_workspace_bytes(d, cap)
+    sel_ws = torch.empty(sel_bytes, **u8)
+    m, b = _time(lambda: nc.nd_sparse_exact_compress(xs[0], d, q, scale, nc.P_INF, s, 0, 0, idx[0],
+                                                     planes[0], count[0], norm[0], cap, sel_ws,
+                                                     sel_bytes), iters)
+    _report(config, "nd_sparse_exact_compress (1 worker)", m, b, d, q * 96.0, peak,
+            {"Gcoord_per_s": round(d / m / 1e6, 1),
+             "note": "four passes over the selection stream (3 digit histograms + mark)"})
+    # TopK then C_nat, K = d / 100, one worker: x is read four times (3 histograms + mark)
+    K = q
+    tidx = torch.empty(K, dtype=torch.int32, device=dev)
+    texp = torch.empty(K, **u8)
+    tsign = torch.empty(4 * ((K + 31) // 32) + 16, **u8)
+    m, b = _time(lambda: nc.nc_topk_compress(xs[0], d, K, 0, 0, tidx, texp, tsign, sel_ws,
+                                             sel_bytes), iters)
+    _report(config, "nc_topk_compress (1 worker)", m, b, d, d * 4.0 + K * 5.125, peak,
+            {"Gcoord_per_s": round(d / m / 1e6, 1), "hbm_bytes_actually_read": d * 16})
+
 
 def main():
     ap = argparse.ArgumentParser()

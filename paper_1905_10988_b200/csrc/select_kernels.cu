@@ -1,0 +1,527 @@
+// Selection of exactly q coordinates on the device, for sm_100a:
+//   * the sparsifier with exactly q non-zeros (the paper's S^q: a uniformly random subset of
+//     size q; here the q coordinates with the smallest selection-stream words), followed by
+//     D_nat^{p,s} of Def. 3 in the compact list format;
+//   * TopK followed by C_nat (the "TopK-C_nat" composition of the experiments): the K entries of
+//     largest magnitude, each with the 9-bit code of Def. 1.
+//
+// Both are "the q smallest 32-bit keys, equal keys by ascending index" (key = the stream word,
+// or the complemented magnitude bits).  Most-significant-digit radix select, no sort and no
+// waiting between blocks:
+//   hist x3   : histogram of the next digit (11, 11, 10 bits) over the keys that match the
+//               digits fixed so far; per-block shared-memory histogram, flushed with integer atomics
+//   choose x3 : one block finds the digit bin holding the q-th key and fixes it
+//   mark      : per 1024-element tile the masks "key < T" and "key == T" (T = the q-th key)
+//   scan      : exclusive offsets of the per-block counts of "== T"
+//   resolve   : final mask = "< T" plus the first r of the "== T" in index order; per-block
+//               kept counts (and norm partials for the sparsifier)
+// then the compaction kernels shared with the independent-selection sparsifier, or the TopK emit.
+// Keys are recomputed (Philox) or re-read (x) in every pass; nothing of size d except the two
+// bit masks is stored.
+#include "sparse_common.cuh"
+
+namespace natcomp {
+
+constexpr int kSelBins = 2048;
+constexpr int kSelPasses = 3;
+
+__host__ __device__ constexpr int sel_shift(int pass) { return pass == 0 ? 21 : pass == 1 ? 10 : 0; }
+__host__ __device__ constexpr int sel_bins(int pass) { return pass == 2 ? 1024 : 2048; }
+// mask of the key bits fixed before this pass
+__host__ __device__ constexpr uint32_t sel_fixed(int pass) {
+    return pass == 0 ? 0u : pass == 1 ? 0xFFE00000u : 0xFFFFFC00u;
+}
+
+struct SelectState {
+    uint32_t prefix;        // digits fixed so far; after the last pass the q-th smallest key T
+    uint32_t pad;
+    uint64_t remaining;     // how many keys to take among those matching the prefix
+};
+
+struct SelectWorkspace {
+    uint32_t* eqmask;       // tiles * 32 words
+    uint32_t* eq_block;     // one per block of 8 tiles
+    uint32_t* hist;         // kSelPasses * kSelBins
+    SelectState* state;
+    uint32_t* count;        // listed entries (TopK)
+};
+
+inline size_t select_extra_bytes(uint64_t d) {
+    const uint64_t t = sparse_tiles(d);
+    return round_up16(t * 128) + round_up16(t * 4) + (size_t)kSelPasses * kSelBins * 4 + 64;
+}
+
+__host__ __device__ inline SelectWorkspace select_ws_carve(char* p, uint64_t d) {
+    const uint64_t t = sparse_tiles(d);
+    SelectWorkspace w;
+    w.eqmask = reinterpret_cast<uint32_t*>(p);   p += round_up16(t * 128);
+    w.eq_block = reinterpret_cast<uint32_t*>(p); p += round_up16(t * 4);
+    w.hist = reinterpret_cast<uint32_t*>(p);     p += (size_t)kSelPasses * kSelBins * 4;
+    w.state = reinterpret_cast<SelectState*>(p);
+    w.count = reinterpret_cast<uint32_t*>(p + 32);
+    return w;
+}
+
+// ---- key sources: the 4 keys of elements base + k*128 + 4*lane + {0..3} ----------------------
+struct StreamKeys {          // selection-stream word of the coordinate
+    uint32_t worker;
+    PhiloxKeys keys;
+    struct Tile {
+        PhiloxTile pt;
+        uint32_t q_lo;
+    };
+    __device__ __forceinline__ Tile tile(uint64_t base, int lane) const {
+        Tile t;
+        t.pt = philox_tile((uint32_t)(base >> 34), worker, kDomainSelect, keys);
+        t.q_lo = (uint32_t)(base >> 2) + (uint32_t)lane;
+        return t;
+    }
+    __device__ __forceinline__ void load(const Tile& t, uint64_t, int, int k, uint64_t,
+                                         uint32_t (&out)[4]) const {
+        stream_words4_tile(t.q_lo + (uint32_t)(k * 32), t.pt, keys, out);
+    }
+};
+
+struct MagnitudeKeys {       // largest |x| first: complement of the magnitude bits
+    const float* x;
+    struct Tile {};
+    __device__ __forceinline__ Tile tile(uint64_t, int) const { return Tile(); }
+    __device__ __forceinline__ void load(const Tile&, uint64_t base, int lane, int k, uint64_t d,
+                                         uint32_t (&out)[4]) const {
+        const uint64_t j = base + (uint64_t)(k * 128 + lane * 4);
+        if (j + 4 <= d) {
+            const uint4 v = ld_stream_u4(x + j);
+            out[0] = ~(v.x & 0x7FFFFFFFu);
+            out[1] = ~(v.y & 0x7FFFFFFFu);
+            out[2] = ~(v.z & 0x7FFFFFFFu);
+            out[3] = ~(v.w & 0x7FFFFFFFu);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                out[c] = (j + c < d) ? ~(__float_as_uint(x[j + c]) & 0x7FFFFFFFu) : 0xFFFFFFFFu;
+        }
+    }
+};
+
+// bits of the load layout (bit 4k+c <-> element k*128 + 4*lane + c) that lie inside [0, d)
+__device__ __forceinline__ uint32_t valid_nibbles(uint64_t base, int lane, uint64_t d) {
+    if (base + kTile <= d) return 0xFFFFFFFFu;
+    uint32_t v = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (base + (uint64_t)(k * 128 + lane * 4 + c) < d) v |= 1u << (4 * k + c);
+    }
+    return v;
+}
+
+__global__ void select_init_kernel(SelectWorkspace ws, const uint64_t q) {
+    for (int i = threadIdx.x; i < kSelPasses * kSelBins; i += blockDim.x) ws.hist[i] = 0u;
+    if (threadIdx.x == 0) {
+        ws.state->prefix = 0u;
+        ws.state->pad = 0u;
+        ws.state->remaining = q;
+        *ws.count = 0u;
+    }
+}
+
+// persistent blocks: block b takes the groups of 8 tiles b, b + gridDim.x, ...
+template <class Src, int PASS>
+__global__ void __launch_bounds__(kBlockThreads)
+select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws) {
+    constexpr int bins = sel_bins(PASS);
+    constexpr int shift = sel_shift(PASS);
+    constexpr uint32_t fixed = sel_fixed(PASS);
+    __shared__ uint32_t s_hist[bins];
+    for (int i = threadIdx.x; i < bins; i += kBlockThreads) s_hist[i] = 0u;
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const uint32_t prefix = PASS == 0 ? 0u : ws.state->prefix;
+    const uint64_t groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    for (uint64_t g = blockIdx.x; g < groups; g += gridDim.x) {
+        const uint64_t base = (g * kWarpsPerBlock + (threadIdx.x >> 5)) * kTile;
+        if (base >= d) continue;
+        const uint32_t valid = valid_nibbles(base, lane, d);
+        const typename Src::Tile t = src.tile(base, lane);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t key[4];
+            src.load(t, base, lane, k, d, key);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if ((key[c] & fixed) == prefix && ((valid >> (4 * k + c)) & 1u))
+                    atomicAdd(&s_hist[(key[c] >> shift) & (uint32_t)(bins - 1)], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    uint32_t* __restrict__ hist = ws.hist + PASS * kSelBins;
+    for (int i = threadIdx.x; i < bins; i += kBlockThreads) {
+        const uint32_t v = s_hist[i];
+        if (v) atomicAdd(&hist[i], v);
+    }
+}
+
+// one block of 1024 threads, two bins each: the bin in which the cumulative count reaches
+// `remaining` becomes the next digit
+template <int PASS>
+__global__ void __launch_bounds__(kScanThreads) select_choose_kernel(const SelectWorkspace ws) {
+    constexpr int bins = sel_bins(PASS);
+    const uint32_t* __restrict__ hist = ws.hist + PASS * kSelBins;
+    __shared__ uint64_t s_sum[kScanThreads];
+    const int t = threadIdx.x;
+    const uint32_t h0 = (2 * t < bins) ? hist[2 * t] : 0u;
+    const uint32_t h1 = (2 * t + 1 < bins) ? hist[2 * t + 1] : 0u;
+    s_sum[t] = (uint64_t)h0 + h1;
+    __syncthreads();
+    for (int o = 1; o < kScanThreads; o <<= 1) {
+        const uint64_t v = (t >= o) ? s_sum[t - o] : 0ull;
+        __syncthreads();
+        s_sum[t] += v;
+        __syncthreads();
+    }
+    const uint64_t remaining = ws.state->remaining;
+    const uint64_t before = s_sum[t] - h0 - h1;         // keys in lower bins
+    __syncthreads();                                    // everyone has read the state
+    if (remaining > before && remaining <= before + h0) {
+        ws.state->prefix |= (uint32_t)(2 * t) << sel_shift(PASS);
+        ws.state->remaining = remaining - before;
+    } else if (remaining > before + h0 && remaining <= before + h0 + h1) {
+        ws.state->prefix |= (uint32_t)(2 * t + 1) << sel_shift(PASS);
+        ws.state->remaining = remaining - before - h0;
+    }
+}
+
+// grid: ceil(tiles / warps per block); one tile per warp
+template <class Src>
+__global__ void __launch_bounds__(kBlockThreads)
+select_mark_kernel(const Src src, const uint64_t d, uint32_t* __restrict__ less_mask,
+                   const SelectWorkspace ws) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const uint64_t base = tile * kTile;
+    const bool active = base < d;
+    const uint32_t T = ws.state->prefix;
+    __shared__ uint32_t s_eq[kWarpsPerBlock];
+    uint32_t less = 0, equal = 0;
+    if (active) {
+        const typename Src::Tile t = src.tile(base, lane);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t key[4];
+            src.load(t, base, lane, k, d, key);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                less |= (key[c] < T ? 1u : 0u) << (4 * k + c);
+                equal |= (key[c] == T ? 1u : 0u) << (4 * k + c);
+            }
+        }
+        const uint32_t valid = valid_nibbles(base, lane, d);
+        less &= valid;
+        equal &= valid;
+    }
+    const uint32_t lw = canonical_mask_word(less, lane);
+    const uint32_t ew = canonical_mask_word(equal, lane);
+    if (active) {
+        less_mask[tile * 32 + lane] = lw;
+        ws.eqmask[tile * 32 + lane] = ew;
+    }
+    const uint32_t ne = warp_sum_u(__popc(ew));
+    if (lane == 0) s_eq[warp] = ne;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t c = 0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) c += s_eq[w];
+        ws.eq_block[blockIdx.x] = c;
+    }
+}
+
+// one block: in-place exclusive scan of n counts; the total goes to *total if it is not null
+__global__ void __launch_bounds__(kScanThreads)
+select_scan_counts_kernel(uint32_t* __restrict__ counts, const uint64_t n,
+                          uint32_t* __restrict__ total) {
+    __shared__ uint32_t s_cnt[kScanThreads];
+    const int t = threadIdx.x;
+    const uint64_t per = (n + kScanThreads - 1) / kScanThreads;
+    const uint64_t t0 = (uint64_t)t * per;
+    const uint64_t t1 = (t0 + per < n) ? t0 + per : n;
+    uint32_t c = 0;
+    for (uint64_t i = t0; i < t1; ++i) c += counts[i];
+    s_cnt[t] = c;
+    __syncthreads();
+    for (int o = 1; o < kScanThreads; o <<= 1) {
+        const uint32_t v = (t >= o) ? s_cnt[t - o] : 0u;
+        __syncthreads();
+        s_cnt[t] += v;
+        __syncthreads();
+    }
+    uint32_t run = s_cnt[t] - c;
+    for (uint64_t i = t0; i < t1; ++i) {
+        const uint32_t v = counts[i];
+        counts[i] = run;
+        run += v;
+    }
+    if (t == kScanThreads - 1 && total) *total = s_cnt[t];
+}
+
+// grid: ceil(tiles / warps per block).  mask <- "< T" | first r of "== T"; per-block kept counts;
+// with kNorm also the norm partials of the scaled kept entries (P as in the sparsifier).
+template <int P, bool kNorm>
+__global__ void __launch_bounds__(kBlockThreads)
+select_resolve_kernel(const float* __restrict__ x, const uint64_t d, const float scale,
+                      const SparseWorkspace sp, const SelectWorkspace ws) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const uint64_t base = tile * kTile;
+    const bool active = base < d;
+    __shared__ uint32_t s_eq[kWarpsPerBlock];
+    __shared__ uint32_t s_kept[kWarpsPerBlock];
+    uint32_t word = active ? sp.bitmask[tile * 32 + lane] : 0u;
+    uint32_t ew = active ? ws.eqmask[tile * 32 + lane] : 0u;
+    const uint32_t ne = __popc(ew);
+    uint32_t incl = ne;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_eq[warp] = incl;
+    __syncthreads();
+    uint64_t rank0 = (uint64_t)ws.eq_block[blockIdx.x] + (incl - ne);   // rank of this lane's first
+    for (int w = 0; w < warp; ++w) rank0 += s_eq[w];
+    const uint64_t r = ws.state->remaining;
+    const uint32_t allowed = (r > rank0) ? (uint32_t)min((uint64_t)ne, r - rank0) : 0u;
+    uint32_t left = ne;
+    while (left > allowed) {                 // drop the highest-index ties beyond the first r
+        ew &= ~(0x80000000u >> __clz(ew));
+        --left;
+    }
+    word |= ew;
+    if (active) sp.bitmask[tile * 32 + lane] = word;
+    if (kNorm) {
+        kept_count_and_partial<P>(word, lane, x, base, scale, sp.block_count, sp.block_partial);
+    } else {
+        const uint32_t kept = warp_sum_u(__popc(word));
+        if (lane == 0) s_kept[warp] = kept;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t c = 0;
+            for (int w = 0; w < kWarpsPerBlock; ++w) c += s_kept[w];
+            sp.block_count[blockIdx.x] = c;
+        }
+    }
+}
+
+// grid: ceil(tiles / warps per block).  Lists the selected entries in index order: index, the
+// exponent byte of C_nat(x_j) (Def. 1; stream of coordinate j) and one sign byte for the packer.
+__global__ void __launch_bounds__(kBlockThreads)
+topk_emit_kernel(const float* __restrict__ x, const uint64_t d, const uint32_t worker,
+                 const __grid_constant__ PhiloxKeys keys, const uint64_t cap,
+                 uint32_t* __restrict__ idx, uint8_t* __restrict__ exp, const SparseWorkspace sp) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const uint64_t base = tile * kTile;
+    const bool active = base < d;
+    __shared__ uint32_t s_tile[kWarpsPerBlock];
+    __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
+    uint16_t* list = s_list[warp];
+    const uint32_t word = active ? sp.bitmask[tile * 32 + lane] : 0u;
+    const uint32_t cnt = warp_list_positions(word, lane, list);
+    if (lane == 0) s_tile[warp] = cnt;
+    __syncthreads();
+    uint64_t k0 = (uint64_t)sp.block_count[blockIdx.x];
+    for (int w = 0; w < warp; ++w) k0 += s_tile[w];
+    for (uint32_t t = lane; t < cnt; t += 32) {
+        const uint64_t k = k0 + t;
+        if (k >= cap) break;
+        const uint64_t j = base + list[t];
+        const uint32_t bits = __float_as_uint(x[j]);
+        const uint32_t r23 = stream_word_at(j, worker, kDomainCnat, keys) & 0x7FFFFFu;
+        const uint32_t e = (bits >> 23) & 0xFFu;
+        const uint32_t m = bits & 0x7FFFFFu;
+        // up with probability m / 2^23; 2^127 and above saturate, inf and NaN give byte 255
+        const uint32_t byte = (e >= 254u) ? e : e + (r23 < m ? 1u : 0u);
+        idx[k] = (uint32_t)j;
+        exp[k] = (uint8_t)byte;
+        sp.tmp_codes[k] = (uint8_t)(bits >> 31);
+    }
+}
+
+// one warp per 32 listed entries: sign bytes -> one word of the sign plane
+__global__ void __launch_bounds__(kBlockThreads)
+topk_pack_sign_kernel(const uint8_t* __restrict__ sign_bytes, const uint64_t listed,
+                      uint32_t* __restrict__ sign) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t group = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    if (group * 32 >= listed) return;
+    const uint64_t k = group * 32 + lane;
+    const uint32_t b = (k < listed) ? sign_bytes[k] : 0u;
+    const uint32_t wv = __ballot_sync(0xFFFFFFFFu, b & 1u);
+    if (lane == 0) sign[group] = wv;
+}
+
+// grid: ceil(count / threads)
+__global__ void __launch_bounds__(kBlockThreads)
+topk_decode_accumulate_kernel(const uint32_t* __restrict__ idx, const uint8_t* __restrict__ exp,
+                              const uint32_t* __restrict__ sign, const uint64_t count,
+                              const uint64_t d, float* __restrict__ acc) {
+    const uint64_t k = (uint64_t)blockIdx.x * kBlockThreads + threadIdx.x;
+    if (k >= count) return;
+    const uint32_t j = idx[k];
+    if (j >= d) return;
+    const uint32_t bits = ((uint32_t)exp[k] << 23) | (((sign[k >> 5] >> (k & 31)) & 1u) << 31);
+    acc[j] = __fadd_rn(acc[j], __uint_as_float(bits));
+}
+
+// zero count, norm and planes: the q = 0 sparsifier
+__global__ void __launch_bounds__(kBlockThreads)
+select_empty_kernel(uint32_t* __restrict__ planes, const uint64_t words,
+                    uint32_t* __restrict__ count, float* __restrict__ norm) {
+    const uint64_t i = (uint64_t)blockIdx.x * kBlockThreads + threadIdx.x;
+    if (i < words) planes[i] = 0u;
+    if (i == 0) {
+        *count = 0u;
+        *norm = 0.f;
+    }
+}
+
+// hist/choose passes, mark, scan of the tie counts: leaves T and r in the state, "< T" in the
+// sparsifier bitmask and "== T" in the tie mask
+template <class Src>
+static void run_select(const Src& src, uint64_t d, uint64_t q, const SparseWorkspace& sp,
+                       const SelectWorkspace& ws, int sm_count, cudaStream_t stream) {
+    const uint64_t groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const unsigned pgrid = (unsigned)(groups < (uint64_t)sm_count * 8 ? groups
+                                                                      : (uint64_t)sm_count * 8);
+    select_init_kernel<<<1, kScanThreads, 0, stream>>>(ws, q);
+    select_hist_kernel<Src, 0><<<pgrid, kBlockThreads, 0, stream>>>(src, d, ws);
+    select_choose_kernel<0><<<1, kScanThreads, 0, stream>>>(ws);
+    select_hist_kernel<Src, 1><<<pgrid, kBlockThreads, 0, stream>>>(src, d, ws);
+    select_choose_kernel<1><<<1, kScanThreads, 0, stream>>>(ws);
+    select_hist_kernel<Src, 2><<<pgrid, kBlockThreads, 0, stream>>>(src, d, ws);
+    select_choose_kernel<2><<<1, kScanThreads, 0, stream>>>(ws);
+    select_mark_kernel<Src><<<(unsigned)groups, kBlockThreads, 0, stream>>>(src, d, sp.bitmask, ws);
+    select_scan_counts_kernel<<<1, kScanThreads, 0, stream>>>(ws.eq_block, groups, nullptr);
+}
+
+static int sm_count_of_current_device() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1)
+            v = 148;
+        cached[dev] = v;
+    }
+    return cached[dev];
+}
+
+}  // namespace natcomp
+
+using namespace natcomp;
+
+extern "C" {
+
+size_t nc_select_workspace_bytes(size_t d, size_t cap) {
+    return sparse_ws_bytes(d, cap) + select_extra_bytes(d);
+}
+
+nc_status nd_sparse_exact_compress(const float* x, size_t d, uint64_t q, float scale, int p, int s,
+                                   uint64_t seed, uint32_t worker, uint32_t* idx,
+                                   uint32_t* planes, uint32_t* count, float* norm, size_t cap,
+                                   void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (!x || !idx || !planes || !count || !norm || s < 1 || s > 8 || cap < 1)
+        return NC_ERR_INVALID;
+    if (p != 1 && p != 2 && p != NC_P_INF) return NC_ERR_UNSUPPORTED;
+    if (d == 0) return NC_OK;
+    if (d > 0xFFFFFFFFull) return NC_ERR_INVALID;
+    if (!workspace) return NC_ERR_INVALID;
+    if (!aligned16(workspace)) return NC_ERR_ALIGN;
+    if (!aligned32(x) || !aligned16(idx) || !aligned16(planes) || !aligned4(count) ||
+        !aligned4(norm))
+        return NC_ERR_ALIGN;
+    if (workspace_bytes < nc_select_workspace_bytes(d, cap)) return NC_ERR_WORKSPACE;
+    if (q > d) q = d;
+    if (q == 0) {
+        const uint64_t words = ((cap + 31) / 32) * (uint64_t)(code_value_bits(s) + 1);
+        select_empty_kernel<<<(unsigned)((words + kBlockThreads - 1) / kBlockThreads),
+                              kBlockThreads, 0, stream>>>(planes, words, count, norm);
+        return launch_status();
+    }
+    char* wsp = reinterpret_cast<char*>(workspace);
+    const SparseWorkspace sp = sparse_ws_carve(wsp, d);
+    const SelectWorkspace ws = select_ws_carve(wsp + sparse_ws_bytes(d, cap), d);
+    const PhiloxKeys keys = make_philox_keys(seed);
+    StreamKeys src;
+    src.worker = worker;
+    src.keys = keys;
+    run_select(src, d, q, sp, ws, sm_count_of_current_device(), stream);
+    const unsigned grid = (unsigned)((sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    if (p == 1)
+        select_resolve_kernel<1, true><<<grid, kBlockThreads, 0, stream>>>(x, d, scale, sp, ws);
+    else if (p == 2)
+        select_resolve_kernel<2, true><<<grid, kBlockThreads, 0, stream>>>(x, d, scale, sp, ws);
+    else
+        select_resolve_kernel<NC_P_INF, true><<<grid, kBlockThreads, 0, stream>>>(x, d, scale, sp,
+                                                                                  ws);
+    SparseBatch batch;
+    batch.x[0] = x;
+    batch.idx[0] = idx;
+    batch.codes[0] = reinterpret_cast<uint8_t*>(planes);
+    batch.count[0] = count;
+    batch.norm[0] = norm;
+    batch.worker[0] = worker;
+    sparse_compact_finish(batch, d, scale, p, s, keys, cap, wsp, sparse_ws_bytes(d, cap), 1,
+                          stream);
+    return launch_status();
+}
+
+nc_status nc_topk_compress(const float* x, size_t d, uint64_t K, uint64_t seed, uint32_t worker,
+                           uint32_t* idx, uint8_t* exp, uint32_t* sign, void* workspace,
+                           size_t workspace_bytes, cudaStream_t stream) {
+    if (!x || !idx || !exp || !sign) return NC_ERR_INVALID;
+    if (d > 0xFFFFFFFFull) return NC_ERR_INVALID;
+    if (K > d) K = d;
+    if (d == 0 || K == 0) return NC_OK;
+    if (!workspace) return NC_ERR_INVALID;
+    if (!aligned16(workspace)) return NC_ERR_ALIGN;
+    if (!aligned32(x) || !aligned16(idx) || !aligned16(exp) || !aligned16(sign))
+        return NC_ERR_ALIGN;
+    if (workspace_bytes < nc_select_workspace_bytes(d, K)) return NC_ERR_WORKSPACE;
+    char* wsp = reinterpret_cast<char*>(workspace);
+    const SparseWorkspace sp = sparse_ws_carve(wsp, d);
+    const SelectWorkspace ws = select_ws_carve(wsp + sparse_ws_bytes(d, K), d);
+    MagnitudeKeys src;
+    src.x = x;
+    run_select(src, d, K, sp, ws, sm_count_of_current_device(), stream);
+    const uint64_t groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    select_resolve_kernel<NC_P_INF, false><<<(unsigned)groups, kBlockThreads, 0, stream>>>(
+        x, d, 1.0f, sp, ws);
+    select_scan_counts_kernel<<<1, kScanThreads, 0, stream>>>(sp.block_count, groups, ws.count);
+    topk_emit_kernel<<<(unsigned)groups, kBlockThreads, 0, stream>>>(
+        x, d, worker, make_philox_keys(seed), K, idx, exp, sp);
+    const uint64_t sgroups = (K + 31) / 32;
+    topk_pack_sign_kernel<<<(unsigned)((sgroups + kWarpsPerBlock - 1) / kWarpsPerBlock),
+                            kBlockThreads, 0, stream>>>(sp.tmp_codes, K, sign);
+    return launch_status();
+}
+
+nc_status nc_topk_decode_accumulate(const uint32_t* idx, const uint8_t* exp, const uint32_t* sign,
+                                    size_t count, size_t d, float* acc, cudaStream_t stream) {
+    if (!idx || !exp || !sign || !acc) return NC_ERR_INVALID;
+    if (d > 0xFFFFFFFFull || count > 0xFFFFFFFFull) return NC_ERR_INVALID;
+    if (count == 0 || d == 0) return NC_OK;
+    if (!aligned16(idx) || !aligned16(exp) || !aligned16(sign) || !aligned32(acc))
+        return NC_ERR_ALIGN;
+    const unsigned grid = (unsigned)((count + kBlockThreads - 1) / kBlockThreads);
+    topk_decode_accumulate_kernel<<<grid, kBlockThreads, 0, stream>>>(idx, exp, sign, count, d,
+                                                                      acc);
+    return launch_status();
+}
+
+}  // extern "C"

@@ -1,0 +1,185 @@
+// Pieces shared by the sparsifier kernels (independent per-coordinate selection) and the
+// exact-count selection kernels (radix select): argument blocks, workspace layout, warp helpers,
+// the level rounding of Def. 3 for a single gathered entry, and the host routine that turns a
+// selection bitmask into the compact list.
+#pragma once
+#include "common.cuh"
+#include "philox.cuh"
+
+namespace natcomp {
+
+constexpr int kScanThreads = 1024;
+
+struct SparseBatch {
+    const float* x[NC_MAX_WORKERS];
+    uint32_t* idx[NC_MAX_WORKERS];
+    uint8_t* codes[NC_MAX_WORKERS];
+    uint32_t* count[NC_MAX_WORKERS];
+    float* norm[NC_MAX_WORKERS];
+    uint32_t worker[NC_MAX_WORKERS];
+};
+
+struct SparseWorkspace {
+    uint32_t* bitmask;      // tiles * 32 words
+    uint32_t* block_count;   // one per block of 8 tiles (the exclusive offset after the scan)
+    uint64_t* block_partial; // one per block of 8 tiles
+    uint8_t* tmp_codes;     // cap bytes
+};
+
+__host__ __device__ inline uint64_t sparse_tiles(uint64_t d) { return (d + kTile - 1) / kTile; }
+
+inline size_t sparse_ws_bytes(uint64_t d, uint64_t cap) {
+    const uint64_t t = sparse_tiles(d);
+    return round_up16(t * 128) + round_up16(t * 4) + round_up16(t * 8) + round_up16(cap);
+}
+
+__host__ __device__ inline SparseWorkspace sparse_ws_carve(void* ws, uint64_t d) {
+    const uint64_t t = sparse_tiles(d);
+    char* p = reinterpret_cast<char*>(ws);
+    SparseWorkspace w;
+    w.bitmask = reinterpret_cast<uint32_t*>(p);      p += round_up16(t * 128);
+    w.block_count = reinterpret_cast<uint32_t*>(p);   p += round_up16(t * 4);
+    w.block_partial = reinterpret_cast<uint64_t*>(p); p += round_up16(t * 8);
+    w.tmp_codes = reinterpret_cast<uint8_t*>(p);
+    return w;
+}
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+__device__ __forceinline__ uint32_t warp_max_u(uint32_t v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ uint32_t warp_sum_u(uint32_t v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// Lists the set bits of a 1024-bit tile mask (lane l holds word l) in ascending order into the
+// warp's shared-memory list as in-tile positions; returns how many there are.  After this the
+// t-th kept entry can be handled by lane t mod 32, so the gathers from x run in parallel
+// instead of one dependent load per set bit of a lane's own word.
+__device__ __forceinline__ uint32_t warp_list_positions(uint32_t word, int lane,
+                                                        uint16_t* __restrict__ list) {
+    const uint32_t cnt = __popc(word);
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    uint32_t at = incl - cnt;
+    while (word) {
+        const int bit = __ffs(word) - 1;
+        word &= word - 1;
+        list[at++] = (uint16_t)(lane * 32 + bit);
+    }
+    __syncwarp();
+    return __shfl_sync(0xFFFFFFFFu, incl, 31);
+}
+
+// A lane's 32 per-element bits in the load layout (bit 4k+c <-> element k*128 + 4*lane + c of
+// the tile) -> canonical order: lane l returns the word of elements 32l .. 32l+31.
+__device__ __forceinline__ uint32_t canonical_mask_word(uint32_t nib, int lane) {
+    const uint32_t word = transpose_nibbles_8x8(nib, lane);   // lane 8g+k holds word 4k+g
+    return __shfl_sync(0xFFFFFFFFu, word, 8 * (lane & 3) + (lane >> 2));
+}
+
+// For one tile per warp (all warps of the block must call): gathers the kept entries of the
+// tile (mask word of lane l = elements 32l..32l+31), accumulates the norm partial of the scaled
+// kept entries, and thread 0 writes the block's kept count and partial.  P = 1, 2 or NC_P_INF.
+template <int P>
+__device__ __forceinline__ void kept_count_and_partial(const uint32_t word, const int lane,
+                                                       const float* __restrict__ x,
+                                                       const uint64_t base, const float scale,
+                                                       uint32_t* __restrict__ block_count,
+                                                       uint64_t* __restrict__ block_partial) {
+    __shared__ uint32_t s_cnt[kWarpsPerBlock];
+    __shared__ uint64_t s_part[kWarpsPerBlock];
+    __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
+    uint16_t* list = s_list[threadIdx.x >> 5];
+    const uint32_t cnt = warp_list_positions(word, lane, list);
+    double dsum = 0.0;
+    uint32_t vmax = 0;
+    for (uint32_t t = lane; t < cnt; t += 32) {
+        const float xs = __fmul_rn(scale, x[base + list[t]]);
+        const uint32_t a = __float_as_uint(xs) & 0x7FFFFFFFu;
+        if (P == NC_P_INF) vmax = max(vmax, a);
+        else if (P == 1) dsum += (double)__uint_as_float(a);
+        else dsum = fma((double)xs, (double)xs, dsum);
+    }
+    uint64_t part;
+    if (P == NC_P_INF) part = (uint64_t)warp_max_u(vmax);
+    else part = (uint64_t)__double_as_longlong(warp_sum_d(dsum));
+    if (lane == 0) {
+        s_cnt[threadIdx.x >> 5] = cnt;
+        s_part[threadIdx.x >> 5] = part;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t c = 0, m = 0;
+        double sum = 0.0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) {     // fixed order
+            c += s_cnt[w];
+            if (P == NC_P_INF) m = max(m, (uint32_t)s_part[w]);
+            else sum += __longlong_as_double((long long)s_part[w]);
+        }
+        block_count[blockIdx.x] = c;
+        block_partial[blockIdx.x] =
+            (P == NC_P_INF) ? (uint64_t)m : (uint64_t)__double_as_longlong(sum);
+    }
+}
+
+struct Scale {
+    float rinv;
+    uint32_t smax;
+};
+
+__device__ __forceinline__ Scale make_scale(float norm, int s) {
+    Scale r;
+    const bool ok = (norm >= 1.17549435e-38f) && (norm <= 3.40282347e38f);
+    r.rinv = ok ? __fdiv_rn(1.0f, norm) : 0.f;
+    r.smax = ok ? (uint32_t)s : 0u;
+    return r;
+}
+
+// same rounding rule as the dense dithering kernel (Def. 3, natural levels)
+__device__ __forceinline__ uint32_t sparse_level_code(uint32_t bits, uint32_t rnd, const Scale sc,
+                                                      float pow2s) {
+    const float ax = __uint_as_float(bits & 0x7FFFFFFFu);
+    const float y = __fmul_rn(ax, sc.rinv);
+    const float z = __fmul_rn(y, pow2s);
+    float w = z;
+    if (z < 2.0f) w = __fmaf_rz(z, 0.5f, 1.0f);
+    const uint32_t t = __float_as_uint(w) + (~rnd & 0x7FFFFFu) - 0x3F800000u;
+    return min(t >> 23, sc.smax);
+}
+
+__host__ __device__ inline int code_value_bits(int s) {
+    int nb = 0;
+    while ((1 << nb) < s) ++nb;
+    return nb;
+}
+
+// the stream word of element j (any domain), for gathered entries
+__device__ __forceinline__ uint32_t stream_word_at(uint64_t j, uint32_t worker, uint32_t domain,
+                                                   const PhiloxKeys& keys) {
+    uint32_t r4[4];
+    stream_words4(j >> 2, worker, domain, keys, r4);
+    return (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1] : (j & 3) == 2 ? r4[2] : r4[3];
+}
+
+// Given, per worker, the selection bitmask, the per-block kept counts and the norm partials in
+// the workspace (what the select kernels leave): norm, level rounding, dropping of level-0
+// entries, index list and code planes of the compact format.  Defined with the sparsifier
+// kernels; launches only.
+void sparse_compact_finish(const SparseBatch& batch, uint64_t d, float scale, int p, int s,
+                           const PhiloxKeys& keys, uint64_t cap, char* ws, uint64_t ws_stride,
+                           int n, cudaStream_t stream);
+
+}  // namespace natcomp

@@ -13,85 +13,9 @@
 //            block + prefix popcount inside the tile; writes the index list and one code byte
 //            per entry
 //   pack   : two code bytes -> one byte of 4-bit codes
-#include "common.cuh"
-#include "philox.cuh"
+#include "sparse_common.cuh"
 
 namespace natcomp {
-
-constexpr int kScanThreads = 1024;
-
-struct SparseBatch {
-    const float* x[NC_MAX_WORKERS];
-    uint32_t* idx[NC_MAX_WORKERS];
-    uint8_t* codes[NC_MAX_WORKERS];
-    uint32_t* count[NC_MAX_WORKERS];
-    float* norm[NC_MAX_WORKERS];
-    uint32_t worker[NC_MAX_WORKERS];
-};
-
-struct SparseWorkspace {
-    uint32_t* bitmask;      // tiles * 32 words
-    uint32_t* block_count;   // one per block of 8 tiles (the exclusive offset after the scan)
-    uint64_t* block_partial; // one per block of 8 tiles
-    uint8_t* tmp_codes;     // cap bytes
-};
-
-__host__ __device__ inline uint64_t sparse_tiles(uint64_t d) { return (d + kTile - 1) / kTile; }
-
-inline size_t sparse_ws_bytes(uint64_t d, uint64_t cap) {
-    const uint64_t t = sparse_tiles(d);
-    return round_up16(t * 128) + round_up16(t * 4) + round_up16(t * 8) + round_up16(cap);
-}
-
-__host__ __device__ inline SparseWorkspace sparse_ws_carve(void* ws, uint64_t d) {
-    const uint64_t t = sparse_tiles(d);
-    char* p = reinterpret_cast<char*>(ws);
-    SparseWorkspace w;
-    w.bitmask = reinterpret_cast<uint32_t*>(p);      p += round_up16(t * 128);
-    w.block_count = reinterpret_cast<uint32_t*>(p);   p += round_up16(t * 4);
-    w.block_partial = reinterpret_cast<uint64_t*>(p); p += round_up16(t * 8);
-    w.tmp_codes = reinterpret_cast<uint8_t*>(p);
-    return w;
-}
-
-__device__ __forceinline__ double warp_sum_d(double v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
-}
-__device__ __forceinline__ uint32_t warp_max_u(uint32_t v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
-    return v;
-}
-__device__ __forceinline__ uint32_t warp_sum_u(uint32_t v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
-}
-
-// Lists the set bits of a 1024-bit tile mask (lane l holds word l) in ascending order into the
-// warp's shared-memory list as in-tile positions; returns how many there are.  After this the
-// t-th kept entry can be handled by lane t mod 32, so the gathers from x run in parallel
-// instead of one dependent load per set bit of a lane's own word.
-__device__ __forceinline__ uint32_t warp_list_positions(uint32_t word, int lane,
-                                                        uint16_t* __restrict__ list) {
-    const uint32_t cnt = __popc(word);
-    uint32_t incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    uint32_t at = incl - cnt;
-    while (word) {
-        const int bit = __ffs(word) - 1;
-        word &= word - 1;
-        list[at++] = (uint16_t)(lane * 32 + bit);
-    }
-    __syncwarp();
-    return __shfl_sync(0xFFFFFFFFu, incl, 31);
-}
 
 // grid: ceil(tiles / warps per block)
 template <int P>
@@ -108,12 +32,6 @@ sparse_select_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d
     const uint32_t worker = batch.worker[blockIdx.y];
     const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
     uint32_t* __restrict__ bitmask = ws.bitmask;
-    __shared__ uint32_t s_cnt[kWarpsPerBlock];
-    __shared__ uint64_t s_part[kWarpsPerBlock];
-
-    __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
-    uint16_t* list = s_list[threadIdx.x >> 5];
-
     // phase 1: the 1024 selection bits of the tile, no memory traffic
     uint32_t nib = 0;        // bit 4k+c <-> element base + k*128 + 4*lane + c
     const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainSelect, keys);
@@ -146,42 +64,11 @@ sparse_select_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d
             }
         }
     }
-    // canonical order: after the transpose lane 8g+k holds word 4k+g; bring word l to lane l
-    uint32_t word = transpose_nibbles_8x8(nib, lane);
-    word = __shfl_sync(0xFFFFFFFFu, word, 8 * (lane & 3) + (lane >> 2));
+    const uint32_t word = canonical_mask_word(nib, lane);
     if (active) bitmask[tile * 32 + lane] = word;
 
     // phase 2: gather the kept entries, spread evenly over the lanes
-    const uint32_t cnt = warp_list_positions(word, lane, list);
-    double dsum = 0.0;
-    uint32_t vmax = 0;
-    for (uint32_t t = lane; t < cnt; t += 32) {
-        const float xs = __fmul_rn(scale, x[base + list[t]]);
-        const uint32_t a = __float_as_uint(xs) & 0x7FFFFFFFu;
-        if (P == NC_P_INF) vmax = max(vmax, a);
-        else if (P == 1) dsum += (double)__uint_as_float(a);
-        else dsum = fma((double)xs, (double)xs, dsum);
-    }
-    uint64_t part;
-    if (P == NC_P_INF) part = (uint64_t)warp_max_u(vmax);
-    else part = (uint64_t)__double_as_longlong(warp_sum_d(dsum));
-    if (lane == 0) {
-        s_cnt[threadIdx.x >> 5] = cnt;
-        s_part[threadIdx.x >> 5] = part;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t c = 0, m = 0;
-        double sum = 0.0;
-        for (int w = 0; w < kWarpsPerBlock; ++w) {     // fixed order
-            c += s_cnt[w];
-            if (P == NC_P_INF) m = max(m, (uint32_t)s_part[w]);
-            else sum += __longlong_as_double((long long)s_part[w]);
-        }
-        ws.block_count[blockIdx.x] = c;
-        ws.block_partial[blockIdx.x] =
-            (P == NC_P_INF) ? (uint64_t)m : (uint64_t)__double_as_longlong(sum);
-    }
+    kept_count_and_partial<P>(word, lane, x, base, scale, ws.block_count, ws.block_partial);
 }
 
 // one block: exclusive scan of the per-block counts (in place), total count, norm
@@ -242,31 +129,6 @@ sparse_scan_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
         else r = (float)sqrt(s_sum[0]);
         *norm = r;
     }
-}
-
-struct Scale {
-    float rinv;
-    uint32_t smax;
-};
-
-__device__ __forceinline__ Scale make_scale(float norm, int s) {
-    Scale r;
-    const bool ok = (norm >= 1.17549435e-38f) && (norm <= 3.40282347e38f);
-    r.rinv = ok ? __fdiv_rn(1.0f, norm) : 0.f;
-    r.smax = ok ? (uint32_t)s : 0u;
-    return r;
-}
-
-// same rounding rule as the dense dithering kernel (Def. 3, natural levels)
-__device__ __forceinline__ uint32_t sparse_level_code(uint32_t bits, uint32_t rnd, const Scale sc,
-                                                      float pow2s) {
-    const float ax = __uint_as_float(bits & 0x7FFFFFFFu);
-    const float y = __fmul_rn(ax, sc.rinv);
-    const float z = __fmul_rn(y, pow2s);
-    float w = z;
-    if (z < 2.0f) w = __fmaf_rz(z, 0.5f, 1.0f);
-    const uint32_t t = __float_as_uint(w) + (~rnd & 0x7FFFFFu) - 0x3F800000u;
-    return min(t >> 23, sc.smax);
 }
 
 // grid: ceil(tiles / warps per block)
@@ -353,6 +215,16 @@ sparse_decode_accumulate_kernel(const uint32_t* __restrict__ idx, const uint8_t*
     acc[j] = __fadd_rn(acc[j], __fmul_rn(nv, __uint_as_float(pb)));
 }
 
+static void launch_scan(const SparseBatch& batch, uint64_t d, int p, char* ws, uint64_t ws_stride,
+                        int n, cudaStream_t stream) {
+    const dim3 sgrid(1, (unsigned)n);
+    if (p == 1) sparse_scan_kernel<1><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
+    else if (p == 2)
+        sparse_scan_kernel<2><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
+    else
+        sparse_scan_kernel<NC_P_INF><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
+}
+
 }  // namespace natcomp
 
 using namespace natcomp;
@@ -400,20 +272,16 @@ nc_status nd_sparse_compress_batch(const float* const* xs, size_t d, uint64_t ke
     const PhiloxKeys keys = make_philox_keys(seed);
     const bool keep_none = keep_threshold == 0;
     const uint32_t neg_thr = (uint32_t)(0ull - keep_threshold);   // 2^32 - threshold (mod 2^32)
-    const dim3 sgrid(1, (unsigned)n);
-    if (p == 1) {
+    if (p == 1)
         sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
                                                                     scale, keys, ws, ws_stride);
-        sparse_scan_kernel<1><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
-    } else if (p == 2) {
+    else if (p == 2)
         sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
                                                                     scale, keys, ws, ws_stride);
-        sparse_scan_kernel<2><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
-    } else {
+    else
         sparse_select_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
             batch, d, neg_thr, keep_none, scale, keys, ws, ws_stride);
-        sparse_scan_kernel<NC_P_INF><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
-    }
+    launch_scan(batch, d, p, ws, ws_stride, n, stream);
     sparse_emit_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap, ws,
                                                            ws_stride);
     const uint64_t pack_threads = round_up16((cap + 1) / 2);
@@ -462,12 +330,6 @@ nc_status nd_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes,
 //   emit_compact  : index list + one code byte per surviving entry
 //   pack_planes   : 32 code bytes -> nb + 1 plane words (warp ballots)
 namespace natcomp {
-
-__host__ __device__ inline int code_value_bits(int s) {
-    int nb = 0;
-    while ((1 << nb) < s) ++nb;
-    return nb;
-}
 
 // grid: (ceil(tiles / warps per block), n workers)
 __global__ void __launch_bounds__(kBlockThreads)
@@ -607,6 +469,28 @@ sparse_compact_decode_accumulate_kernel(const uint32_t* __restrict__ idx,
 
 }  // namespace natcomp
 
+namespace natcomp {
+
+void sparse_compact_finish(const SparseBatch& batch, uint64_t d, float scale, int p, int s,
+                           const PhiloxKeys& keys, uint64_t cap, char* ws, uint64_t ws_stride,
+                           int n, cudaStream_t stream) {
+    const uint64_t tiles = sparse_tiles(d);
+    const dim3 grid((unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
+    launch_scan(batch, d, p, ws, ws_stride, n, stream);          // norm (and the kept count)
+    sparse_round_filter_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, ws,
+                                                                   ws_stride);
+    // second scan: offsets and count of the surviving entries (the norm partials are unchanged)
+    launch_scan(batch, d, p, ws, ws_stride, n, stream);
+    sparse_emit_compact_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap,
+                                                                   ws, ws_stride);
+    const uint64_t groups = (cap + 31) / 32;
+    const dim3 pgrid((unsigned)((groups + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
+    sparse_pack_planes_kernel<<<pgrid, kBlockThreads, 0, stream>>>(batch, d, cap, s, ws,
+                                                                   ws_stride);
+}
+
+}  // namespace natcomp
+
 extern "C" {
 
 size_t nd_sparse_plane_bytes(size_t cap, int s) {
@@ -647,37 +531,19 @@ nc_status nd_sparse_compact_compress_batch(const float* const* xs, size_t d,
     char* ws = reinterpret_cast<char*>(workspace);
     const uint64_t tiles = sparse_tiles(d);
     const dim3 grid((unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
-    const dim3 sgrid(1, (unsigned)n);
     const PhiloxKeys keys = make_philox_keys(seed);
     const bool keep_none = keep_threshold == 0;
     const uint32_t neg_thr = (uint32_t)(0ull - keep_threshold);
-    if (p == 1) {
+    if (p == 1)
         sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
                                                                     scale, keys, ws, ws_stride);
-        sparse_scan_kernel<1><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
-    } else if (p == 2) {
+    else if (p == 2)
         sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
                                                                     scale, keys, ws, ws_stride);
-        sparse_scan_kernel<2><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
-    } else {
+    else
         sparse_select_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
             batch, d, neg_thr, keep_none, scale, keys, ws, ws_stride);
-        sparse_scan_kernel<NC_P_INF><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
-    }
-    sparse_round_filter_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, ws,
-                                                                   ws_stride);
-    // second scan: offsets and count of the surviving entries (the norm partials are unchanged)
-    if (p == 1) sparse_scan_kernel<1><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
-    else if (p == 2)
-        sparse_scan_kernel<2><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
-    else
-        sparse_scan_kernel<NC_P_INF><<<sgrid, kScanThreads, 0, stream>>>(batch, d, ws, ws_stride);
-    sparse_emit_compact_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap,
-                                                                   ws, ws_stride);
-    const uint64_t groups = (cap + 31) / 32;
-    const dim3 pgrid((unsigned)((groups + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
-    sparse_pack_planes_kernel<<<pgrid, kBlockThreads, 0, stream>>>(batch, d, cap, s, ws,
-                                                                   ws_stride);
+    sparse_compact_finish(batch, d, scale, p, s, keys, cap, ws, ws_stride, n, stream);
     return launch_status();
 }
 
