@@ -159,8 +159,8 @@ def run_sparse(config, n, d, iters, peak, s=4):
                                                      sel_bytes), iters)
     _report(config, "nd_sparse_exact_compress (1 worker)", m, b, d, q * 96.0, peak,
             {"Gcoord_per_s": round(d / m / 1e6, 1),
-             "note": "four passes over the selection stream (3 digit histograms + mark)"})
-    # TopK then C_nat, K = d / 100, one worker: x is read four times (3 histograms + mark)
+             "note": "two sweeps over the selection stream (digit histogram, mark) + candidate list"})
+    # TopK then C_nat, K = d / 100, one worker: x is read three times (2 histograms + mark)
     K = q
     tidx = torch.empty(K, dtype=torch.int32, device=dev)
     texp = torch.empty(K, **u8)
@@ -168,7 +168,7 @@ def run_sparse(config, n, d, iters, peak, s=4):
     m, b = _time(lambda: nc.nc_topk_compress(xs[0], d, K, 0, 0, tidx, texp, tsign, sel_ws,
                                              sel_bytes), iters)
     _report(config, "nc_topk_compress (1 worker)", m, b, d, d * 4.0 + K * 5.125, peak,
-            {"Gcoord_per_s": round(d / m / 1e6, 1), "hbm_bytes_actually_read": d * 16})
+            {"Gcoord_per_s": round(d / m / 1e6, 1), "hbm_bytes_actually_read": d * 12})
 
 
 def main():

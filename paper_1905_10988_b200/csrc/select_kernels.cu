@@ -11,7 +11,10 @@
 //   hist x3   : histogram of the next digit (11, 11, 10 bits) over the keys that match the
 //               digits fixed so far; per-block shared-memory histogram, flushed with integer atomics
 //   choose x3 : one block finds the digit bin holding the q-th key and fixes it
+//               (if few keys share the digits fixed after pass 0 or 1, the later passes are
+//               skipped on the device and those keys are collected as candidates instead)
 //   mark      : per 1024-element tile the masks "key < T" and "key == T" (T = the q-th key)
+//   candidates: one block finishes the selection on the collected (key, coordinate) pairs
 //   scan      : exclusive offsets of the per-block counts of "== T"
 //   resolve   : final mask = "< T" plus the first r of the "== T" in index order; per-block
 //               kept counts (and norm partials for the sparsifier)
@@ -32,9 +35,11 @@ __host__ __device__ constexpr uint32_t sel_fixed(int pass) {
     return pass == 0 ? 0u : pass == 1 ? 0xFFE00000u : 0xFFFFFC00u;
 }
 
+constexpr uint32_t kCandCap = 1u << 18;      // candidate list entries (8 bytes each)
+
 struct SelectState {
     uint32_t prefix;        // digits fixed so far; after the last pass the q-th smallest key T
-    uint32_t pad;
+    uint32_t mode;          // 0: all three digit passes; 1 / 2: candidates collected after pass 0 / 1
     uint64_t remaining;     // how many keys to take among those matching the prefix
 };
 
@@ -44,11 +49,14 @@ struct SelectWorkspace {
     uint32_t* hist;         // kSelPasses * kSelBins
     SelectState* state;
     uint32_t* count;        // listed entries (TopK)
+    uint32_t* cand_count;
+    uint2* cand;            // kCandCap pairs (key, coordinate)
 };
 
 inline size_t select_extra_bytes(uint64_t d) {
     const uint64_t t = sparse_tiles(d);
-    return round_up16(t * 128) + round_up16(t * 4) + (size_t)kSelPasses * kSelBins * 4 + 64;
+    return round_up16(t * 128) + round_up16(t * 4) + (size_t)kSelPasses * kSelBins * 4 + 64 +
+           (size_t)kCandCap * 8;
 }
 
 __host__ __device__ inline SelectWorkspace select_ws_carve(char* p, uint64_t d) {
@@ -59,6 +67,8 @@ __host__ __device__ inline SelectWorkspace select_ws_carve(char* p, uint64_t d) 
     w.hist = reinterpret_cast<uint32_t*>(p);     p += (size_t)kSelPasses * kSelBins * 4;
     w.state = reinterpret_cast<SelectState*>(p);
     w.count = reinterpret_cast<uint32_t*>(p + 32);
+    w.cand_count = reinterpret_cast<uint32_t*>(p + 36);
+    w.cand = reinterpret_cast<uint2*>(p + 64);
     return w;
 }
 
@@ -79,6 +89,12 @@ struct StreamKeys {          // selection-stream word of the coordinate
     __device__ __forceinline__ void load(const Tile& t, uint64_t, int, int k, uint64_t,
                                          uint32_t (&out)[4]) const {
         stream_words4_tile(t.q_lo + (uint32_t)(k * 32), t.pt, keys, out);
+    }
+    // the key of element k*128 + 4*lane + c of the tile alone (recomputed)
+    __device__ __forceinline__ uint32_t key_at(const Tile& t, uint64_t, int, int k, int c) const {
+        uint32_t out[4];
+        stream_words4_tile(t.q_lo + (uint32_t)(k * 32), t.pt, keys, out);
+        return c == 0 ? out[0] : c == 1 ? out[1] : c == 2 ? out[2] : out[3];
     }
 };
 
@@ -101,6 +117,10 @@ struct MagnitudeKeys {       // largest |x| first: complement of the magnitude b
                 out[c] = (j + c < d) ? ~(__float_as_uint(x[j + c]) & 0x7FFFFFFFu) : 0xFFFFFFFFu;
         }
     }
+    __device__ __forceinline__ uint32_t key_at(const Tile&, uint64_t base, int lane, int k,
+                                               int c) const {
+        return ~(__float_as_uint(x[base + (uint64_t)(k * 128 + lane * 4 + c)]) & 0x7FFFFFFFu);
+    }
 };
 
 // bits of the load layout (bit 4k+c <-> element k*128 + 4*lane + c) that lie inside [0, d)
@@ -120,9 +140,10 @@ __global__ void select_init_kernel(SelectWorkspace ws, const uint64_t q) {
     for (int i = threadIdx.x; i < kSelPasses * kSelBins; i += blockDim.x) ws.hist[i] = 0u;
     if (threadIdx.x == 0) {
         ws.state->prefix = 0u;
-        ws.state->pad = 0u;
+        ws.state->mode = 0u;
         ws.state->remaining = q;
         *ws.count = 0u;
+        *ws.cand_count = 0u;
     }
 }
 
@@ -133,6 +154,8 @@ select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws) {
     constexpr int bins = sel_bins(PASS);
     constexpr int shift = sel_shift(PASS);
     constexpr uint32_t fixed = sel_fixed(PASS);
+    // candidates already collected: the remaining digits are found on the candidate list
+    if (PASS > 0 && ws.state->mode != 0u) return;
     __shared__ uint32_t s_hist[bins];
     for (int i = threadIdx.x; i < bins; i += kBlockThreads) s_hist[i] = 0u;
     __syncthreads();
@@ -164,10 +187,13 @@ select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws) {
 }
 
 // one block of 1024 threads, two bins each: the bin in which the cumulative count reaches
-// `remaining` becomes the next digit
+// `remaining` becomes the next digit.  If few enough keys share the digits fixed so far (passes 0
+// and 1), the remaining passes over all d keys are skipped: the mark kernel collects those keys
+// and the candidate kernel finishes the selection on the list.
 template <int PASS>
 __global__ void __launch_bounds__(kScanThreads) select_choose_kernel(const SelectWorkspace ws) {
     constexpr int bins = sel_bins(PASS);
+    if (PASS > 0 && ws.state->mode != 0u) return;
     const uint32_t* __restrict__ hist = ws.hist + PASS * kSelBins;
     __shared__ uint64_t s_sum[kScanThreads];
     const int t = threadIdx.x;
@@ -184,16 +210,21 @@ __global__ void __launch_bounds__(kScanThreads) select_choose_kernel(const Selec
     const uint64_t remaining = ws.state->remaining;
     const uint64_t before = s_sum[t] - h0 - h1;         // keys in lower bins
     __syncthreads();                                    // everyone has read the state
-    if (remaining > before && remaining <= before + h0) {
-        ws.state->prefix |= (uint32_t)(2 * t) << sel_shift(PASS);
-        ws.state->remaining = remaining - before;
-    } else if (remaining > before + h0 && remaining <= before + h0 + h1) {
-        ws.state->prefix |= (uint32_t)(2 * t + 1) << sel_shift(PASS);
-        ws.state->remaining = remaining - before - h0;
+    int pick = -1;
+    if (remaining > before && remaining <= before + h0) pick = 0;
+    else if (remaining > before + h0 && remaining <= before + h0 + h1) pick = 1;
+    if (pick >= 0) {
+        ws.state->prefix |= (uint32_t)(2 * t + pick) << sel_shift(PASS);
+        ws.state->remaining = remaining - before - (pick ? h0 : 0u);
+        if (PASS < 2 && (pick ? h1 : h0) <= kCandCap) ws.state->mode = (uint32_t)(PASS + 1);
     }
 }
 
-// grid: ceil(tiles / warps per block); one tile per warp
+// grid: ceil(tiles / warps per block); one tile per warp.  With sh = 0 (all digits fixed) the
+// masks are "key < T" and "key == T"; with candidates (sh = 21 or 10 undecided low bits) they are
+// "fixed digits below the prefix" and, instead of a tie mask, the keys whose fixed digits equal
+// the prefix go to the candidate list: one reservation on the global counter per block, the
+// (rare) candidate keys recomputed one by one.
 template <class Src>
 __global__ void __launch_bounds__(kBlockThreads)
 select_mark_kernel(const Src src, const uint64_t d, uint32_t* __restrict__ less_mask,
@@ -203,19 +234,24 @@ select_mark_kernel(const Src src, const uint64_t d, uint32_t* __restrict__ less_
     const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
     const uint64_t base = tile * kTile;
     const bool active = base < d;
-    const uint32_t T = ws.state->prefix;
+    const uint32_t mode = ws.state->mode;
+    const int sh = mode == 0u ? 0 : mode == 1u ? 21 : 10;
+    const uint32_t T = ws.state->prefix >> sh;
     __shared__ uint32_t s_eq[kWarpsPerBlock];
+    __shared__ uint32_t s_base;
     uint32_t less = 0, equal = 0;
+    typename Src::Tile t;
     if (active) {
-        const typename Src::Tile t = src.tile(base, lane);
+        t = src.tile(base, lane);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             uint32_t key[4];
             src.load(t, base, lane, k, d, key);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                less |= (key[c] < T ? 1u : 0u) << (4 * k + c);
-                equal |= (key[c] == T ? 1u : 0u) << (4 * k + c);
+                const uint32_t hi = key[c] >> sh;
+                less |= (hi < T ? 1u : 0u) << (4 * k + c);
+                equal |= (hi == T ? 1u : 0u) << (4 * k + c);
             }
         }
         const uint32_t valid = valid_nibbles(base, lane, d);
@@ -223,18 +259,136 @@ select_mark_kernel(const Src src, const uint64_t d, uint32_t* __restrict__ less_
         equal &= valid;
     }
     const uint32_t lw = canonical_mask_word(less, lane);
-    const uint32_t ew = canonical_mask_word(equal, lane);
+    const uint32_t ew = (mode == 0u) ? canonical_mask_word(equal, lane) : 0u;
     if (active) {
         less_mask[tile * 32 + lane] = lw;
         ws.eqmask[tile * 32 + lane] = ew;
     }
-    const uint32_t ne = warp_sum_u(__popc(ew));
-    if (lane == 0) s_eq[warp] = ne;
+    // ties (mode 0) or candidates (modes 1, 2) of this lane, then of the warps before it
+    const uint32_t mine = __popc(equal);
+    uint32_t incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_eq[warp] = incl;
     __syncthreads();
+    uint32_t block_total = 0, before = incl - mine;
+    for (int w = 0; w < kWarpsPerBlock; ++w) {
+        if (w < warp) before += s_eq[w];
+        block_total += s_eq[w];
+    }
+    if (mode == 0u) {
+        if (threadIdx.x == 0) ws.eq_block[blockIdx.x] = block_total;
+        return;
+    }
     if (threadIdx.x == 0) {
-        uint32_t c = 0;
-        for (int w = 0; w < kWarpsPerBlock; ++w) c += s_eq[w];
-        ws.eq_block[blockIdx.x] = c;
+        ws.eq_block[blockIdx.x] = 0u;
+        s_base = block_total ? atomicAdd(ws.cand_count, block_total) : 0u;
+    }
+    __syncthreads();
+    uint32_t at = s_base + before;
+    while (equal) {
+        const int bit = __ffs(equal) - 1;
+        equal &= equal - 1;
+        if (at < kCandCap)
+            ws.cand[at] = make_uint2(src.key_at(t, base, lane, bit >> 2, bit & 3),
+                                     (uint32_t)(base + (uint64_t)((bit >> 2) * 128 + lane * 4 + (bit & 3))));
+        ++at;
+    }
+}
+
+// One block.  Finishes the selection on the candidate list: the `remaining` smallest pairs
+// (key, coordinate) among the candidates are selected, digit by digit over the undecided key bits
+// and then, only while equal keys remain undecided, over the coordinate bits; stops as soon as a
+// digit bin is taken whole.  Selected coordinates are set in the mask.
+__global__ void __launch_bounds__(kScanThreads)
+select_candidates_kernel(uint32_t* __restrict__ mask, const SelectWorkspace ws) {
+    const uint32_t mode = ws.state->mode;
+    if (mode == 0u) return;
+    __shared__ uint32_t s_hist[kSelBins];
+    __shared__ uint32_t s_scan[kScanThreads];
+    __shared__ unsigned long long s_prefix;
+    __shared__ uint32_t s_remaining, s_done;
+    const int t = threadIdx.x;
+    const uint32_t n = min(*ws.cand_count, kCandCap);
+    const uint2* __restrict__ cand = ws.cand;
+    if (t == 0) {
+        s_prefix = (unsigned long long)ws.state->prefix << 32;
+        s_remaining = (uint32_t)ws.state->remaining;
+        s_done = 0u;
+    }
+    __syncthreads();
+    // digit positions in the 64-bit pair (key << 32 | coordinate): shift, width
+    const int shifts[5] = {42, 32, 21, 10, 0};
+    const int widths[5] = {11, 10, 11, 11, 10};
+    int final_shift = 0;
+    for (int pass = (mode == 1u ? 0 : 1); pass < 5; ++pass) {
+        const int shift = shifts[pass];
+        const int bins = 1 << widths[pass];
+        for (int i = t; i < kSelBins; i += kScanThreads) s_hist[i] = 0u;
+        __syncthreads();
+        const unsigned long long prefix = s_prefix;
+        const int above = shift + widths[pass];
+        for (uint32_t i0 = t; i0 < n; i0 += 8 * kScanThreads) {      // 8 loads in flight
+            uint2 e[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const uint32_t i = i0 + u * kScanThreads;
+                e[u] = (i < n) ? cand[i] : make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const unsigned long long v = ((unsigned long long)e[u].x << 32) | e[u].y;
+                if (i0 + u * kScanThreads < n && (v >> above) == (prefix >> above))
+                    atomicAdd(&s_hist[(uint32_t)(v >> shift) & (uint32_t)(bins - 1)], 1u);
+            }
+        }
+        __syncthreads();
+        const uint32_t h0 = (2 * t < bins) ? s_hist[2 * t] : 0u;
+        const uint32_t h1 = (2 * t + 1 < bins) ? s_hist[2 * t + 1] : 0u;
+        s_scan[t] = h0 + h1;
+        __syncthreads();
+        for (int o = 1; o < kScanThreads; o <<= 1) {
+            const uint32_t v = (t >= o) ? s_scan[t - o] : 0u;
+            __syncthreads();
+            s_scan[t] += v;
+            __syncthreads();
+        }
+        const uint32_t remaining = s_remaining;
+        const uint32_t before = s_scan[t] - h0 - h1;
+        __syncthreads();
+        int pick = -1;
+        if (remaining > before && remaining <= before + h0) pick = 0;
+        else if (remaining > before + h0 && remaining <= before + h0 + h1) pick = 1;
+        if (pick >= 0) {
+            const uint32_t lower = before + (pick ? h0 : 0u);
+            s_prefix = prefix | ((unsigned long long)(2 * t + pick) << shift);
+            s_remaining = remaining - lower;
+            if ((pick ? h1 : h0) == remaining - lower) s_done = 1u;      // the bin is taken whole
+        }
+        __syncthreads();
+        final_shift = shift;
+        if (s_done) break;
+    }
+    // pairs are distinct, so the loop ends with s_done set at the latest after the last pass
+    const unsigned long long limit = s_prefix >> final_shift;
+    const unsigned long long fixed_hi = s_prefix >> (mode == 1u ? 53 : 42);
+    for (uint32_t i0 = t; i0 < n; i0 += 8 * kScanThreads) {
+        uint2 e[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t i = i0 + u * kScanThreads;
+            e[u] = (i < n) ? cand[i] : make_uint2(0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const unsigned long long v = ((unsigned long long)e[u].x << 32) | e[u].y;
+            if (i0 + u * kScanThreads < n && (v >> (mode == 1u ? 53 : 42)) == fixed_hi &&
+                (v >> final_shift) <= limit)
+                atomicOr(&mask[e[u].y >> 5], 1u << (e[u].y & 31u));
+        }
     }
 }
 
@@ -242,28 +396,8 @@ select_mark_kernel(const Src src, const uint64_t d, uint32_t* __restrict__ less_
 __global__ void __launch_bounds__(kScanThreads)
 select_scan_counts_kernel(uint32_t* __restrict__ counts, const uint64_t n,
                           uint32_t* __restrict__ total) {
-    __shared__ uint32_t s_cnt[kScanThreads];
-    const int t = threadIdx.x;
-    const uint64_t per = (n + kScanThreads - 1) / kScanThreads;
-    const uint64_t t0 = (uint64_t)t * per;
-    const uint64_t t1 = (t0 + per < n) ? t0 + per : n;
-    uint32_t c = 0;
-    for (uint64_t i = t0; i < t1; ++i) c += counts[i];
-    s_cnt[t] = c;
-    __syncthreads();
-    for (int o = 1; o < kScanThreads; o <<= 1) {
-        const uint32_t v = (t >= o) ? s_cnt[t - o] : 0u;
-        __syncthreads();
-        s_cnt[t] += v;
-        __syncthreads();
-    }
-    uint32_t run = s_cnt[t] - c;
-    for (uint64_t i = t0; i < t1; ++i) {
-        const uint32_t v = counts[i];
-        counts[i] = run;
-        run += v;
-    }
-    if (t == kScanThreads - 1 && total) *total = s_cnt[t];
+    const uint32_t sum = block_exclusive_scan_inplace(counts, n);
+    if (threadIdx.x == 0 && total) *total = sum;
 }
 
 // grid: ceil(tiles / warps per block).  mask <- "< T" | first r of "== T"; per-block kept counts;
@@ -405,6 +539,7 @@ static void run_select(const Src& src, uint64_t d, uint64_t q, const SparseWorks
     select_hist_kernel<Src, 2><<<pgrid, kBlockThreads, 0, stream>>>(src, d, ws);
     select_choose_kernel<2><<<1, kScanThreads, 0, stream>>>(ws);
     select_mark_kernel<Src><<<(unsigned)groups, kBlockThreads, 0, stream>>>(src, d, sp.bitmask, ws);
+    select_candidates_kernel<<<1, kScanThreads, 0, stream>>>(sp.bitmask, ws);
     select_scan_counts_kernel<<<1, kScanThreads, 0, stream>>>(ws.eq_block, groups, nullptr);
 }
 

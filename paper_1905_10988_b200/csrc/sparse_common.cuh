@@ -174,6 +174,57 @@ __device__ __forceinline__ uint32_t stream_word_at(uint64_t j, uint32_t worker, 
     return (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1] : (j & 3) == 2 ? r4[2] : r4[3];
 }
 
+// One block of kScanThreads threads: in-place exclusive scan of counts[0, n); every thread gets
+// the total.  Chunks of 4 * kScanThreads values, one coalesced 16-byte load per thread and chunk
+// (the array is 16-byte aligned and allocated up to a multiple of 4 entries).
+__device__ __forceinline__ uint32_t block_exclusive_scan_inplace(uint32_t* __restrict__ counts,
+                                                                 const uint64_t n) {
+    __shared__ uint32_t s_warp[32];
+    const int t = threadIdx.x;
+    const int lane = t & 31;
+    const int warp = t >> 5;
+    uint32_t carry = 0;
+    for (uint64_t c0 = 0; c0 < n; c0 += 4ull * kScanThreads) {
+        const uint64_t i = c0 + 4ull * t;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (i < n) v = *reinterpret_cast<const uint4*>(counts + i);
+        if (i + 1 >= n) v.y = 0u;
+        if (i + 2 >= n) v.z = 0u;
+        if (i + 3 >= n) v.w = 0u;
+        const uint32_t sum = v.x + v.y + v.z + v.w;
+        uint32_t incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += u;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            uint32_t w = s_warp[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, w, o);
+                if (lane >= o) w += u;
+            }
+            s_warp[lane] = w;
+        }
+        __syncthreads();
+        const uint32_t run = carry + (warp ? s_warp[warp - 1] : 0u) + incl - sum;
+        if (i < n) {
+            uint4 o;
+            o.x = run;
+            o.y = o.x + v.x;
+            o.z = o.y + v.y;
+            o.w = o.z + v.z;
+            *reinterpret_cast<uint4*>(counts + i) = o;
+        }
+        carry += s_warp[31];
+        __syncthreads();
+    }
+    return carry;
+}
+
 // Given, per worker, the selection bitmask, the per-block kept counts and the norm partials in
 // the workspace (what the select kernels leave): norm, level rounding, dropping of level-0
 // entries, index list and code planes of the compact format.  Defined with the sparsifier

@@ -82,31 +82,18 @@ sparse_scan_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
     const uint64_t* __restrict__ tile_partial = ws.block_partial;
     uint32_t* __restrict__ count = batch.count[blockIdx.y];
     float* __restrict__ norm = batch.norm[blockIdx.y];
-    __shared__ uint32_t s_cnt[kScanThreads];
     __shared__ double s_sum[kScanThreads];
     __shared__ uint32_t s_max[kScanThreads];
     const int t = threadIdx.x;
-    const uint64_t per = (tiles + kScanThreads - 1) / kScanThreads;
-    const uint64_t t0 = (uint64_t)t * per;
-    const uint64_t t1 = (t0 + per < tiles) ? t0 + per : tiles;
-    uint32_t c = 0, m = 0;
+    uint32_t m = 0;
     double s = 0.0;
-    for (uint64_t i = t0; i < t1; ++i) {
-        c += tile_count[i];
+    for (uint64_t i = t; i < tiles; i += kScanThreads) {     // fixed order per thread
         if (P == NC_P_INF) m = max(m, (uint32_t)tile_partial[i]);
         else s += __longlong_as_double((long long)tile_partial[i]);
     }
-    s_cnt[t] = c;
     s_sum[t] = s;
     s_max[t] = m;
     __syncthreads();
-    // inclusive Hillis-Steele scan of the per-thread counts
-    for (int o = 1; o < kScanThreads; o <<= 1) {
-        const uint32_t v = (t >= o) ? s_cnt[t - o] : 0u;
-        __syncthreads();
-        s_cnt[t] += v;
-        __syncthreads();
-    }
     // fixed-shape tree for the norm partials
     for (int o = kScanThreads / 2; o > 0; o >>= 1) {
         if (t < o) {
@@ -115,14 +102,9 @@ sparse_scan_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
         }
         __syncthreads();
     }
-    uint32_t run = s_cnt[t] - c;     // exclusive prefix of this thread's chunk
-    for (uint64_t i = t0; i < t1; ++i) {
-        const uint32_t v = tile_count[i];
-        tile_count[i] = run;
-        run += v;
-    }
+    const uint32_t total = block_exclusive_scan_inplace(tile_count, tiles);
     if (t == 0) {
-        *count = s_cnt[kScanThreads - 1];
+        *count = total;
         float r;
         if (P == NC_P_INF) r = __uint_as_float(s_max[0]);
         else if (P == 1) r = (float)s_sum[0];

@@ -135,6 +135,31 @@ def test_topk_ties_specials_and_decode_accumulate():
     assert np.array_equal(idx.numpy(np.uint32)[:77], np.arange(77, dtype=np.uint32))
 
 
+@pytest.mark.parametrize("kind", ["one_binade_slice", "all_equal", "two_values"])
+def test_topk_every_selection_route(kind):
+    # the device picks between three routes by how many keys share the leading digits of the
+    # K-th key: candidates after the first digit (the cases above), candidates after the second
+    # digit (more than 2^18 keys share the first 11 key bits), and all three digit passes with
+    # ties broken by index (more than 2^18 keys equal in the first 22 bits)
+    rng = np.random.default_rng(12)
+    d = (1 << 20) + 77
+    if kind == "one_binade_slice":
+        x = (1.0 + rng.random(d) * 0.0624).astype(np.float32)
+        x *= rng.choice(np.float32([-1, 1]), d)
+        K = 5000
+    elif kind == "all_equal":
+        x = np.full(d, 0.75, np.float32)
+        K = 300_001
+    else:
+        x = np.where(rng.random(d) < 0.4, np.float32(2.0), np.float32(-1.0)).astype(np.float32)
+        K = int((x == 2.0).sum()) + 123_456          # all the 2.0 and the first 123,456 of the -1.0
+    idx, exp, sign, listed = _gpu_topk(x, K, 4, 9)
+    i_ref, e_ref, s_ref = oracle.topk_compress(x, K, 4, 9)
+    assert np.array_equal(idx.numpy(np.uint32)[:listed], i_ref)
+    assert np.array_equal(exp.numpy(np.uint8)[:listed], e_ref)
+    assert np.array_equal(sign.numpy(np.uint32)[:s_ref.size], s_ref)
+
+
 def test_exact_and_topk_on_config5_shape_sampled():
     # d = 2^26 of the sparse workload (the full 2^28 case is timed by the config bench): exact
     # count and threshold property checked in full, listed entries against the oracle on a prefix
