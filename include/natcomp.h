@@ -273,6 +273,38 @@ nc_status nc8_aggregate(const uint8_t* const* codes, int n, size_t d, float* out
 nc_status nc8_aggregate_compress(const uint8_t* const* codes, int n, size_t d, uint64_t seed,
                                  uint32_t master, uint8_t* out_code, cudaStream_t stream);
 
+/* ---- 16-bit inputs ---------------------------------------------------------------------------
+ * C_nat (Def. 1) of a bfloat16 or binary16 vector.  Such a value is a binary32 value, so the
+ * operator is the binary32 rule of Sec. 2 on the exactly converted input: same 9-bit code, same
+ * planes and same stream (seed, worker, domain 0, j) as nc_compress; the up-probability is the
+ * 7- or 10-bit mantissa fraction (for a binary16 subnormal: its fraction of the binade).
+ * x: device pointer to 16-bit patterns, 16-byte aligned.  dtype NC_DTYPE_F32 forwards to
+ * nc_compress; other values give NC_ERR_UNSUPPORTED. */
+enum { NC_DTYPE_F32 = 0, NC_DTYPE_BF16 = 1, NC_DTYPE_F16 = 2 };
+nc_status nc_compress_typed(const void* x, int dtype, size_t d, uint64_t seed, uint32_t worker,
+                            uint8_t* exp, uint32_t* sign, cudaStream_t stream);
+nc_status nc_compress_typed_batch(const void* const* xs, int dtype, size_t d, uint64_t seed,
+                                  const uint32_t* workers, uint8_t* const* exps,
+                                  uint32_t* const* signs, int n, cudaStream_t stream);
+
+/* ---- binary64 inputs: 12-bit codes -------------------------------------------------------------
+ * Sec. 2: "11 bits for the exponent and 1 for the sign".  C_nat (Def. 1) of a binary64 vector with
+ * a 52-bit threshold: r52 = (low 23 bits of the stream word (seed, worker, domain 0, j)) << 29 |
+ * (stream word (seed, worker, domain 3, j) >> 3); round up iff r52 < the 52-bit mantissa field.
+ * Planes: exp_lo[j] = low 8 bits of the rounded 11-bit exponent field (nc_exp_bytes(d) bytes);
+ * hi: 4 bits per entry, (sign << 3) | (exponent field >> 8), entry j in nibble j mod 2 of byte
+ * j / 2 (nd_level_bytes(d) bytes).  Padding bytes are written as 0.  Subnormals round to +-0 or
+ * +-2^-1022, 2^1023 and above stay, +-inf and NaN give exponent field 2047.  x 32-byte aligned. */
+nc_status nc64_compress(const double* x, size_t d, uint64_t seed, uint32_t worker, uint8_t* exp_lo,
+                        uint8_t* hi, cudaStream_t stream);
+nc_status nc64_compress_batch(const double* const* xs, size_t d, uint64_t seed,
+                              const uint32_t* workers, uint8_t* const* exp_los,
+                              uint8_t* const* his, int n, cudaStream_t stream);
+/* Master side (Algorithm 1, aggregate): out[j] = sum over the n workers, in that order, of the
+ * decoded values, binary64 adds starting from +0.  out: double[d], 32-byte aligned. */
+nc_status nc64_aggregate(const uint8_t* const* exp_los, const uint8_t* const* his, int n, size_t d,
+                         double* out, cudaStream_t stream);
+
 /* ---- exactly q kept coordinates: S^q then D_nat, and TopK then C_nat -------------------------
  * The sparsifier definition of the appendix with exactly q non-zeros ("S^q": xi a uniformly random
  * subset of size q, probabilities q/d), composed with D_nat^{p,s} (Def. 3, Thm. 3), and the

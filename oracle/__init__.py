@@ -412,3 +412,63 @@ def topk_decode_accumulate(idx, exp, sign, acc) -> None:
     assert acc.dtype == np.float32 and acc.flags.c_contiguous
     _topk_decode_accumulate(_p(idx, _u32p), _p(exp, _u8p), _p(sign, _u32p), idx.size,
                             _p(acc, _f32p))
+
+
+_u16p = C.POINTER(C.c_uint16)
+_nc_compress_typed = _sig("orc_nc_compress_typed", None, _u16p, C.c_int, C.c_uint64, C.c_uint64,
+                          C.c_uint32, _u8p, _u32p)
+_values_of_16bit = _sig("orc_values_of_16bit", None, _u16p, C.c_int, C.c_uint64, _f32p)
+DTYPE_BF16, DTYPE_F16 = 1, 2
+
+
+def nc_compress_typed(x16, dtype: int, seed: int, worker: int):
+    """C_nat of bfloat16 (dtype 1) or binary16 (dtype 2) bit patterns: exponent bytes, sign words."""
+    x16 = _arr(x16, np.uint16)
+    exp = np.zeros(x16.size, np.uint8)
+    sign = np.zeros((x16.size + 31) // 32, np.uint32)
+    _nc_compress_typed(_p(x16, _u16p), dtype, x16.size, seed, worker, _p(exp, _u8p),
+                       _p(sign, _u32p))
+    return exp, sign
+
+
+def values_of_16bit(x16, dtype: int) -> np.ndarray:
+    x16 = _arr(x16, np.uint16)
+    out = np.zeros(x16.size, np.float32)
+    _values_of_16bit(_p(x16, _u16p), dtype, x16.size, _p(out, _f32p))
+    return out
+
+
+_u64p = C.POINTER(C.c_uint64)
+_nc64_compress = _sig("orc_nc64_compress", None, _f64p, C.c_uint64, C.c_uint64, C.c_uint32, _u8p,
+                      _u8p)
+_nc64_aggregate = _sig("orc_nc64_aggregate", None, C.POINTER(_u8p), C.POINTER(_u8p), C.c_int,
+                       C.c_uint64, _f64p)
+_cnat64_values = _sig("orc_cnat64_values", None, _f64p, _u64p, C.c_uint64, _f64p)
+
+
+def nc64_compress(x, seed: int, worker: int):
+    """C_nat of a binary64 vector: low exponent bytes and the (sign, high exponent) nibble plane."""
+    x = _arr(x, np.float64)
+    exp_lo = np.zeros(x.size, np.uint8)
+    hi = np.zeros((x.size + 1) // 2, np.uint8)
+    _nc64_compress(_p(x, _f64p), x.size, seed, worker, _p(exp_lo, _u8p), _p(hi, _u8p))
+    return exp_lo, hi
+
+
+def nc64_aggregate(exp_los, his, d: int) -> np.ndarray:
+    n = len(exp_los)
+    exp_los = [_arr(e, np.uint8) for e in exp_los]
+    his = [_arr(h, np.uint8) for h in his]
+    ea = (_u8p * n)(*[_p(e, _u8p) for e in exp_los])
+    ha = (_u8p * n)(*[_p(h, _u8p) for h in his])
+    out = np.zeros(d, np.float64)
+    _nc64_aggregate(ea, ha, n, d, _p(out, _f64p))
+    return out
+
+
+def cnat64_values(t, r52) -> np.ndarray:
+    t = _arr(t, np.float64)
+    r52 = _arr(r52, np.uint64)
+    out = np.zeros(t.size, np.float64)
+    _cnat64_values(_p(t, _f64p), _p(r52, _u64p), t.size, _p(out, _f64p))
+    return out

@@ -735,4 +735,122 @@ void orc_topk_decode_accumulate(const uint32_t* idx, const uint8_t* exp, const u
     }
 }
 
+// ---- 16-bit inputs ----------------------------------------------------------------------
+// The real value of a bfloat16 (8-bit exponent, 7-bit mantissa) or binary16 (5-bit exponent,
+// 10-bit mantissa) pattern, by the format definition.  Both are exactly representable in binary32.
+static float value_of_16bit(uint16_t h, int dtype) {
+    const int sign = h >> 15;
+    double a;
+    if (dtype == 1) {                                   // bfloat16
+        const int e = (h >> 7) & 0xFF, m = h & 0x7F;
+        if (e == 0xFF) a = m ? std::numeric_limits<double>::quiet_NaN()
+                             : std::numeric_limits<double>::infinity();
+        else if (e == 0) a = std::ldexp((double)m / 128.0, -126);
+        else a = std::ldexp(1.0 + (double)m / 128.0, e - 127);
+    } else {                                            // binary16
+        const int e = (h >> 10) & 0x1F, m = h & 0x3FF;
+        if (e == 0x1F) a = m ? std::numeric_limits<double>::quiet_NaN()
+                             : std::numeric_limits<double>::infinity();
+        else if (e == 0) a = std::ldexp((double)m / 1024.0, -14);
+        else a = std::ldexp(1.0 + (double)m / 1024.0, e - 15);
+    }
+    return (float)(sign ? -a : a);
+}
+
+// C_nat (Def. 1) of 16-bit inputs: the operator on the real value, coded as for binary32.
+void orc_nc_compress_typed(const uint16_t* x, int dtype, uint64_t d, uint64_t seed,
+                           uint32_t worker, uint8_t* exp, uint32_t* sign) {
+    std::memset(sign, 0, (size_t)((d + 31) / 32) * 4);
+    for (uint64_t j = 0; j < d; ++j) {
+        const float t = value_of_16bit(x[j], dtype);
+        const uint32_t r23 = stream_word(seed, worker, 0u, j) & 0x7FFFFFu;
+        uint32_t sb;
+        cnat_code(cnat_value(t, r23), &exp[j], &sb);
+        sign[j / 32] |= sb << (j % 32);
+    }
+}
+
+void orc_values_of_16bit(const uint16_t* x, int dtype, uint64_t d, float* out) {
+    for (uint64_t j = 0; j < d; ++j) out[j] = value_of_16bit(x[j], dtype);
+}
+
+// ---- binary64 inputs: 11-bit exponent + sign ---------------------------------------------
+// Def. 1 on a binary64 t ("11 bits for the exponent and 1 for the sign", Sec. 2).  The mantissa has
+// 52 bits, so the threshold needs 52 random bits: r52 = (low 23 bits of the domain-0 word of
+// element j) * 2^29 + (domain-3 word of element j) / 8, "up" iff r52 < (1 - p(t)) * 2^52.
+// Edge policy as for binary32 with the binary64 limits (subnormals bracket [0, 2^-1022],
+// 2^1023 and above never round up, inf / NaN give exponent field 2047).
+static double cnat64_value(double t, uint64_t r52) {
+    if (t == 0.0) return t;
+    if (std::isnan(t) || std::isinf(t))
+        return std::copysign(std::numeric_limits<double>::infinity(), t);
+    const double a = std::fabs(t);
+    double lo, hi;
+    if (a < 0x1p-1022) {
+        lo = 0.0;
+        hi = 0x1p-1022;
+    } else {
+        const int fl = std::ilogb(a);
+        lo = std::ldexp(1.0, fl);
+        if (fl >= 1023) return std::copysign(lo, t);
+        hi = std::ldexp(1.0, fl + 1);
+    }
+    const double p_up = (a - lo) / (hi - lo);            // exact: a - lo and a power of two
+    const bool up = (double)r52 < p_up * 0x1p52;          // both sides exact integers below 2^53
+    return std::copysign(up ? hi : lo, t);
+}
+
+static uint64_t stream_r52(uint64_t seed, uint32_t worker, uint64_t j) {
+    const uint64_t top = stream_word(seed, worker, 0u, j) & 0x7FFFFFu;
+    const uint64_t low = stream_word(seed, worker, 3u, j) >> 3;
+    return (top << 29) | low;
+}
+
+// 12-bit code of +-0, +-2^k, +-inf: 11-bit biased exponent and the sign
+static void cnat64_code(double value, uint32_t* e11, uint32_t* sign_bit) {
+    *sign_bit = std::signbit(value) ? 1u : 0u;
+    const double a = std::fabs(value);
+    if (a == 0.0) *e11 = 0;
+    else if (std::isinf(a)) *e11 = 2047;
+    else *e11 = (uint32_t)(std::ilogb(a) + 1023);
+}
+
+// exp_lo[j] = low 8 bits of the exponent field; nibble (j mod 2) of hi[j / 2] = sign * 8 +
+// (exponent field >> 8)
+void orc_nc64_compress(const double* x, uint64_t d, uint64_t seed, uint32_t worker,
+                       uint8_t* exp_lo, uint8_t* hi) {
+    std::memset(hi, 0, (size_t)((d + 1) / 2));
+    for (uint64_t j = 0; j < d; ++j) {
+        uint32_t e11, sb;
+        cnat64_code(cnat64_value(x[j], stream_r52(seed, worker, j)), &e11, &sb);
+        exp_lo[j] = (uint8_t)(e11 & 0xFFu);
+        hi[j / 2] |= (uint8_t)(((sb << 3) | (e11 >> 8)) << (4 * (j % 2)));
+    }
+}
+
+static double cnat64_decode(uint32_t e11, uint32_t sign_bit) {
+    double a;
+    if (e11 == 0) a = 0.0;
+    else if (e11 == 2047) a = std::numeric_limits<double>::infinity();
+    else a = std::ldexp(1.0, (int)e11 - 1023);
+    return sign_bit ? -a : a;
+}
+
+// out[j] = sum over the workers, in worker order, of the decoded values (binary64 adds from +0)
+void orc_nc64_aggregate(const uint8_t* const* exp_lo, const uint8_t* const* hi, int n, uint64_t d,
+                        double* out) {
+    for (uint64_t j = 0; j < d; ++j) {
+        double acc = 0.0;
+        for (int i = 0; i < n; ++i) {
+            const uint32_t nib = (hi[i][j / 2] >> (4 * (j % 2))) & 0xFu;
+            acc = acc + cnat64_decode(((nib & 7u) << 8) | exp_lo[i][j], nib >> 3);
+        }
+        out[j] = acc;
+    }
+}
+
+void orc_cnat64_values(const double* t, const uint64_t* r52, uint64_t n, double* out) {
+    for (uint64_t i = 0; i < n; ++i) out[i] = cnat64_value(t[i], r52[i]);
+}
+
 }  // extern "C"

@@ -38,7 +38,8 @@ EXPORTS = (
     "nd_sparse_plane_bytes", "nd_sparse_compact_compress", "nd_sparse_compact_compress_batch",
     "nd_sparse_compact_decode_accumulate", "nc8_compress", "nc8_compress_batch", "nc8_aggregate",
     "nc8_aggregate_compress", "nc_select_workspace_bytes", "nd_sparse_exact_compress",
-    "nc_topk_compress", "nc_topk_decode_accumulate",
+    "nc_topk_compress", "nc_topk_decode_accumulate", "nc_compress_typed",
+    "nc_compress_typed_batch", "nc64_compress", "nc64_compress_batch", "nc64_aggregate",
 )
 
 
@@ -399,3 +400,49 @@ def nc_topk_decode_accumulate(idx, exp, sign, count, d, acc, stream=None) -> Non
     _check("nc_topk_decode_accumulate",
            _nc_topk_decode_accumulate(_ptr(idx), _ptr(exp), _ptr(sign), count, d, _ptr(acc),
                                       _stream(stream)))
+
+
+# ---- 16-bit inputs ----------------------------------------------------------------------------
+DTYPE_F32, DTYPE_BF16, DTYPE_F16 = 0, 1, 2
+_nc_compress_typed = _sig("nc_compress_typed", C.c_int, _vp, C.c_int, _sz, C.c_uint64, C.c_uint32,
+                          _vp, _vp, _vp)
+_nc_compress_typed_batch = _sig("nc_compress_typed_batch", C.c_int, C.POINTER(_vp), C.c_int, _sz,
+                                C.c_uint64, C.POINTER(C.c_uint32), C.POINTER(_vp), C.POINTER(_vp),
+                                C.c_int, _vp)
+
+
+def nc_compress_typed(x, dtype, d, seed, worker, exp, sign, stream=None) -> None:
+    _check("nc_compress_typed", _nc_compress_typed(_ptr(x), dtype, d, seed, worker, _ptr(exp),
+                                                   _ptr(sign), _stream(stream)))
+
+
+def nc_compress_typed_batch(xs, dtype, d, seed, workers, exps, signs, n, stream=None) -> None:
+    w = (C.c_uint32 * n)(*[int(v) for v in workers])
+    _check("nc_compress_typed_batch",
+           _nc_compress_typed_batch(_ptrs(xs), dtype, d, seed, w, _ptrs(exps), _ptrs(signs), n,
+                                    _stream(stream)))
+
+
+# ---- binary64 inputs: 12-bit codes ------------------------------------------------------------
+_nc64_compress = _sig("nc64_compress", C.c_int, _vp, _sz, C.c_uint64, C.c_uint32, _vp, _vp, _vp)
+_nc64_compress_batch = _sig("nc64_compress_batch", C.c_int, C.POINTER(_vp), _sz, C.c_uint64,
+                            C.POINTER(C.c_uint32), C.POINTER(_vp), C.POINTER(_vp), C.c_int, _vp)
+_nc64_aggregate = _sig("nc64_aggregate", C.c_int, C.POINTER(_vp), C.POINTER(_vp), C.c_int, _sz,
+                       _vp, _vp)
+
+
+def nc64_compress(x, d, seed, worker, exp_lo, hi, stream=None) -> None:
+    _check("nc64_compress", _nc64_compress(_ptr(x), d, seed, worker, _ptr(exp_lo), _ptr(hi),
+                                           _stream(stream)))
+
+
+def nc64_compress_batch(xs, d, seed, workers, exp_los, his, n, stream=None) -> None:
+    w = (C.c_uint32 * n)(*[int(v) for v in workers])
+    _check("nc64_compress_batch",
+           _nc64_compress_batch(_ptrs(xs), d, seed, w, _ptrs(exp_los), _ptrs(his), n,
+                                _stream(stream)))
+
+
+def nc64_aggregate(exp_los, his, n, d, out, stream=None) -> None:
+    _check("nc64_aggregate", _nc64_aggregate(_ptrs(exp_los), _ptrs(his), n, d, _ptr(out),
+                                             _stream(stream)))

@@ -73,6 +73,15 @@ def run_cnat(config, n, d, make_vector, iters, peak, with_sum=True):
     _report(config, "nc8_compress_batch (8-bit codes)", m, b, n * d, n * d * 5.0, peak)
     m, b = _time(lambda: nc.nc8_aggregate(es, n, d, out), iters)
     _report(config, "nc8_aggregate (int64 sums)", m, b, d, d * (1.0 * n + 4), peak)
+    # 16-bit inputs (the same operator on bfloat16 / binary16 gradients): 2 + 1.125 bytes per entry
+    for name, tdt, code in (("bf16", torch.bfloat16, nc.DTYPE_BF16),
+                            ("f16", torch.float16, nc.DTYPE_F16)):
+        xh = [x.to(tdt) for x in xs]
+        m, b = _time(lambda: nc.nc_compress_typed_batch(xh, code, d, 0, workers, es, ss, n), iters)
+        _report(config, "nc_compress_typed_batch (%s inputs)" % name, m, b, n * d, n * d * 3.125,
+                peak, {"note": "generator-bound: the multiplier-pipe ceiling is about 1860-2070 "
+                               "Gelem/s, the HBM roof 2093 Gelem/s"})
+        del xh
     if with_sum:
         m, b = _time(lambda: nc.nc_sum_fp32(xs, n, d, out), iters)
         _report(config, "nc_sum_fp32 (uncompressed reference point)", m, b, d, d * (4 * n + 4),

@@ -10,6 +10,9 @@
 // random bits, v + (~r23 & 0x7FFFFF) carries into the exponent field iff r23 < mantissa, i.e.
 // with probability m (Sec. 2: round up with probability m).  The add is suppressed for biased
 // exponents 254 and 255 (saturation / inf / NaN policy).
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "philox.cuh"
 
@@ -160,6 +163,67 @@ nc_compress_kernel(const __grid_constant__ CompressBatch batch, const uint64_t d
     }
     cnat_ragged_tile<kDet>([&](uint64_t j) { return __float_as_uint(x[j]); }, base, d,
                            batch.worker[w], keys, batch.exp[w], batch.sign[w], lane);
+}
+
+// ---- 16-bit inputs --------------------------------------------------------------------
+// bfloat16 and binary16 values are binary32 values, so C_nat of such an input is the binary32
+// rule applied to the exactly converted value: the up-probability m (7 or 10 mantissa bits, or a
+// binary16 subnormal's fraction) is compared with r23 at full width.  Same tile layout; a lane
+// loads 4 consecutive 16-bit elements (8 bytes) per step and widens them.
+struct Compress16Batch {
+    const uint16_t* x[NC_MAX_WORKERS];
+    uint8_t* exp[NC_MAX_WORKERS];
+    uint32_t* sign[NC_MAX_WORKERS];
+    uint32_t worker[NC_MAX_WORKERS];
+};
+
+template <int DT>
+__device__ __forceinline__ uint32_t widen16(uint32_t h) {          // one element, low 16 bits
+    if (DT == NC_DTYPE_BF16) return h << 16;
+    // the conversion may return a canonical NaN: the sign bit is taken from the input
+    const uint32_t f = __float_as_uint(__half2float(__ushort_as_half((unsigned short)h)));
+    return (f & 0x7FFFFFFFu) | ((h & 0x8000u) << 16);
+}
+
+template <int DT>
+__device__ __forceinline__ void widen16x2(uint32_t w, uint32_t& lo, uint32_t& hi) {
+    if (DT == NC_DTYPE_BF16) {
+        lo = w << 16;
+        hi = w & 0xFFFF0000u;
+    } else {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w));
+        lo = (__float_as_uint(f.x) & 0x7FFFFFFFu) | ((w << 16) & 0x80000000u);   // sign of a NaN
+        hi = (__float_as_uint(f.y) & 0x7FFFFFFFu) | (w & 0x80000000u);
+    }
+}
+
+// grid: (ceil(tiles / warps per block), n workers)
+template <int DT>
+__global__ void __launch_bounds__(kBlockThreads)
+nc_compress16_kernel(const __grid_constant__ Compress16Batch batch, const uint64_t d,
+                     const __grid_constant__ PhiloxKeys keys) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t base = tile * kTile;
+    if (base >= d) return;
+    const int w = blockIdx.y;
+    const uint16_t* __restrict__ x = batch.x[w];
+    if (base + kTile <= d) {
+        const uint2* xv = reinterpret_cast<const uint2*>(x + base);
+        uint2 h[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) h[k] = __ldcs(xv + k * 32 + lane);
+        uint4 u[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            widen16x2<DT>(h[k].x, u[k].x, u[k].y);
+            widen16x2<DT>(h[k].y, u[k].z, u[k].w);
+        }
+        cnat_full_tile<false>(u, base, batch.worker[w], keys, batch.exp[w], batch.sign[w], lane);
+        return;
+    }
+    cnat_ragged_tile<false>([&](uint64_t j) { return widen16<DT>(x[j]); }, base, d,
+                            batch.worker[w], keys, batch.exp[w], batch.sign[w], lane);
 }
 
 // value of a 9-bit code: exponent byte in byte `BYTE` of `e4`, sign in bit 0 of `s`
@@ -351,6 +415,41 @@ nc_status nc_compress_nearest(const float* x, size_t d, uint8_t* exp, uint32_t* 
 nc_status nc_compress(const float* x, size_t d, uint64_t seed, uint32_t worker, uint8_t* exp,
                       uint32_t* sign, cudaStream_t stream) {
     return nc_compress_batch(&x, d, seed, &worker, &exp, &sign, 1, stream);
+}
+
+nc_status nc_compress_typed_batch(const void* const* xs, int dtype, size_t d, uint64_t seed,
+                                  const uint32_t* workers, uint8_t* const* exps,
+                                  uint32_t* const* signs, int n, cudaStream_t stream) {
+    if (dtype == NC_DTYPE_F32)
+        return nc_compress_batch(reinterpret_cast<const float* const*>(xs), d, seed, workers, exps,
+                                 signs, n, stream);
+    if (dtype != NC_DTYPE_BF16 && dtype != NC_DTYPE_F16) return NC_ERR_UNSUPPORTED;
+    if (!xs || !workers || !exps || !signs || n < 1 || n > NC_MAX_WORKERS) return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    Compress16Batch batch;
+    for (int i = 0; i < n; ++i) {
+        if (!xs[i] || !exps[i] || !signs[i]) return NC_ERR_INVALID;
+        if (!aligned16(xs[i]) || !aligned16(exps[i]) || !aligned16(signs[i])) return NC_ERR_ALIGN;
+        batch.x[i] = reinterpret_cast<const uint16_t*>(xs[i]);
+        batch.exp[i] = exps[i];
+        batch.sign[i] = signs[i];
+        batch.worker[i] = workers[i];
+    }
+    const PhiloxKeys keys = make_philox_keys(seed);
+    dim3 grid(tile_blocks(d), (unsigned)n);
+    if (dtype == NC_DTYPE_BF16)
+        nc_compress16_kernel<NC_DTYPE_BF16><<<grid, kBlockThreads, 0, stream>>>(batch, (uint64_t)d,
+                                                                               keys);
+    else
+        nc_compress16_kernel<NC_DTYPE_F16><<<grid, kBlockThreads, 0, stream>>>(batch, (uint64_t)d,
+                                                                              keys);
+    return launch_status();
+}
+
+nc_status nc_compress_typed(const void* x, int dtype, size_t d, uint64_t seed, uint32_t worker,
+                            uint8_t* exp, uint32_t* sign, cudaStream_t stream) {
+    return nc_compress_typed_batch(&x, dtype, d, seed, &worker, &exp, &sign, 1, stream);
 }
 
 nc_status nc_aggregate(const uint8_t* const* exps, const uint32_t* const* signs, int n, size_t d,

@@ -72,8 +72,12 @@ __host__ __device__ inline SelectWorkspace select_ws_carve(char* p, uint64_t d) 
     return w;
 }
 
-// ---- key sources: the 4 keys of elements base + k*128 + 4*lane + {0..3} ----------------------
+// ---- key sources: load(k) gives the 4 keys of in-tile positions pos(lane, k, 0..3) ------------
+// Stream keys are computed, not loaded, so a lane takes 32 consecutive coordinates and its 32
+// per-key bits are a word of the tile mask as they are; keys read from memory keep the coalesced
+// layout of the other kernels and their bits are transposed.
 struct StreamKeys {          // selection-stream word of the coordinate
+    static constexpr bool kCanonical = true;
     uint32_t worker;
     PhiloxKeys keys;
     struct Tile {
@@ -83,22 +87,23 @@ struct StreamKeys {          // selection-stream word of the coordinate
     __device__ __forceinline__ Tile tile(uint64_t base, int lane) const {
         Tile t;
         t.pt = philox_tile((uint32_t)(base >> 34), worker, kDomainSelect, keys);
-        t.q_lo = (uint32_t)(base >> 2) + (uint32_t)lane;
+        t.q_lo = (uint32_t)(base >> 2) + (uint32_t)(lane * 8);
         return t;
     }
     __device__ __forceinline__ void load(const Tile& t, uint64_t, int, int k, uint64_t,
                                          uint32_t (&out)[4]) const {
-        stream_words4_tile(t.q_lo + (uint32_t)(k * 32), t.pt, keys, out);
+        stream_words4_tile(t.q_lo + (uint32_t)k, t.pt, keys, out);
     }
     // the key of element k*128 + 4*lane + c of the tile alone (recomputed)
     __device__ __forceinline__ uint32_t key_at(const Tile& t, uint64_t, int, int k, int c) const {
         uint32_t out[4];
-        stream_words4_tile(t.q_lo + (uint32_t)(k * 32), t.pt, keys, out);
+        stream_words4_tile(t.q_lo + (uint32_t)k, t.pt, keys, out);
         return c == 0 ? out[0] : c == 1 ? out[1] : c == 2 ? out[2] : out[3];
     }
 };
 
 struct MagnitudeKeys {       // largest |x| first: complement of the magnitude bits
+    static constexpr bool kCanonical = false;
     const float* x;
     struct Tile {};
     __device__ __forceinline__ Tile tile(uint64_t, int) const { return Tile(); }
@@ -123,7 +128,14 @@ struct MagnitudeKeys {       // largest |x| first: complement of the magnitude b
     }
 };
 
-// bits of the load layout (bit 4k+c <-> element k*128 + 4*lane + c) that lie inside [0, d)
+// in-tile position of key c of load k
+template <class Src>
+__device__ __forceinline__ int key_pos(int lane, int k, int c) {
+    return Src::kCanonical ? lane * 32 + 4 * k + c : k * 128 + lane * 4 + c;
+}
+
+// bits 4k+c of a lane whose keys lie inside [0, d)
+template <class Src>
 __device__ __forceinline__ uint32_t valid_nibbles(uint64_t base, int lane, uint64_t d) {
     if (base + kTile <= d) return 0xFFFFFFFFu;
     uint32_t v = 0;
@@ -131,9 +143,15 @@ __device__ __forceinline__ uint32_t valid_nibbles(uint64_t base, int lane, uint6
     for (int k = 0; k < 8; ++k) {
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-            if (base + (uint64_t)(k * 128 + lane * 4 + c) < d) v |= 1u << (4 * k + c);
+            if (base + (uint64_t)key_pos<Src>(lane, k, c) < d) v |= 1u << (4 * k + c);
     }
     return v;
+}
+
+// per-key bits of a lane -> word `lane` of the tile mask
+template <class Src>
+__device__ __forceinline__ uint32_t mask_word(uint32_t nib, int lane) {
+    return Src::kCanonical ? nib : canonical_mask_word(nib, lane);
 }
 
 __global__ void select_init_kernel(SelectWorkspace ws, const uint64_t q) {
@@ -165,7 +183,7 @@ select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws) {
     for (uint64_t g = blockIdx.x; g < groups; g += gridDim.x) {
         const uint64_t base = (g * kWarpsPerBlock + (threadIdx.x >> 5)) * kTile;
         if (base >= d) continue;
-        const uint32_t valid = valid_nibbles(base, lane, d);
+        const uint32_t valid = valid_nibbles<Src>(base, lane, d);
         const typename Src::Tile t = src.tile(base, lane);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -254,12 +272,12 @@ select_mark_kernel(const Src src, const uint64_t d, uint32_t* __restrict__ less_
                 equal |= (hi == T ? 1u : 0u) << (4 * k + c);
             }
         }
-        const uint32_t valid = valid_nibbles(base, lane, d);
+        const uint32_t valid = valid_nibbles<Src>(base, lane, d);
         less &= valid;
         equal &= valid;
     }
-    const uint32_t lw = canonical_mask_word(less, lane);
-    const uint32_t ew = (mode == 0u) ? canonical_mask_word(equal, lane) : 0u;
+    const uint32_t lw = mask_word<Src>(less, lane);
+    const uint32_t ew = (mode == 0u) ? mask_word<Src>(equal, lane) : 0u;
     if (active) {
         less_mask[tile * 32 + lane] = lw;
         ws.eqmask[tile * 32 + lane] = ew;
@@ -294,7 +312,7 @@ select_mark_kernel(const Src src, const uint64_t d, uint32_t* __restrict__ less_
         equal &= equal - 1;
         if (at < kCandCap)
             ws.cand[at] = make_uint2(src.key_at(t, base, lane, bit >> 2, bit & 3),
-                                     (uint32_t)(base + (uint64_t)((bit >> 2) * 128 + lane * 4 + (bit & 3))));
+                                     (uint32_t)(base + (uint64_t)key_pos<Src>(lane, bit >> 2, bit & 3)));
         ++at;
     }
 }

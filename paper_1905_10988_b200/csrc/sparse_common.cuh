@@ -49,15 +49,12 @@ __device__ __forceinline__ double warp_sum_d(double v) {
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
     return v;
 }
+// warp-wide integer reductions: one redux instruction each
 __device__ __forceinline__ uint32_t warp_max_u(uint32_t v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
-    return v;
+    return __reduce_max_sync(0xFFFFFFFFu, v);
 }
 __device__ __forceinline__ uint32_t warp_sum_u(uint32_t v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
+    return __reduce_add_sync(0xFFFFFFFFu, v);
 }
 
 // Lists the set bits of a 1024-bit tile mask (lane l holds word l) in ascending order into the
@@ -103,15 +100,31 @@ __device__ __forceinline__ void kept_count_and_partial(const uint32_t word, cons
     __shared__ uint64_t s_part[kWarpsPerBlock];
     __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
     uint16_t* list = s_list[threadIdx.x >> 5];
-    const uint32_t cnt = warp_list_positions(word, lane, list);
+    const uint32_t cnt = warp_sum_u(__popc(word));
     double dsum = 0.0;
     uint32_t vmax = 0;
-    for (uint32_t t = lane; t < cnt; t += 32) {
-        const float xs = __fmul_rn(scale, x[base + list[t]]);
-        const uint32_t a = __float_as_uint(xs) & 0x7FFFFFFFu;
-        if (P == NC_P_INF) vmax = max(vmax, a);
-        else if (P == 1) dsum += (double)__uint_as_float(a);
-        else dsum = fma((double)xs, (double)xs, dsum);
+    if (cnt <= 96u) {
+        // few kept entries (the 1 % workloads): every lane walks the bits of its own word
+        uint32_t w = word;
+        while (w) {
+            const int bit = __ffs(w) - 1;
+            w &= w - 1;
+            const float xs = __fmul_rn(scale, x[base + (uint64_t)(lane * 32 + bit)]);
+            const uint32_t a = __float_as_uint(xs) & 0x7FFFFFFFu;
+            if (P == NC_P_INF) vmax = max(vmax, a);
+            else if (P == 1) dsum += (double)__uint_as_float(a);
+            else dsum = fma((double)xs, (double)xs, dsum);
+        }
+    } else {
+        // many: list the positions so that the gathers spread evenly over the lanes
+        warp_list_positions(word, lane, list);
+        for (uint32_t t = lane; t < cnt; t += 32) {
+            const float xs = __fmul_rn(scale, x[base + list[t]]);
+            const uint32_t a = __float_as_uint(xs) & 0x7FFFFFFFu;
+            if (P == NC_P_INF) vmax = max(vmax, a);
+            else if (P == 1) dsum += (double)__uint_as_float(a);
+            else dsum = fma((double)xs, (double)xs, dsum);
+        }
     }
     uint64_t part;
     if (P == NC_P_INF) part = (uint64_t)warp_max_u(vmax);

@@ -32,19 +32,20 @@ sparse_select_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d
     const uint32_t worker = batch.worker[blockIdx.y];
     const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
     uint32_t* __restrict__ bitmask = ws.bitmask;
-    // phase 1: the 1024 selection bits of the tile, no memory traffic
-    uint32_t nib = 0;        // bit 4k+c <-> element base + k*128 + 4*lane + c
+    // phase 1: the 1024 selection bits of the tile, no memory traffic.  Lane l draws the eight
+    // counter groups of elements 32l .. 32l+31, so its 32 bits are word l of the tile mask.
+    uint32_t word = 0;
     const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainSelect, keys);
     if (active && !keep_none) {
         // coordinate j is dropped iff word >= threshold, i.e. iff word + (2^32 - threshold)
         // carries out of 32 bits.  The drop bits are shifted in straight from that carry: two
         // integer instructions per coordinate on top of the generator.
-        const uint32_t q_lo = (uint32_t)(base >> 2) + (uint32_t)lane;
+        const uint32_t q_lo = (uint32_t)(base >> 2) + (uint32_t)(lane * 8);
         uint32_t drop = 0;
 #pragma unroll
         for (int k = 7; k >= 0; --k) {
             uint32_t rnd[4];
-            stream_words4_tile(q_lo + (uint32_t)(k * 32), pt, keys, rnd);
+            stream_words4_tile(q_lo + (uint32_t)k, pt, keys, rnd);
 #pragma unroll
             for (int c = 3; c >= 0; --c) {
                 uint32_t tmp;
@@ -53,18 +54,13 @@ sparse_select_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d
                     : "r"(rnd[c]), "r"(neg_thr));
             }
         }
-        nib = ~drop;
+        word = ~drop;
         if (base + kTile > d) {          // ragged last tile: clear the bits past the end
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (base + (uint64_t)(k * 128 + lane * 4 + c) >= d) nib &= ~(1u << (4 * k + c));
-                }
-            }
+            const uint64_t first = base + (uint64_t)(lane * 32);
+            if (first >= d) word = 0u;
+            else if (first + 32 > d) word &= (1u << (uint32_t)(d - first)) - 1u;
         }
     }
-    const uint32_t word = canonical_mask_word(nib, lane);
     if (active) bitmask[tile * 32 + lane] = word;
 
     // phase 2: gather the kept entries, spread evenly over the lanes
@@ -332,23 +328,36 @@ sparse_round_filter_kernel(const __grid_constant__ SparseBatch batch, const uint
     __shared__ uint32_t s_cnt[kWarpsPerBlock];
     uint16_t* list = s_list[warp];
     const uint32_t word = active ? ws.bitmask[tile * 32 + lane] : 0u;
-    s_mask[warp][lane] = word;
-    const uint32_t cnt = warp_list_positions(word, lane, list);     // ends with __syncwarp
+    const uint32_t cnt = warp_sum_u(__popc(word));
     const Scale sc = make_scale(*batch.norm[blockIdx.y], s);
     const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
-    for (uint32_t t = lane; t < cnt; t += 32) {
-        const uint32_t pos = list[t];
-        const uint64_t j = base + pos;
-        const float xs = __fmul_rn(scale, x[j]);
-        uint32_t r4[4];
-        stream_words4(j >> 2, worker, kDomainDnat, keys, r4);
-        const uint32_t r = (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1]
-                         : (j & 3) == 2 ? r4[2] : r4[3];
-        if (sparse_level_code(__float_as_uint(xs), r, sc, pow2s) == 0u)
-            atomicAnd(&s_mask[warp][pos >> 5], ~(1u << (pos & 31)));
+    uint32_t kept;
+    if (cnt <= 96u) {
+        // few kept entries: every lane walks the bits of its own word
+        kept = word;
+        uint32_t w = word;
+        while (w) {
+            const int bit = __ffs(w) - 1;
+            w &= w - 1;
+            const uint64_t j = base + (uint64_t)(lane * 32 + bit);
+            const float xs = __fmul_rn(scale, x[j]);
+            const uint32_t r = stream_word_at(j, worker, kDomainDnat, keys);
+            if (sparse_level_code(__float_as_uint(xs), r, sc, pow2s) == 0u) kept &= ~(1u << bit);
+        }
+    } else {
+        s_mask[warp][lane] = word;
+        warp_list_positions(word, lane, list);     // ends with __syncwarp
+        for (uint32_t t = lane; t < cnt; t += 32) {
+            const uint32_t pos = list[t];
+            const uint64_t j = base + pos;
+            const float xs = __fmul_rn(scale, x[j]);
+            const uint32_t r = stream_word_at(j, worker, kDomainDnat, keys);
+            if (sparse_level_code(__float_as_uint(xs), r, sc, pow2s) == 0u)
+                atomicAnd(&s_mask[warp][pos >> 5], ~(1u << (pos & 31)));
+        }
+        __syncwarp();
+        kept = s_mask[warp][lane];
     }
-    __syncwarp();
-    const uint32_t kept = s_mask[warp][lane];
     if (active) ws.bitmask[tile * 32 + lane] = kept;
     const uint32_t total = warp_sum_u(__popc(kept));
     if (lane == 0) s_cnt[warp] = total;

@@ -26,7 +26,7 @@ def nc():
 def _declared_functions():
     src = open(HEADER).read()
     src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    names = re.findall(r"\b(n[cd]8?_[a-z0-9_]+)\s*\(", src)
+    names = re.findall(r"\b(n[cd](?:8|64)?_[a-z0-9_]+)\s*\(", src)
     return sorted(set(names))
 
 
