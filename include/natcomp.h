@@ -218,6 +218,21 @@ nc_status nd_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes,
                                       const uint32_t* count, const float* norm, int s, size_t d,
                                       size_t cap, float* acc, cudaStream_t stream);
 
+/* ---- sparse update without an index list --------------------------------------------------
+ * With independent selection the kept set is a function of (seed, worker, keep_threshold), so a
+ * receiver that knows them can regenerate it instead of receiving idx ("next" item of the type /
+ * mode variants: the wire carries count, norm and the 4-bit codes only, 0.5 byte per kept entry).
+ * Applies the output of nd_sparse_compress made with the same d, keep_threshold, seed and worker:
+ * the k-th code goes to the k-th kept coordinate in ascending order, k < min(*count, cap);
+ * acc[j] <- acc[j] + sign * fl32(norm * 2^(c - s)).  Cost: one pass of the selection generator
+ * over d.  workspace: nd_sparse_regen_workspace_bytes(d) bytes, 16-byte aligned. */
+size_t nd_sparse_regen_workspace_bytes(size_t d);
+nc_status nd_sparse_regen_decode_accumulate(const uint8_t* codes, const uint32_t* count,
+                                            const float* norm, size_t d, uint64_t keep_threshold,
+                                            int s, uint64_t seed, uint32_t worker, size_t cap,
+                                            float* acc, void* workspace, size_t workspace_bytes,
+                                            cudaStream_t stream);
+
 /* ---- compact sparse format: zero levels dropped, codes as bit planes ------------------------
  * Same operator as nd_sparse_compress (sparsifier definition + Def. 3, composition of Thm. 3), in
  * the format "index list + log2(s)+1 bits per listed entry" that the paper's bit counts for

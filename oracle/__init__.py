@@ -472,3 +472,17 @@ def cnat64_values(t, r52) -> np.ndarray:
     out = np.zeros(t.size, np.float64)
     _cnat64_values(_p(t, _f64p), _p(r52, _u64p), t.size, _p(out, _f64p))
     return out
+
+
+_sparse_regen_decode_accumulate = _sig("orc_sparse_regen_decode_accumulate", None, _u8p,
+                                       C.c_uint64, C.c_float, C.c_uint64, C.c_uint64, C.c_int,
+                                       C.c_uint64, C.c_uint32, _f32p)
+
+
+def sparse_regen_decode_accumulate(codes, count: int, nrm, keep_threshold: int, s: int, seed: int,
+                                   worker: int, acc) -> None:
+    """Apply the listed 4-bit codes to the kept coordinates regenerated from the seed."""
+    codes = _arr(codes, np.uint8)
+    assert acc.dtype == np.float32 and acc.flags.c_contiguous
+    _sparse_regen_decode_accumulate(_p(codes, _u8p), count, float(nrm), acc.size, keep_threshold, s,
+                                    seed, worker, _p(acc, _f32p))

@@ -853,4 +853,21 @@ void orc_cnat64_values(const double* t, const uint64_t* r52, uint64_t n, double*
     for (uint64_t i = 0; i < n; ++i) out[i] = cnat64_value(t[i], r52[i]);
 }
 
+// ---- receiver-side regeneration of the kept set --------------------------------------------
+// With independent selection the kept set is a function of (seed, worker, threshold) alone, so
+// the index list need not travel: the receiver walks the coordinates, regenerates "kept iff
+// stream word (domain 2, j) < threshold" and pairs the k-th kept coordinate with the k-th code of
+// the listed 4-bit form (orc_sparse_compress).  Only the first `count` kept coordinates are applied.
+void orc_sparse_regen_decode_accumulate(const uint8_t* codes, uint64_t count, float norm,
+                                        uint64_t d, uint64_t keep_threshold, int s, uint64_t seed,
+                                        uint32_t worker, float* acc) {
+    uint64_t k = 0;
+    for (uint64_t j = 0; j < d && k < count; ++j) {
+        if ((uint64_t)stream_word(seed, worker, 2u, j) >= keep_threshold) continue;
+        const uint32_t code = (codes[k / 2] >> (4 * (k % 2))) & 0xFu;
+        acc[j] = acc[j] + nd_decode_value((int)(code & 7u), s, norm, code >> 3);
+        ++k;
+    }
+}
+
 }  // extern "C"

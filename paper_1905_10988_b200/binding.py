@@ -40,6 +40,7 @@ EXPORTS = (
     "nc8_aggregate_compress", "nc_select_workspace_bytes", "nd_sparse_exact_compress",
     "nc_topk_compress", "nc_topk_decode_accumulate", "nc_compress_typed",
     "nc_compress_typed_batch", "nc64_compress", "nc64_compress_batch", "nc64_aggregate",
+    "nd_sparse_regen_workspace_bytes", "nd_sparse_regen_decode_accumulate",
 )
 
 
@@ -446,3 +447,22 @@ def nc64_compress_batch(xs, d, seed, workers, exp_los, his, n, stream=None) -> N
 def nc64_aggregate(exp_los, his, n, d, out, stream=None) -> None:
     _check("nc64_aggregate", _nc64_aggregate(_ptrs(exp_los), _ptrs(his), n, d, _ptr(out),
                                              _stream(stream)))
+
+
+# ---- sparse update without an index list (kept set regenerated from the seed) -----------------
+_nd_sparse_regen_workspace_bytes = _sig("nd_sparse_regen_workspace_bytes", _sz, _sz)
+_nd_sparse_regen_decode_accumulate = _sig("nd_sparse_regen_decode_accumulate", C.c_int, _vp, _vp,
+                                          _vp, _sz, C.c_uint64, C.c_int, C.c_uint64, C.c_uint32,
+                                          _sz, _vp, _vp, _sz, _vp)
+
+
+def nd_sparse_regen_workspace_bytes(d: int) -> int:
+    return int(_nd_sparse_regen_workspace_bytes(d))
+
+
+def nd_sparse_regen_decode_accumulate(codes, count, norm, d, keep_threshold, s, seed, worker, cap,
+                                      acc, workspace, workspace_bytes, stream=None) -> None:
+    _check("nd_sparse_regen_decode_accumulate",
+           _nd_sparse_regen_decode_accumulate(_ptr(codes), _ptr(count), _ptr(norm), d,
+                                              keep_threshold, s, seed, worker, cap, _ptr(acc),
+                                              _ptr(workspace), workspace_bytes, _stream(stream)))

@@ -88,6 +88,23 @@ def run_cnat(config, n, d, make_vector, iters, peak, with_sum=True):
                 peak)
 
 
+def run_cnat64(config, n, d, iters, peak):
+    dev = "cuda"
+    u8 = dict(dtype=torch.uint8, device=dev)
+    g = torch.Generator(device=dev)
+    g.manual_seed(64)
+    xs = [torch.randn(d, dtype=torch.float64, device=dev, generator=g) * 1e-3 for _ in range(n)]
+    es = [torch.empty(nc.nc_exp_bytes(d), **u8) for _ in range(n)]
+    hs = [torch.empty(nc.nd_level_bytes(d), **u8) for _ in range(n)]
+    out = torch.empty(d, dtype=torch.float64, device=dev)
+    workers = list(range(n))
+    m, b = _time(lambda: nc.nc64_compress_batch(xs, d, 0, workers, es, hs, n), iters)
+    _report(config, "nc64_compress_batch (binary64, 12-bit codes)", m, b, n * d, n * d * 9.5, peak,
+            {"n": n, "d": d})
+    m, b = _time(lambda: nc.nc64_aggregate(es, hs, n, d, out), iters)
+    _report(config, "nc64_aggregate", m, b, d, d * (1.5 * n + 8), peak)
+
+
 def run_dnat(config, n, sizes, iters, peak, p=2, s=8):
     dev = "cuda"
     u8 = dict(dtype=torch.uint8, device=dev)
@@ -139,6 +156,20 @@ def run_sparse(config, n, d, iters, peak, s=4):
 
     m, b = _time(accumulate, iters)
     _report(config, "nd_sparse_decode_accumulate x n", m, b, n * kept, n * kept * 68.5, peak)
+
+    # the same update without the index list: the master regenerates the kept set from the seed
+    rws_bytes = nc.nd_sparse_regen_workspace_bytes(d)
+    rws = torch.empty(rws_bytes, **u8)
+
+    def accumulate_regen():
+        for w in range(n):
+            nc.nd_sparse_regen_decode_accumulate(codes[w], count[w], norm[w], d, thr, s, 0, w, cap,
+                                                 acc, rws, rws_bytes)
+
+    m, b = _time(accumulate_regen, iters)
+    _report(config, "nd_sparse_regen_decode_accumulate x n (no index list)", m, b, n * kept,
+            n * kept * 64.5, peak, {"Gcoord_per_s": round(n * d / m / 1e6, 1),
+                                    "wire_bytes_per_kept_entry": 0.5})
 
     # the compact format: level-0 entries dropped, 3-bit codes as bit planes
     planes = [torch.empty(nc.nd_sparse_plane_bytes(cap, s), **u8) for _ in range(n)]
@@ -198,6 +229,7 @@ def main():
         d = sum(sizes)
         run_cnat("c2", 8, d, lambda w: workloads.config2_vector(w, "cuda", sizes), args.iters,
                  peak)
+        run_cnat64("c2", 8, d, args.iters, peak)
     elif args.config == "c3":
         run_dnat("c3", 8, workloads.resnet50_tensor_sizes(), args.iters, peak)
     elif args.config == "c4":

@@ -567,3 +567,136 @@ nc_status nd_sparse_compact_decode_accumulate(const uint32_t* idx, const uint32_
 }
 
 }  // extern "C"
+
+// ---- receiver-side regeneration of the kept set: no index list on the wire ------------------
+//
+// With independent selection the kept set depends on (seed, worker, threshold) only.  The master
+// regenerates the selection mask with the same generator, scans the per-block counts, and pairs
+// the k-th kept coordinate with the k-th code of the listed 4-bit form.
+//   regen_mask  : the select kernel's phase 1 alone (mask + per-block kept counts)
+//   regen_scan  : one block, exclusive offsets
+//   regen_apply : acc[j_k] += decode(code_k) for k < min(count, cap)
+namespace natcomp {
+
+// grid: ceil(tiles / warps per block)
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_regen_mask_kernel(const uint64_t d, const uint32_t neg_thr, const bool keep_none,
+                         const uint32_t worker, const __grid_constant__ PhiloxKeys keys,
+                         const SparseWorkspace ws) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const uint64_t base = tile * kTile;
+    const bool active = base < d;
+    __shared__ uint32_t s_cnt[kWarpsPerBlock];
+    uint32_t word = 0;
+    if (active && !keep_none) {
+        const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainSelect, keys);
+        const uint32_t q_lo = (uint32_t)(base >> 2) + (uint32_t)(lane * 8);
+        uint32_t drop = 0;
+#pragma unroll
+        for (int k = 7; k >= 0; --k) {
+            uint32_t rnd[4];
+            stream_words4_tile(q_lo + (uint32_t)k, pt, keys, rnd);
+#pragma unroll
+            for (int c = 3; c >= 0; --c) {
+                uint32_t tmp;
+                asm("add.cc.u32 %1, %2, %3;\n\taddc.u32 %0, %0, %0;"
+                    : "+r"(drop), "=r"(tmp)
+                    : "r"(rnd[c]), "r"(neg_thr));
+            }
+        }
+        word = ~drop;
+        if (base + kTile > d) {
+            const uint64_t first = base + (uint64_t)(lane * 32);
+            if (first >= d) word = 0u;
+            else if (first + 32 > d) word &= (1u << (uint32_t)(d - first)) - 1u;
+        }
+    }
+    if (active) ws.bitmask[tile * 32 + lane] = word;
+    const uint32_t cnt = warp_sum_u(__popc(word));
+    if (lane == 0) s_cnt[warp] = cnt;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t c = 0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) c += s_cnt[w];
+        ws.block_count[blockIdx.x] = c;
+    }
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+sparse_regen_scan_kernel(uint32_t* __restrict__ counts, const uint64_t n) {
+    block_exclusive_scan_inplace(counts, n);
+}
+
+// grid: ceil(tiles / warps per block)
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_regen_apply_kernel(const uint8_t* __restrict__ codes, const uint32_t* __restrict__ count,
+                          const float* __restrict__ norm, const int s, const uint64_t d,
+                          const uint64_t cap, float* __restrict__ acc, const SparseWorkspace ws) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const uint64_t base = tile * kTile;
+    const bool active = base < d;
+    __shared__ uint32_t s_tile[kWarpsPerBlock];
+    uint32_t word = active ? ws.bitmask[tile * 32 + lane] : 0u;
+    const uint32_t mine = __popc(word);
+    uint32_t incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_tile[warp] = incl;
+    __syncthreads();
+    uint64_t k = (uint64_t)ws.block_count[blockIdx.x] + (incl - mine);
+    for (int w = 0; w < warp; ++w) k += s_tile[w];
+    const uint64_t total = min((uint64_t)*count, cap);
+    float nv = *norm;
+    if (!(fabsf(nv) <= 3.40282347e38f)) nv = 0.f;
+    while (word && k < total) {
+        const int bit = __ffs(word) - 1;
+        word &= word - 1;
+        const uint64_t j = base + (uint64_t)(lane * 32 + bit);
+        const uint32_t code = (codes[k >> 1] >> (4 * (k & 1))) & 0xFu;
+        const uint32_t c = code & 7u;
+        const uint32_t pb = (c ? ((c + 127u - (uint32_t)s) << 23) : 0u) | ((code >> 3) << 31);
+        acc[j] = __fadd_rn(acc[j], __fmul_rn(nv, __uint_as_float(pb)));
+        ++k;
+    }
+}
+
+}  // namespace natcomp
+
+extern "C" {
+
+size_t nd_sparse_regen_workspace_bytes(size_t d) { return sparse_ws_bytes(d, 0); }
+
+nc_status nd_sparse_regen_decode_accumulate(const uint8_t* codes, const uint32_t* count,
+                                            const float* norm, size_t d, uint64_t keep_threshold,
+                                            int s, uint64_t seed, uint32_t worker, size_t cap,
+                                            float* acc, void* workspace, size_t workspace_bytes,
+                                            cudaStream_t stream) {
+    if (!codes || !count || !norm || !acc || s < 1 || s > 7 || cap < 1 ||
+        keep_threshold > ((uint64_t)1 << 32))
+        return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > 0xFFFFFFFFull) return NC_ERR_INVALID;
+    if (!workspace) return NC_ERR_INVALID;
+    if (!aligned16(workspace) || !aligned16(codes) || !aligned32(acc) || !aligned4(count) ||
+        !aligned4(norm))
+        return NC_ERR_ALIGN;
+    if (workspace_bytes < sparse_ws_bytes(d, 0)) return NC_ERR_WORKSPACE;
+    const SparseWorkspace ws = sparse_ws_carve(workspace, d);
+    const uint64_t groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const uint32_t neg_thr = (uint32_t)(0ull - keep_threshold);
+    sparse_regen_mask_kernel<<<(unsigned)groups, kBlockThreads, 0, stream>>>(
+        d, neg_thr, keep_threshold == 0, worker, make_philox_keys(seed), ws);
+    sparse_regen_scan_kernel<<<1, kScanThreads, 0, stream>>>(ws.block_count, groups);
+    sparse_regen_apply_kernel<<<(unsigned)groups, kBlockThreads, 0, stream>>>(
+        codes, count, norm, s, d, cap, acc, ws);
+    return launch_status();
+}
+
+}  // extern "C"
