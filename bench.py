@@ -297,7 +297,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--only", default=None, choices=list(HotPath.GROUPS),
                     help="profiling aid: time one call group alone")
     ap.add_argument("--workers", type=int, default=N_WORKERS,

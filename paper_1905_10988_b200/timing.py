@@ -30,30 +30,47 @@ def replica_worker_ids(rank: int, n_workers: int):
 def e2e_host_steps(nc, hp, steps: int) -> dict:
     """Runs `steps` steps with the inputs in pinned host memory: every step copies the n
     gradient vectors host -> device through the C ABI, runs the whole path, and copies the
-    three aggregates back to pinned host memory.  Returns ms per step and bytes moved."""
+    three aggregates back to pinned host memory.  Returns ms per step and bytes moved.
+
+    Two streams: the upload and the kernels of step i run on one, the download of its results on
+    the other, so that the download of step i overlaps the upload of step i + 1 (PCIe is full
+    duplex).  The kernels of step i + 1 wait until the download of step i has read the outputs.
+    The timed region runs from the first upload to the end of the last download."""
     n, d = hp.n, hp.d
     host_x = [torch.empty(d, dtype=torch.float32, pin_memory=True) for _ in range(n)]
     for w in range(n):
         host_x[w].copy_(hp.x[w])
     host_out = [torch.empty(d, dtype=torch.float32, pin_memory=True) for _ in range(3)]
     torch.cuda.synchronize()
+    s_main = torch.cuda.Stream()
+    s_out = torch.cuda.Stream()
+    state = {"downloaded": None}
 
     def one_step():
-        for w in range(n):
-            nc.nc_copy_to_device(hp.x[w], host_x[w], 4 * d)
-        hp.step()
-        for dst, src in zip(host_out, (hp.out_nc, hp.out_nd, hp.out_sp)):
-            nc.nc_copy_to_host(dst, src, 4 * d)
+        with torch.cuda.stream(s_main):
+            for w in range(n):
+                nc.nc_copy_to_device(hp.x[w], host_x[w], 4 * d)
+            if state["downloaded"] is not None:
+                s_main.wait_event(state["downloaded"])      # outputs may be overwritten now
+            hp.step()
+            computed = torch.cuda.Event()
+            computed.record(s_main)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(computed)
+            for dst, src in zip(host_out, (hp.out_nc, hp.out_nd, hp.out_sp)):
+                nc.nc_copy_to_host(dst, src, 4 * d)
+            state["downloaded"] = torch.cuda.Event()
+            state["downloaded"].record(s_out)
 
     one_step()                                   # warm-up
     torch.cuda.synchronize()
     e0 = torch.cuda.Event(enable_timing=True)
     e1 = torch.cuda.Event(enable_timing=True)
-    e0.record()
+    e0.record(s_main)
     for _ in range(steps):
         one_step()
-    e1.record()
+    e1.record(s_out)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
     return {"ms_per_step": ms, "h2d_bytes_per_step": 4 * d * n, "d2h_bytes_per_step": 4 * d * 3,
-            "steps": steps}
+            "steps": steps, "overlap": "download of step i overlaps upload of step i+1"}
