@@ -6,7 +6,7 @@ ResNet-50-shaped workload (n = 8 workers, d = 25,557,032 fp32 entries in 161 buc
   C_nat  : nc_compress_batch (8 workers, one launch) + nc_aggregate
   D_nat  : nd_compress x 8 (p = 2, s = 8, per-bucket norms) + nd_aggregate
   sparse : nd_sparse_compact_compress_batch (keep 1 %, p = inf, s = 4, 3-bit codes)
-           + nd_sparse_compact_decode_accumulate x 8
+           + nd_sparse_compact_aggregate (all workers, one launch)
   ref    : nc_sum_fp32 (uncompressed 8-way sum, the reference point)
 The metric is worker-entries taken through the whole path per second (n * d per step).
 Inputs (818 MB) are larger than the 126 MB L2, so no flush is needed between steps.
@@ -159,8 +159,8 @@ class HotPath:
         self.out_sp = torch.empty(d, **f32)
         self.out_sum = torch.empty(d, **f32)
         # nc_compress_batch 1, nc_aggregate 1, nd_compress_batch 3, nd_aggregate 1,
-        # nd_sparse_compact_compress_batch 6, nd_sparse_compact_decode_accumulate n, nc_sum_fp32 1
-        self.launches_per_step = 1 + 1 + 3 + 1 + 6 + n + 1
+        # nd_sparse_compact_compress_batch 6, nd_sparse_compact_aggregate 1, nc_sum_fp32 1
+        self.launches_per_step = 1 + 1 + 3 + 1 + 6 + 1 + 1
         self.seed = 0
 
     def step(self, marks=None):
@@ -200,11 +200,8 @@ class HotPath:
                                                 self.sws_bytes)
         mark("sparse_compress")
         if want("sparse_accumulate"):
-            self.out_sp.zero_()
-            for w in range(n):
-                nc.nd_sparse_compact_decode_accumulate(self.idx[w], self.codes[w], self.count[w],
-                                                       self.snorm[w], S_SPARSE, d, self.cap,
-                                                       self.out_sp)
+            nc.nd_sparse_compact_aggregate(self.idx, self.codes, self.count, self.snorm, n,
+                                           S_SPARSE, d, self.cap, self.out_sp)
         mark("sparse_accumulate")
         if want("sum_fp32"):
             nc.nc_sum_fp32(self.x, n, d, self.out_sum)
@@ -222,7 +219,8 @@ class HotPath:
             # kept entries are read as 32-byte sectors in three passes (norm, filter, emit);
             # about half of them survive the level-0 filter and are listed (4 B index + 3 bits)
             "sparse_compress": n * kept * (3 * 32 + 0.5 * 4.375),
-            "sparse_accumulate": 4 * d + n * kept * 0.5 * (4.375 + 64),
+            # dense output written once; the listed entries (about half of the kept) read once
+            "sparse_accumulate": 4 * d + n * kept * 0.5 * 4.375,
             "sum_fp32": d * (4 * n + 4),
         }
 

@@ -262,6 +262,15 @@ nc_status nd_sparse_compact_decode_accumulate(const uint32_t* idx, const uint32_
                                               size_t d, size_t cap, float* acc,
                                               cudaStream_t stream);
 
+/* Master side, all workers in one call (Algorithm 1, aggregate): out[j] = sum over the n workers,
+ * in that order and starting from +0, of their decoded entries at coordinate j; coordinates no
+ * list mentions get +0.  Every index list must be ascending (as the compressors write it);
+ * entries k >= min(*count, cap) are ignored.  out: float[d], 32-byte aligned, overwritten. */
+nc_status nd_sparse_compact_aggregate(const uint32_t* const* idxs, const uint32_t* const* planes,
+                                      const uint32_t* const* counts, const float* const* norms,
+                                      int n, int s, size_t d, size_t cap, float* out,
+                                      cudaStream_t stream);
+
 /* ---- the paper's 8-bit wire format and integer aggregation ----------------------------------
  * Experimental set-up appendix ("1 bit for the sign ... clip the exponents in the range -50~10 ...
  * the remaining one bit is used to represent zeros", "64-bit integers to store the intermediate

@@ -41,6 +41,7 @@ EXPORTS = (
     "nc_topk_compress", "nc_topk_decode_accumulate", "nc_compress_typed",
     "nc_compress_typed_batch", "nc64_compress", "nc64_compress_batch", "nc64_aggregate",
     "nd_sparse_regen_workspace_bytes", "nd_sparse_regen_decode_accumulate",
+    "nd_sparse_compact_aggregate",
 )
 
 
@@ -466,3 +467,15 @@ def nd_sparse_regen_decode_accumulate(codes, count, norm, d, keep_threshold, s, 
            _nd_sparse_regen_decode_accumulate(_ptr(codes), _ptr(count), _ptr(norm), d,
                                               keep_threshold, s, seed, worker, cap, _ptr(acc),
                                               _ptr(workspace), workspace_bytes, _stream(stream)))
+
+
+_nd_sparse_compact_aggregate = _sig("nd_sparse_compact_aggregate", C.c_int, C.POINTER(_vp),
+                                    C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.c_int,
+                                    C.c_int, _sz, _sz, _vp, _vp)
+
+
+def nd_sparse_compact_aggregate(idxs, planes, counts, norms, n, s, d, cap, out,
+                                stream=None) -> None:
+    _check("nd_sparse_compact_aggregate",
+           _nd_sparse_compact_aggregate(_ptrs(idxs), _ptrs(planes), _ptrs(counts), _ptrs(norms),
+                                        n, s, d, cap, _ptr(out), _stream(stream)))

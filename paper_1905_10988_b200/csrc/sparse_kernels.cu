@@ -604,6 +604,7 @@ sparse_regen_mask_kernel(const uint64_t d, const uint32_t neg_thr, const bool ke
                 asm("add.cc.u32 %1, %2, %3;\n\taddc.u32 %0, %0, %0;"
                     : "+r"(drop), "=r"(tmp)
                     : "r"(rnd[c]), "r"(neg_thr));
+                (void)tmp;
             }
         }
         word = ~drop;
@@ -696,6 +697,149 @@ nc_status nd_sparse_regen_decode_accumulate(const uint8_t* codes, const uint32_t
     sparse_regen_scan_kernel<<<1, kScanThreads, 0, stream>>>(ws.block_count, groups);
     sparse_regen_apply_kernel<<<(unsigned)groups, kBlockThreads, 0, stream>>>(
         codes, count, norm, s, d, cap, acc, ws);
+    return launch_status();
+}
+
+}  // extern "C"
+
+// ---- master side, all workers in one launch: dense sum of n compact lists --------------------
+//
+// out[j] = sum over the workers, in worker order and starting from +0, of their decoded entries
+// at coordinate j (Algorithm 1, aggregate).  A block owns a range of 8192 coordinates and keeps
+// it in shared memory: every worker's entries that fall into the range are found by a warp-wide
+// 32-ary search in its ascending index list and applied there, workers separated by a barrier so
+// that the order of the fp32 additions is fixed; the range is then written out once, coalesced.
+// No read-modify-write of global memory and no zero fill beforehand.
+namespace natcomp {
+
+constexpr int kAggRange = 8192;
+
+struct SparseLists {
+    const uint32_t* idx[NC_MAX_WORKERS];
+    const uint32_t* planes[NC_MAX_WORKERS];
+    const uint32_t* count[NC_MAX_WORKERS];
+    const float* norm[NC_MAX_WORKERS];
+};
+
+// first k in [lo, hi) with idx[k] >= key (hi if none), given idx[k] < key for all k < lo;
+// all lanes of the warp take part
+__device__ __forceinline__ uint32_t warp_lower_bound(const uint32_t* __restrict__ idx, uint32_t lo,
+                                                     uint32_t hi, uint32_t key, int lane) {
+    while (hi - lo > 32u) {
+        const uint32_t step = (hi - lo + 31u) / 32u;
+        const uint32_t probe = lo + (uint32_t)lane * step;      // lane 0 probes lo
+        const bool below = probe < hi && idx[probe] < key;
+        const uint32_t m = __ballot_sync(0xFFFFFFFFu, below);   // a prefix of the lanes
+        const uint32_t cnt = __popc(m);
+        if (cnt == 0u) return lo;                // idx[lo] >= key
+        const uint32_t nlo = lo + (cnt - 1u) * step + 1u;       // idx[nlo - 1] < key
+        const uint32_t nhi = min(hi, lo + cnt * step);          // idx[nhi] >= key, or nhi = hi
+        lo = nlo;
+        hi = nhi;
+    }
+    const uint32_t probe = lo + (uint32_t)lane;
+    const bool below = probe < hi && idx[probe] < key;
+    return lo + __popc(__ballot_sync(0xFFFFFFFFu, below));
+}
+
+// decoded value of listed entry k of a compact list
+__device__ __forceinline__ float compact_entry_value(const uint32_t* __restrict__ planes,
+                                                     uint32_t k, int nb, int s, float nv) {
+    const uint32_t* pw = planes + (uint64_t)(k >> 5) * (uint64_t)(nb + 1);
+    uint32_t code = 0;
+    for (int b = 0; b <= nb; ++b) code |= ((pw[b] >> (k & 31)) & 1u) << b;
+    const uint32_t level = (code & ((1u << nb) - 1u)) + 1u;
+    const uint32_t pb = ((level + 127u - (uint32_t)s) << 23) | ((code >> nb) << 31);
+    return __fmul_rn(nv, __uint_as_float(pb));
+}
+
+// grid: ceil(d / kAggRange).  Warp t of the block serves workers t, t + 8, ...: it finds the
+// worker's entries of the range and preloads up to kAggPre of them per lane, so the loads of
+// eight workers are in flight together; the additions then happen worker by worker.
+constexpr int kAggPre = 4;
+
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_compact_aggregate_kernel(const __grid_constant__ SparseLists lists, const int n, const int s,
+                                const uint64_t d, const uint64_t cap, float* __restrict__ out) {
+    __shared__ float s_val[kAggRange];
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t r0 = (uint64_t)blockIdx.x * kAggRange;
+    const uint64_t r1 = min(r0 + (uint64_t)kAggRange, d);
+    for (int i = threadIdx.x; i < kAggRange; i += kBlockThreads) s_val[i] = 0.f;
+    const int nb = code_value_bits(s);
+    for (int w0 = 0; w0 < n; w0 += kWarpsPerBlock) {
+        const int w = w0 + warp;
+        uint32_t lo = 0, hi = 0;
+        uint32_t pj[kAggPre];
+        float pv[kAggPre];
+        float nv = 0.f;
+        const uint32_t* __restrict__ idx = nullptr;
+        const uint32_t* __restrict__ planes = nullptr;
+        if (w < n) {
+            idx = lists.idx[w];
+            planes = lists.planes[w];
+            nv = *lists.norm[w];
+            if (!(fabsf(nv) <= 3.40282347e38f)) nv = 0.f;
+            const uint32_t total = (uint32_t)min((uint64_t)*lists.count[w], cap);
+            lo = warp_lower_bound(idx, 0u, total, (uint32_t)r0, lane);
+            // ascending distinct indices: at most kAggRange entries fall into the range
+            const uint32_t lim = (uint32_t)min((uint64_t)total, (uint64_t)lo + kAggRange);
+            hi = (r1 > 0xFFFFFFFFull) ? total : warp_lower_bound(idx, lo, lim, (uint32_t)r1, lane);
+#pragma unroll
+            for (int e = 0; e < kAggPre; ++e) {
+                const uint32_t k = lo + (uint32_t)(e * 32 + lane);
+                pj[e] = 0xFFFFFFFFu;
+                pv[e] = 0.f;
+                if (k < hi) {
+                    pj[e] = idx[k] - (uint32_t)r0;
+                    pv[e] = compact_entry_value(planes, k, nb, s, nv);
+                }
+            }
+        }
+        for (int t = 0; t < kWarpsPerBlock; ++t) {
+            __syncthreads();                     // fixes the order of the additions (and the fill)
+            if (t != warp || w >= n) continue;
+#pragma unroll
+            for (int e = 0; e < kAggPre; ++e)
+                if (pj[e] != 0xFFFFFFFFu) s_val[pj[e]] = __fadd_rn(s_val[pj[e]], pv[e]);
+            for (uint32_t k = lo + (uint32_t)(kAggPre * 32 + lane); k < hi; k += 32) {
+                float* cell = &s_val[idx[k] - (uint32_t)r0];
+                *cell = __fadd_rn(*cell, compact_entry_value(planes, k, nb, s, nv));
+            }
+        }
+    }
+    __syncthreads();
+    for (uint64_t i = threadIdx.x; r0 + i < r1; i += kBlockThreads) out[r0 + i] = s_val[i];
+}
+
+}  // namespace natcomp
+
+extern "C" {
+
+nc_status nd_sparse_compact_aggregate(const uint32_t* const* idxs, const uint32_t* const* planes,
+                                      const uint32_t* const* counts, const float* const* norms,
+                                      int n, int s, size_t d, size_t cap, float* out,
+                                      cudaStream_t stream) {
+    if (!idxs || !planes || !counts || !norms || !out || n < 1 || n > NC_MAX_WORKERS || s < 1 ||
+        s > 8 || cap < 1)
+        return NC_ERR_INVALID;
+    if (d == 0) return NC_OK;
+    if (d > 0xFFFFFFFFull || cap > 0xFFFFFFFFull) return NC_ERR_INVALID;
+    if (!aligned32(out)) return NC_ERR_ALIGN;
+    SparseLists lists;
+    for (int i = 0; i < n; ++i) {
+        if (!idxs[i] || !planes[i] || !counts[i] || !norms[i]) return NC_ERR_INVALID;
+        if (!aligned16(idxs[i]) || !aligned16(planes[i]) || !aligned4(counts[i]) ||
+            !aligned4(norms[i]))
+            return NC_ERR_ALIGN;
+        lists.idx[i] = idxs[i];
+        lists.planes[i] = planes[i];
+        lists.count[i] = counts[i];
+        lists.norm[i] = norms[i];
+    }
+    const unsigned grid = (unsigned)((d + kAggRange - 1) / kAggRange);
+    sparse_compact_aggregate_kernel<<<grid, kBlockThreads, 0, stream>>>(lists, n, s, d, cap, out);
     return launch_status();
 }
 

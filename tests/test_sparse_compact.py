@@ -178,3 +178,53 @@ def test_config5_full_size_compact_one_worker():
     ref = np.zeros(d, np.float32)
     oracle.sparse_compact_decode_accumulate(i_ref, p_ref, c_ref, n_ref, s, ref)
     assert np.array_equal(acc.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("n,d,thr,scale,cap_frac", [(1, 5, 1 << 32, 1.0, 1.0),
+                                                    (3, 8192, 1 << 30, 4.0, 1.0),
+                                                    (4, 300_000, THR * 8, 12.5, 1.0),
+                                                    (8, (1 << 20) + 77, THR, SCALE, 1.0),
+                                                    (16, 50_001, 1 << 31, 2.0, 0.1),
+                                                    (64, 20_000, 1 << 32, 1.0, 1.0)])
+def test_gpu_compact_aggregate_one_launch_matches_oracle(n, d, thr, scale, cap_frac):
+    # dense sum of n compact lists in worker order; equals the oracle's zero fill followed by the
+    # per-worker decode-accumulate, and the GPU's own per-worker calls
+    import torch
+    import paper_1905_10988_b200 as nc
+    from gpu_util import Guarded, dev
+    rng = np.random.default_rng(n * 7 + d)
+    s = 4
+    cap = max(int(d * cap_frac), 1)
+    xs = [rng.standard_normal(d).astype(np.float32) for _ in range(n)]
+    workers = list(range(20, 20 + n))
+    idx = [Guarded(4 * cap) for _ in range(n)]
+    planes = [Guarded(nc.nd_sparse_plane_bytes(cap, s)) for _ in range(n)]
+    count = [Guarded(4) for _ in range(n)]
+    norm = [Guarded(4) for _ in range(n)]
+    ws_bytes = nc.nd_sparse_batch_workspace_bytes(d, cap, n)
+    ws = Guarded(ws_bytes)
+    nc.nd_sparse_compact_compress_batch([dev(x) for x in xs], d, thr, scale, nc.P_INF, s, 9,
+                                        workers, [g.buf for g in idx], [g.buf for g in planes],
+                                        [g.buf for g in count], [g.buf for g in norm], cap, n,
+                                        ws.buf, ws_bytes)
+    out = Guarded(4 * d)
+    out.buf.fill_(0x7F)                                  # the call must overwrite everything
+    nc.nd_sparse_compact_aggregate([g.buf for g in idx], [g.buf for g in planes],
+                                   [g.buf for g in count], [g.buf for g in norm], n, s, d, cap,
+                                   out.buf)
+    acc = Guarded(4 * d)
+    acc.buf.zero_()
+    for i in range(n):
+        nc.nd_sparse_compact_decode_accumulate(idx[i].buf, planes[i].buf, count[i].buf,
+                                               norm[i].buf, s, d, cap, acc.buf)
+    torch.cuda.synchronize()
+    out.check()
+    ref = np.zeros(d, np.float32)
+    for i in range(n):
+        i_ref, p_ref, c_ref, n_ref = oracle.sparse_compact_compress(xs[i], thr, scale,
+                                                                    oracle.P_INF, s, 9,
+                                                                    workers[i], cap=cap)
+        oracle.sparse_compact_decode_accumulate(i_ref, p_ref, min(c_ref, cap), n_ref, s, ref)
+    assert np.array_equal(out.numpy(np.uint32), ref.view(np.uint32))
+    assert np.array_equal(out.numpy(np.uint32), acc.numpy(np.uint32))
