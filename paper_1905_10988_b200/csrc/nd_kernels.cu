@@ -250,8 +250,9 @@ __device__ __forceinline__ uint32_t level_code(uint32_t bits, uint32_t rnd, cons
                                                float pow2s) {
     const float y = __fmul_rn(fabsf(__uint_as_float(bits)), sc.rinv);   // |x| is an operand modifier
     const float z = __fmul_rn(y, pow2s);
-    float w = z;
-    if (z < 2.0f) w = __fmaf_rz(z, 0.5f, 1.0f);
+    // below 2 the bottom interval [0, 2^(1-s)] is mapped onto [1, 2): w = 1 + z/2 (> z there);
+    // from 2 on 1 + z/2 <= z, so one max selects the right branch
+    const float w = fmaxf(z, __fmaf_rz(z, 0.5f, 1.0f));
     const uint32_t t = __float_as_uint(w) + (~rnd & 0x7FFFFFu) - 0x3F800000u;
     return min(t >> 23, sc.smax);
 }
@@ -260,8 +261,9 @@ __device__ __forceinline__ uint32_t level_code(uint32_t bits, uint32_t rnd, cons
 __device__ __forceinline__ uint32_t level_code_scaled(uint32_t bits, uint32_t rnd, float rinv_s,
                                                       uint32_t smax) {
     const float z = __fmul_rn(fabsf(__uint_as_float(bits)), rinv_s);
-    float w = z;
-    if (z < 2.0f) w = __fmaf_rz(z, 0.5f, 1.0f);
+    // below 2 the bottom interval [0, 2^(1-s)] is mapped onto [1, 2): w = 1 + z/2 (> z there);
+    // from 2 on 1 + z/2 <= z, so one max selects the right branch
+    const float w = fmaxf(z, __fmaf_rz(z, 0.5f, 1.0f));
     const uint32_t t = __float_as_uint(w) + (~rnd & 0x7FFFFFu) - 0x3F800000u;
     return min(t >> 23, smax);
 }

@@ -148,6 +148,14 @@ __device__ __forceinline__ void kept_count_and_partial(const uint32_t word, cons
     }
 }
 
+// drop <- 2 * drop + carry(word + neg_thr): shifts in a 1 iff word >= 2^32 - neg_thr, i.e. iff the
+// coordinate's stream word is not below the keep threshold
+__device__ __forceinline__ void shift_in_drop_bit(uint32_t& drop, uint32_t word, uint32_t neg_thr) {
+    asm("{\n\t.reg .u32 t;\n\tadd.cc.u32 t, %1, %2;\n\taddc.u32 %0, %0, %0;\n\t}"
+        : "+r"(drop)
+        : "r"(word), "r"(neg_thr));
+}
+
 struct Scale {
     float rinv;
     uint32_t smax;
@@ -167,8 +175,9 @@ __device__ __forceinline__ uint32_t sparse_level_code(uint32_t bits, uint32_t rn
     const float ax = __uint_as_float(bits & 0x7FFFFFFFu);
     const float y = __fmul_rn(ax, sc.rinv);
     const float z = __fmul_rn(y, pow2s);
-    float w = z;
-    if (z < 2.0f) w = __fmaf_rz(z, 0.5f, 1.0f);
+    // below 2 the bottom interval [0, 2^(1-s)] is mapped onto [1, 2): w = 1 + z/2 (> z there);
+    // from 2 on 1 + z/2 <= z, so one max selects the right branch
+    const float w = fmaxf(z, __fmaf_rz(z, 0.5f, 1.0f));
     const uint32_t t = __float_as_uint(w) + (~rnd & 0x7FFFFFu) - 0x3F800000u;
     return min(t >> 23, sc.smax);
 }

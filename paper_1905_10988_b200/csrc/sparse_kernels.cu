@@ -47,12 +47,7 @@ sparse_select_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d
             uint32_t rnd[4];
             stream_words4_tile(q_lo + (uint32_t)k, pt, keys, rnd);
 #pragma unroll
-            for (int c = 3; c >= 0; --c) {
-                uint32_t tmp;
-                asm("add.cc.u32 %1, %2, %3;\n\taddc.u32 %0, %0, %0;"
-                    : "+r"(drop), "=r"(tmp)
-                    : "r"(rnd[c]), "r"(neg_thr));
-            }
+            for (int c = 3; c >= 0; --c) shift_in_drop_bit(drop, rnd[c], neg_thr);
         }
         word = ~drop;
         if (base + kTile > d) {          // ragged last tile: clear the bits past the end
@@ -599,13 +594,7 @@ sparse_regen_mask_kernel(const uint64_t d, const uint32_t neg_thr, const bool ke
             uint32_t rnd[4];
             stream_words4_tile(q_lo + (uint32_t)k, pt, keys, rnd);
 #pragma unroll
-            for (int c = 3; c >= 0; --c) {
-                uint32_t tmp;
-                asm("add.cc.u32 %1, %2, %3;\n\taddc.u32 %0, %0, %0;"
-                    : "+r"(drop), "=r"(tmp)
-                    : "r"(rnd[c]), "r"(neg_thr));
-                (void)tmp;
-            }
+            for (int c = 3; c >= 0; --c) shift_in_drop_bit(drop, rnd[c], neg_thr);
         }
         word = ~drop;
         if (base + kTile > d) {
