@@ -217,6 +217,10 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--peak-gbs", type=float, default=HBM_PEAK_FALLBACK,
                     help="HBM bandwidth the fractions are quoted against")
+    ap.add_argument("--workers", type=int, default=0,
+                    help="override the number of simulated workers (smaller cases for profiling)")
+    ap.add_argument("--log2-d", type=int, default=0,
+                    help="override the vector length of c5 with 2^LOG2_D")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device")
@@ -227,16 +231,17 @@ def main():
     elif args.config == "c2":
         sizes = workloads.resnet50_tensor_sizes()
         d = sum(sizes)
-        run_cnat("c2", 8, d, lambda w: workloads.config2_vector(w, "cuda", sizes), args.iters,
+        n = args.workers or 8
+        run_cnat("c2", n, d, lambda w: workloads.config2_vector(w, "cuda", sizes), args.iters,
                  peak)
-        run_cnat64("c2", 8, d, args.iters, peak)
+        run_cnat64("c2", n, d, args.iters, peak)
     elif args.config == "c3":
         run_dnat("c3", 8, workloads.resnet50_tensor_sizes(), args.iters, peak)
     elif args.config == "c4":
         d = sum(workloads.bert_large_bucket_sizes())
         run_cnat("c4", 16, d, lambda w: workloads.config4_vector(w, d, "cuda"), args.iters, peak)
     else:
-        run_sparse("c5", 8, 1 << 28, args.iters, peak)
+        run_sparse("c5", args.workers or 8, 1 << (args.log2_d or 28), args.iters, peak)
 
 
 if __name__ == "__main__":

@@ -228,3 +228,38 @@ def test_gpu_compact_aggregate_one_launch_matches_oracle(n, d, thr, scale, cap_f
         oracle.sparse_compact_decode_accumulate(i_ref, p_ref, min(c_ref, cap), n_ref, s, ref)
     assert np.array_equal(out.numpy(np.uint32), ref.view(np.uint32))
     assert np.array_equal(out.numpy(np.uint32), acc.numpy(np.uint32))
+
+
+@pytest.mark.gpu
+def test_compact_bench_launch_configuration_full_size():
+    # exactly what the benchmark step runs for the sparse part: 8 workers, d = 25,557,032, one
+    # batch compress call and one aggregate call; every output compared in full
+    import torch
+    import paper_1905_10988_b200 as nc
+    n, s = 8, 4
+    sizes = workloads.resnet50_tensor_sizes()
+    d = sum(sizes)
+    cap = int(d * 0.0125)
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    xd = [workloads.config2_vector(w, "cuda", sizes) for w in range(n)]
+    idx = [torch.empty(cap, dtype=torch.int32, device="cuda") for _ in range(n)]
+    planes = [torch.empty(nc.nd_sparse_plane_bytes(cap, s), **u8) for _ in range(n)]
+    count = [torch.zeros(1, dtype=torch.int32, device="cuda") for _ in range(n)]
+    norm = [torch.zeros(1, dtype=torch.float32, device="cuda") for _ in range(n)]
+    ws_bytes = nc.nd_sparse_batch_workspace_bytes(d, cap, n)
+    ws = torch.empty(ws_bytes, **u8)
+    nc.nd_sparse_compact_compress_batch(xd, d, THR, SCALE, nc.P_INF, s, 0, list(range(n)), idx,
+                                        planes, count, norm, cap, n, ws, ws_bytes)
+    out = torch.empty(d, dtype=torch.float32, device="cuda")
+    nc.nd_sparse_compact_aggregate(idx, planes, count, norm, n, s, d, cap, out)
+    torch.cuda.synchronize()
+    ref = np.zeros(d, np.float32)
+    for w in range(n):
+        i_ref, p_ref, c_ref, n_ref = oracle.sparse_compact_compress(xd[w].cpu().numpy(), THR, SCALE,
+                                                                    oracle.P_INF, s, 0, w, cap=cap)
+        cnt = int(count[w].cpu().numpy().view(np.uint32)[0])
+        assert cnt == c_ref <= cap and float(norm[w].cpu()[0]) == float(n_ref)
+        assert np.array_equal(idx[w][:cnt].cpu().numpy().view(np.uint32), i_ref)
+        assert np.array_equal(planes[w].cpu().numpy().view(np.uint32)[:p_ref.size], p_ref)
+        oracle.sparse_compact_decode_accumulate(i_ref, p_ref, c_ref, n_ref, s, ref)
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), ref.view(np.uint32))
