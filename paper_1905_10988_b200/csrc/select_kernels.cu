@@ -183,8 +183,23 @@ select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws) {
     for (uint64_t g = blockIdx.x; g < groups; g += gridDim.x) {
         const uint64_t base = (g * kWarpsPerBlock + (threadIdx.x >> 5)) * kTile;
         if (base >= d) continue;
-        const uint32_t valid = valid_nibbles<Src>(base, lane, d);
         const typename Src::Tile t = src.tile(base, lane);
+        if (Src::kCanonical && base + kTile <= d) {
+            // computed keys, full tile: no validity test (this variant is bound by instruction
+            // issue; the loaded-key variant is bound by memory and keeps the smaller code)
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                uint32_t key[4];
+                src.load(t, base, lane, k, d, key);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if ((key[c] & fixed) == prefix)
+                        atomicAdd(&s_hist[(key[c] >> shift) & (uint32_t)(bins - 1)], 1u);
+                }
+            }
+            continue;
+        }
+        const uint32_t valid = valid_nibbles<Src>(base, lane, d);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             uint32_t key[4];
@@ -547,8 +562,24 @@ template <class Src>
 static void run_select(const Src& src, uint64_t d, uint64_t q, const SparseWorkspace& sp,
                        const SelectWorkspace& ws, int sm_count, cudaStream_t stream) {
     const uint64_t groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    const unsigned pgrid = (unsigned)(groups < (uint64_t)sm_count * 8 ? groups
-                                                                      : (uint64_t)sm_count * 8);
+    // persistent grid: exactly the blocks that are resident together (a partial second wave would
+    // run at the end with most SMs idle)
+    static int per_sm[64] = {0};
+    int dev = 0;
+    int resident = 4;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
+        if (per_sm[dev] == 0) {
+            int v = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, select_hist_kernel<Src, 0>,
+                                                              kBlockThreads, 0) != cudaSuccess ||
+                v < 1)
+                v = 4;
+            per_sm[dev] = v;
+        }
+        resident = per_sm[dev];
+    }
+    const uint64_t cap_blocks = (uint64_t)sm_count * (uint64_t)resident;
+    const unsigned pgrid = (unsigned)(groups < cap_blocks ? groups : cap_blocks);
     select_init_kernel<<<1, kScanThreads, 0, stream>>>(ws, q);
     select_hist_kernel<Src, 0><<<pgrid, kBlockThreads, 0, stream>>>(src, d, ws);
     select_choose_kernel<0><<<1, kScanThreads, 0, stream>>>(ws);
