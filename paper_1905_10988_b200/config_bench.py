@@ -190,6 +190,11 @@ def run_sparse(config, n, d, iters, peak, s=4):
     m, b = _time(accumulate_compact, iters)
     _report(config, "nd_sparse_compact_decode_accumulate x n", m, b, listed, listed * 68.4, peak)
 
+    m, b = _time(lambda: nc.nd_sparse_compact_aggregate(idx, planes, count, norm, n, s, d, cap,
+                                                        acc), iters)
+    _report(config, "nd_sparse_compact_aggregate (all workers, one launch, dense output)", m, b,
+            listed, 4.0 * d + listed * 4.375, peak)
+
     # exactly q = d / 100 kept coordinates (radix select over the selection words), one worker
     q = d // 100
     sel_bytes = nc.nc_select_workspace_bytes(d, cap)
