@@ -40,10 +40,10 @@ UNIT = "Gelem/s"
 
 # Per-launch DRAM traffic of the dominant kernel (nc_compress_kernel, 8-worker batch launch):
 # dram__bytes_read.sum + dram__bytes_write.sum of the 2-worker capture summarised in
-# profiles/nc_compress_c2_2workers.md (204.48 MB + 28.95 MB), scaled by 4 to the 8-worker launch
+# profiles/nc_compress_c2_2workers.md (204.48 MB + 31.59 MB), scaled by 4 to the 8-worker launch
 # (traffic is proportional to the number of workers).  The write part is below the 28.75 MB per
 # worker that the kernel stores because some output is still dirty in L2 when the kernel ends.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * (204_482_048 + 28_953_600)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * (204_482_816 + 31_589_376)
 
 
 def measured_hbm_peak():
