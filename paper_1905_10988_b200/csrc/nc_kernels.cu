@@ -233,10 +233,76 @@ __device__ __forceinline__ float decode9(uint32_t e4, uint32_t s) {
     return __uint_as_float(__funnelshift_r(hi, s, 1));                // (hi >> 1) | (s << 31)
 }
 
+// Staging of the workers' planes for the aggregation sweep: the 1024 exponent bytes and 32 sign
+// words of a tile are copied global -> shared with cp.async (16 bytes per lane and copy), three
+// workers ahead of the one being decoded, in a ring that is private to the warp.  The loads of
+// several workers are in flight without holding registers, so the sweep is not bound by the
+// latency of one worker's loads.
+constexpr int kAggStages = 4;
+
+struct AggStage {
+    uint32_t e[256];     // exponent bytes of the tile, word k*32 + l = lane l's group k
+    uint32_t s[32];      // sign words of the tile
+};
+
+__device__ __forceinline__ void agg_stage_issue(AggStage* st, const uint8_t* __restrict__ exp_tile,
+                                                const uint32_t* __restrict__ sign_tile,
+                                                const int lane) {
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&st->e[lane * 4]);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(exp_tile + lane * 16)
+                 : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 512u),
+                 "l"(exp_tile + 512 + lane * 16)
+                 : "memory");
+    if (lane < 8) {
+        const uint32_t dsts = (uint32_t)__cvta_generic_to_shared(&st->s[lane * 4]);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dsts),
+                     "l"(sign_tile + lane * 4)
+                     : "memory");
+    }
+}
+
 // acc[k] += decoded values of workers 0..n-1, in that order, for one full tile
 __device__ __forceinline__ void aggregate_full_tile(const PackedPlanes& planes, const int n,
                                                     const uint64_t base, float4 (&acc)[8],
                                                     const int lane) {
+    __shared__ __align__(16) AggStage s_ring[kWarpsPerBlock][kAggStages];
+    AggStage* ring = s_ring[threadIdx.x >> 5];
+    const int sh = 4 * (lane & 7);
+#pragma unroll
+    for (int j = 0; j < kAggStages - 1; ++j) {
+        if (j < n) agg_stage_issue(&ring[j], planes.exp[j] + base, planes.sign[j] + (base >> 5), lane);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    for (int i = 0; i < n; ++i) {
+        const int ahead = i + kAggStages - 1;
+        if (ahead < n)
+            agg_stage_issue(&ring[ahead % kAggStages], planes.exp[ahead] + base,
+                            planes.sign[ahead] + (base >> 5), lane);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group %0;" ::"n"(kAggStages - 1) : "memory");
+        __syncwarp();                                   // worker i's planes are in the ring
+        const AggStage* st = &ring[i % kAggStages];
+        const uint32_t sw = st->s[lane];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t e = st->e[k * 32 + lane];
+            // sign word (k, g) lives in lane 4k+g; this lane needs group g = lane / 8
+            const uint32_t s = __shfl_sync(0xFFFFFFFFu, sw, k * 4 + (lane >> 3)) >> sh;
+            acc[k].x += decode9<0>(e, s);
+            acc[k].y += decode9<1>(e, s >> 1);
+            acc[k].z += decode9<2>(e, s >> 2);
+            acc[k].w += decode9<3>(e, s >> 3);
+        }
+        __syncwarp();                                   // the stage may be overwritten now
+    }
+}
+
+// The same sweep with plain loads, for the kernel that compresses the sum again: that one is
+// bound by its own generator and packing work, and the shared-memory ring only costs it residency.
+__device__ __forceinline__ void aggregate_full_tile_direct(const PackedPlanes& planes, const int n,
+                                                           const uint64_t base, float4 (&acc)[8],
+                                                           const int lane) {
     const int sh = 4 * (lane & 7);
     for (int i = 0; i < n; ++i) {
         const uint32_t* ev = reinterpret_cast<const uint32_t*>(planes.exp[i] + base);
@@ -246,7 +312,6 @@ __device__ __forceinline__ void aggregate_full_tile(const PackedPlanes& planes, 
         for (int k = 0; k < 8; ++k) e[k] = ld_stream_u32(ev + k * 32 + lane);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            // sign word (k, g) lives in lane 4k+g; this lane needs group g = lane / 8
             const uint32_t s = __shfl_sync(0xFFFFFFFFu, sw, k * 4 + (lane >> 3)) >> sh;
             acc[k].x += decode9<0>(e[k], s);
             acc[k].y += decode9<1>(e[k], s >> 1);
@@ -270,7 +335,7 @@ __device__ __forceinline__ float aggregate_element(const PackedPlanes& planes, c
 // out[j] = (init + v_0j) + v_1j + ... ; init = +0 (aggregate) or acc[j] (decode-accumulate).
 // grid: ceil(tiles / warps per block)
 template <bool kFromAcc>
-__global__ void __launch_bounds__(kBlockThreads, 5)
+__global__ void __launch_bounds__(kBlockThreads, 4)
 nc_aggregate_kernel(const __grid_constant__ PackedPlanes planes, const int n, const uint64_t d,
                     float* __restrict__ out) {
     const int lane = threadIdx.x & 31;
@@ -311,7 +376,7 @@ nc_aggregate_compress_kernel(const __grid_constant__ PackedPlanes planes, const 
         float4 acc[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        aggregate_full_tile(planes, n, base, acc, lane);
+        aggregate_full_tile_direct(planes, n, base, acc, lane);
         uint4 u[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k)
