@@ -216,3 +216,38 @@ def test_config4_full_size_sampled():
     x2 = sum(float((x.double() ** 2).sum()) for x in xd)
     assert err2 <= x2 / 8 * 1.02
     assert err2 >= x2 / 8 * 0.3
+
+
+def test_beyond_2_to_34_entries_sampled():
+    # one vector of 2^34 + 2^20 + 77 entries (69 GB): tile bases above 2^32 (64-bit addressing)
+    # and above 2^34, where the high word of the generator's counter becomes non-zero; sampled
+    # slices against the oracle, which takes the offset of a slice as its first element index
+    d = (1 << 34) + (1 << 20) + 77
+    free, _ = torch.cuda.mem_get_info()
+    if free < 110 * (1 << 30):
+        pytest.skip("needs ~90 GB of free device memory")
+    x = torch.empty(d, dtype=torch.float32, device="cuda")
+    g = torch.Generator(device="cuda")
+    g.manual_seed(34)
+    chunk = 1 << 28
+    for a in range(0, d, chunk):
+        x[a:min(d, a + chunk)].normal_(0.0, 1e-3, generator=g)
+    e = torch.empty(nc.nc_exp_bytes(d), dtype=torch.uint8, device="cuda")
+    s = torch.empty(nc.nc_sign_bytes(d), dtype=torch.uint8, device="cuda")
+    nc.nc_compress(x, d, 5, 9, e, s)
+    torch.cuda.synchronize()
+    length = 4096
+    offs = [0, (1 << 32) - 2048, (1 << 32), (1 << 33) + 1024 * 777, (1 << 34) - 2048, (1 << 34),
+            (1 << 34) + 1024 * 500, ((d - length) // 32) * 32]
+    for o in offs:
+        hi = min(d, o + length)
+        e_ref, s_ref = oracle.nc_compress(x[o:hi].cpu().numpy(), 5, 9, j0=o)
+        assert np.array_equal(e[o:hi].cpu().numpy(), e_ref), o
+        sw = s.view(torch.int32)[o // 32:(hi + 31) // 32].cpu().numpy().view(np.uint32)
+        assert np.array_equal(sw, s_ref), o
+    # the two sides of 2^34 draw from different counter blocks: same inputs, different rounding
+    a = e[(1 << 34) - 4096:(1 << 34)].cpu().numpy()
+    b = e[(1 << 34):(1 << 34) + 4096].cpu().numpy()
+    assert not np.array_equal(a, b)
+    del x, e, s
+    torch.cuda.empty_cache()

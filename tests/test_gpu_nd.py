@@ -273,3 +273,59 @@ def test_one_element_buckets_and_many_empty_buckets():
     off2 = sorted([0] + list(rng.integers(0, d, 40)) * 3 + [d])
     norms, level, sign = gpu_nd_compress(dev(x), off2, 1, 4, seed=5, worker=0)
     check_against_oracle(x, off2, 1, 4, 5, 0, norms, level, sign, slack=2)
+
+
+def test_beyond_2_to_32_entries_sampled():
+    # one vector of 2^32 + 2^21 + 13 entries (17 GB) in three buckets whose boundaries sit at odd
+    # places around 2^31 and 2^32: 64-bit element indices in the norm pass, the rounding pass and
+    # the aggregate.  Norms against float64 sums on the device data, level and sign planes on
+    # sampled slices against the oracle (given the norm, slice offset as first element index).
+    d = (1 << 32) + (1 << 21) + 13
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 * (1 << 30):
+        pytest.skip("needs ~50 GB of free device memory")
+    p, s = 2, 8
+    off = [0, (1 << 31) + 5, (1 << 32) + 1029, d]
+    B = 3
+    off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
+    x = torch.empty(d, dtype=torch.float32, device="cuda")
+    g = torch.Generator(device="cuda")
+    g.manual_seed(32)
+    chunk = 1 << 28
+    for a in range(0, d, chunk):
+        x[a:min(d, a + chunk)].normal_(0.0, 1e-3, generator=g)
+    ws_bytes = nc.nd_workspace_bytes(d, B)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    norms = torch.empty(B, dtype=torch.float32, device="cuda")
+    level = torch.empty(nc.nd_level_bytes(d), dtype=torch.uint8, device="cuda")
+    sign = torch.empty(nc.nc_sign_bytes(d), dtype=torch.uint8, device="cuda")
+    nc.nd_compress(x, d, off_dev, B, p, s, 3, 1, norms, level, sign, ws, ws_bytes)
+    out = torch.empty(d, dtype=torch.float32, device="cuda")
+    nc.nd_aggregate([norms], [level], [sign], 1, d, off_dev, B, s, out)
+    torch.cuda.synchronize()
+    gn = norms.cpu().numpy()
+    for b in range(B):
+        sq = 0.0
+        for a in range(off[b], off[b + 1], chunk):
+            sq += float((x[a:min(off[b + 1], a + chunk)].double() ** 2).sum())
+        assert abs(float(gn[b]) - sq ** 0.5) <= NORM_RTOL * sq ** 0.5
+    length = 4096
+    # (slice start, bucket): inside each bucket, on both sides of 2^32, and the ragged tail
+    picks = [(0, 0), ((1 << 31) - 4096, 0), ((1 << 31) + 32, 1), ((1 << 32) - 4096, 1),
+             ((1 << 32), 1), ((1 << 32) + 2048, 2), (((d - length) // 32) * 32, 2)]
+    for o, b in picks:
+        hi = min(d, o + length, off[b + 1])
+        assert off[b] <= o and hi <= off[b + 1]
+        xs = x[o:hi].cpu().numpy()
+        _, l_ref, s_ref = oracle.nd_compress(xs, [0, hi - o], p, s, 3, 1, given_norms=gn[b:b + 1],
+                                             j0=o)
+        m = hi - o                                  # a slice may end inside a byte / sign word
+        lv = level[o // 2:(hi + 1) // 2].cpu().numpy()
+        assert np.array_equal(unpack_nibbles(lv, m), unpack_nibbles(l_ref, m)), o
+        sw = sign.view(torch.int32)[o // 32:(hi + 31) // 32].cpu().numpy().view(np.uint32)
+        k = np.arange(m)
+        assert np.array_equal((sw[k // 32] >> (k % 32)) & 1, (s_ref[k // 32] >> (k % 32)) & 1), o
+        want = oracle.nd_aggregate([gn[b:b + 1]], [l_ref], [s_ref], [0, hi - o], s, hi - o)
+        assert np.array_equal(out[o:hi].cpu().numpy().view(np.uint32), want.view(np.uint32)), o
+    del x, level, sign, out, ws
+    torch.cuda.empty_cache()
