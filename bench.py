@@ -404,7 +404,16 @@ def main():
                 "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind,
                 "unit": "GB/s", "frac": round(achieved / peak, 4),
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
-                "algorithmic_bytes_per_launch": alg[dom]}
+                "algorithmic_bytes_per_launch": alg[dom],
+                # the second resource of this kernel: the generator needs 18 wide 32x32->64
+                # multiplies per 4 entries, and a sub-partition issues one per 4 cycles:
+                # 148 SMs x 4 x 32 lanes x f_SM / 4 / 4.5 entries per second at the sampled SM clock
+                "generator_view": {
+                    "achieved_Gelem_per_s": round(units_per_step / group_ms[dom] / 1e6, 1),
+                    "multiplier_pipe_peak_Gelem_per_s": round(
+                        148 * 4 * 32 * (clocks.get("sm_mhz") or 1965) * 1e6 / 4 / 4.5 / 1e9, 1)}}
+    gv = roofline["generator_view"]
+    gv["frac"] = round(gv["achieved_Gelem_per_s"] / gv["multiplier_pipe_peak_Gelem_per_s"], 4)
 
     # end to end: host buffers -> device -> whole path -> aggregates back on the host
     e2e = None
