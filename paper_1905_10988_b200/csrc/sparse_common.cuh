@@ -80,6 +80,31 @@ __device__ __forceinline__ uint32_t warp_list_positions(uint32_t word, int lane,
     return __shfl_sync(0xFFFFFFFFu, incl, 31);
 }
 
+// Lists of kept positions for a group of 8 tiles (8192 coordinates, the unit of the per-block
+// counts): at 1 % density a single tile has about ten kept entries, so the sparse passes give a
+// warp a whole group and work on the listed entries with all lanes busy.
+constexpr uint32_t kGroupListCap = 2048;      // >= kTile: one tile always fits into an empty list
+
+// appends the positions (inside the group, tile w) of the set bits of `word` (lane l = word l of
+// the tile) to list[at ..]; returns how many
+__device__ __forceinline__ uint32_t group_list_append(uint32_t word, int lane, int w,
+                                                      uint16_t* __restrict__ list, uint32_t at) {
+    const uint32_t cnt = __popc(word);
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    uint32_t pos = at + incl - cnt;
+    while (word) {
+        const int bit = __ffs(word) - 1;
+        word &= word - 1;
+        list[pos++] = (uint16_t)(w * kTile + lane * 32 + bit);
+    }
+    return __shfl_sync(0xFFFFFFFFu, incl, 31);
+}
+
 // A lane's 32 per-element bits in the load layout (bit 4k+c <-> element k*128 + 4*lane + c of
 // the tile) -> canonical order: lane l returns the word of elements 32l .. 32l+31.
 __device__ __forceinline__ uint32_t canonical_mask_word(uint32_t nib, int lane) {

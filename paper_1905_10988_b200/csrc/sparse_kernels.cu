@@ -62,6 +62,109 @@ sparse_select_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d
     kept_count_and_partial<P>(word, lane, x, base, scale, ws.block_count, ws.block_partial);
 }
 
+// The same pass with one warp per group of 8 tiles: an eighth of the per-tile bookkeeping, used
+// when there are enough groups to fill the GPU many times over (otherwise the coarser work
+// units cost more in the last, partly filled wave than they save).
+// grid: (ceil(tile groups / warps per block), n workers); one warp per group of 8 tiles
+// (8192 coordinates, the unit of the per-block counts and norm partials)
+template <int P>
+__global__ void __launch_bounds__(kBlockThreads)
+sparse_select_group_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
+                           const uint32_t neg_thr, const bool keep_none, const float scale,
+                           const __grid_constant__ PhiloxKeys keys, char* __restrict__ ws_all,
+                           const uint64_t ws_stride) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t tiles = sparse_tiles(d);
+    const uint64_t groups = (tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const uint64_t grp = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    if (grp >= groups) return;
+    const uint64_t tile0 = grp * kWarpsPerBlock;
+    const uint64_t gbase = tile0 * kTile;
+    const float* __restrict__ x = batch.x[blockIdx.y];
+    const uint32_t worker = batch.worker[blockIdx.y];
+    const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
+    __shared__ uint16_t s_list[kWarpsPerBlock][kGroupListCap];
+    uint16_t* list = s_list[warp];
+
+    double dsum = 0.0;
+    uint32_t vmax = 0;
+    auto take = [&](float xv) {
+        const float xs = __fmul_rn(scale, xv);
+        const uint32_t a = __float_as_uint(xs) & 0x7FFFFFFFu;
+        if (P == NC_P_INF) vmax = max(vmax, a);
+        else if (P == 1) dsum += (double)__uint_as_float(a);
+        else dsum = fma((double)xs, (double)xs, dsum);
+    };
+    // gathers the listed entries (all loads of the usual short list are issued before any is used)
+    auto flush = [&](uint32_t cnt) {
+        __syncwarp();
+        if (cnt <= 4u * 32u) {
+            float xv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t t = (uint32_t)(e * 32 + lane);
+                xv[e] = (t < cnt) ? x[gbase + list[t]] : 0.f;       // +0 adds nothing to any norm
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) take(xv[e]);
+        } else {
+            for (uint32_t t = lane; t < cnt; t += 32) take(x[gbase + list[t]]);
+        }
+        __syncwarp();
+    };
+
+    // phase 1 per tile: the 1024 selection bits, no memory traffic.  Lane l draws the eight
+    // counter groups of elements 32l .. 32l+31, so its 32 bits are word l of the tile mask.
+    // phase 2: the kept positions of the whole group are listed and gathered together.
+    uint32_t cnt = 0, kept = 0;
+#pragma unroll 1
+    for (int w = 0; w < kWarpsPerBlock; ++w) {
+        const uint64_t tile = tile0 + w;
+        const uint64_t base = tile * kTile;
+        if (base >= d) break;
+        uint32_t word = 0;
+        if (!keep_none) {
+            // coordinate j is dropped iff word >= threshold, i.e. iff word + (2^32 - threshold)
+            // carries out of 32 bits.  The drop bits are shifted in straight from that carry:
+            // two integer instructions per coordinate on top of the generator.
+            const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainSelect, keys);
+            const uint32_t q_lo = (uint32_t)(base >> 2) + (uint32_t)(lane * 8);
+            uint32_t drop = 0;
+#pragma unroll
+            for (int k = 7; k >= 0; --k) {
+                uint32_t rnd[4];
+                stream_words4_tile(q_lo + (uint32_t)k, pt, keys, rnd);
+#pragma unroll
+                for (int c = 3; c >= 0; --c) shift_in_drop_bit(drop, rnd[c], neg_thr);
+            }
+            word = ~drop;
+            if (base + kTile > d) {          // ragged last tile: clear the bits past the end
+                const uint64_t first = base + (uint64_t)(lane * 32);
+                if (first >= d) word = 0u;
+                else if (first + 32 > d) word &= (1u << (uint32_t)(d - first)) - 1u;
+            }
+        }
+        ws.bitmask[tile * 32 + lane] = word;
+        const uint32_t tile_cnt = warp_sum_u(__popc(word));
+        if (cnt + tile_cnt > kGroupListCap) {
+            flush(cnt);
+            cnt = 0;
+        }
+        group_list_append(word, lane, w, list, cnt);
+        cnt += tile_cnt;
+        kept += tile_cnt;
+    }
+    flush(cnt);
+    uint64_t part;
+    if (P == NC_P_INF) part = (uint64_t)warp_max_u(vmax);
+    else part = (uint64_t)__double_as_longlong(warp_sum_d(dsum));
+    if (lane == 0) {
+        ws.block_count[grp] = kept;
+        ws.block_partial[grp] = part;
+    }
+}
+
 // one block: exclusive scan of the per-block counts (in place), total count, norm
 template <int P>
 __global__ void __launch_bounds__(kScanThreads)
@@ -188,6 +291,40 @@ sparse_decode_accumulate_kernel(const uint32_t* __restrict__ idx, const uint8_t*
     acc[j] = __fadd_rn(acc[j], __fmul_rn(nv, __uint_as_float(pb)));
 }
 
+static void launch_select(const SparseBatch& batch, uint64_t d, uint64_t keep_threshold,
+                          float scale, int p, const PhiloxKeys& keys, char* ws, uint64_t ws_stride,
+                          int n, cudaStream_t stream) {
+    const uint64_t tile_groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const bool keep_none = keep_threshold == 0;
+    const uint32_t neg_thr = (uint32_t)(0ull - keep_threshold);   // 2^32 - threshold (mod 2^32)
+    // one warp per group needs about 150 SMs x 48 resident warps x 8 groups to balance
+    const bool by_group = tile_groups * (uint64_t)n >= 57000;
+    if (by_group) {
+        const dim3 grid((unsigned)((tile_groups + kWarpsPerBlock - 1) / kWarpsPerBlock),
+                        (unsigned)n);
+        if (p == 1)
+            sparse_select_group_kernel<1><<<grid, kBlockThreads, 0, stream>>>(
+                batch, d, neg_thr, keep_none, scale, keys, ws, ws_stride);
+        else if (p == 2)
+            sparse_select_group_kernel<2><<<grid, kBlockThreads, 0, stream>>>(
+                batch, d, neg_thr, keep_none, scale, keys, ws, ws_stride);
+        else
+            sparse_select_group_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
+                batch, d, neg_thr, keep_none, scale, keys, ws, ws_stride);
+        return;
+    }
+    const dim3 grid((unsigned)tile_groups, (unsigned)n);
+    if (p == 1)
+        sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
+                                                                    scale, keys, ws, ws_stride);
+    else if (p == 2)
+        sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
+                                                                    scale, keys, ws, ws_stride);
+    else
+        sparse_select_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
+            batch, d, neg_thr, keep_none, scale, keys, ws, ws_stride);
+}
+
 static void launch_scan(const SparseBatch& batch, uint64_t d, int p, char* ws, uint64_t ws_stride,
                         int n, cudaStream_t stream) {
     const dim3 sgrid(1, (unsigned)n);
@@ -243,17 +380,7 @@ nc_status nd_sparse_compress_batch(const float* const* xs, size_t d, uint64_t ke
     const uint64_t tiles = sparse_tiles(d);
     const dim3 grid((unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
     const PhiloxKeys keys = make_philox_keys(seed);
-    const bool keep_none = keep_threshold == 0;
-    const uint32_t neg_thr = (uint32_t)(0ull - keep_threshold);   // 2^32 - threshold (mod 2^32)
-    if (p == 1)
-        sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
-                                                                    scale, keys, ws, ws_stride);
-    else if (p == 2)
-        sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
-                                                                    scale, keys, ws, ws_stride);
-    else
-        sparse_select_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
-            batch, d, neg_thr, keep_none, scale, keys, ws, ws_stride);
+    launch_select(batch, d, keep_threshold, scale, p, keys, ws, ws_stride, n, stream);
     launch_scan(batch, d, p, ws, ws_stride, n, stream);
     sparse_emit_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap, ws,
                                                            ws_stride);
@@ -304,7 +431,13 @@ nc_status nd_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes,
 //   pack_planes   : 32 code bytes -> nb + 1 plane words (warp ballots)
 namespace natcomp {
 
-// grid: (ceil(tiles / warps per block), n workers)
+// The level filter and the emit pass give one warp a whole group of 8 tiles (8192 coordinates,
+// the unit of the per-block counts): at 1 % density a single tile has about ten kept entries, so
+// a warp per tile leaves most lanes idle and pays its fixed costs per ten entries.  The warp loads
+// the 8 x 32 mask words at once, lists the kept positions of the group in shared memory (flushing
+// whenever the next tile would not fit, so any density works) and handles the listed entries with
+// all lanes busy.  No block barrier.
+// grid: (ceil(tile groups / warps per block), n workers); one warp per group of 8 tiles
 __global__ void __launch_bounds__(kBlockThreads)
 sparse_round_filter_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
                            const float scale, const int s,
@@ -312,59 +445,82 @@ sparse_round_filter_kernel(const __grid_constant__ SparseBatch batch, const uint
                            const uint64_t ws_stride) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
-    const uint64_t base = tile * kTile;
-    const bool active = base < d;
+    const uint64_t tiles = sparse_tiles(d);
+    const uint64_t groups = (tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const uint64_t grp = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    if (grp >= groups) return;
+    const uint64_t tile0 = grp * kWarpsPerBlock;
+    const uint64_t gbase = tile0 * kTile;
     const float* __restrict__ x = batch.x[blockIdx.y];
     const uint32_t worker = batch.worker[blockIdx.y];
     const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
-    __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
-    __shared__ uint32_t s_mask[kWarpsPerBlock][32];
-    __shared__ uint32_t s_cnt[kWarpsPerBlock];
+    __shared__ uint16_t s_list[kWarpsPerBlock][kGroupListCap];
+    __shared__ uint32_t s_mask[kWarpsPerBlock][kWarpsPerBlock * 32];
     uint16_t* list = s_list[warp];
-    const uint32_t word = active ? ws.bitmask[tile * 32 + lane] : 0u;
-    const uint32_t cnt = warp_sum_u(__popc(word));
+    uint32_t* mask = s_mask[warp];
+    uint32_t word[kWarpsPerBlock];
+#pragma unroll
+    for (int w = 0; w < kWarpsPerBlock; ++w)
+        word[w] = (tile0 + w < tiles) ? ws.bitmask[(tile0 + w) * 32 + lane] : 0u;
+#pragma unroll
+    for (int w = 0; w < kWarpsPerBlock; ++w) mask[w * 32 + lane] = word[w];
     const Scale sc = make_scale(*batch.norm[blockIdx.y], s);
     const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
-    uint32_t kept;
-    if (cnt <= 96u) {
-        // few kept entries: every lane walks the bits of its own word
-        kept = word;
-        uint32_t w = word;
-        while (w) {
-            const int bit = __ffs(w) - 1;
-            w &= w - 1;
-            const uint64_t j = base + (uint64_t)(lane * 32 + bit);
-            const float xs = __fmul_rn(scale, x[j]);
-            const uint32_t r = stream_word_at(j, worker, kDomainDnat, keys);
-            if (sparse_level_code(__float_as_uint(xs), r, sc, pow2s) == 0u) kept &= ~(1u << bit);
-        }
-    } else {
-        s_mask[warp][lane] = word;
-        warp_list_positions(word, lane, list);     // ends with __syncwarp
-        for (uint32_t t = lane; t < cnt; t += 32) {
-            const uint32_t pos = list[t];
-            const uint64_t j = base + pos;
-            const float xs = __fmul_rn(scale, x[j]);
-            const uint32_t r = stream_word_at(j, worker, kDomainDnat, keys);
-            if (sparse_level_code(__float_as_uint(xs), r, sc, pow2s) == 0u)
-                atomicAnd(&s_mask[warp][pos >> 5], ~(1u << (pos & 31)));
+    __syncwarp();
+
+    auto round_one = [&](uint32_t p, float xv) {
+        const float xs = __fmul_rn(scale, xv);
+        const uint32_t r = stream_word_at(gbase + p, worker, kDomainDnat, keys);
+        if (sparse_level_code(__float_as_uint(xs), r, sc, pow2s) == 0u)
+            atomicAnd(&mask[p >> 5], ~(1u << (p & 31)));
+    };
+    auto flush = [&](uint32_t cnt) {
+        __syncwarp();
+        if (cnt <= 4u * 32u) {
+            // the usual case: all gathers of the group are issued before any is used
+            uint32_t pp[4];
+            float xv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t t = (uint32_t)(e * 32 + lane);
+                pp[e] = (t < cnt) ? (uint32_t)list[t] : 0xFFFFFFFFu;
+                xv[e] = (t < cnt) ? x[gbase + pp[e]] : 0.f;
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (pp[e] != 0xFFFFFFFFu) round_one(pp[e], xv[e]);
+        } else {
+            for (uint32_t t = lane; t < cnt; t += 32) {
+                const uint32_t p = list[t];
+                round_one(p, x[gbase + p]);
+            }
         }
         __syncwarp();
-        kept = s_mask[warp][lane];
+    };
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int w = 0; w < kWarpsPerBlock; ++w) {
+        const uint32_t tile_cnt = warp_sum_u(__popc(word[w]));
+        if (cnt + tile_cnt > kGroupListCap) {
+            flush(cnt);
+            cnt = 0;
+        }
+        group_list_append(word[w], lane, w, list, cnt);
+        cnt += tile_cnt;
     }
-    if (active) ws.bitmask[tile * 32 + lane] = kept;
-    const uint32_t total = warp_sum_u(__popc(kept));
-    if (lane == 0) s_cnt[warp] = total;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t c = 0;
-        for (int w = 0; w < kWarpsPerBlock; ++w) c += s_cnt[w];
-        ws.block_count[blockIdx.x] = c;
+    flush(cnt);
+    uint32_t total = 0;
+#pragma unroll
+    for (int w = 0; w < kWarpsPerBlock; ++w) {
+        const uint32_t kept = mask[w * 32 + lane];
+        if (tile0 + w < tiles) ws.bitmask[(tile0 + w) * 32 + lane] = kept;
+        total += __popc(kept);
     }
+    total = warp_sum_u(total);
+    if (lane == 0) ws.block_count[grp] = total;
 }
 
-// grid: (ceil(tiles / warps per block), n workers)
+// grid: (ceil(tile groups / warps per block), n workers); one warp per group of 8 tiles
 __global__ void __launch_bounds__(kBlockThreads)
 sparse_emit_compact_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
                            const float scale, const int s,
@@ -372,40 +528,74 @@ sparse_emit_compact_kernel(const __grid_constant__ SparseBatch batch, const uint
                            char* __restrict__ ws_all, const uint64_t ws_stride) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
-    const uint64_t base = tile * kTile;
-    const bool active = base < d;
+    const uint64_t tiles = sparse_tiles(d);
+    const uint64_t groups = (tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const uint64_t grp = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    if (grp >= groups) return;
+    const uint64_t tile0 = grp * kWarpsPerBlock;
+    const uint64_t gbase = tile0 * kTile;
     const float* __restrict__ x = batch.x[blockIdx.y];
     const uint32_t worker = batch.worker[blockIdx.y];
     const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
     uint32_t* __restrict__ idx = batch.idx[blockIdx.y];
-    __shared__ uint32_t s_tile[kWarpsPerBlock];
-    __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
+    __shared__ uint16_t s_list[kWarpsPerBlock][kGroupListCap];
     uint16_t* list = s_list[warp];
-    const uint32_t word = active ? ws.bitmask[tile * 32 + lane] : 0u;
-    const uint32_t cnt = warp_list_positions(word, lane, list);
-    if (lane == 0) s_tile[warp] = cnt;
-    __syncthreads();
-    uint64_t k0 = (uint64_t)ws.block_count[blockIdx.x];
-    for (int w = 0; w < warp; ++w) k0 += s_tile[w];
-    if (cnt == 0) return;
+    uint32_t word[kWarpsPerBlock];
+#pragma unroll
+    for (int w = 0; w < kWarpsPerBlock; ++w)
+        word[w] = (tile0 + w < tiles) ? ws.bitmask[(tile0 + w) * 32 + lane] : 0u;
+    uint64_t k0 = (uint64_t)ws.block_count[grp];          // listed entries before this group
     const Scale sc = make_scale(*batch.norm[blockIdx.y], s);
     const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
     const int nb = code_value_bits(s);
-    for (uint32_t t = lane; t < cnt; t += 32) {
-        const uint64_t k = k0 + t;
-        if (k >= cap) break;
-        const uint64_t j = base + list[t];
-        const float xs = __fmul_rn(scale, x[j]);
+
+    auto emit_one = [&](uint64_t k, uint32_t p, float xv) {
+        const uint64_t j = gbase + p;
+        const float xs = __fmul_rn(scale, xv);
         const uint32_t bits = __float_as_uint(xs);
-        uint32_t r4[4];
-        stream_words4(j >> 2, worker, kDomainDnat, keys, r4);
-        const uint32_t r = (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1]
-                         : (j & 3) == 2 ? r4[2] : r4[3];
+        const uint32_t r = stream_word_at(j, worker, kDomainDnat, keys);
         const uint32_t level = sparse_level_code(bits, r, sc, pow2s);   // >= 1 after the filter
         idx[k] = (uint32_t)j;
         ws.tmp_codes[k] = (uint8_t)(((bits >> 31) << nb) | (level - 1u));
+    };
+    auto flush = [&](uint32_t cnt) {
+        __syncwarp();
+        if (cnt <= 4u * 32u) {
+            uint32_t pp[4];
+            float xv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t t = (uint32_t)(e * 32 + lane);
+                const bool on = t < cnt && k0 + t < cap;
+                pp[e] = on ? (uint32_t)list[t] : 0xFFFFFFFFu;
+                xv[e] = on ? x[gbase + pp[e]] : 0.f;
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (pp[e] != 0xFFFFFFFFu) emit_one(k0 + (uint32_t)(e * 32 + lane), pp[e], xv[e]);
+        } else {
+            for (uint32_t t = lane; t < cnt; t += 32) {
+                const uint64_t k = k0 + t;
+                if (k >= cap) break;
+                const uint32_t p = list[t];
+                emit_one(k, p, x[gbase + p]);
+            }
+        }
+        __syncwarp();
+        k0 += cnt;
+    };
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int w = 0; w < kWarpsPerBlock; ++w) {
+        const uint32_t tile_cnt = warp_sum_u(__popc(word[w]));
+        if (cnt + tile_cnt > kGroupListCap) {
+            flush(cnt);
+            cnt = 0;
+        }
+        group_list_append(word[w], lane, w, list, cnt);
+        cnt += tile_cnt;
     }
+    flush(cnt);
 }
 
 // one warp per 32 listed entries; grid: (ceil(groups / warps per block), n workers)
@@ -460,15 +650,15 @@ namespace natcomp {
 void sparse_compact_finish(const SparseBatch& batch, uint64_t d, float scale, int p, int s,
                            const PhiloxKeys& keys, uint64_t cap, char* ws, uint64_t ws_stride,
                            int n, cudaStream_t stream) {
-    const uint64_t tiles = sparse_tiles(d);
-    const dim3 grid((unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
+    const uint64_t tile_groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const dim3 ggrid((unsigned)((tile_groups + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
     launch_scan(batch, d, p, ws, ws_stride, n, stream);          // norm (and the kept count)
-    sparse_round_filter_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, ws,
-                                                                   ws_stride);
+    sparse_round_filter_kernel<<<ggrid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, ws,
+                                                                    ws_stride);
     // second scan: offsets and count of the surviving entries (the norm partials are unchanged)
     launch_scan(batch, d, p, ws, ws_stride, n, stream);
-    sparse_emit_compact_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap,
-                                                                   ws, ws_stride);
+    sparse_emit_compact_kernel<<<ggrid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap,
+                                                                    ws, ws_stride);
     const uint64_t groups = (cap + 31) / 32;
     const dim3 pgrid((unsigned)((groups + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
     sparse_pack_planes_kernel<<<pgrid, kBlockThreads, 0, stream>>>(batch, d, cap, s, ws,
@@ -515,20 +705,8 @@ nc_status nd_sparse_compact_compress_batch(const float* const* xs, size_t d,
     const uint64_t ws_stride = sparse_ws_bytes(d, cap);
     if (workspace_bytes < (size_t)n * ws_stride) return NC_ERR_WORKSPACE;
     char* ws = reinterpret_cast<char*>(workspace);
-    const uint64_t tiles = sparse_tiles(d);
-    const dim3 grid((unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
     const PhiloxKeys keys = make_philox_keys(seed);
-    const bool keep_none = keep_threshold == 0;
-    const uint32_t neg_thr = (uint32_t)(0ull - keep_threshold);
-    if (p == 1)
-        sparse_select_kernel<1><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
-                                                                    scale, keys, ws, ws_stride);
-    else if (p == 2)
-        sparse_select_kernel<2><<<grid, kBlockThreads, 0, stream>>>(batch, d, neg_thr, keep_none,
-                                                                    scale, keys, ws, ws_stride);
-    else
-        sparse_select_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
-            batch, d, neg_thr, keep_none, scale, keys, ws, ws_stride);
+    launch_select(batch, d, keep_threshold, scale, p, keys, ws, ws_stride, n, stream);
     sparse_compact_finish(batch, d, scale, p, s, keys, cap, ws, ws_stride, n, stream);
     return launch_status();
 }
