@@ -207,48 +207,81 @@ sparse_scan_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
     }
 }
 
-// grid: ceil(tiles / warps per block)
+// grid: (ceil(tile groups / warps per block), n workers); one warp per group of 8 tiles
 __global__ void __launch_bounds__(kBlockThreads)
 sparse_emit_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d, const float scale,
                    const int s, const __grid_constant__ PhiloxKeys keys, const uint64_t cap,
                    char* __restrict__ ws_all, const uint64_t ws_stride) {
     const int lane = threadIdx.x & 31;
-    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    const uint64_t base = tile * kTile;
-    const bool active = base < d;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t tiles = sparse_tiles(d);
+    const uint64_t groups = (tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const uint64_t grp = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    if (grp >= groups) return;
+    const uint64_t tile0 = grp * kWarpsPerBlock;
+    const uint64_t gbase = tile0 * kTile;
     const float* __restrict__ x = batch.x[blockIdx.y];
     const uint32_t worker = batch.worker[blockIdx.y];
     const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
-    const uint32_t* __restrict__ bitmask = ws.bitmask;
-    const float* __restrict__ norm = batch.norm[blockIdx.y];
     uint32_t* __restrict__ idx = batch.idx[blockIdx.y];
     uint8_t* __restrict__ tmp_codes = ws.tmp_codes;
-    __shared__ uint32_t s_tile[kWarpsPerBlock];
-    __shared__ uint16_t s_list[kWarpsPerBlock][kTile];
-    uint16_t* list = s_list[threadIdx.x >> 5];
-    const uint32_t word = active ? bitmask[tile * 32 + lane] : 0u;
-    const uint32_t cnt = warp_list_positions(word, lane, list);
-    if (lane == 0) s_tile[threadIdx.x >> 5] = cnt;        // kept entries of this tile
-    __syncthreads();
-    uint64_t k0 = (uint64_t)ws.block_count[blockIdx.x];
-    for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) k0 += s_tile[w];
-    if (cnt == 0) return;
-    const Scale sc = make_scale(*norm, s);
+    __shared__ uint16_t s_list[kWarpsPerBlock][kGroupListCap];
+    uint16_t* list = s_list[warp];
+    uint32_t word[kWarpsPerBlock];
+#pragma unroll
+    for (int w = 0; w < kWarpsPerBlock; ++w)
+        word[w] = (tile0 + w < tiles) ? ws.bitmask[(tile0 + w) * 32 + lane] : 0u;
+    uint64_t k0 = (uint64_t)ws.block_count[grp];          // kept entries before this group
+    const Scale sc = make_scale(*batch.norm[blockIdx.y], s);
     const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
-    for (uint32_t t = lane; t < cnt; t += 32) {      // the t-th kept entry of the tile
-        const uint64_t k = k0 + t;
-        if (k >= cap) break;
-        const uint64_t j = base + list[t];
-        const float xs = __fmul_rn(scale, x[j]);
+
+    auto emit_one = [&](uint64_t k, uint32_t p, float xv) {
+        const uint64_t j = gbase + p;
+        const float xs = __fmul_rn(scale, xv);
         const uint32_t bits = __float_as_uint(xs);
-        uint32_t r4[4];
-        stream_words4(j >> 2, worker, kDomainDnat, keys, r4);
-        const uint32_t r = (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1]
-                         : (j & 3) == 2 ? r4[2] : r4[3];
+        const uint32_t r = stream_word_at(j, worker, kDomainDnat, keys);
         const uint32_t code = sparse_level_code(bits, r, sc, pow2s);
         idx[k] = (uint32_t)j;
         tmp_codes[k] = (uint8_t)(((bits >> 31) << 3) | code);
+    };
+    auto flush = [&](uint32_t cnt) {
+        __syncwarp();
+        if (cnt <= 4u * 32u) {
+            uint32_t pp[4];
+            float xv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t t = (uint32_t)(e * 32 + lane);
+                const bool on = t < cnt && k0 + t < cap;
+                pp[e] = on ? (uint32_t)list[t] : 0xFFFFFFFFu;
+                xv[e] = on ? x[gbase + pp[e]] : 0.f;
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (pp[e] != 0xFFFFFFFFu) emit_one(k0 + (uint32_t)(e * 32 + lane), pp[e], xv[e]);
+        } else {
+            for (uint32_t t = lane; t < cnt; t += 32) {
+                const uint64_t k = k0 + t;
+                if (k >= cap) break;
+                const uint32_t p = list[t];
+                emit_one(k, p, x[gbase + p]);
+            }
+        }
+        __syncwarp();
+        k0 += cnt;
+    };
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int w = 0; w < kWarpsPerBlock; ++w) {
+        const uint32_t tile_cnt = warp_sum_u(__popc(word[w]));
+        if (cnt + tile_cnt > kGroupListCap) {
+            flush(cnt);
+            cnt = 0;
+        }
+        group_list_append(word[w], lane, w, list, cnt);
+        cnt += tile_cnt;
     }
+    flush(cnt);
 }
 
 // thread t -> output byte t; zero padding up to the next multiple of 16 bytes
@@ -377,13 +410,13 @@ nc_status nd_sparse_compress_batch(const float* const* xs, size_t d, uint64_t ke
     const uint64_t ws_stride = sparse_ws_bytes(d, cap);
     if (workspace_bytes < (size_t)n * ws_stride) return NC_ERR_WORKSPACE;
     char* ws = reinterpret_cast<char*>(workspace);
-    const uint64_t tiles = sparse_tiles(d);
-    const dim3 grid((unsigned)((tiles + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
     const PhiloxKeys keys = make_philox_keys(seed);
     launch_select(batch, d, keep_threshold, scale, p, keys, ws, ws_stride, n, stream);
     launch_scan(batch, d, p, ws, ws_stride, n, stream);
-    sparse_emit_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap, ws,
-                                                           ws_stride);
+    const uint64_t tile_groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const dim3 ggrid((unsigned)((tile_groups + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
+    sparse_emit_kernel<<<ggrid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap, ws,
+                                                            ws_stride);
     const uint64_t pack_threads = round_up16((cap + 1) / 2);
     const dim3 pgrid((unsigned)((pack_threads + kBlockThreads - 1) / kBlockThreads), (unsigned)n);
     sparse_pack_kernel<<<pgrid, kBlockThreads, 0, stream>>>(batch, d, cap, ws, ws_stride);
