@@ -316,13 +316,21 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
                 stream_words4_tile(q + 1, pt, keys, r4);
                 rnd[4] = r4[0]; rnd[5] = r4[1]; rnd[6] = r4[2]; rnd[7] = r4[3];
             }
+            // The codes are packed as nib = nib * 16 + e with e = code + 127 (the biased exponent
+            // after the carry, clamped), and 127 * 0x11111111 is taken off the word at the end:
+            // the arithmetic is linear mod 2^32, so the result is the packed codes exactly, the
+            // per-entry subtraction is gone and the packing is multiply-add work, which runs
+            // beside the integer pipe that bounds this kernel.
             uint32_t nib = 0;
 #pragma unroll
             for (int c = 7; c >= 0; --c) {
-                nib = (nib << 4) | level_code_scaled(u[it].v[c], rnd[c], rinv_s, sc.smax);
+                const float z = __fmul_rn(fabsf(__uint_as_float(u[it].v[c])), rinv_s);
+                const float w = fmaxf(z, __fmaf_rz(z, 0.5f, 1.0f));       // see level_code_scaled
+                const uint32_t e = (__float_as_uint(w) + (~rnd[c] & 0x7FFFFFu)) >> 23;
+                nib = nib * 16u + min(e, sc.smax + 127u);
                 sbytes = __funnelshift_l(u[it].v[c], sbytes, 1);
             }
-            st_stream_u32(lv + it * 32 + lane, nib);
+            st_stream_u32(lv + it * 32 + lane, nib - 127u * 0x11111111u);
         }
         // lane 4g+i holds byte i of sign word (it, g) = word it*8 + g of the tile
         const uint32_t word = transpose_bytes_4x4(sbytes, lane);
