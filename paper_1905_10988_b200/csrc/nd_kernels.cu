@@ -299,8 +299,12 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
     // level code 0.  If rinv * 2^s overflows (norm below 2^(s-126)) the general path is used.
     const BucketScale sc0 = bucket_scale(norms[b], s);
     const float rinv_s = __fmul_rn(sc0.rinv, pow2s);
-    if (full && __ldg(off + b + 1) >= base + kTile && rinv_s <= 3.40282347e38f) {
-        const BucketScale sc = sc0;
+    // No clamp of the code in this path: the norm was computed from the same entries, so
+    // |x| <= norm, |x| * rinv <= 1 + 2^-24 rounds to at most 1 (a tie goes to the even mantissa 0)
+    // and z <= 2^s has a zero mantissa at the top exponent, which the random increment cannot carry
+    // out of.  A degenerate bucket (norm 0, subnormal or not finite; all codes 0) takes the
+    // general path, which clamps.
+    if (full && __ldg(off + b + 1) >= base + kTile && rinv_s <= 3.40282347e38f && sc0.smax != 0u) {
         uint32_t* lv = reinterpret_cast<uint32_t*>(level + (base >> 1));
         const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainDnat, keys);
         const uint32_t q_lo = (uint32_t)(base >> 2) + (uint32_t)(lane * 2);
@@ -317,7 +321,7 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
                 rnd[4] = r4[0]; rnd[5] = r4[1]; rnd[6] = r4[2]; rnd[7] = r4[3];
             }
             // The codes are packed as nib = nib * 16 + e with e = code + 127 (the biased exponent
-            // after the carry, clamped), and 127 * 0x11111111 is taken off the word at the end:
+            // after the carry), and 127 * 0x11111111 is taken off the word at the end:
             // the arithmetic is linear mod 2^32, so the result is the packed codes exactly, the
             // per-entry subtraction is gone and the packing is multiply-add work, which runs
             // beside the integer pipe that bounds this kernel.
@@ -327,7 +331,7 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
                 const float z = __fmul_rn(fabsf(__uint_as_float(u[it].v[c])), rinv_s);
                 const float w = fmaxf(z, __fmaf_rz(z, 0.5f, 1.0f));       // see level_code_scaled
                 const uint32_t e = (__float_as_uint(w) + (~rnd[c] & 0x7FFFFFu)) >> 23;
-                nib = nib * 16u + min(e, sc.smax + 127u);
+                nib = nib * 16u + e;
                 sbytes = __funnelshift_l(u[it].v[c], sbytes, 1);
             }
             st_stream_u32(lv + it * 32 + lane, nib - 127u * 0x11111111u);
