@@ -272,24 +272,50 @@ select_mark_kernel(const Src src, const uint64_t d, uint32_t* __restrict__ less_
     const uint32_t T = ws.state->prefix >> sh;
     __shared__ uint32_t s_eq[kWarpsPerBlock];
     __shared__ uint32_t s_base;
+    // "fixed digits >= T" is "key >= T << sh", "fixed digits > T" is "key >= (T + 1) << sh"; both
+    // comparisons are the carry of key + (2^32 - bound), shifted straight into a bit register
+    // (two integer instructions each).  T << sh = 0 never carries and means "always"; a second
+    // bound of 2^32 gives the addend 0, which never carries, as it should.
+    const uint32_t lo_bound = T << sh;
+    const uint32_t neg_lo = 0u - lo_bound;
+    const uint32_t neg_hi = (uint32_t)(0ull - (((unsigned long long)T + 1ull) << sh));
     uint32_t less = 0, equal = 0;
     typename Src::Tile t;
     if (active) {
         t = src.tile(base, lane);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            uint32_t key[4];
-            src.load(t, base, lane, k, d, key);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t hi = key[c] >> sh;
-                less |= (hi < T ? 1u : 0u) << (4 * k + c);
-                equal |= (hi == T ? 1u : 0u) << (4 * k + c);
-            }
-        }
         const uint32_t valid = valid_nibbles<Src>(base, lane, d);
-        less &= valid;
-        equal &= valid;
+        if (Src::kCanonical) {
+            // computed keys: the pass is bound by instruction issue, the carry form is shorter
+            uint32_t ge_lo = 0, ge_hi = 0;
+#pragma unroll
+            for (int k = 7; k >= 0; --k) {
+                uint32_t key[4];
+                src.load(t, base, lane, k, d, key);
+#pragma unroll
+                for (int c = 3; c >= 0; --c) {
+                    shift_in_drop_bit(ge_lo, key[c], neg_lo);
+                    shift_in_drop_bit(ge_hi, key[c], neg_hi);
+                }
+            }
+            if (lo_bound == 0u) ge_lo = 0xFFFFFFFFu;
+            less = ~ge_lo & valid;
+            equal = ge_lo & ~ge_hi & valid;
+        } else {
+            // loaded keys: the pass is bound by memory; plain comparisons, loads in ascending order
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                uint32_t key[4];
+                src.load(t, base, lane, k, d, key);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t hi = key[c] >> sh;
+                    less |= (hi < T ? 1u : 0u) << (4 * k + c);
+                    equal |= (hi == T ? 1u : 0u) << (4 * k + c);
+                }
+            }
+            less &= valid;
+            equal &= valid;
+        }
     }
     const uint32_t lw = mask_word<Src>(less, lane);
     const uint32_t ew = (mode == 0u) ? mask_word<Src>(equal, lane) : 0u;
