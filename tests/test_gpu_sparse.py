@@ -195,3 +195,64 @@ def test_sparse_bench_launch_configuration_sampled():
         assert np.array_equal(codes[w][:(cnt + 1) // 2].cpu().numpy(), c_ref)
         oracle.sparse_decode_accumulate(i_ref, c_ref, count_ref, n_ref, s, ref)
     assert np.array_equal(acc.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+
+
+def test_sparse_near_the_largest_d_properties():
+    # d = 2^32 - 5 (the sparse calls store 32-bit indices): 17 GB of input, keep 1 %.  The oracle
+    # cannot walk 4.3 G coordinates in a test, so the output is checked through what is unique and
+    # local: the count against its binomial law, ascending in-range indices, the norm against the
+    # maximum over the listed entries, and in sampled windows the kept set ("stream word < T") and
+    # the codes (given the norm).
+    d = (1 << 32) - 5
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * (1 << 30):
+        pytest.skip("needs ~25 GB of free device memory")
+    s, seed, worker = 4, 11, 6
+    thr, scale = workloads.KEEP_1PCT_THRESHOLD, workloads.KEEP_1PCT_SCALE
+    cap = int(d * 0.0102)
+    x = torch.empty(d, dtype=torch.float32, device="cuda")
+    g = torch.Generator(device="cuda")
+    g.manual_seed(321)
+    chunk = 1 << 28
+    for a in range(0, d, chunk):
+        x[a:min(d, a + chunk)].normal_(0.0, 1.0, generator=g)
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    idx = torch.empty(cap, dtype=torch.int32, device="cuda")
+    codes = torch.empty((cap + 1) // 2 + 16, **u8)
+    count = torch.zeros(1, dtype=torch.int32, device="cuda")
+    norm = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ws_bytes = nc.nd_sparse_workspace_bytes(d, cap)
+    ws = torch.empty(ws_bytes, **u8)
+    nc.nd_sparse_compress(x, d, thr, scale, nc.P_INF, s, seed, worker, idx, codes, count, norm,
+                          cap, ws, ws_bytes)
+    torch.cuda.synchronize()
+    cnt = int(count.cpu().numpy().view(np.uint32)[0])
+    prob = thr / 2.0 ** 32
+    assert abs(cnt - d * prob) < 6 * (d * prob * (1 - prob)) ** 0.5 and cnt <= cap
+    ih = idx[:cnt].cpu().numpy().view(np.uint32).astype(np.int64)
+    assert np.all(np.diff(ih) > 0) and ih[0] >= 0 and ih[-1] < d
+    nrm = float(norm.cpu()[0])
+    kept_max = 0.0
+    for a in range(0, cnt, 1 << 24):
+        sel = idx[a:min(cnt, a + (1 << 24))].to(torch.int64) & 0xFFFFFFFF
+        kept_max = max(kept_max, float((x[sel] * scale).abs().max()))
+    assert nrm == kept_max
+    ch = codes[:(cnt + 1) // 2].cpu().numpy()
+    W = 1 << 16
+    rinv = np.float32(1.0) / np.float32(nrm)
+    for o in (0, (1 << 31) - W // 2, (1 << 32) - (1 << 20), ((d - W) // 4) * 4):
+        hi = min(d, o + W)
+        words = oracle.stream_words(seed, worker, 2, o, hi - o).astype(np.uint64)
+        kept = o + np.nonzero(words < thr)[0]
+        a, b = np.searchsorted(ih, o), np.searchsorted(ih, hi)
+        assert np.array_equal(ih[a:b], kept)
+        xs = (x[o:hi].cpu().numpy()[kept - o] * np.float32(scale)).astype(np.float32)
+        y = (np.abs(xs) * rinv).astype(np.float32)
+        r23 = oracle.stream_words(seed, worker, 1, o, hi - o)[kept - o] & 0x7FFFFF
+        lev = oracle.nd_level_codes(y.astype(np.float64), r23, s)
+        k = np.arange(a, b)
+        got = (ch[k // 2] >> (4 * (k % 2))) & 0xF
+        assert np.array_equal(got & 7, lev)
+        assert np.array_equal(got >> 3, (xs.view(np.uint32) >> 31).astype(np.uint8))
+    del x, idx, codes, ws
+    torch.cuda.empty_cache()
