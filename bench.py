@@ -207,6 +207,28 @@ class HotPath:
             nc.nc_sum_fp32(self.x, n, d, self.out_sum)
         mark("sum_fp32")
 
+    STREAM_GROUPS = (("nc_compress", "nc_aggregate"), ("nd_compress", "nd_aggregate"),
+                     ("sparse_compress", "sparse_accumulate"), ("sum_fp32",))
+
+    def step_on_streams(self, streams):
+        """The same step with its four independent call chains on four streams (fork from the
+        current stream, join back into it): the HBM-bound and the integer-bound kernels of
+        different chains overlap at their tails."""
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        keep = self.only
+        for stream, chain in zip(streams, self.STREAM_GROUPS):
+            stream.wait_event(fork)
+            with torch.cuda.stream(stream):
+                for g in chain:
+                    self.only = g
+                    self.step()
+            done = torch.cuda.Event()
+            done.record(stream)
+            main.wait_event(done)
+        self.only = keep
+
     def algorithmic_bytes(self):
         """Compulsory HBM bytes per call group (per step)."""
         n, d = self.n, self.d
@@ -415,6 +437,24 @@ def main():
     gv = roofline["generator_view"]
     gv["frac"] = round(gv["achieved_Gelem_per_s"] / gv["multiplier_pipe_peak_Gelem_per_s"], 4)
 
+    # the same step with its independent call chains on four streams (reported beside `value`,
+    # which stays the single-stream figure the per-group times belong to)
+    streams = [torch.cuda.Stream() for _ in HotPath.STREAM_GROUPS]
+    k_conc = min(args.steps, 100)
+    for _ in range(3):
+        hp.step_on_streams(streams)
+    torch.cuda.synchronize()
+    c0 = torch.cuda.Event(enable_timing=True)
+    c1 = torch.cuda.Event(enable_timing=True)
+    c0.record()
+    for _ in range(k_conc):
+        hp.step_on_streams(streams)
+    c1.record()
+    torch.cuda.synchronize()
+    conc_ms = timing.max_over_ranks(c0.elapsed_time(c1) / k_conc, dist, device)
+    concurrent = {"ms_per_step": conc_ms, "streams": len(streams), "steps": k_conc,
+                  "value": world * units_per_step / (conc_ms * 1e-3) / 1e9, "unit": UNIT}
+
     # end to end: host buffers -> device -> whole path -> aggregates back on the host
     e2e = None
     if args.e2e_steps > 0:
@@ -443,6 +483,7 @@ def main():
                        "l2": "inputs are 818 MB per replica, larger than the 126 MB L2; no flush",
                        "multi_gpu": "replicas only"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": hp.launches_per_step * args.steps,
+            "concurrent_streams": concurrent,
             "roofline": roofline, "cpu_baseline": cpu, "kernels": kernels,
         }
         print(json.dumps(line))
