@@ -269,7 +269,7 @@ __device__ __forceinline__ uint32_t level_code_scaled(uint32_t bits, uint32_t rn
 }
 
 // grid: ceil(tiles / warps per block)
-__global__ void __launch_bounds__(kBlockThreads, 5)
+__global__ void __launch_bounds__(kBlockThreads, 4)
 nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d,
                      const uint64_t* __restrict__ off, const int B, const int s,
                      const __grid_constant__ PhiloxKeys keys,
