@@ -39,6 +39,20 @@ inline bool aligned4(const void* p) { return ((uintptr_t)p & 3u) == 0; }
 
 __host__ __device__ inline size_t round_up16(size_t v) { return (v + 15) & ~(size_t)15; }
 
+// SM count of the current device (looked up once per device)
+inline int device_sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1)
+            v = 148;
+        cached[dev] = v;
+    }
+    return cached[dev];
+}
+
 inline nc_status launch_status() {
     return cudaPeekAtLastError() == cudaSuccess ? NC_OK : NC_ERR_CUDA;
 }

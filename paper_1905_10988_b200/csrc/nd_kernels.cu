@@ -128,27 +128,15 @@ struct NormAcc {
     }
 };
 
-// grid: (ceil(tiles / warps per block), n workers); worker w uses slots + w * slot_stride
+// norm partial(s) of one tile; `u` holds the tile's entries if it is full
 template <int P>
-__global__ void __launch_bounds__(kBlockThreads)
-nd_norm_partials_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d,
-                        const uint64_t* __restrict__ off, const int B,
-                        uint64_t* __restrict__ slots_all, const uint64_t slot_stride,
-                        uint32_t* __restrict__ tile_bucket) {
-    const int lane = threadIdx.x & 31;
-    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+__device__ __forceinline__ void norm_tile(const float* __restrict__ x, uint64_t* __restrict__ slots,
+                                          const uint64_t tile, const uint64_t d,
+                                          const uint64_t* __restrict__ off, const int B,
+                                          uint32_t* __restrict__ tile_bucket, const V8 (&u)[4],
+                                          const bool full, const int lane) {
     const uint64_t base = tile * kTile;
-    if (base >= d) return;
-    const float* __restrict__ x = batch.x[blockIdx.y];
-    uint64_t* __restrict__ slots = slots_all + (uint64_t)blockIdx.y * slot_stride;
-    const uint64_t end = (base + kTile <= d) ? base + kTile : d;
-    const bool full = (base + kTile <= d);
-
-    V8 u[4];
-    if (full) {
-#pragma unroll
-        for (int it = 0; it < 4; ++it) u[it] = ld_stream_v8(x + base + it * 256 + lane * 8);
-    }
+    const uint64_t end = full ? base + kTile : d;
     int b = find_bucket(off, B, base);
     if (lane == 0) tile_bucket[tile] = (uint32_t)b;
 
@@ -182,6 +170,45 @@ nd_norm_partials_kernel(const __grid_constant__ DitherBatch batch, const uint64_
             ++b;
             while (__ldg(off + b + 1) <= pos) ++b;   // skip empty buckets
         }
+    }
+}
+
+// Persistent warps: a warp takes the tiles w, w + W, w + 2W, ... (W = warps in the grid row) and
+// loads the next tile before it reduces the current one, so every warp always has 4 KB in flight.
+// grid: (blocks resident on the device, n workers); worker w uses slots + w * slot_stride
+template <int P>
+__global__ void __launch_bounds__(kBlockThreads, 2)
+nd_norm_partials_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d,
+                        const uint64_t* __restrict__ off, const int B,
+                        uint64_t* __restrict__ slots_all, const uint64_t slot_stride,
+                        uint32_t* __restrict__ tile_bucket) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t tiles = (d + kTile - 1) / kTile;
+    const uint64_t stride = (uint64_t)gridDim.x * kWarpsPerBlock;
+    uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    if (tile >= tiles) return;
+    const float* __restrict__ x = batch.x[blockIdx.y];
+    uint64_t* __restrict__ slots = slots_all + (uint64_t)blockIdx.y * slot_stride;
+    V8 u[4], nx[4];
+    bool full = (tile + 1) * kTile <= d;
+    if (full) {
+#pragma unroll
+        for (int it = 0; it < 4; ++it) u[it] = ld_stream_v8(x + tile * kTile + it * 256 + lane * 8);
+    }
+    for (;;) {
+        const uint64_t next = tile + stride;
+        const bool next_full = next < tiles && (next + 1) * kTile <= d;
+        if (next_full) {
+#pragma unroll
+            for (int it = 0; it < 4; ++it)
+                nx[it] = ld_stream_v8(x + next * kTile + it * 256 + lane * 8);
+        }
+        norm_tile<P>(x, slots, tile, d, off, B, tile_bucket, u, full, lane);
+        if (next >= tiles) break;
+        tile = next;
+        full = next_full;
+#pragma unroll
+        for (int it = 0; it < 4; ++it) u[it] = nx[it];
     }
 }
 
@@ -563,19 +590,21 @@ nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bu
     uint64_t* slots = reinterpret_cast<uint64_t*>(workspace);
     uint32_t* tile_bucket = reinterpret_cast<uint32_t*>(slots + (uint64_t)n * slot_stride);
     const dim3 grid(nd_tile_blocks(d), (unsigned)n);
+    const unsigned resident = 2u * (unsigned)device_sm_count();
+    const dim3 ngrid(nd_tile_blocks(d) < resident ? nd_tile_blocks(d) : resident, (unsigned)n);
     const dim3 fgrid((unsigned)B, (unsigned)n);
     if (p == 1) {
-        nd_norm_partials_kernel<1><<<grid, kBlockThreads, 0, stream>>>(
+        nd_norm_partials_kernel<1><<<ngrid, kBlockThreads, 0, stream>>>(
             batch, d, bucket_off, B, slots, slot_stride, tile_bucket);
         nd_norm_finalize_kernel<1><<<fgrid, kBlockThreads, 0, stream>>>(batch, bucket_off, B,
                                                                         slots, slot_stride);
     } else if (p == 2) {
-        nd_norm_partials_kernel<2><<<grid, kBlockThreads, 0, stream>>>(
+        nd_norm_partials_kernel<2><<<ngrid, kBlockThreads, 0, stream>>>(
             batch, d, bucket_off, B, slots, slot_stride, tile_bucket);
         nd_norm_finalize_kernel<2><<<fgrid, kBlockThreads, 0, stream>>>(batch, bucket_off, B,
                                                                         slots, slot_stride);
     } else {
-        nd_norm_partials_kernel<NC_P_INF><<<grid, kBlockThreads, 0, stream>>>(
+        nd_norm_partials_kernel<NC_P_INF><<<ngrid, kBlockThreads, 0, stream>>>(
             batch, d, bucket_off, B, slots, slot_stride, tile_bucket);
         nd_norm_finalize_kernel<NC_P_INF><<<fgrid, kBlockThreads, 0, stream>>>(
             batch, bucket_off, B, slots, slot_stride);
