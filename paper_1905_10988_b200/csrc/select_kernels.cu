@@ -47,6 +47,7 @@ struct SelectWorkspace {
     uint32_t* eqmask;       // tiles * 32 words
     uint32_t* eq_block;     // one per block of 8 tiles
     uint32_t* hist;         // kSelPasses * kSelBins
+    uint32_t* hist2;        // 3 * kSelBins: second digit of the keys in the three guessed first bins
     SelectState* state;
     uint32_t* count;        // listed entries (TopK)
     uint32_t* cand_count;
@@ -55,7 +56,7 @@ struct SelectWorkspace {
 
 inline size_t select_extra_bytes(uint64_t d) {
     const uint64_t t = sparse_tiles(d);
-    return round_up16(t * 128) + round_up16(t * 4) + (size_t)kSelPasses * kSelBins * 4 + 64 +
+    return round_up16(t * 128) + round_up16(t * 4) + (size_t)(kSelPasses + 3) * kSelBins * 4 + 64 +
            (size_t)kCandCap * 8;
 }
 
@@ -65,6 +66,7 @@ __host__ __device__ inline SelectWorkspace select_ws_carve(char* p, uint64_t d) 
     w.eqmask = reinterpret_cast<uint32_t*>(p);   p += round_up16(t * 128);
     w.eq_block = reinterpret_cast<uint32_t*>(p); p += round_up16(t * 4);
     w.hist = reinterpret_cast<uint32_t*>(p);     p += (size_t)kSelPasses * kSelBins * 4;
+    w.hist2 = reinterpret_cast<uint32_t*>(p);    p += (size_t)3 * kSelBins * 4;
     w.state = reinterpret_cast<SelectState*>(p);
     w.count = reinterpret_cast<uint32_t*>(p + 32);
     w.cand_count = reinterpret_cast<uint32_t*>(p + 36);
@@ -155,7 +157,7 @@ __device__ __forceinline__ uint32_t mask_word(uint32_t nib, int lane) {
 }
 
 __global__ void select_init_kernel(SelectWorkspace ws, const uint64_t q) {
-    for (int i = threadIdx.x; i < kSelPasses * kSelBins; i += blockDim.x) ws.hist[i] = 0u;
+    for (int i = threadIdx.x; i < (kSelPasses + 3) * kSelBins; i += blockDim.x) ws.hist[i] = 0u;
     if (threadIdx.x == 0) {
         ws.state->prefix = 0u;
         ws.state->mode = 0u;
@@ -166,19 +168,27 @@ __global__ void select_init_kernel(SelectWorkspace ws, const uint64_t q) {
 }
 
 // persistent blocks: block b takes the groups of 8 tiles b, b + gridDim.x, ...
-template <class Src, int PASS>
+// With a guess g of the first digit of the q-th key (stream keys are uniform, so g = q * 2048 / d
+// is right to within one bin), pass 0 also counts the second digit of the keys whose first digit
+// is g - 1, g or g + 1: the choose kernel can then fix 22 key bits at once and the candidate list
+// shrinks from d / 2^11 to d / 2^22 keys.  A wrong guess only loses that shortcut.
+template <class Src, int PASS, bool kGuess = false>
 __global__ void __launch_bounds__(kBlockThreads)
-select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws) {
+select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws, const int guess = 0) {
     constexpr int bins = sel_bins(PASS);
     constexpr int shift = sel_shift(PASS);
     constexpr uint32_t fixed = sel_fixed(PASS);
     // candidates already collected: the remaining digits are found on the candidate list
     if (PASS > 0 && ws.state->mode != 0u) return;
     __shared__ uint32_t s_hist[bins];
+    __shared__ uint32_t s_hist2[kGuess ? 3 * kSelBins : 1];
     for (int i = threadIdx.x; i < bins; i += kBlockThreads) s_hist[i] = 0u;
+    if (kGuess)
+        for (int i = threadIdx.x; i < 3 * kSelBins; i += kBlockThreads) s_hist2[i] = 0u;
     __syncthreads();
     const int lane = threadIdx.x & 31;
     const uint32_t prefix = PASS == 0 ? 0u : ws.state->prefix;
+    const uint32_t guess_lo = kGuess ? (uint32_t)(guess - 1) << 21 : 0u;    // first key of bin g - 1
     const uint64_t groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
     for (uint64_t g = blockIdx.x; g < groups; g += gridDim.x) {
         const uint64_t base = (g * kWarpsPerBlock + (threadIdx.x >> 5)) * kTile;
@@ -195,6 +205,8 @@ select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws) {
                 for (int c = 0; c < 4; ++c) {
                     if ((key[c] & fixed) == prefix)
                         atomicAdd(&s_hist[(key[c] >> shift) & (uint32_t)(bins - 1)], 1u);
+                    if (kGuess && key[c] - guess_lo < (3u << 21))
+                        atomicAdd(&s_hist2[(key[c] - guess_lo) >> 10], 1u);
                 }
             }
             continue;
@@ -206,8 +218,11 @@ select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws) {
             src.load(t, base, lane, k, d, key);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                if ((key[c] & fixed) == prefix && ((valid >> (4 * k + c)) & 1u))
+                if ((key[c] & fixed) == prefix && ((valid >> (4 * k + c)) & 1u)) {
                     atomicAdd(&s_hist[(key[c] >> shift) & (uint32_t)(bins - 1)], 1u);
+                    if (kGuess && key[c] - guess_lo < (3u << 21))
+                        atomicAdd(&s_hist2[(key[c] - guess_lo) >> 10], 1u);
+                }
             }
         }
     }
@@ -217,6 +232,12 @@ select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws) {
         const uint32_t v = s_hist[i];
         if (v) atomicAdd(&hist[i], v);
     }
+    if (kGuess) {
+        for (int i = threadIdx.x; i < 3 * kSelBins; i += kBlockThreads) {
+            const uint32_t v = s_hist2[i];
+            if (v) atomicAdd(&ws.hist2[i], v);
+        }
+    }
 }
 
 // one block of 1024 threads, two bins each: the bin in which the cumulative count reaches
@@ -224,14 +245,17 @@ select_hist_kernel(const Src src, const uint64_t d, const SelectWorkspace ws) {
 // and 1), the remaining passes over all d keys are skipped: the mark kernel collects those keys
 // and the candidate kernel finishes the selection on the list.
 template <int PASS>
-__global__ void __launch_bounds__(kScanThreads) select_choose_kernel(const SelectWorkspace ws) {
+__global__ void __launch_bounds__(kScanThreads)
+select_choose_kernel(const SelectWorkspace ws, const int guess = -1) {
     constexpr int bins = sel_bins(PASS);
     if (PASS > 0 && ws.state->mode != 0u) return;
     const uint32_t* __restrict__ hist = ws.hist + PASS * kSelBins;
     __shared__ uint64_t s_sum[kScanThreads];
+    __shared__ int s_pick;
     const int t = threadIdx.x;
-    const uint32_t h0 = (2 * t < bins) ? hist[2 * t] : 0u;
-    const uint32_t h1 = (2 * t + 1 < bins) ? hist[2 * t + 1] : 0u;
+    uint32_t h0 = (2 * t < bins) ? hist[2 * t] : 0u;
+    uint32_t h1 = (2 * t + 1 < bins) ? hist[2 * t + 1] : 0u;
+    if (t == 0) s_pick = -1;
     s_sum[t] = (uint64_t)h0 + h1;
     __syncthreads();
     for (int o = 1; o < kScanThreads; o <<= 1) {
@@ -240,8 +264,8 @@ __global__ void __launch_bounds__(kScanThreads) select_choose_kernel(const Selec
         s_sum[t] += v;
         __syncthreads();
     }
-    const uint64_t remaining = ws.state->remaining;
-    const uint64_t before = s_sum[t] - h0 - h1;         // keys in lower bins
+    uint64_t remaining = ws.state->remaining;
+    uint64_t before = s_sum[t] - h0 - h1;               // keys in lower bins
     __syncthreads();                                    // everyone has read the state
     int pick = -1;
     if (remaining > before && remaining <= before + h0) pick = 0;
@@ -250,6 +274,34 @@ __global__ void __launch_bounds__(kScanThreads) select_choose_kernel(const Selec
         ws.state->prefix |= (uint32_t)(2 * t + pick) << sel_shift(PASS);
         ws.state->remaining = remaining - before - (pick ? h0 : 0u);
         if (PASS < 2 && (pick ? h1 : h0) <= kCandCap) ws.state->mode = (uint32_t)(PASS + 1);
+        s_pick = 2 * t + pick;
+    }
+    if (PASS != 0 || guess < 0) return;
+    // second digit from the guessed rows, if the first digit is one of the three guessed bins
+    __syncthreads();
+    const int row = s_pick - (guess - 1);
+    if (s_pick < 0 || row < 0 || row > 2) return;
+    const uint32_t* __restrict__ hist2 = ws.hist2 + row * kSelBins;
+    h0 = hist2[2 * t];
+    h1 = hist2[2 * t + 1];
+    s_sum[t] = (uint64_t)h0 + h1;
+    __syncthreads();
+    for (int o = 1; o < kScanThreads; o <<= 1) {
+        const uint64_t v = (t >= o) ? s_sum[t - o] : 0ull;
+        __syncthreads();
+        s_sum[t] += v;
+        __syncthreads();
+    }
+    remaining = ws.state->remaining;                    // what is left inside the first bin
+    before = s_sum[t] - h0 - h1;
+    __syncthreads();
+    pick = -1;
+    if (remaining > before && remaining <= before + h0) pick = 0;
+    else if (remaining > before + h0 && remaining <= before + h0 + h1) pick = 1;
+    if (pick >= 0 && (pick ? h1 : h0) <= kCandCap) {
+        ws.state->prefix |= (uint32_t)(2 * t + pick) << sel_shift(1);
+        ws.state->remaining = remaining - before - (pick ? h0 : 0u);
+        ws.state->mode = 2u;                            // candidates share 22 fixed bits
     }
 }
 
@@ -586,7 +638,8 @@ select_empty_kernel(uint32_t* __restrict__ planes, const uint64_t words,
 // sparsifier bitmask and "== T" in the tie mask
 template <class Src>
 static void run_select(const Src& src, uint64_t d, uint64_t q, const SparseWorkspace& sp,
-                       const SelectWorkspace& ws, int sm_count, cudaStream_t stream) {
+                       const SelectWorkspace& ws, int sm_count, cudaStream_t stream,
+                       int guess = -1) {
     const uint64_t groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
     // persistent grid: exactly the blocks that are resident together (a partial second wave would
     // run at the end with most SMs idle)
@@ -607,8 +660,11 @@ static void run_select(const Src& src, uint64_t d, uint64_t q, const SparseWorks
     const uint64_t cap_blocks = (uint64_t)sm_count * (uint64_t)resident;
     const unsigned pgrid = (unsigned)(groups < cap_blocks ? groups : cap_blocks);
     select_init_kernel<<<1, kScanThreads, 0, stream>>>(ws, q);
-    select_hist_kernel<Src, 0><<<pgrid, kBlockThreads, 0, stream>>>(src, d, ws);
-    select_choose_kernel<0><<<1, kScanThreads, 0, stream>>>(ws);
+    if (guess >= 0)
+        select_hist_kernel<Src, 0, true><<<pgrid, kBlockThreads, 0, stream>>>(src, d, ws, guess);
+    else
+        select_hist_kernel<Src, 0><<<pgrid, kBlockThreads, 0, stream>>>(src, d, ws);
+    select_choose_kernel<0><<<1, kScanThreads, 0, stream>>>(ws, guess);
     select_hist_kernel<Src, 1><<<pgrid, kBlockThreads, 0, stream>>>(src, d, ws);
     select_choose_kernel<1><<<1, kScanThreads, 0, stream>>>(ws);
     select_hist_kernel<Src, 2><<<pgrid, kBlockThreads, 0, stream>>>(src, d, ws);
@@ -670,7 +726,10 @@ nc_status nd_sparse_exact_compress(const float* x, size_t d, uint64_t q, float s
     StreamKeys src;
     src.worker = worker;
     src.keys = keys;
-    run_select(src, d, q, sp, ws, sm_count_of_current_device(), stream);
+    // stream keys are uniform: the q-th smallest lies in first-digit bin q * 2048 / d, give or take one
+    int guess = (int)((unsigned __int128)q * 2048u / d);
+    guess = guess < 1 ? 1 : (guess > 2046 ? 2046 : guess);
+    run_select(src, d, q, sp, ws, sm_count_of_current_device(), stream, guess);
     const unsigned grid = (unsigned)((sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock);
     if (p == 1)
         select_resolve_kernel<1, true><<<grid, kBlockThreads, 0, stream>>>(x, d, scale, sp, ws);
