@@ -506,57 +506,127 @@ select_candidates_kernel(uint32_t* __restrict__ mask, const SelectWorkspace ws) 
 // one block: in-place exclusive scan of n counts; the total goes to *total if it is not null
 __global__ void __launch_bounds__(kScanThreads)
 select_scan_counts_kernel(uint32_t* __restrict__ counts, const uint64_t n,
-                          uint32_t* __restrict__ total) {
+                          uint32_t* __restrict__ total, const SelectState* skip_unless_mode0) {
+    // the tie counts are only needed when all three digit passes ran
+    if (skip_unless_mode0 && skip_unless_mode0->mode != 0u) return;
     const uint32_t sum = block_exclusive_scan_inplace(counts, n);
     if (threadIdx.x == 0 && total) *total = sum;
 }
 
-// grid: ceil(tiles / warps per block).  mask <- "< T" | first r of "== T"; per-block kept counts;
-// with kNorm also the norm partials of the scaled kept entries (P as in the sparsifier).
-template <int P, bool kNorm>
+// grid: ceil(tiles / warps per block).  Only when all three digit passes ran (mode 0): mask <-
+// "< T" | the first r of "== T" in index order.  In the candidate modes the candidate kernel has
+// already set the selected candidates in the mask and there is nothing to do.
 __global__ void __launch_bounds__(kBlockThreads)
-select_resolve_kernel(const float* __restrict__ x, const uint64_t d, const float scale,
-                      const SparseWorkspace sp, const SelectWorkspace ws) {
+select_resolve_kernel(const uint64_t d, const SparseWorkspace sp, const SelectWorkspace ws) {
+    if (ws.state->mode != 0u) return;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
-    const uint64_t base = tile * kTile;
-    const bool active = base < d;
     __shared__ uint32_t s_eq[kWarpsPerBlock];
-    __shared__ uint32_t s_kept[kWarpsPerBlock];
-    uint32_t word = active ? sp.bitmask[tile * 32 + lane] : 0u;
-    uint32_t ew = active ? ws.eqmask[tile * 32 + lane] : 0u;
-    const uint32_t ne = __popc(ew);
-    uint32_t incl = ne;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) s_eq[warp] = incl;
-    __syncthreads();
-    uint64_t rank0 = (uint64_t)ws.eq_block[blockIdx.x] + (incl - ne);   // rank of this lane's first
-    for (int w = 0; w < warp; ++w) rank0 += s_eq[w];
     const uint64_t r = ws.state->remaining;
-    const uint32_t allowed = (r > rank0) ? (uint32_t)min((uint64_t)ne, r - rank0) : 0u;
-    uint32_t left = ne;
-    while (left > allowed) {                 // drop the highest-index ties beyond the first r
-        ew &= ~(0x80000000u >> __clz(ew));
-        --left;
-    }
-    word |= ew;
-    if (active) sp.bitmask[tile * 32 + lane] = word;
-    if (kNorm) {
-        kept_count_and_partial<P>(word, lane, x, base, scale, sp.block_count, sp.block_partial);
-    } else {
-        const uint32_t kept = warp_sum_u(__popc(word));
-        if (lane == 0) s_kept[warp] = kept;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t c = 0;
-            for (int w = 0; w < kWarpsPerBlock; ++w) c += s_kept[w];
-            sp.block_count[blockIdx.x] = c;
+    const uint64_t groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    for (uint64_t g = blockIdx.x; g < groups; g += gridDim.x) {      // a few blocks: the usual
+        const uint64_t tile = g * kWarpsPerBlock + warp;             // early exit costs nothing
+        const uint64_t base = tile * kTile;
+        const bool active = base < d;
+        uint32_t word = active ? sp.bitmask[tile * 32 + lane] : 0u;
+        uint32_t ew = active ? ws.eqmask[tile * 32 + lane] : 0u;
+        const uint32_t ne = __popc(ew);
+        uint32_t incl = ne;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += v;
         }
+        __syncthreads();                                             // s_eq of the last round is read
+        if (lane == 31) s_eq[warp] = incl;
+        __syncthreads();
+        uint64_t rank0 = (uint64_t)ws.eq_block[g] + (incl - ne);     // rank of this lane's first
+        for (int w = 0; w < warp; ++w) rank0 += s_eq[w];
+        const uint32_t allowed = (r > rank0) ? (uint32_t)min((uint64_t)ne, r - rank0) : 0u;
+        uint32_t left = ne;
+        while (left > allowed) {             // drop the highest-index ties beyond the first r
+            ew &= ~(0x80000000u >> __clz(ew));
+            --left;
+        }
+        word |= ew;
+        if (active) sp.bitmask[tile * 32 + lane] = word;
+    }
+}
+
+// grid: ceil(tile groups / warps per block); one warp per group of 8 tiles.  Per-group kept count
+// of the final mask and, with kNorm, the norm partial of the scaled kept entries (P as in the
+// sparsifier): what the compaction kernels shared with the sparsifier expect from a select pass.
+template <int P, bool kNorm>
+__global__ void __launch_bounds__(kBlockThreads)
+select_group_partial_kernel(const float* __restrict__ x, const uint64_t d, const float scale,
+                            const SparseWorkspace sp) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint64_t tiles = sparse_tiles(d);
+    const uint64_t groups = (tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const uint64_t grp = (uint64_t)blockIdx.x * kWarpsPerBlock + warp;
+    if (grp >= groups) return;
+    const uint64_t tile0 = grp * kWarpsPerBlock;
+    const uint64_t gbase = tile0 * kTile;
+    __shared__ uint16_t s_list[kNorm ? kWarpsPerBlock : 1][kNorm ? kGroupListCap : 1];
+    uint32_t word[kWarpsPerBlock];
+#pragma unroll
+    for (int w = 0; w < kWarpsPerBlock; ++w)
+        word[w] = (tile0 + w < tiles) ? sp.bitmask[(tile0 + w) * 32 + lane] : 0u;
+    uint32_t kept = 0;
+    double dsum = 0.0;
+    uint32_t vmax = 0;
+    if (kNorm) {
+        uint16_t* list = s_list[warp];
+        auto take = [&](float xv) {
+            const float xs = __fmul_rn(scale, xv);
+            const uint32_t a = __float_as_uint(xs) & 0x7FFFFFFFu;
+            if (P == NC_P_INF) vmax = max(vmax, a);
+            else if (P == 1) dsum += (double)__uint_as_float(a);
+            else dsum = fma((double)xs, (double)xs, dsum);
+        };
+        auto flush = [&](uint32_t cnt) {
+            __syncwarp();
+            if (cnt <= 4u * 32u) {
+                float xv[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t t = (uint32_t)(e * 32 + lane);
+                    xv[e] = (t < cnt) ? x[gbase + list[t]] : 0.f;   // +0 adds nothing to any norm
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) take(xv[e]);
+            } else {
+                for (uint32_t t = lane; t < cnt; t += 32) take(x[gbase + list[t]]);
+            }
+            __syncwarp();
+        };
+        uint32_t cnt = 0;
+#pragma unroll
+        for (int w = 0; w < kWarpsPerBlock; ++w) {
+            const uint32_t tile_cnt = warp_sum_u(__popc(word[w]));
+            if (cnt + tile_cnt > kGroupListCap) {
+                flush(cnt);
+                cnt = 0;
+            }
+            group_list_append(word[w], lane, w, list, cnt);
+            cnt += tile_cnt;
+            kept += tile_cnt;
+        }
+        flush(cnt);
+    } else {
+#pragma unroll
+        for (int w = 0; w < kWarpsPerBlock; ++w) kept += __popc(word[w]);
+        kept = warp_sum_u(kept);
+    }
+    uint64_t part = 0;
+    if (kNorm) {
+        if (P == NC_P_INF) part = (uint64_t)warp_max_u(vmax);
+        else part = (uint64_t)__double_as_longlong(warp_sum_d(dsum));
+    }
+    if (lane == 0) {
+        sp.block_count[grp] = kept;
+        if (kNorm) sp.block_partial[grp] = part;
     }
 }
 
@@ -671,7 +741,8 @@ static void run_select(const Src& src, uint64_t d, uint64_t q, const SparseWorks
     select_choose_kernel<2><<<1, kScanThreads, 0, stream>>>(ws);
     select_mark_kernel<Src><<<(unsigned)groups, kBlockThreads, 0, stream>>>(src, d, sp.bitmask, ws);
     select_candidates_kernel<<<1, kScanThreads, 0, stream>>>(sp.bitmask, ws);
-    select_scan_counts_kernel<<<1, kScanThreads, 0, stream>>>(ws.eq_block, groups, nullptr);
+    select_scan_counts_kernel<<<1, kScanThreads, 0, stream>>>(ws.eq_block, groups, nullptr,
+                                                              ws.state);
 }
 
 static int sm_count_of_current_device() {
@@ -731,13 +802,17 @@ nc_status nd_sparse_exact_compress(const float* x, size_t d, uint64_t q, float s
     guess = guess < 1 ? 1 : (guess > 2046 ? 2046 : guess);
     run_select(src, d, q, sp, ws, sm_count_of_current_device(), stream, guess);
     const unsigned grid = (unsigned)((sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    const uint64_t tile_groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const unsigned ggrid = (unsigned)((tile_groups + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    select_resolve_kernel<<<min(grid, 4u * (unsigned)sm_count_of_current_device()), kBlockThreads, 0,
+                            stream>>>(d, sp, ws);
     if (p == 1)
-        select_resolve_kernel<1, true><<<grid, kBlockThreads, 0, stream>>>(x, d, scale, sp, ws);
+        select_group_partial_kernel<1, true><<<ggrid, kBlockThreads, 0, stream>>>(x, d, scale, sp);
     else if (p == 2)
-        select_resolve_kernel<2, true><<<grid, kBlockThreads, 0, stream>>>(x, d, scale, sp, ws);
+        select_group_partial_kernel<2, true><<<ggrid, kBlockThreads, 0, stream>>>(x, d, scale, sp);
     else
-        select_resolve_kernel<NC_P_INF, true><<<grid, kBlockThreads, 0, stream>>>(x, d, scale, sp,
-                                                                                  ws);
+        select_group_partial_kernel<NC_P_INF, true><<<ggrid, kBlockThreads, 0, stream>>>(x, d,
+                                                                                        scale, sp);
     SparseBatch batch;
     batch.x[0] = x;
     batch.idx[0] = idx;
@@ -769,9 +844,13 @@ nc_status nc_topk_compress(const float* x, size_t d, uint64_t K, uint64_t seed, 
     src.x = x;
     run_select(src, d, K, sp, ws, sm_count_of_current_device(), stream);
     const uint64_t groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    select_resolve_kernel<NC_P_INF, false><<<(unsigned)groups, kBlockThreads, 0, stream>>>(
-        x, d, 1.0f, sp, ws);
-    select_scan_counts_kernel<<<1, kScanThreads, 0, stream>>>(sp.block_count, groups, ws.count);
+    select_resolve_kernel<<<(unsigned)min(groups, (uint64_t)(4 * sm_count_of_current_device())),
+                            kBlockThreads, 0, stream>>>(d, sp, ws);
+    select_group_partial_kernel<NC_P_INF, false>
+        <<<(unsigned)((groups + kWarpsPerBlock - 1) / kWarpsPerBlock), kBlockThreads, 0, stream>>>(
+            x, d, 1.0f, sp);
+    select_scan_counts_kernel<<<1, kScanThreads, 0, stream>>>(sp.block_count, groups, ws.count,
+                                                              nullptr);
     topk_emit_kernel<<<(unsigned)groups, kBlockThreads, 0, stream>>>(
         x, d, worker, make_philox_keys(seed), K, idx, exp, sp);
     const uint64_t sgroups = (K + 31) / 32;
