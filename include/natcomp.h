@@ -123,6 +123,17 @@ nc_status nc_aggregate_compress(const uint8_t* const* exps, const uint32_t* cons
                                 size_t d, uint64_t seed, uint32_t master, uint8_t* out_exp,
                                 uint32_t* out_sign, cudaStream_t stream);
 
+/* The same for a shard of a longer vector (the master's work split over several devices, each
+ * owning a range of coordinates): the d entries are the coordinates first_index .. first_index+d-1
+ * of the whole vector and the rounding uses the stream of (seed, master, first_index + j), so the
+ * shards' outputs put side by side equal one nc_aggregate_compress over the whole vector.
+ * first_index must be a multiple of 1024 (NC_ERR_INVALID otherwise); every pointer addresses the
+ * shard's own first entry. */
+nc_status nc_aggregate_compress_shard(const uint8_t* const* exps, const uint32_t* const* signs,
+                                      int n, size_t d, uint64_t first_index, uint64_t seed,
+                                      uint32_t master, uint8_t* out_exp, uint32_t* out_sign,
+                                      cudaStream_t stream);
+
 /* Reference point (the "no compression" baseline of Table 1): out[j] <- ((+0 + x_0j) + x_1j) + ...
  * xs: host array of n device pointers to fp32[d]. */
 nc_status nc_sum_fp32(const float* const* xs, int n, size_t d, float* out, cudaStream_t stream);

@@ -41,7 +41,7 @@ EXPORTS = (
     "nc_topk_compress", "nc_topk_decode_accumulate", "nc_compress_typed",
     "nc_compress_typed_batch", "nc64_compress", "nc64_compress_batch", "nc64_aggregate",
     "nd_sparse_regen_workspace_bytes", "nd_sparse_regen_decode_accumulate",
-    "nd_sparse_compact_aggregate",
+    "nd_sparse_compact_aggregate", "nc_aggregate_compress_shard",
 )
 
 
@@ -134,6 +134,18 @@ def nc_aggregate_compress(exps, signs, n, d, seed, master, out_exp, out_sign, st
     _check("nc_aggregate_compress",
            _nc_aggregate_compress(_ptrs(exps), _ptrs(signs), n, d, seed, master, _ptr(out_exp),
                                   _ptr(out_sign), _stream(stream)))
+
+
+_nc_aggregate_compress_shard = _sig("nc_aggregate_compress_shard", C.c_int, C.POINTER(_vp),
+                                    C.POINTER(_vp), C.c_int, _sz, C.c_uint64, C.c_uint64,
+                                    C.c_uint32, _vp, _vp, _vp)
+
+
+def nc_aggregate_compress_shard(exps, signs, n, d, first_index, seed, master, out_exp, out_sign,
+                                stream=None) -> None:
+    _check("nc_aggregate_compress_shard",
+           _nc_aggregate_compress_shard(_ptrs(exps), _ptrs(signs), n, d, first_index, seed,
+                                        master, _ptr(out_exp), _ptr(out_sign), _stream(stream)))
 
 
 _nc_compress_nearest = _sig("nc_compress_nearest", C.c_int, _vp, _sz, _vp, _vp, _vp)

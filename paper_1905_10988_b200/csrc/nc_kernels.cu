@@ -362,15 +362,18 @@ nc_aggregate_kernel(const __grid_constant__ PackedPlanes planes, const int n, co
 
 // Master side with compression of the aggregate (Algorithm 1: g = C_M(sum_i Delta_i) with
 // C_M = C_nat): the fp32 sum never leaves the registers, only its 9-bit code is written.
-// grid: ceil(tiles / warps per block)
+// The call covers the elements [first, d) of a longer vector (first a multiple of the tile size):
+// every pointer is the address element 0 of that vector would have, so that the stream index and
+// the memory index of an element are the same number.
+// grid: ceil(tiles in [first, d) / warps per block)
 __global__ void __launch_bounds__(kBlockThreads)
 nc_aggregate_compress_kernel(const __grid_constant__ PackedPlanes planes, const int n,
-                             const uint64_t d, const uint32_t master,
+                             const uint64_t first, const uint64_t d, const uint32_t master,
                              const __grid_constant__ PhiloxKeys keys, uint8_t* __restrict__ exp,
                              uint32_t* __restrict__ sign) {
     const int lane = threadIdx.x & 31;
     const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    const uint64_t base = tile * kTile;
+    const uint64_t base = first + tile * kTile;
     if (base >= d) return;
     if (base + kTile <= d) {
         float4 acc[8];
@@ -535,25 +538,39 @@ nc_status nc_aggregate(const uint8_t* const* exps, const uint32_t* const* signs,
     return launch_status();
 }
 
-nc_status nc_aggregate_compress(const uint8_t* const* exps, const uint32_t* const* signs, int n,
-                                size_t d, uint64_t seed, uint32_t master, uint8_t* out_exp,
-                                uint32_t* out_sign, cudaStream_t stream) {
+nc_status nc_aggregate_compress_shard(const uint8_t* const* exps, const uint32_t* const* signs,
+                                      int n, size_t d, uint64_t first_index, uint64_t seed,
+                                      uint32_t master, uint8_t* out_exp, uint32_t* out_sign,
+                                      cudaStream_t stream) {
     if (!exps || !signs || !out_exp || !out_sign || n < 1 || n > NC_MAX_WORKERS)
         return NC_ERR_INVALID;
+    if (first_index % kTile != 0) return NC_ERR_INVALID;
     if (d == 0) return NC_OK;
-    if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
+    if (d > ((uint64_t)1 << 40) || first_index > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
     if (!aligned16(out_exp) || !aligned16(out_sign)) return NC_ERR_ALIGN;
+    // the kernel indexes by position in the whole vector: move every pointer back by the shard's
+    // offset (first_index bytes of exponents, first_index / 8 bytes of sign words)
+    const uintptr_t exp_back = (uintptr_t)first_index, sign_back = (uintptr_t)(first_index / 8);
     PackedPlanes planes;
     for (int i = 0; i < n; ++i) {
         if (!exps[i] || !signs[i]) return NC_ERR_INVALID;
         if (!aligned16(exps[i]) || !aligned16(signs[i])) return NC_ERR_ALIGN;
-        planes.exp[i] = exps[i];
-        planes.sign[i] = signs[i];
+        planes.exp[i] = reinterpret_cast<const uint8_t*>((uintptr_t)exps[i] - exp_back);
+        planes.sign[i] = reinterpret_cast<const uint32_t*>((uintptr_t)signs[i] - sign_back);
     }
     const PhiloxKeys keys = make_philox_keys(seed);
     nc_aggregate_compress_kernel<<<tile_blocks(d), kBlockThreads, 0, stream>>>(
-        planes, n, (uint64_t)d, master, keys, out_exp, out_sign);
+        planes, n, first_index, first_index + (uint64_t)d, master, keys,
+        reinterpret_cast<uint8_t*>((uintptr_t)out_exp - exp_back),
+        reinterpret_cast<uint32_t*>((uintptr_t)out_sign - sign_back));
     return launch_status();
+}
+
+nc_status nc_aggregate_compress(const uint8_t* const* exps, const uint32_t* const* signs, int n,
+                                size_t d, uint64_t seed, uint32_t master, uint8_t* out_exp,
+                                uint32_t* out_sign, cudaStream_t stream) {
+    return nc_aggregate_compress_shard(exps, signs, n, d, 0, seed, master, out_exp, out_sign,
+                                       stream);
 }
 
 nc_status nc_decode_accumulate(const uint8_t* exp, const uint32_t* sign, size_t d, float* acc,

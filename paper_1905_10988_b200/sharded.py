@@ -1,0 +1,157 @@
+"""Algorithm 1 with the master's work split over the GPUs of one node: every rank is a worker
+(Delta_i = C_nat(g_i)) and the master of one contiguous range of coordinates.
+
+    compress        each rank codes its whole vector once (9 bits per entry); the random stream is
+                    indexed by the position in the whole vector, so nothing depends on the split
+    exchange        rank r needs the codes of its range from every rank: either an all-to-all of
+                    the two code planes over NCCL ("collective"), or no copy at all: the aggregate
+                    kernel reads the peers' planes in place through peer-mapped pointers
+                    ("peer", plain loads over NVLink; planes live in symmetric memory)
+    aggregate       nc_aggregate over the n = world code shards in rank order 0..world-1: the
+                    same sum, bit for bit, as one GPU aggregating n simulated workers
+    return          all-gather of the fp32 range, or, with master compression (g = C_M(Delta),
+                    C_M = C_nat), of its 9-bit code followed by one decode launch
+
+All arithmetic runs in the library's kernels; this module only owns buffers, slices them and
+calls the collectives.  `codec` is the module that provides nc_compress, nc_aggregate and
+nc_aggregate_compress_shard (the CUDA binding unless a test injects another).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import torch
+
+TILE = 1024                      # shards start on a tile boundary: 16-byte aligned plane slices
+MASTER_WORKER_ID = 0xFFFF0000    # stream id of C_M, outside the range of worker ranks
+
+
+@dataclass(frozen=True)
+class ShardPlan:
+    """Equal shards of a whole number of tiles; the last ranks' shards may reach past d (their
+    surplus entries are coded as zeros and dropped at the end)."""
+    d: int
+    world: int
+
+    def __post_init__(self):
+        if self.d < 1 or self.world < 1 or self.world > 64:
+            raise ValueError("need d >= 1 and 1 <= world <= 64")
+
+    @property
+    def shard(self) -> int:
+        per = -(-self.d // self.world)
+        return -(-per // TILE) * TILE
+
+    @property
+    def padded(self) -> int:
+        return self.shard * self.world
+
+    def first(self, rank: int) -> int:
+        return rank * self.shard
+
+    def owned(self, rank: int):
+        """[lo, hi) of the coordinates inside [0, d) that rank aggregates (empty if lo == hi)."""
+        lo = min(self.first(rank), self.d)
+        return lo, min(lo + self.shard, self.d)
+
+
+class NaturalAllReduce:
+    """sum_i C_nat(g_i) over the ranks of `group`, every rank receiving the full result.
+
+    transport = "collective": code planes move by all_to_all_single.
+    transport = "peer":       planes are allocated in symmetric memory and read in place by the
+                              aggregate kernel (needs CUDA peer access between all ranks).
+    """
+
+    def __init__(self, d: int, dist, group=None, *, seed: int = 0, transport: str = "collective",
+                 master_compress: bool = False, device=None, codec=None):
+        if transport not in ("collective", "peer"):
+            raise ValueError("transport must be 'collective' or 'peer'")
+        if codec is None:
+            from . import binding as codec          # fails loudly without the built library
+        self.codec = codec
+        self.dist = dist
+        self.group = group
+        self.rank = dist.get_rank(group)
+        self.world = dist.get_world_size(group)
+        self.plan = ShardPlan(d, self.world)
+        self.seed = seed
+        self.transport = transport
+        self.master_compress = master_compress
+        self.device = torch.device(device if device is not None else "cuda")
+        P, S = self.plan.padded, self.plan.shard
+        dev = self.device
+        self._symm = None
+        if transport == "peer":
+            import torch.distributed._symmetric_memory as symm_mem
+            # one allocation for both planes: exponents, then sign bytes
+            self._send = symm_mem.empty(P + P // 8, dtype=torch.uint8, device=dev)
+            self._send.zero_()
+            self._symm = symm_mem.rendezvous(self._send, group if group is not None
+                                             else dist.group.WORLD)
+        else:
+            self._send = torch.zeros(P + P // 8, dtype=torch.uint8, device=dev)
+            self._recv = torch.empty(P + P // 8, dtype=torch.uint8, device=dev)
+        self.exp_send = self._send[:P]
+        self.sign_send = self._send[P:]
+        if master_compress:
+            self._mine = torch.empty(S + S // 8, dtype=torch.uint8, device=dev)
+            self._all = torch.empty(P + P // 8, dtype=torch.uint8, device=dev)
+        else:
+            self._out_shard = torch.empty(S, dtype=torch.float32, device=dev)
+        self.out = torch.empty(P, dtype=torch.float32, device=dev)
+
+    # ---- the exchange: where rank r finds the codes of its range, one (exp, sign) per rank ----
+    def _shards_by_collective(self):
+        P, S, W = self.plan.padded, self.plan.shard, self.world
+        exp_recv, sign_recv = self._recv[:P], self._recv[P:]
+        self.dist.all_to_all_single(exp_recv, self.exp_send, group=self.group)
+        self.dist.all_to_all_single(sign_recv, self.sign_send, group=self.group)
+        exps = [exp_recv[i * S:(i + 1) * S] for i in range(W)]
+        signs = [sign_recv[i * (S // 8):(i + 1) * (S // 8)] for i in range(W)]
+        return exps, signs
+
+    def _shards_in_peer_memory(self):
+        P, S, W, r = self.plan.padded, self.plan.shard, self.world, self.rank
+        self._symm.barrier(channel=0)               # every rank's planes are written
+        exps, signs = [], []
+        for i in range(W):
+            buf = self._symm.get_buffer(i, (P + P // 8,), torch.uint8)
+            exps.append(buf[r * S:(r + 1) * S])
+            signs.append(buf[P + r * (S // 8):P + (r + 1) * (S // 8)])
+        return exps, signs
+
+    def __call__(self, g: torch.Tensor) -> torch.Tensor:
+        plan, W, r, c = self.plan, self.world, self.rank, self.codec
+        if g.numel() != plan.d or g.dtype != torch.float32:
+            raise ValueError("expected an fp32 vector of %d entries" % plan.d)
+        P, S = plan.padded, plan.shard
+        c.nc_compress(g, plan.d, self.seed, r, self.exp_send, self.sign_send)
+        if self.transport == "peer":
+            exps, signs = self._shards_in_peer_memory()
+        else:
+            exps, signs = self._shards_by_collective()
+        if self.master_compress:
+            my_exp, my_sign = self._mine[:S], self._mine[S:]
+            c.nc_aggregate_compress_shard(exps, signs, W, S, plan.first(r), self.seed,
+                                          MASTER_WORKER_ID, my_exp, my_sign)
+            if self.transport == "peer":
+                self._symm.barrier(channel=1)       # peers have read my planes: free to rewrite
+            all_exp, all_sign = self._all[:P], self._all[P:]
+            self.dist.all_gather_into_tensor(all_exp, my_exp, group=self.group)
+            self.dist.all_gather_into_tensor(all_sign, my_sign, group=self.group)
+            c.nc_aggregate([all_exp], [all_sign], 1, plan.d, self.out)
+        else:
+            c.nc_aggregate(exps, signs, W, S, self._out_shard)
+            if self.transport == "peer":
+                self._symm.barrier(channel=1)
+            self.dist.all_gather_into_tensor(self.out, self._out_shard, group=self.group)
+        return self.out[:plan.d]
+
+    def wire_bytes_per_rank(self) -> dict:
+        """Bytes a rank sends per call (its own shard stays local)."""
+        P, S, W = self.plan.padded, self.plan.shard, self.world
+        planes = (P + P // 8) * (W - 1) // W
+        back = (S + S // 8 if self.master_compress else 4 * S) * (W - 1)
+        return {"codes_out": planes, "result_out": back,
+                "uncompressed_ring_allreduce": 2 * 4 * P * (W - 1) // W}

@@ -1,0 +1,253 @@
+"""Algorithm 1 with the master sharded over the ranks (paper_1905_10988_b200.sharded).
+
+Host logic (shard plan, buffer slicing, order of the collectives) runs here as gloo ranks on CPU
+with the oracle injected as the codec; on a GPU the same flow runs with the CUDA codec: as one
+NCCL rank, and as four ranks emulated by host threads that exchange through host-side barriers
+(no kernel waits on another).  Expected values come from the oracle on the whole vectors:
+sum_i C_nat(g_i) in rank order, optionally followed by C_M = C_nat with the master's stream."""
+import os
+import socket
+import sys
+import threading
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import oracle
+from paper_1905_10988_b200.sharded import MASTER_WORKER_ID, NaturalAllReduce, ShardPlan
+
+SEED = 0x5EED1905
+
+
+def gradient(rank: int, d: int) -> np.ndarray:
+    rng = np.random.default_rng(1000 + rank)
+    x = (rng.standard_normal(d) * 10.0 ** rng.uniform(-4, 1, d)).astype(np.float32)
+    x[rng.random(d) < 0.02] = 0.0
+    return x
+
+
+def expected(d: int, world: int, master_compress: bool) -> np.ndarray:
+    planes = [oracle.nc_compress(gradient(r, d), SEED, r) for r in range(world)]
+    total = oracle.nc_aggregate([p[0] for p in planes], [p[1] for p in planes], d)
+    if not master_compress:
+        return total
+    e, s = oracle.nc_compress(total, SEED, MASTER_WORKER_ID)
+    return oracle.nc_aggregate([e], [s], d)
+
+
+def same_bits(a, b) -> bool:
+    return np.array_equal(np.asarray(a, np.float32).view(np.uint32),
+                          np.asarray(b, np.float32).view(np.uint32))
+
+
+# ---- shard plan -------------------------------------------------------------------------------
+@pytest.mark.parametrize("d,world", [(1, 1), (1, 4), (1024, 2), (1025, 2), (5000, 3),
+                                     (25_557_032, 8), (2 ** 28, 64)])
+def test_shard_plan_covers_every_coordinate_once(d, world):
+    plan = ShardPlan(d, world)
+    assert plan.shard % 1024 == 0 and plan.padded >= d
+    assert plan.padded - d < world * 1024 + world          # no more than a tile per rank wasted
+    hi_prev = 0
+    for r in range(world):
+        lo, hi = plan.owned(r)
+        assert lo == hi_prev and lo <= hi <= d
+        assert plan.first(r) % 1024 == 0
+        hi_prev = hi
+    assert hi_prev == d
+
+
+def test_shard_plan_rejects_bad_arguments():
+    with pytest.raises(ValueError):
+        ShardPlan(0, 2)
+    with pytest.raises(ValueError):
+        ShardPlan(10, 65)
+
+
+# ---- the oracle as codec (CPU tensors) --------------------------------------------------------
+class OracleCodec:
+    @staticmethod
+    def nc_compress(x, d, seed, worker, exp, sign):
+        e, s = oracle.nc_compress(x.numpy()[:d], seed, worker)
+        exp.numpy()[:d] = e
+        sign.numpy().view(np.uint32)[:s.size] = s
+
+    @staticmethod
+    def nc_aggregate(exps, signs, n, d, out):
+        out.numpy()[:d] = oracle.nc_aggregate([e.numpy()[:d] for e in exps[:n]],
+                                              [s.numpy().view(np.uint32) for s in signs[:n]], d)
+
+    @staticmethod
+    def nc_aggregate_compress_shard(exps, signs, n, d, first, seed, master, out_exp, out_sign):
+        total = oracle.nc_aggregate([e.numpy()[:d] for e in exps[:n]],
+                                    [s.numpy().view(np.uint32) for s in signs[:n]], d)
+        e, s = oracle.nc_compress(total, seed, master, j0=first)
+        out_exp.numpy()[:d] = e
+        out_sign.numpy().view(np.uint32)[:s.size] = s
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _gloo_rank(rank, world, port, d, master_compress, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ar = NaturalAllReduce(d, dist, seed=SEED, master_compress=master_compress, device="cpu",
+                          codec=OracleCodec)
+    g = torch.from_numpy(gradient(rank, d))
+    first = ar(g).numpy().copy()
+    second = ar(g).numpy().copy()                   # buffers are reused: a second call agrees
+    out.put((rank, first, second, ar.wire_bytes_per_rank()))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world,d,master_compress", [(2, 5000, False), (2, 5000, True),
+                                                     (3, 7 * 1024 + 5, True), (2, 3, False)])
+def test_gloo_ranks_reproduce_the_single_master_result(world, d, master_compress):
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_gloo_rank, args=(r, world, port, d, master_compress, out))
+             for r in range(world)]
+    for p in procs:
+        p.start()
+    got = [out.get(timeout=180) for _ in range(world)]
+    for p in procs:
+        p.join(timeout=180)
+        assert p.exitcode == 0
+    want = expected(d, world, master_compress)
+    for rank, first, second, wire in got:
+        assert same_bits(first, want), "rank %d differs from the single-master result" % rank
+        assert same_bits(second, want)
+        assert wire["codes_out"] < wire["uncompressed_ring_allreduce"]
+
+
+# ---- CUDA codec -------------------------------------------------------------------------------
+@pytest.mark.gpu
+def test_aggregate_compress_shards_side_by_side_equal_the_whole_vector():
+    import paper_1905_10988_b200 as nc
+    d, n = 6 * 1024 + 37, 3
+    xs = [torch.from_numpy(gradient(r, d)).cuda() for r in range(n)]
+    exps = [torch.zeros(nc.nc_exp_bytes(d) + 1024, dtype=torch.uint8, device="cuda") for _ in xs]
+    signs = [torch.zeros(nc.nc_sign_bytes(d) + 128, dtype=torch.uint8, device="cuda") for _ in xs]
+    for r in range(n):
+        nc.nc_compress(xs[r], d, SEED, r, exps[r], signs[r])
+    whole_e = torch.zeros(nc.nc_exp_bytes(d), dtype=torch.uint8, device="cuda")
+    whole_s = torch.zeros(nc.nc_sign_bytes(d), dtype=torch.uint8, device="cuda")
+    nc.nc_aggregate_compress(exps, signs, n, d, SEED, 77, whole_e, whole_s)
+    parts_e = torch.full_like(whole_e, 0xCD)
+    parts_s = torch.full_like(whole_s, 0xCD)
+    for first, length in ((0, 2048), (2048, 3072), (5120, d - 5120)):
+        nc.nc_aggregate_compress_shard([e[first:] for e in exps], [s[first // 8:] for s in signs],
+                                       n, length, first, SEED, 77, parts_e[first:],
+                                       parts_s[first // 8:])
+    torch.cuda.synchronize()
+    assert torch.equal(parts_e, whole_e) and torch.equal(parts_s, whole_s)
+    # and against the oracle
+    planes = [oracle.nc_compress(x.cpu().numpy(), SEED, r) for r, x in enumerate(xs)]
+    total = oracle.nc_aggregate([p[0] for p in planes], [p[1] for p in planes], d)
+    e, s = oracle.nc_compress(total, SEED, 77)
+    assert np.array_equal(whole_e.cpu().numpy()[:d], e)
+    assert np.array_equal(whole_s.cpu().numpy().view(np.uint32)[:s.size], s)
+    with pytest.raises(nc.NatcompError):
+        nc.nc_aggregate_compress_shard(exps, signs, n, 64, 512, SEED, 77, parts_e, parts_s)
+
+
+class ThreadFabric:
+    """The two collectives of the flow among `world` host threads of one process that share one
+    device and one stream: a thread publishes its tensor, waits at a host barrier, copies its
+    part of everybody's tensor.  Stream order equals enqueue order, so no device-side wait."""
+
+    def __init__(self, world):
+        self.world = world
+        self.local = threading.local()
+        self.barrier = threading.Barrier(world)
+        self.slots = [None] * world
+
+    def get_rank(self, group=None):
+        return self.local.rank
+
+    def get_world_size(self, group=None):
+        return self.world
+
+    def _publish(self, t):
+        self.slots[self.local.rank] = t
+        self.barrier.wait()
+
+    def all_to_all_single(self, out, inp, group=None):
+        self._publish(inp)
+        n = inp.numel() // self.world
+        r = self.local.rank
+        for i in range(self.world):
+            out[i * n:(i + 1) * n].copy_(self.slots[i][r * n:(r + 1) * n])
+        self.barrier.wait()
+
+    def all_gather_into_tensor(self, out, inp, group=None):
+        self._publish(inp)
+        n = inp.numel()
+        for i in range(self.world):
+            out[i * n:(i + 1) * n].copy_(self.slots[i])
+        self.barrier.wait()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("master_compress", [False, True])
+@pytest.mark.parametrize("world,d", [(4, 300_000), (3, 5 * 1024 + 1)])
+def test_cuda_codec_four_emulated_ranks(world, d, master_compress):
+    fabric = ThreadFabric(world)
+    results, errors = [None] * world, []
+
+    def run(rank):
+        try:
+            fabric.local.rank = rank
+            torch.cuda.set_device(0)
+            ar = NaturalAllReduce(d, fabric, seed=SEED, master_compress=master_compress)
+            g = torch.from_numpy(gradient(rank, d)).cuda()
+            ar(g)
+            out = ar(g)
+            torch.cuda.synchronize()
+            results[rank] = out.cpu().numpy()
+        except Exception as e:                                  # surfaces in the main thread
+            errors.append(e)
+            fabric.barrier.abort()
+
+    threads = [threading.Thread(target=run, args=(r,)) for r in range(world)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=300)
+    assert not errors, errors
+    want = expected(d, world, master_compress)
+    for r in range(world):
+        assert same_bits(results[r], want), "rank %d" % r
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("transport", ["collective", "peer"])
+def test_cuda_codec_one_nccl_rank(transport):
+    d = 200_000
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(_free_port())
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda:0"))
+    try:
+        for master_compress in (False, True):
+            ar = NaturalAllReduce(d, dist, seed=SEED, transport=transport,
+                                  master_compress=master_compress, device="cuda:0")
+            out = ar(torch.from_numpy(gradient(0, d)).cuda())
+            torch.cuda.synchronize()
+            assert same_bits(out.cpu().numpy(), expected(d, 1, master_compress))
+    finally:
+        dist.destroy_process_group()
