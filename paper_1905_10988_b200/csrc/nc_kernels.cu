@@ -226,11 +226,17 @@ nc_compress16_kernel(const __grid_constant__ Compress16Batch batch, const uint64
                             batch.worker[w], keys, batch.exp[w], batch.sign[w], lane);
 }
 
-// value of a 9-bit code: exponent byte in byte `BYTE` of `e4`, sign in bit 0 of `s`
+// value of a 9-bit code: exponent byte in byte `BYTE` of `e4`, sign in bit `BYTE` of `s4` (4 valid
+// bits, the rest zero).  The exponent byte is shifted to bits 30..23 and the sign bit to bit 31;
+// one three-input logic operation takes bits 30..23 from the first and everything else from the
+// second, so what the shifts drag along is dropped.
 template <int BYTE>
-__device__ __forceinline__ float decode9(uint32_t e4, uint32_t s) {
-    const uint32_t hi = __byte_perm(e4, 0u, 0x0444 | (BYTE << 12));   // exponent -> bits 24..31
-    return __uint_as_float(__funnelshift_r(hi, s, 1));                // (hi >> 1) | (s << 31)
+__device__ __forceinline__ float decode9(uint32_t e4, uint32_t s4) {
+    const uint32_t a = BYTE == 3 ? (e4 >> 1) : (e4 << (23 - 8 * BYTE));
+    const uint32_t b = s4 << (31 - BYTE);
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xCA;" : "=r"(r) : "r"(0x7F800000u), "r"(a), "r"(b));
+    return __uint_as_float(r);
 }
 
 // Staging of the workers' planes for the aggregation sweep: the 1024 exponent bytes and 32 sign
@@ -288,11 +294,11 @@ __device__ __forceinline__ void aggregate_full_tile(const PackedPlanes& planes, 
         for (int k = 0; k < 8; ++k) {
             const uint32_t e = st->e[k * 32 + lane];
             // sign word (k, g) lives in lane 4k+g; this lane needs group g = lane / 8
-            const uint32_t s = __shfl_sync(0xFFFFFFFFu, sw, k * 4 + (lane >> 3)) >> sh;
+            const uint32_t s = (__shfl_sync(0xFFFFFFFFu, sw, k * 4 + (lane >> 3)) >> sh) & 0xFu;
             acc[k].x += decode9<0>(e, s);
-            acc[k].y += decode9<1>(e, s >> 1);
-            acc[k].z += decode9<2>(e, s >> 2);
-            acc[k].w += decode9<3>(e, s >> 3);
+            acc[k].y += decode9<1>(e, s);
+            acc[k].z += decode9<2>(e, s);
+            acc[k].w += decode9<3>(e, s);
         }
         __syncwarp();                                   // the stage may be overwritten now
     }
@@ -312,11 +318,11 @@ __device__ __forceinline__ void aggregate_full_tile_direct(const PackedPlanes& p
         for (int k = 0; k < 8; ++k) e[k] = ld_stream_u32(ev + k * 32 + lane);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            const uint32_t s = __shfl_sync(0xFFFFFFFFu, sw, k * 4 + (lane >> 3)) >> sh;
+            const uint32_t s = (__shfl_sync(0xFFFFFFFFu, sw, k * 4 + (lane >> 3)) >> sh) & 0xFu;
             acc[k].x += decode9<0>(e[k], s);
-            acc[k].y += decode9<1>(e[k], s >> 1);
-            acc[k].z += decode9<2>(e[k], s >> 2);
-            acc[k].w += decode9<3>(e[k], s >> 3);
+            acc[k].y += decode9<1>(e[k], s);
+            acc[k].z += decode9<2>(e[k], s);
+            acc[k].w += decode9<3>(e[k], s);
         }
     }
 }

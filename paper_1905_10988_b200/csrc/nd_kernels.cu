@@ -420,10 +420,17 @@ __device__ __forceinline__ void level_exp_bytes(uint32_t nib8, uint32_t kexp, ui
     hi4 = b + mb * kexp;
 }
 
-template <int BYTE>
-__device__ __forceinline__ float pow2_signed(uint32_t e4, uint32_t s) {
-    const uint32_t hi = __byte_perm(e4, 0u, 0x0444 | (BYTE << 12));
-    return __uint_as_float(__funnelshift_r(hi, s, 1));
+// +-2^(c-s) (or +-0) of entry K of a group of eight: the exponent byte BYTE of e4 moved to bits
+// 30..23, the sign bit K of sg8 (8 valid bits, the rest zero) moved to bit 31, merged by one
+// three-input logic operation that takes bits 30..23 from the first and the rest from the second
+// operand.  Whatever else the shifts drag along lands in bits that the merge does not take.
+template <int BYTE, int K>
+__device__ __forceinline__ float pow2_signed(uint32_t e4, uint32_t sg8) {
+    const uint32_t a = BYTE == 3 ? (e4 >> 1) : (e4 << (23 - 8 * BYTE));
+    const uint32_t b = sg8 << (31 - K);
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xCA;" : "=r"(r) : "r"(0x7F800000u), "r"(a), "r"(b));
+    return __uint_as_float(r);
 }
 
 // fl32(norm * p) followed by a separate binary32 add (p = +-2^(c-s) or +-0)
@@ -489,7 +496,8 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
             if (!(fabsf(norm) <= 3.40282347e38f)) norm = 0.f;   // codes of such a bucket are 0
 #pragma unroll
             for (int it = 0; it < 4; ++it) {
-                const uint32_t sg = __shfl_sync(0xFFFFFFFFu, sw, it * 8 + (lane >> 2)) >> sh;
+                const uint32_t sg =
+                    (__shfl_sync(0xFFFFFFFFu, sw, it * 8 + (lane >> 2)) >> sh) & 0xFFu;
                 uint32_t lo4, hi4;
                 if ((nb[it] & 0x88888888u) == 0u) {
                     lo4 = __byte_perm(tbl_lo, tbl_hi, nb[it] & 0xFFFFu);
@@ -498,14 +506,14 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
                     level_exp_bytes(nb[it], kexp, lo4, hi4);
                 }
                 float* a = reinterpret_cast<float*>(acc[it].v);
-                a[0] = add_scaled(a[0], norm, pow2_signed<0>(lo4, sg));
-                a[1] = add_scaled(a[1], norm, pow2_signed<1>(lo4, sg >> 1));
-                a[2] = add_scaled(a[2], norm, pow2_signed<2>(lo4, sg >> 2));
-                a[3] = add_scaled(a[3], norm, pow2_signed<3>(lo4, sg >> 3));
-                a[4] = add_scaled(a[4], norm, pow2_signed<0>(hi4, sg >> 4));
-                a[5] = add_scaled(a[5], norm, pow2_signed<1>(hi4, sg >> 5));
-                a[6] = add_scaled(a[6], norm, pow2_signed<2>(hi4, sg >> 6));
-                a[7] = add_scaled(a[7], norm, pow2_signed<3>(hi4, sg >> 7));
+                a[0] = add_scaled(a[0], norm, pow2_signed<0, 0>(lo4, sg));
+                a[1] = add_scaled(a[1], norm, pow2_signed<1, 1>(lo4, sg));
+                a[2] = add_scaled(a[2], norm, pow2_signed<2, 2>(lo4, sg));
+                a[3] = add_scaled(a[3], norm, pow2_signed<3, 3>(lo4, sg));
+                a[4] = add_scaled(a[4], norm, pow2_signed<0, 4>(hi4, sg));
+                a[5] = add_scaled(a[5], norm, pow2_signed<1, 5>(hi4, sg));
+                a[6] = add_scaled(a[6], norm, pow2_signed<2, 6>(hi4, sg));
+                a[7] = add_scaled(a[7], norm, pow2_signed<3, 7>(hi4, sg));
             }
 #pragma unroll
             for (int it = 0; it < 4; ++it) nb[it] = nb_n[it];
