@@ -438,6 +438,39 @@ __device__ __forceinline__ float add_scaled(float acc, float norm, float p) {
     return __fadd_rn(acc, __fmul_rn(norm, p));
 }
 
+// One worker's contribution to the 1024 entries of a tile.  The caller guarantees
+// |norm| >= 2^(s-126): every product norm * 2^(c-s), c >= 1, is then a normal number, hence exact,
+// and one fused multiply-add gives the bits of the multiplication followed by the addition.
+// kWide: some code of the tile is above 7, the exponent bytes come from arithmetic instead of the
+// byte-permute table.
+template <bool kWide>
+__device__ __forceinline__ void add_worker_tile(V8 (&acc)[4], const uint32_t (&nb)[4],
+                                                const uint32_t sw, const float norm,
+                                                const uint32_t tbl_lo, const uint32_t tbl_hi,
+                                                const uint32_t kexp, const int lane) {
+    const int sh = 8 * (lane & 3);
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const uint32_t sg = (__shfl_sync(0xFFFFFFFFu, sw, it * 8 + (lane >> 2)) >> sh) & 0xFFu;
+        uint32_t lo4, hi4;
+        if (kWide) {
+            level_exp_bytes(nb[it], kexp, lo4, hi4);
+        } else {
+            lo4 = __byte_perm(tbl_lo, tbl_hi, nb[it]);
+            hi4 = __byte_perm(tbl_lo, tbl_hi, nb[it] >> 16);
+        }
+        float* a = reinterpret_cast<float*>(acc[it].v);
+        a[0] = __fmaf_rn(norm, pow2_signed<0, 0>(lo4, sg), a[0]);
+        a[1] = __fmaf_rn(norm, pow2_signed<1, 1>(lo4, sg), a[1]);
+        a[2] = __fmaf_rn(norm, pow2_signed<2, 2>(lo4, sg), a[2]);
+        a[3] = __fmaf_rn(norm, pow2_signed<3, 3>(lo4, sg), a[3]);
+        a[4] = __fmaf_rn(norm, pow2_signed<0, 4>(hi4, sg), a[4]);
+        a[5] = __fmaf_rn(norm, pow2_signed<1, 5>(hi4, sg), a[5]);
+        a[6] = __fmaf_rn(norm, pow2_signed<2, 6>(hi4, sg), a[6]);
+        a[7] = __fmaf_rn(norm, pow2_signed<3, 7>(hi4, sg), a[7]);
+    }
+}
+
 // grid: ceil(tiles / warps per block)
 template <bool kFromAcc>
 __global__ void __launch_bounds__(kBlockThreads)
@@ -445,13 +478,26 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
                     const uint64_t* __restrict__ off, const int B, const int s,
                     float* __restrict__ out) {
     const int lane = threadIdx.x & 31;
-    const uint64_t tile = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t tile = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const uint64_t base = tile * kTile;
     if (base >= d) return;
     const bool full = (base + kTile <= d);
     int b = find_bucket(off, B, base);
 
-    if (full && __ldg(off + b + 1) >= base + kTile) {
+    // The vector path needs a whole tile inside one bucket whose norms are all finite and either
+    // zero or at least 2^(s-126) (see add_worker_tile); anything else takes the scalar path.
+    bool vector = full && __ldg(off + b + 1) >= base + kTile;
+    if (vector) {
+        const float fused_min = __uint_as_float((uint32_t)(s + 1) << 23);   // 2^(s-126)
+        bool ok = true;
+        for (int i = lane; i < n; i += 32) {
+            const float a = fabsf(__ldg(planes.norms[i] + b));
+            ok = ok && (a == 0.f || (a >= fused_min && a <= 3.40282347e38f));
+        }
+        vector = __all_sync(0xFFFFFFFFu, ok);
+    }
+
+    if (vector) {
         V8 acc[4];
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
@@ -462,7 +508,6 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
             }
         }
         const uint32_t kexp = (uint32_t)(127 - s);
-        const int sh = 8 * (lane & 3);
         // exponent bytes of 2^(c-s) for c = 0..7 (0 for c = 0): a byte-permute with the four level
         // nibbles as selector looks four of them up at once; codes 8..15 take the arithmetic path
         uint32_t tbl_lo = 0, tbl_hi = 0;
@@ -493,28 +538,11 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
 #pragma unroll
                 for (int it = 0; it < 4; ++it) nb_n[it] = ld_stream_u32(lv + it * 32 + lane);
             }
-            if (!(fabsf(norm) <= 3.40282347e38f)) norm = 0.f;   // codes of such a bucket are 0
-#pragma unroll
-            for (int it = 0; it < 4; ++it) {
-                const uint32_t sg =
-                    (__shfl_sync(0xFFFFFFFFu, sw, it * 8 + (lane >> 2)) >> sh) & 0xFFu;
-                uint32_t lo4, hi4;
-                if ((nb[it] & 0x88888888u) == 0u) {
-                    lo4 = __byte_perm(tbl_lo, tbl_hi, nb[it] & 0xFFFFu);
-                    hi4 = __byte_perm(tbl_lo, tbl_hi, nb[it] >> 16);
-                } else {
-                    level_exp_bytes(nb[it], kexp, lo4, hi4);
-                }
-                float* a = reinterpret_cast<float*>(acc[it].v);
-                a[0] = add_scaled(a[0], norm, pow2_signed<0, 0>(lo4, sg));
-                a[1] = add_scaled(a[1], norm, pow2_signed<1, 1>(lo4, sg));
-                a[2] = add_scaled(a[2], norm, pow2_signed<2, 2>(lo4, sg));
-                a[3] = add_scaled(a[3], norm, pow2_signed<3, 3>(lo4, sg));
-                a[4] = add_scaled(a[4], norm, pow2_signed<0, 4>(hi4, sg));
-                a[5] = add_scaled(a[5], norm, pow2_signed<1, 5>(hi4, sg));
-                a[6] = add_scaled(a[6], norm, pow2_signed<2, 6>(hi4, sg));
-                a[7] = add_scaled(a[7], norm, pow2_signed<3, 7>(hi4, sg));
-            }
+            const uint32_t high = (nb[0] | nb[1] | nb[2] | nb[3]) & 0x88888888u;
+            if (__any_sync(0xFFFFFFFFu, high != 0u))
+                add_worker_tile<true>(acc, nb, sw, norm, tbl_lo, tbl_hi, kexp, lane);
+            else
+                add_worker_tile<false>(acc, nb, sw, norm, tbl_lo, tbl_hi, kexp, lane);
 #pragma unroll
             for (int it = 0; it < 4; ++it) nb[it] = nb_n[it];
             sw = sw_n;
@@ -549,6 +577,15 @@ inline unsigned nd_tile_blocks(uint64_t d) {
 }
 
 inline uint64_t nd_tiles(uint64_t d) { return (d + kTile - 1) / kTile; }
+
+// The aggregate kernel runs in small blocks: a block's life is long (n workers per tile), and
+// with 8 warps per block the blocks left over after the last full wave kept a quarter of the SMs
+// busy while the rest idled.
+constexpr int kAggregateThreads = 64;
+inline unsigned nd_aggregate_blocks(uint64_t d) {
+    const uint64_t per = kAggregateThreads / 32;
+    return (unsigned)((nd_tiles(d) + per - 1) / per);
+}
 
 }  // namespace natcomp
 
@@ -657,7 +694,7 @@ nc_status nd_aggregate(const float* const* norms, const uint8_t* const* levels,
     DitherPlanes planes;
     const nc_status st = nd_check_planes(norms, levels, signs, n, &planes);
     if (st != NC_OK) return st;
-    nd_aggregate_kernel<false><<<nd_tile_blocks(d), kBlockThreads, 0, stream>>>(
+    nd_aggregate_kernel<false><<<nd_aggregate_blocks(d), kAggregateThreads, 0, stream>>>(
         planes, n, (uint64_t)d, bucket_off, B, s, out);
     return launch_status();
 }
@@ -673,7 +710,7 @@ nc_status nd_decode_accumulate(const float* norms, const uint8_t* level, const u
     DitherPlanes planes;
     const nc_status st = nd_check_planes(&norms, &level, &sign, 1, &planes);
     if (st != NC_OK) return st;
-    nd_aggregate_kernel<true><<<nd_tile_blocks(d), kBlockThreads, 0, stream>>>(
+    nd_aggregate_kernel<true><<<nd_aggregate_blocks(d), kAggregateThreads, 0, stream>>>(
         planes, 1, (uint64_t)d, bucket_off, B, s, acc);
     return launch_status();
 }
