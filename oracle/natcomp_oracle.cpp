@@ -770,6 +770,25 @@ void orc_nc_compress_typed(const uint16_t* x, int dtype, uint64_t d, uint64_t se
     }
 }
 
+// C_nat (Def. 1) of bfloat16 inputs with a short random threshold.  A bfloat16 value has 7
+// mantissa bits, so its up-probability m = 1 - p(t) is a multiple of 1/128 and 7 random bits
+// decide the rounding exactly: "up" iff r7 < m * 128.  The draw is r7 = low 7 bits of byte
+// (j mod 4) of the stream word with index j / 4 in domain 4 (so one generator block of four words
+// serves 16 entries).  Written as the binary32 rule with r23 = r7 * 2^16: the threshold
+// m * 2^23 of a bfloat16 value is a multiple of 2^16.  Codes and edge cases as for binary32.
+void orc_nc_compress_bf16_r8(const uint16_t* x, uint64_t d, uint64_t seed, uint32_t worker,
+                             uint8_t* exp, uint32_t* sign) {
+    std::memset(sign, 0, (size_t)((d + 31) / 32) * 4);
+    for (uint64_t j = 0; j < d; ++j) {
+        const float t = value_of_16bit(x[j], 1);
+        const uint32_t word = stream_word(seed, worker, 4u, j / 4);
+        const uint32_t r7 = (word >> (8 * (j % 4))) & 0x7Fu;
+        uint32_t sb;
+        cnat_code(cnat_value(t, r7 << 16), &exp[j], &sb);
+        sign[j / 32] |= sb << (j % 32);
+    }
+}
+
 void orc_values_of_16bit(const uint16_t* x, int dtype, uint64_t d, float* out) {
     for (uint64_t j = 0; j < d; ++j) out[j] = value_of_16bit(x[j], dtype);
 }

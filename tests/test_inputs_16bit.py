@@ -90,3 +90,103 @@ def test_gpu_typed_batch_and_aggregate_round_trip():
     assert np.array_equal(out.cpu().numpy().view(np.uint32), want.view(np.uint32))
     with pytest.raises(nc.NatcompError):
         nc.nc_compress_typed(xd[0], 9, d, 1, 0, es[0], ss[0])
+
+
+# ---- bfloat16 with 7-bit thresholds: one stream byte per entry --------------------------------
+def test_bf16_short_threshold_rounds_up_in_exactly_m_of_128_draws():
+    # every finite bfloat16 pattern against every 7-bit draw: the number of draws that round up
+    # is the mantissa field (so P(up) = m exactly), and the mean over the draws is the value itself
+    h = _all_patterns()
+    t = oracle.values_of_16bit(h, BF16)
+    e_field = (h >> 7) & 0xFF
+    m_field = (h & 0x7F).astype(np.int64)
+    finite = e_field < 254                       # 254: never up (saturation); 255: inf / NaN
+    ups = np.zeros(h.size, np.int64)
+    total = np.zeros(h.size, np.float64)
+    lo_e, _ = oracle.cnat_codes(t, np.full(h.size, 127 << 16, np.uint32))   # r7 = 127: never up
+    for r7 in range(128):
+        vals = oracle.cnat_values(t, np.full(h.size, r7 << 16, np.uint32))
+        e, _ = oracle.cnat_codes(t, np.full(h.size, r7 << 16, np.uint32))
+        ups += (e != lo_e)
+        total += np.where(finite, vals.astype(np.float64), 0.0)
+    assert np.array_equal(ups[finite], m_field[finite])
+    assert np.all(ups[~finite] == 0)
+    want = np.where(finite, t.astype(np.float64), 0.0)
+    assert np.array_equal(total / 128.0, want)           # exact: sums of 128 powers of two
+
+
+def test_bf16_short_threshold_stream_mapping():
+    # entry j draws byte (j mod 4) of stream word j / 4 of domain 4 (the word stream itself is
+    # pinned by the generator's known answers); the codes are those of the binary32 rule with
+    # r23 = r7 * 2^16
+    rng = np.random.default_rng(11)
+    d = 4099
+    h = rng.integers(0, 1 << 16, d).astype(np.uint16)
+    seed, worker = 0xABCDEF0123, 9
+    words = oracle.stream_words(seed, worker, 4, 0, (d + 3) // 4)
+    j = np.arange(d)
+    r7 = (words[j // 4] >> (8 * (j % 4)).astype(np.uint32)) & 0x7F
+    e_want, s_want = oracle.cnat_codes(oracle.values_of_16bit(h, BF16), (r7 << 16).astype(np.uint32))
+    e, s = oracle.nc_compress_bf16_r8(h, seed, worker)
+    assert np.array_equal(e, e_want)
+    bits = (s[j // 32] >> (j % 32).astype(np.uint32)) & 1
+    assert np.array_equal(bits.astype(np.uint8), s_want)
+    # a different stream from the 23-bit variant's (domain 0)
+    e23, _ = oracle.nc_compress_typed(h, BF16, seed, worker)
+    assert not np.array_equal(e, e23)
+
+
+def test_bf16_short_threshold_frequency():
+    d = 1 << 20
+    h = np.full(d, 0x3F80 | 37, np.uint16)               # 1 + 37/128
+    e, _ = oracle.nc_compress_bf16_r8(h, 3, 1)
+    p = 37 / 128
+    assert abs((e == 128).mean() - p) < 5 * np.sqrt(p * (1 - p) / d)
+    assert set(np.unique(e)) == {127, 128}
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d", [1, 5, 31, 1024, 2048, 4097, 65536, 6 * 2048 + 515, (1 << 20) + 33])
+def test_gpu_bf16_short_threshold_matches_oracle(d):
+    import torch
+    import paper_1905_10988_b200 as nc
+    from gpu_util import Guarded, check_nc_planes, dev
+    rng = np.random.default_rng(d)
+    if d == 65536:
+        h = _all_patterns()                       # every pattern, specials included
+    else:
+        x = (rng.standard_normal(d) * 10.0 ** rng.uniform(-6, 3, d)).astype(np.float32)
+        h = (x.view(np.uint32) >> 16).astype(np.uint16)
+        h[rng.random(d) < 0.01] = 0x7F00 | 0x55   # exponent field 254: must not round up
+        h[rng.random(d) < 0.01] = 0x0033          # subnormal
+    e = Guarded(nc.nc_exp_bytes(d))
+    s = Guarded(nc.nc_sign_bytes(d))
+    nc.nc_compress_bf16_r8(dev(h.view(np.int16)), d, 7, 3, e.buf, s.buf)
+    torch.cuda.synchronize()
+    e_ref, s_ref = oracle.nc_compress_bf16_r8(h, 7, 3)
+    check_nc_planes(e, s, d, e_ref, s_ref)
+
+
+@pytest.mark.gpu
+def test_gpu_bf16_short_threshold_batch_aggregate_and_errors():
+    import torch
+    import paper_1905_10988_b200 as nc
+    from gpu_util import dev
+    rng = np.random.default_rng(5)
+    n, d = 3, 200_003
+    hs = [(rng.standard_normal(d).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+          for _ in range(n)]
+    xd = [dev(h.view(np.int16)) for h in hs]
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    es = [torch.empty(nc.nc_exp_bytes(d), **u8) for _ in range(n)]
+    ss = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
+    nc.nc_compress_bf16_r8_batch(xd, d, 1, [5, 6, 7], es, ss, n)
+    out = torch.empty(d, dtype=torch.float32, device="cuda")
+    nc.nc_aggregate(es, ss, n, d, out)
+    torch.cuda.synchronize()
+    refs = [oracle.nc_compress_bf16_r8(h, 1, 5 + i) for i, h in enumerate(hs)]
+    want = oracle.nc_aggregate([r[0] for r in refs], [r[1] for r in refs], d)
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    with pytest.raises(nc.NatcompError):
+        nc.nc_compress_bf16_r8(xd[0][1:], d - 1, 1, 0, es[0], ss[0])       # misaligned input
+    nc.nc_compress_bf16_r8(xd[0], 0, 1, 0, es[0], ss[0])                   # d = 0: nothing to do
