@@ -25,7 +25,8 @@
  * Random stream (the paper fixes none): Philox4x32-10 with
  *   key = (low32(seed), high32(seed)), counter = (low32(q), high32(q), worker, domain),
  *   q = j / 4; element j of a worker's vector uses output word j mod 4, low 23 bits.
- *   domain 0: C_nat, 1: D_nat rounding, 2: sparsifier selection.
+ *   domain 0: C_nat, 1: D_nat rounding, 2: sparsifier selection, 3: low bits of binary64
+ *   thresholds, 4: byte-wide draws of nc_compress_bf16_r8.
  * The stream depends on (seed, worker, j) only, so outputs are reproducible and
  * independent of launch geometry.
  *
@@ -321,6 +322,19 @@ nc_status nc_compress_typed(const void* x, int dtype, size_t d, uint64_t seed, u
 nc_status nc_compress_typed_batch(const void* const* xs, int dtype, size_t d, uint64_t seed,
                                   const uint32_t* workers, uint8_t* const* exps,
                                   uint32_t* const* signs, int n, cudaStream_t stream);
+
+/* bfloat16 inputs with 7-bit thresholds (Def. 1: a bfloat16 value has 7 mantissa bits, so its
+ * up-probability is a multiple of 1/128 and 7 random bits decide the rounding exactly).  Entry j
+ * draws the low 7 bits of byte (j mod 4) of stream word j / 4 of domain 4 and is rounded up iff
+ * the draw is below its mantissa field: one generator block serves 16 entries, which makes the
+ * call memory-bound.  Unbiased like nc_compress_typed, but a different draw, so the two calls give
+ * different (equally distributed) codes.  x: d bfloat16 bit patterns, 32-byte aligned.  Planes,
+ * edge cases and errors as for nc_compress. */
+nc_status nc_compress_bf16_r8(const void* x, size_t d, uint64_t seed, uint32_t worker,
+                              uint8_t* exp, uint32_t* sign, cudaStream_t stream);
+nc_status nc_compress_bf16_r8_batch(const void* const* xs, size_t d, uint64_t seed,
+                                    const uint32_t* workers, uint8_t* const* exps,
+                                    uint32_t* const* signs, int n, cudaStream_t stream);
 
 /* ---- binary64 inputs: 12-bit codes -------------------------------------------------------------
  * Sec. 2: "11 bits for the exponent and 1 for the sign".  C_nat (Def. 1) of a binary64 vector with

@@ -81,6 +81,11 @@ def run_cnat(config, n, d, make_vector, iters, peak, with_sum=True):
         _report(config, "nc_compress_typed_batch (%s inputs)" % name, m, b, n * d, n * d * 3.125,
                 peak, {"note": "generator-bound: the multiplier-pipe ceiling is about 1860-2070 "
                                "Gelem/s, the HBM roof 2093 Gelem/s"})
+        if code == nc.DTYPE_BF16:
+            m, b = _time(lambda: nc.nc_compress_bf16_r8_batch(xh, d, 0, workers, es, ss, n), iters)
+            _report(config, "nc_compress_bf16_r8_batch (bf16 inputs, 7-bit thresholds)", m, b,
+                    n * d, n * d * 3.125, peak,
+                    {"note": "one generator block per 16 entries: memory-bound"})
         del xh
     if with_sum:
         m, b = _time(lambda: nc.nc_sum_fp32(xs, n, d, out), iters)
