@@ -471,22 +471,76 @@ __device__ __forceinline__ void add_worker_tile(V8 (&acc)[4], const uint32_t (&n
     }
 }
 
-// grid: ceil(tiles / warps per block)
+// The same for a piece of 256 entries (8 per lane; base a multiple of 256): one nibble word and one
+// byte of the sign plane per lane and worker.  Used at the end of the vector, see the kernel.
+template <bool kFromAcc>
+__device__ __forceinline__ void aggregate_small_piece(const DitherPlanes& planes, const int n,
+                                                      const uint64_t base, const int b,
+                                                      const uint32_t tbl_lo, const uint32_t tbl_hi,
+                                                      const uint32_t kexp,
+                                                      float* __restrict__ out, const int lane) {
+    V8 acc;
+    if (kFromAcc) acc = ld_stream_v8(out + base + lane * 8);
+    else {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc.v[c] = 0u;
+    }
+    float* a = reinterpret_cast<float*>(acc.v);
+    uint32_t nb = ld_stream_u32(planes.level[0] + (base >> 1) + lane * 4);
+    uint32_t sg = reinterpret_cast<const uint8_t*>(planes.sign[0])[(base >> 3) + lane];
+    float norm = __ldg(planes.norms[0] + b);
+    for (int i = 0; i < n; ++i) {
+        uint32_t nb_n = 0u, sg_n = 0u;
+        float norm_n = 0.f;
+        if (i + 1 < n) {
+            nb_n = ld_stream_u32(planes.level[i + 1] + (base >> 1) + lane * 4);
+            sg_n = reinterpret_cast<const uint8_t*>(planes.sign[i + 1])[(base >> 3) + lane];
+            norm_n = __ldg(planes.norms[i + 1] + b);
+        }
+        uint32_t lo4, hi4;
+        if (__any_sync(0xFFFFFFFFu, (nb & 0x88888888u) != 0u)) {
+            level_exp_bytes(nb, kexp, lo4, hi4);
+        } else {
+            lo4 = __byte_perm(tbl_lo, tbl_hi, nb);
+            hi4 = __byte_perm(tbl_lo, tbl_hi, nb >> 16);
+        }
+        a[0] = __fmaf_rn(norm, pow2_signed<0, 0>(lo4, sg), a[0]);
+        a[1] = __fmaf_rn(norm, pow2_signed<1, 1>(lo4, sg), a[1]);
+        a[2] = __fmaf_rn(norm, pow2_signed<2, 2>(lo4, sg), a[2]);
+        a[3] = __fmaf_rn(norm, pow2_signed<3, 3>(lo4, sg), a[3]);
+        a[4] = __fmaf_rn(norm, pow2_signed<0, 4>(hi4, sg), a[4]);
+        a[5] = __fmaf_rn(norm, pow2_signed<1, 5>(hi4, sg), a[5]);
+        a[6] = __fmaf_rn(norm, pow2_signed<2, 6>(hi4, sg), a[6]);
+        a[7] = __fmaf_rn(norm, pow2_signed<3, 7>(hi4, sg), a[7]);
+        nb = nb_n;
+        sg = sg_n;
+        norm = norm_n;
+    }
+    st_stream_v8(out + base + lane * 8, acc);
+}
+
+// Warps 0 .. big_tiles-1 take one tile of 1024 entries each; the entries after those tiles are cut
+// into pieces of 256, one per warp.  Blocks start in index order, so the small pieces run last
+// and fill the SMs evenly while the grid drains: a warp's life is long here (n workers per tile),
+// and with whole tiles to the end the SMs were busy only three quarters of the kernel's duration.
+// grid: ceil((big_tiles + small pieces) / warps per block)
 template <bool kFromAcc>
 __global__ void __launch_bounds__(kBlockThreads)
 nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, const uint64_t d,
                     const uint64_t* __restrict__ off, const int B, const int s,
-                    float* __restrict__ out) {
+                    const uint64_t big_tiles, float* __restrict__ out) {
     const int lane = threadIdx.x & 31;
-    const uint64_t tile = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const uint64_t base = tile * kTile;
+    const uint64_t warp = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const bool big = warp < big_tiles;
+    const uint64_t len = big ? kTile : kTile / 4;
+    const uint64_t base = big ? warp * kTile : big_tiles * kTile + (warp - big_tiles) * (kTile / 4);
     if (base >= d) return;
-    const bool full = (base + kTile <= d);
+    const bool full = (base + len <= d);
     int b = find_bucket(off, B, base);
 
-    // The vector path needs a whole tile inside one bucket whose norms are all finite and either
+    // The vector path needs a whole piece inside one bucket whose norms are all finite and either
     // zero or at least 2^(s-126) (see add_worker_tile); anything else takes the scalar path.
-    bool vector = full && __ldg(off + b + 1) >= base + kTile;
+    bool vector = full && __ldg(off + b + 1) >= base + len;
     if (vector) {
         const float fused_min = __uint_as_float((uint32_t)(s + 1) << 23);   // 2^(s-126)
         bool ok = true;
@@ -498,15 +552,6 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
     }
 
     if (vector) {
-        V8 acc[4];
-#pragma unroll
-        for (int it = 0; it < 4; ++it) {
-            if (kFromAcc) acc[it] = ld_stream_v8(out + base + it * 256 + lane * 8);
-            else {
-#pragma unroll
-                for (int c = 0; c < 8; ++c) acc[it].v[c] = 0u;
-            }
-        }
         const uint32_t kexp = (uint32_t)(127 - s);
         // exponent bytes of 2^(c-s) for c = 0..7 (0 for c = 0): a byte-permute with the four level
         // nibbles as selector looks four of them up at once; codes 8..15 take the arithmetic path
@@ -515,6 +560,19 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
         for (int c = 1; c < 8; ++c) {
             const uint32_t e = (uint32_t)c + kexp;
             if (c < 4) tbl_lo |= e << (8 * c); else tbl_hi |= e << (8 * (c - 4));
+        }
+        if (!big) {
+            aggregate_small_piece<kFromAcc>(planes, n, base, b, tbl_lo, tbl_hi, kexp, out, lane);
+            return;
+        }
+        V8 acc[4];
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            if (kFromAcc) acc[it] = ld_stream_v8(out + base + it * 256 + lane * 8);
+            else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) acc[it].v[c] = 0u;
+            }
         }
         // software pipeline over the workers: the planes of worker i+1 are in flight while
         // worker i is decoded
@@ -553,8 +611,8 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
         return;
     }
 
-    // tile spans several buckets or is ragged: scalar, per-lane bucket cursor
-    const uint64_t end = full ? base + kTile : d;
+    // the piece spans several buckets or is ragged: scalar, per-lane bucket cursor
+    const uint64_t end = full ? base + len : d;
     uint64_t bend = __ldg(off + b + 1);
     for (uint64_t j = base + lane; j < end; j += 32) {
         while (j >= bend) { ++b; bend = __ldg(off + b + 1); }
@@ -578,13 +636,24 @@ inline unsigned nd_tile_blocks(uint64_t d) {
 
 inline uint64_t nd_tiles(uint64_t d) { return (d + kTile - 1) / kTile; }
 
-// The aggregate kernel runs in small blocks: a block's life is long (n workers per tile), and
-// with 8 warps per block the blocks left over after the last full wave kept a quarter of the SMs
-// busy while the rest idled.
+// The aggregate kernel runs in small blocks (2 warps).  Tiles of 1024 entries except for the last
+// `nd_small_region_tiles` tiles' worth of entries, which are cut into pieces of 256: half a wave
+// of resident warps (4 blocks of 8 warps' worth per SM), and nothing when all tiles are resident
+// at once anyway.
 constexpr int kAggregateThreads = 64;
-inline unsigned nd_aggregate_blocks(uint64_t d) {
+
+inline uint64_t nd_aggregate_big_tiles(uint64_t d) {
+    const uint64_t tiles = nd_tiles(d);
+    const uint64_t resident = (uint64_t)device_sm_count() * 32u;
+    if (tiles <= resident) return tiles;
+    return tiles - resident / 2;
+}
+
+inline unsigned nd_aggregate_blocks(uint64_t d, uint64_t big_tiles) {
+    const uint64_t rest = d > big_tiles * kTile ? d - big_tiles * kTile : 0;
+    const uint64_t warps = big_tiles + (rest + kTile / 4 - 1) / (kTile / 4);
     const uint64_t per = kAggregateThreads / 32;
-    return (unsigned)((nd_tiles(d) + per - 1) / per);
+    return (unsigned)((warps + per - 1) / per);
 }
 
 }  // namespace natcomp
@@ -694,8 +763,9 @@ nc_status nd_aggregate(const float* const* norms, const uint8_t* const* levels,
     DitherPlanes planes;
     const nc_status st = nd_check_planes(norms, levels, signs, n, &planes);
     if (st != NC_OK) return st;
-    nd_aggregate_kernel<false><<<nd_aggregate_blocks(d), kAggregateThreads, 0, stream>>>(
-        planes, n, (uint64_t)d, bucket_off, B, s, out);
+    const uint64_t big_tiles = nd_aggregate_big_tiles(d);
+    nd_aggregate_kernel<false><<<nd_aggregate_blocks(d, big_tiles), kAggregateThreads, 0, stream>>>(
+        planes, n, (uint64_t)d, bucket_off, B, s, big_tiles, out);
     return launch_status();
 }
 
@@ -710,8 +780,9 @@ nc_status nd_decode_accumulate(const float* norms, const uint8_t* level, const u
     DitherPlanes planes;
     const nc_status st = nd_check_planes(&norms, &level, &sign, 1, &planes);
     if (st != NC_OK) return st;
-    nd_aggregate_kernel<true><<<nd_aggregate_blocks(d), kAggregateThreads, 0, stream>>>(
-        planes, 1, (uint64_t)d, bucket_off, B, s, acc);
+    const uint64_t big_tiles = nd_aggregate_big_tiles(d);
+    nd_aggregate_kernel<true><<<nd_aggregate_blocks(d, big_tiles), kAggregateThreads, 0, stream>>>(
+        planes, 1, (uint64_t)d, bucket_off, B, s, big_tiles, acc);
     return launch_status();
 }
 
