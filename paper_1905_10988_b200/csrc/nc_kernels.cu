@@ -372,7 +372,7 @@ nc_aggregate_kernel(const __grid_constant__ PackedPlanes planes, const int n, co
 // every pointer is the address element 0 of that vector would have, so that the stream index and
 // the memory index of an element are the same number.
 // grid: ceil(tiles in [first, d) / warps per block)
-__global__ void __launch_bounds__(kBlockThreads)
+__global__ void __launch_bounds__(kBlockThreads, 4)
 nc_aggregate_compress_kernel(const __grid_constant__ PackedPlanes planes, const int n,
                              const uint64_t first, const uint64_t d, const uint32_t master,
                              const __grid_constant__ PhiloxKeys keys, uint8_t* __restrict__ exp,
