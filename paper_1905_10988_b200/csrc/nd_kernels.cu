@@ -445,13 +445,11 @@ __device__ __forceinline__ float add_scaled(float acc, float norm, float p) {
 // byte-permute table.
 template <bool kWide>
 __device__ __forceinline__ void add_worker_tile(V8 (&acc)[4], const uint32_t (&nb)[4],
-                                                const uint32_t sw, const float norm,
+                                                const uint32_t (&sg)[4], const float norm,
                                                 const uint32_t tbl_lo, const uint32_t tbl_hi,
-                                                const uint32_t kexp, const int lane) {
-    const int sh = 8 * (lane & 3);
+                                                const uint32_t kexp) {
 #pragma unroll
     for (int it = 0; it < 4; ++it) {
-        const uint32_t sg = (__shfl_sync(0xFFFFFFFFu, sw, it * 8 + (lane >> 2)) >> sh) & 0xFFu;
         uint32_t lo4, hi4;
         if (kWide) {
             level_exp_bytes(nb[it], kexp, lo4, hi4);
@@ -460,15 +458,46 @@ __device__ __forceinline__ void add_worker_tile(V8 (&acc)[4], const uint32_t (&n
             hi4 = __byte_perm(tbl_lo, tbl_hi, nb[it] >> 16);
         }
         float* a = reinterpret_cast<float*>(acc[it].v);
-        a[0] = __fmaf_rn(norm, pow2_signed<0, 0>(lo4, sg), a[0]);
-        a[1] = __fmaf_rn(norm, pow2_signed<1, 1>(lo4, sg), a[1]);
-        a[2] = __fmaf_rn(norm, pow2_signed<2, 2>(lo4, sg), a[2]);
-        a[3] = __fmaf_rn(norm, pow2_signed<3, 3>(lo4, sg), a[3]);
-        a[4] = __fmaf_rn(norm, pow2_signed<0, 4>(hi4, sg), a[4]);
-        a[5] = __fmaf_rn(norm, pow2_signed<1, 5>(hi4, sg), a[5]);
-        a[6] = __fmaf_rn(norm, pow2_signed<2, 6>(hi4, sg), a[6]);
-        a[7] = __fmaf_rn(norm, pow2_signed<3, 7>(hi4, sg), a[7]);
+        a[0] = __fmaf_rn(norm, pow2_signed<0, 0>(lo4, sg[it]), a[0]);
+        a[1] = __fmaf_rn(norm, pow2_signed<1, 1>(lo4, sg[it]), a[1]);
+        a[2] = __fmaf_rn(norm, pow2_signed<2, 2>(lo4, sg[it]), a[2]);
+        a[3] = __fmaf_rn(norm, pow2_signed<3, 3>(lo4, sg[it]), a[3]);
+        a[4] = __fmaf_rn(norm, pow2_signed<0, 4>(hi4, sg[it]), a[4]);
+        a[5] = __fmaf_rn(norm, pow2_signed<1, 5>(hi4, sg[it]), a[5]);
+        a[6] = __fmaf_rn(norm, pow2_signed<2, 6>(hi4, sg[it]), a[6]);
+        a[7] = __fmaf_rn(norm, pow2_signed<3, 7>(hi4, sg[it]), a[7]);
     }
+}
+
+// a worker's planes of one tile as a lane holds them: the nibble words of its 4 x 8 entries and,
+// per group of 8, the byte of the sign plane with their sign bits
+struct WorkerTile {
+    uint32_t nb[4];
+    uint32_t sg[4];
+    float norm;
+};
+
+__device__ __forceinline__ void load_worker_tile(WorkerTile& t, const DitherPlanes& planes,
+                                                 const int i, const uint64_t base, const int b,
+                                                 const int lane) {
+    const uint32_t* lv = reinterpret_cast<const uint32_t*>(planes.level[i] + (base >> 1));
+    const uint8_t* sb = reinterpret_cast<const uint8_t*>(planes.sign[i]) + (base >> 3);
+    t.norm = __ldg(planes.norms[i] + b);
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        t.nb[it] = ld_stream_u32(lv + it * 32 + lane);
+        t.sg[it] = sb[it * 32 + lane];
+    }
+}
+
+__device__ __forceinline__ void add_worker(V8 (&acc)[4], const WorkerTile& t,
+                                           const uint32_t tbl_lo, const uint32_t tbl_hi,
+                                           const uint32_t kexp) {
+    const uint32_t high = (t.nb[0] | t.nb[1] | t.nb[2] | t.nb[3]) & 0x88888888u;
+    if (__any_sync(0xFFFFFFFFu, high != 0u))
+        add_worker_tile<true>(acc, t.nb, t.sg, t.norm, tbl_lo, tbl_hi, kexp);
+    else
+        add_worker_tile<false>(acc, t.nb, t.sg, t.norm, tbl_lo, tbl_hi, kexp);
 }
 
 // The same for a piece of 256 entries (8 per lane; base a multiple of 256): one nibble word and one
@@ -574,37 +603,18 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
                 for (int c = 0; c < 8; ++c) acc[it].v[c] = 0u;
             }
         }
-        // software pipeline over the workers: the planes of worker i+1 are in flight while
-        // worker i is decoded
-        uint32_t nb[4], sw;
-        float norm;
-        {
-            const uint32_t* lv = reinterpret_cast<const uint32_t*>(planes.level[0] + (base >> 1));
-            norm = __ldg(planes.norms[0] + b);
-            sw = ld_stream_u32(planes.sign[0] + (base >> 5) + lane);
-#pragma unroll
-            for (int it = 0; it < 4; ++it) nb[it] = ld_stream_u32(lv + it * 32 + lane);
-        }
-        for (int i = 0; i < n; ++i) {
-            uint32_t nb_n[4] = {0u, 0u, 0u, 0u}, sw_n = 0u;
-            float norm_n = 0.f;
-            if (i + 1 < n) {
-                const uint32_t* lv =
-                    reinterpret_cast<const uint32_t*>(planes.level[i + 1] + (base >> 1));
-                norm_n = __ldg(planes.norms[i + 1] + b);
-                sw_n = ld_stream_u32(planes.sign[i + 1] + (base >> 5) + lane);
-#pragma unroll
-                for (int it = 0; it < 4; ++it) nb_n[it] = ld_stream_u32(lv + it * 32 + lane);
+        // software pipeline over the workers, two register sets in turn: the planes of worker
+        // i+1 are in flight while worker i is decoded
+        WorkerTile ta, tb;
+        load_worker_tile(ta, planes, 0, base, b, lane);
+        for (int i = 0; i < n; i += 2) {
+            const bool second = i + 1 < n;
+            if (second) load_worker_tile(tb, planes, i + 1, base, b, lane);
+            add_worker(acc, ta, tbl_lo, tbl_hi, kexp);
+            if (second) {
+                if (i + 2 < n) load_worker_tile(ta, planes, i + 2, base, b, lane);
+                add_worker(acc, tb, tbl_lo, tbl_hi, kexp);
             }
-            const uint32_t high = (nb[0] | nb[1] | nb[2] | nb[3]) & 0x88888888u;
-            if (__any_sync(0xFFFFFFFFu, high != 0u))
-                add_worker_tile<true>(acc, nb, sw, norm, tbl_lo, tbl_hi, kexp, lane);
-            else
-                add_worker_tile<false>(acc, nb, sw, norm, tbl_lo, tbl_hi, kexp, lane);
-#pragma unroll
-            for (int it = 0; it < 4; ++it) nb[it] = nb_n[it];
-            sw = sw_n;
-            norm = norm_n;
         }
 #pragma unroll
         for (int it = 0; it < 4; ++it) st_stream_v8(out + base + it * 256 + lane * 8, acc[it]);
