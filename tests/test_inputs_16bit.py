@@ -190,3 +190,24 @@ def test_gpu_bf16_short_threshold_batch_aggregate_and_errors():
     with pytest.raises(nc.NatcompError):
         nc.nc_compress_bf16_r8(xd[0][1:], d - 1, 1, 0, es[0], ss[0])       # misaligned input
     nc.nc_compress_bf16_r8(xd[0], 0, 1, 0, es[0], ss[0])                   # d = 0: nothing to do
+
+
+@pytest.mark.gpu
+def test_gpu_bf16_short_threshold_full_size_batch():
+    # the benchmark shape: 2 of the 8 workers of the ResNet-50-sized vector in one batch launch,
+    # whole planes compared
+    import torch
+    import paper_1905_10988_b200 as nc
+    d, n = 25_557_032, 2
+    g = torch.Generator(device="cuda").manual_seed(2001)
+    xs = [(torch.randn(d, device="cuda", generator=g) * 1e-3).to(torch.bfloat16) for _ in range(n)]
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    es = [torch.full((nc.nc_exp_bytes(d),), 0xCD, **u8) for _ in range(n)]
+    ss = [torch.full((nc.nc_sign_bytes(d),), 0xCD, **u8) for _ in range(n)]
+    nc.nc_compress_bf16_r8_batch(xs, d, 0, [0, 1], es, ss, n)
+    torch.cuda.synchronize()
+    for w in range(n):
+        h = xs[w].view(torch.int16).cpu().numpy().view(np.uint16)
+        e_ref, s_ref = oracle.nc_compress_bf16_r8(h, 0, w)
+        assert np.array_equal(es[w].cpu().numpy()[:d], e_ref)
+        assert np.array_equal(ss[w].cpu().numpy().view(np.uint32)[:s_ref.size], s_ref)
