@@ -155,3 +155,113 @@ class NaturalAllReduce:
         back = (S + S // 8 if self.master_compress else 4 * S) * (W - 1)
         return {"codes_out": planes, "result_out": back,
                 "uncompressed_ring_allreduce": 2 * 4 * P * (W - 1) // W}
+
+
+def shard_bucket_table(bucket_off, first: int, stop: int):
+    """The buckets that overlap the coordinates [first, stop) of the whole vector, as the
+    aggregate call of that range needs them: (index of the first overlapping bucket, offsets
+    relative to `first`, clipped to the range).  Empty buckets inside the range are kept (their
+    offsets repeat); stop <= first gives (0, [0])."""
+    if stop <= first:
+        return 0, [0]
+    B = len(bucket_off) - 1
+    b0 = 0
+    while b0 + 1 < B and bucket_off[b0 + 1] <= first:
+        b0 += 1
+    local = [0]
+    b = b0
+    while b < B and bucket_off[b] < stop:
+        local.append(min(bucket_off[b + 1], stop) - first)
+        b += 1
+    return b0, local
+
+
+class DitherAllReduce:
+    """sum_i D_nat^{p,s}(g_i) over the ranks of `group` with the master's work split as in
+    NaturalAllReduce.  Every rank codes its whole vector (per-bucket norms, level nibbles, sign
+    bits; the rounding stream is indexed by the position in the whole vector), the norms of all
+    ranks are all-gathered (W * B floats), the level and sign planes of a rank's range are
+    fetched from every rank (all-to-all or peer pointers), and nd_aggregate runs on the range
+    with the bucket table cut to it.  Buckets are never split between compressing ranks, so no
+    partial norms are exchanged; a bucket that straddles two ranges is simply decoded by both
+    with the same norm."""
+
+    def __init__(self, d: int, bucket_off, dist, group=None, *, p: int = 2, s: int = 8,
+                 seed: int = 0, transport: str = "collective", device=None, codec=None):
+        if transport not in ("collective", "peer"):
+            raise ValueError("transport must be 'collective' or 'peer'")
+        bucket_off = [int(v) for v in bucket_off]
+        if bucket_off[0] != 0 or bucket_off[-1] != d or any(
+                a > b for a, b in zip(bucket_off, bucket_off[1:])):
+            raise ValueError("bucket_off must ascend from 0 to d")
+        if codec is None:
+            from . import binding as codec
+        self.codec = codec
+        self.dist = dist
+        self.group = group
+        self.rank = dist.get_rank(group)
+        self.world = dist.get_world_size(group)
+        self.plan = ShardPlan(d, self.world)
+        self.p, self.s, self.seed = p, s, seed
+        self.transport = transport
+        self.device = torch.device(device if device is not None else "cuda")
+        self.B = len(bucket_off) - 1
+        P, S, dev = self.plan.padded, self.plan.shard, self.device
+        nbytes = P // 2 + P // 8                      # level nibbles, then sign bytes
+        self._symm = None
+        if transport == "peer":
+            import torch.distributed._symmetric_memory as symm_mem
+            self._send = symm_mem.empty(nbytes, dtype=torch.uint8, device=dev)
+            self._send.zero_()
+            self._symm = symm_mem.rendezvous(self._send, group if group is not None
+                                             else dist.group.WORLD)
+        else:
+            self._send = torch.zeros(nbytes, dtype=torch.uint8, device=dev)
+            self._recv = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        self.level_send = self._send[:P // 2]
+        self.sign_send = self._send[P // 2:]
+        self.off_dev = torch.tensor(bucket_off, dtype=torch.int64, device=dev)
+        self.norms_mine = torch.zeros(self.B, dtype=torch.float32, device=dev)
+        self.norms_all = torch.zeros(self.world * self.B, dtype=torch.float32, device=dev)
+        self.ws_bytes = int(codec.nd_workspace_bytes(d, self.B))
+        self.ws = torch.empty(max(self.ws_bytes, 16), dtype=torch.uint8, device=dev)
+        lo, hi = self.plan.owned(self.rank)
+        self.owned_len = hi - lo
+        self.b0, local = shard_bucket_table(bucket_off, lo, hi)
+        self.off_local = torch.tensor(local, dtype=torch.int64, device=dev)
+        self.B_local = len(local) - 1
+        self._out_shard = torch.zeros(S, dtype=torch.float32, device=dev)
+        self.out = torch.empty(P, dtype=torch.float32, device=dev)
+
+    def _planes_of_my_range(self):
+        P, S, W, r = self.plan.padded, self.plan.shard, self.world, self.rank
+        if self.transport == "peer":
+            self._symm.barrier(channel=0)
+            levels, signs = [], []
+            for i in range(W):
+                buf = self._symm.get_buffer(i, (P // 2 + P // 8,), torch.uint8)
+                levels.append(buf[r * (S // 2):(r + 1) * (S // 2)])
+                signs.append(buf[P // 2 + r * (S // 8):P // 2 + (r + 1) * (S // 8)])
+            return levels, signs
+        level_recv, sign_recv = self._recv[:P // 2], self._recv[P // 2:]
+        self.dist.all_to_all_single(level_recv, self.level_send, group=self.group)
+        self.dist.all_to_all_single(sign_recv, self.sign_send, group=self.group)
+        return ([level_recv[i * (S // 2):(i + 1) * (S // 2)] for i in range(W)],
+                [sign_recv[i * (S // 8):(i + 1) * (S // 8)] for i in range(W)])
+
+    def __call__(self, g: torch.Tensor) -> torch.Tensor:
+        plan, W, r, c = self.plan, self.world, self.rank, self.codec
+        if g.numel() != plan.d or g.dtype != torch.float32:
+            raise ValueError("expected an fp32 vector of %d entries" % plan.d)
+        c.nd_compress(g, plan.d, self.off_dev, self.B, self.p, self.s, self.seed, r,
+                      self.norms_mine, self.level_send, self.sign_send, self.ws, self.ws_bytes)
+        self.dist.all_gather_into_tensor(self.norms_all, self.norms_mine, group=self.group)
+        levels, signs = self._planes_of_my_range()
+        if self.owned_len > 0:
+            norms = [self.norms_all[i * self.B + self.b0:(i + 1) * self.B] for i in range(W)]
+            c.nd_aggregate(norms, levels, signs, W, self.owned_len, self.off_local, self.B_local,
+                           self.s, self._out_shard)
+        if self.transport == "peer":
+            self._symm.barrier(channel=1)
+        self.dist.all_gather_into_tensor(self.out, self._out_shard, group=self.group)
+        return self.out[:plan.d]

@@ -251,3 +251,151 @@ def test_cuda_codec_one_nccl_rank(transport):
             assert same_bits(out.cpu().numpy(), expected(d, 1, master_compress))
     finally:
         dist.destroy_process_group()
+
+
+# ---- D_nat over the sharded master -------------------------------------------------------------
+from paper_1905_10988_b200.sharded import DitherAllReduce, shard_bucket_table
+
+
+def bucket_table(d: int):
+    rng = np.random.default_rng(d)
+    cuts = sorted(set(int(v) for v in rng.integers(1, d, 7)) | {d // 2})
+    off = [0] + cuts + [d]
+    off.insert(3, off[3])                         # one empty bucket
+    return off
+
+
+def expected_dither(d: int, world: int, off, p: int, s: int) -> np.ndarray:
+    parts = [oracle.nd_compress(gradient(r, d), off, p, s, SEED, r) for r in range(world)]
+    return oracle.nd_aggregate([q[0] for q in parts], [q[1] for q in parts],
+                               [q[2] for q in parts], off, s, d)
+
+
+def test_shard_bucket_table_cuts_the_global_table():
+    off = [0, 100, 100, 3000, 5000]
+    assert shard_bucket_table(off, 0, 2048) == (0, [0, 100, 100, 2048])
+    assert shard_bucket_table(off, 2048, 4096) == (2, [0, 952, 2048])
+    assert shard_bucket_table(off, 4096, 5000) == (3, [0, 904])
+    assert shard_bucket_table(off, 5000, 5000) == (0, [0])
+    assert shard_bucket_table([0, 10], 0, 10) == (0, [0, 10])
+    # every coordinate of every range lands in the bucket the global table gives it
+    off = bucket_table(7000)
+    for world in (1, 2, 3, 5):
+        plan = ShardPlan(7000, world)
+        for r in range(world):
+            lo, hi = plan.owned(r)
+            b0, local = shard_bucket_table(off, lo, hi)
+            assert local[0] == 0 and local[-1] == hi - lo
+            for j in range(lo, hi, 97):
+                want = max(b for b in range(len(off) - 1) if off[b] <= j and j < off[b + 1])
+                got = b0 + max(k for k in range(len(local) - 1)
+                               if local[k] <= j - lo and j - lo < local[k + 1])
+                assert got == want
+
+
+class OracleDitherCodec:
+    @staticmethod
+    def nd_workspace_bytes(d, B):
+        return 16
+
+    @staticmethod
+    def nd_compress(x, d, off, B, p, s, seed, worker, norms, level, sign, ws, wsb):
+        nrm, lv, sg = oracle.nd_compress(x.numpy()[:d], off.numpy().astype(np.uint64), p, s, seed,
+                                         worker)
+        norms.numpy()[:] = nrm
+        level.numpy()[:lv.size] = lv
+        sign.numpy().view(np.uint32)[:sg.size] = sg
+
+    @staticmethod
+    def nd_aggregate(norms, levels, signs, n, d, off, B, s, out):
+        out.numpy()[:d] = oracle.nd_aggregate(
+            [a.numpy()[:B] for a in norms[:n]], [a.numpy()[:(d + 1) // 2] for a in levels[:n]],
+            [a.numpy().view(np.uint32) for a in signs[:n]], off.numpy().astype(np.uint64), s, d)
+
+
+def _gloo_dither_rank(rank, world, port, d, p, s, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ar = DitherAllReduce(d, bucket_table(d), dist, p=p, s=s, seed=SEED, device="cpu",
+                         codec=OracleDitherCodec)
+    g = torch.from_numpy(gradient(rank, d))
+    ar(g)
+    out.put((rank, ar(g).numpy().copy()))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world,d,p,s", [(2, 6000, 2, 8), (3, 5 * 1024 + 77, 0, 4), (2, 900, 1, 3)])
+def test_gloo_ranks_reproduce_the_single_master_dither_sum(world, d, p, s):
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_gloo_dither_rank, args=(r, world, port, d, p, s, out))
+             for r in range(world)]
+    for q in procs:
+        q.start()
+    got = [out.get(timeout=180) for _ in range(world)]
+    for q in procs:
+        q.join(timeout=180)
+        assert q.exitcode == 0
+    want = expected_dither(d, world, bucket_table(d), p, s)
+    for rank, res in got:
+        assert same_bits(res, want), "rank %d differs from the single-master result" % rank
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("world,d,p,s", [(4, 300_000, 0, 4), (3, 5 * 1024 + 1, 0, 8),
+                                         (4, 300_000, 2, 8)])
+def test_cuda_codec_dither_emulated_ranks(world, d, p, s):
+    import paper_1905_10988_b200 as nc
+    off = bucket_table(d)
+    fabric = ThreadFabric(world)
+    results, errors = [None] * world, []
+
+    def run(rank):
+        try:
+            fabric.local.rank = rank
+            torch.cuda.set_device(0)
+            ar = DitherAllReduce(d, off, fabric, p=p, s=s, seed=SEED)
+            g = torch.from_numpy(gradient(rank, d)).cuda()
+            ar(g)
+            out = ar(g)
+            torch.cuda.synchronize()
+            results[rank] = out.cpu().numpy()
+        except Exception as e:
+            errors.append(e)
+            fabric.barrier.abort()
+
+    threads = [threading.Thread(target=run, args=(r,)) for r in range(world)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=300)
+    assert not errors, errors
+    for r in range(1, world):
+        assert same_bits(results[r], results[0])
+    if p == 0:
+        # the max-norm is exact, so the codes and the sum are the oracle's bit for bit
+        assert same_bits(results[0], expected_dither(d, world, off, p, s))
+    else:
+        # p = 2: the norm may differ in the last place, so compare with one GPU aggregating the
+        # same W vectors as simulated workers (the same kernels, unsharded)
+        B = len(off) - 1
+        offd = torch.tensor(off, dtype=torch.int64, device="cuda")
+        u8 = dict(dtype=torch.uint8, device="cuda")
+        norms = [torch.zeros(B, dtype=torch.float32, device="cuda") for _ in range(world)]
+        levels = [torch.zeros(nc.nd_level_bytes(d), **u8) for _ in range(world)]
+        signs = [torch.zeros(nc.nc_sign_bytes(d), **u8) for _ in range(world)]
+        wsb = nc.nd_workspace_bytes(d, B)
+        ws = torch.empty(wsb, **u8)
+        for r in range(world):
+            nc.nd_compress(torch.from_numpy(gradient(r, d)).cuda(), d, offd, B, p, s, SEED, r,
+                           norms[r], levels[r], signs[r], ws, wsb)
+        single = torch.empty(d, dtype=torch.float32, device="cuda")
+        nc.nd_aggregate(norms, levels, signs, world, d, offd, B, s, single)
+        torch.cuda.synchronize()
+        assert same_bits(results[0], single.cpu().numpy())
+        want = expected_dither(d, world, off, p, s)
+        assert np.allclose(results[0], want, rtol=0, atol=1e-5 * np.abs(want).max() + 1e-30) or \
+            np.mean(results[0] != want) < 1e-3
