@@ -117,8 +117,9 @@ def _random_planes(rng, n, d, B, s):
     return norms, levels, signs
 
 
+# the last case has more tiles than are resident at once: its tail runs as 256-entry pieces
 @pytest.mark.parametrize("n,d,s", [(1, 999, 8), (3, 4096, 4), (8, 70001, 8), (16, 5000, 15),
-                                   (64, 2100, 1)])
+                                   (64, 2100, 1), (2, 5_000_333, 8)])
 def test_aggregate_and_decode_accumulate_are_bit_exact(n, d, s):
     rng = np.random.default_rng(n * 7 + d)
     off = workloads.small_bucket_table(d, seed=n + d)
