@@ -43,11 +43,17 @@ __device__ __forceinline__ uint32_t cnat_code8(uint32_t bits, uint32_t rnd) {
     return code8_from_exp(v >> 23, bits >> 31);
 }
 
-__device__ __forceinline__ long long restore8(uint32_t c) {
+// Restores byte K of a word of four codes: +1 or -1 as a 64-bit integer (high word = the sign
+// bit spread by an arithmetic shift, low word = that | 1), shifted left by the 7-bit field (the
+// zero flag makes the shift >= 64, which gives 0).
+template <int K>
+__device__ __forceinline__ long long restore8_of(uint32_t c4) {
+    const int hi = (int)(c4 << (24 - 8 * K)) >> 31;                      // 0 or -1
+    const unsigned long long one =
+        ((unsigned long long)(uint32_t)hi << 32) | (uint32_t)(hi | 1);   // +1 or -1
     unsigned long long v;
-    asm("shl.b64 %0, %1, %2;" : "=l"(v) : "l"(1ull), "r"(c & 0x7Fu));   // shift >= 64 gives 0
-    const long long m = -(long long)(c >> 7);                            // 0 or all ones
-    return ((long long)v ^ m) - m;
+    asm("shl.b64 %0, %1, %2;" : "=l"(v) : "l"(one), "r"((c4 >> (8 * K)) & 0x7Fu));
+    return (long long)v;
 }
 
 // grid: (ceil(tiles / warps per block), n workers)
@@ -109,37 +115,67 @@ __device__ __forceinline__ uint32_t cnat_code8_of_int(long long s, uint32_t rnd)
     return code8_from_exp(biased, sign_bit);
 }
 
+__device__ __forceinline__ void add_codes4(long long* acc, uint32_t c4) {
+    acc[0] += restore8_of<0>(c4);
+    acc[1] += restore8_of<1>(c4);
+    acc[2] += restore8_of<2>(c4);
+    acc[3] += restore8_of<3>(c4);
+}
+
 // kCompress = false: out32[j] = fl32(sum) * 2^-50;  true: out8[j] = code of C_nat(sum)
-// grid: ceil(d / (threads * 4))
+// A thread owns 16 consecutive entries (one 128-bit load per worker, the next worker's load in
+// flight while this one's codes are added).
+// grid: ceil(d / (threads * 16))
 template <bool kCompress>
 __global__ void __launch_bounds__(kBlockThreads)
 nc8_aggregate_kernel(const __grid_constant__ Code8Planes planes, const int n, const uint64_t d,
                      float* __restrict__ out32, uint8_t* __restrict__ out8, const uint32_t master,
                      const __grid_constant__ PhiloxKeys keys) {
-    const uint64_t q = (uint64_t)blockIdx.x * kBlockThreads + threadIdx.x;   // group of 4 entries
-    const uint64_t j0 = q * 4;
-    if (j0 >= round_up16(d)) return;
-    long long acc[4] = {0, 0, 0, 0};
-    if (j0 < d) {
-        for (int i = 0; i < n; ++i) {
-            // planes are padded to 16 bytes, so the 4-byte load stays inside the plane
-            const uint32_t c4 = ld_stream_u32(planes.code[i] + j0);
+    const uint64_t j0 = ((uint64_t)blockIdx.x * kBlockThreads + threadIdx.x) * 16;
+    if (j0 >= d) return;          // the plane's padding up to 16 bytes lies in the last group
+    long long acc[16];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) acc[c] += restore8((c4 >> (8 * c)) & 0xFFu);
-        }
+    for (int c = 0; c < 16; ++c) acc[c] = 0;
+    // planes are padded to 16 bytes, so the 16-byte load stays inside the plane
+    uint4 cur = ld_stream_u4(planes.code[0] + j0);
+    for (int i = 0; i < n; ++i) {
+        uint4 nxt = make_uint4(0u, 0u, 0u, 0u);
+        if (i + 1 < n) nxt = ld_stream_u4(planes.code[i + 1] + j0);
+        add_codes4(acc + 0, cur.x);
+        add_codes4(acc + 4, cur.y);
+        add_codes4(acc + 8, cur.z);
+        add_codes4(acc + 12, cur.w);
+        cur = nxt;
     }
     if (!kCompress) {
+        if (j0 + 16 <= d) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (j0 + c < d) out32[j0 + c] = __fmul_rn(__ll2float_rn(acc[c]), 8.8817841970012523e-16f);
+            for (int g = 0; g < 4; ++g) {
+                float4 o;
+                o.x = __fmul_rn(__ll2float_rn(acc[4 * g + 0]), 8.8817841970012523e-16f);
+                o.y = __fmul_rn(__ll2float_rn(acc[4 * g + 1]), 8.8817841970012523e-16f);
+                o.z = __fmul_rn(__ll2float_rn(acc[4 * g + 2]), 8.8817841970012523e-16f);
+                o.w = __fmul_rn(__ll2float_rn(acc[4 * g + 3]), 8.8817841970012523e-16f);
+                __stcs(reinterpret_cast<float4*>(out32 + j0) + g, o);
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+                if (j0 + c < d)
+                    out32[j0 + c] = __fmul_rn(__ll2float_rn(acc[c]), 8.8817841970012523e-16f);
+        }
     } else {
-        uint32_t rnd[4] = {0u, 0u, 0u, 0u};
-        if (j0 < d) stream_words4(q, master, kDomainCnat, keys, rnd);
-        uint32_t c4 = 0;
+        uint32_t c4[4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (j0 + c < d) c4 |= cnat_code8_of_int(acc[c], rnd[c]) << (8 * c);
-        *reinterpret_cast<uint32_t*>(out8 + j0) = c4;          // zero padding past d
+        for (int g = 0; g < 4; ++g) {
+            uint32_t rnd[4];
+            stream_words4((j0 >> 2) + g, master, kDomainCnat, keys, rnd);
+            c4[g] = 0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (j0 + 4 * g + c < d) c4[g] |= cnat_code8_of_int(acc[4 * g + c], rnd[c]) << (8 * c);
+        }
+        st_stream_u4(out8 + j0, make_uint4(c4[0], c4[1], c4[2], c4[3]));   // zero padding past d
     }
 }
 
@@ -193,7 +229,7 @@ nc_status nc8_aggregate(const uint8_t* const* codes, int n, size_t d, float* out
     Code8Planes planes;
     const nc_status st = nc8_planes(codes, n, &planes);
     if (st != NC_OK) return st;
-    const uint64_t groups = round_up16(d) / 4;
+    const uint64_t groups = round_up16(d) / 16;
     const unsigned grid = (unsigned)((groups + kBlockThreads - 1) / kBlockThreads);
     const PhiloxKeys keys = make_philox_keys(0);
     nc8_aggregate_kernel<false><<<grid, kBlockThreads, 0, stream>>>(planes, n, (uint64_t)d, out,
@@ -210,7 +246,7 @@ nc_status nc8_aggregate_compress(const uint8_t* const* codes, int n, size_t d, u
     Code8Planes planes;
     const nc_status st = nc8_planes(codes, n, &planes);
     if (st != NC_OK) return st;
-    const uint64_t groups = round_up16(d) / 4;
+    const uint64_t groups = round_up16(d) / 16;
     const unsigned grid = (unsigned)((groups + kBlockThreads - 1) / kBlockThreads);
     const PhiloxKeys keys = make_philox_keys(seed);
     nc8_aggregate_kernel<true><<<grid, kBlockThreads, 0, stream>>>(planes, n, (uint64_t)d, nullptr,
