@@ -445,6 +445,20 @@ def nc_compress_bf16_r8(x16, seed: int, worker: int):
     return exp, sign
 
 
+_nc_compress_f16_r16 = _sig("orc_nc_compress_f16_r16", None, _u16p, C.c_uint64, C.c_uint64,
+                            C.c_uint32, _u8p, _u32p)
+
+
+def nc_compress_f16_r16(x16, seed: int, worker: int):
+    """C_nat of binary16 bit patterns with 10-bit thresholds drawn from one stream half-word per
+    entry (domain 5): exponent bytes, sign words."""
+    x16 = _arr(x16, np.uint16)
+    exp = np.zeros(x16.size, np.uint8)
+    sign = np.zeros((x16.size + 31) // 32, np.uint32)
+    _nc_compress_f16_r16(_p(x16, _u16p), x16.size, seed, worker, _p(exp, _u8p), _p(sign, _u32p))
+    return exp, sign
+
+
 def values_of_16bit(x16, dtype: int) -> np.ndarray:
     x16 = _arr(x16, np.uint16)
     out = np.zeros(x16.size, np.float32)

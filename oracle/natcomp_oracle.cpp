@@ -789,6 +789,25 @@ void orc_nc_compress_bf16_r8(const uint16_t* x, uint64_t d, uint64_t seed, uint3
     }
 }
 
+// C_nat (Def. 1) of binary16 inputs with a short random threshold.  A binary16 value has 10
+// mantissa bits (a subnormal has fewer), so its up-probability m = 1 - p(t) is a multiple of
+// 1/1024 and 10 random bits decide the rounding exactly: "up" iff r10 < m * 1024.  The draw is
+// r10 = low 10 bits of half-word (j mod 2) of the stream word with index j / 2 in domain 5 (one
+// generator block of four words serves 8 entries).  Written as the binary32 rule with
+// r23 = r10 * 2^13: the threshold m * 2^23 of a binary16 value is a multiple of 2^13.
+void orc_nc_compress_f16_r16(const uint16_t* x, uint64_t d, uint64_t seed, uint32_t worker,
+                             uint8_t* exp, uint32_t* sign) {
+    std::memset(sign, 0, (size_t)((d + 31) / 32) * 4);
+    for (uint64_t j = 0; j < d; ++j) {
+        const float t = value_of_16bit(x[j], 2);
+        const uint32_t word = stream_word(seed, worker, 5u, j / 2);
+        const uint32_t r10 = (word >> (16 * (j % 2))) & 0x3FFu;
+        uint32_t sb;
+        cnat_code(cnat_value(t, r10 << 13), &exp[j], &sb);
+        sign[j / 32] |= sb << (j % 32);
+    }
+}
+
 void orc_values_of_16bit(const uint16_t* x, int dtype, uint64_t d, float* out) {
     for (uint64_t j = 0; j < d; ++j) out[j] = value_of_16bit(x[j], dtype);
 }

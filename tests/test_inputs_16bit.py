@@ -211,3 +211,92 @@ def test_gpu_bf16_short_threshold_full_size_batch():
         e_ref, s_ref = oracle.nc_compress_bf16_r8(h, 0, w)
         assert np.array_equal(es[w].cpu().numpy()[:d], e_ref)
         assert np.array_equal(ss[w].cpu().numpy().view(np.uint32)[:s_ref.size], s_ref)
+
+
+# ---- binary16 with 10-bit thresholds: one stream half-word per entry ---------------------------
+def test_f16_short_threshold_rounds_up_in_exactly_m_of_1024_draws():
+    # every finite binary16 pattern against every 10-bit draw: the draws that round up number
+    # m * 1024 (the mantissa field of a normal value, the normalised fraction of a subnormal), and
+    # the mean over the draws is the value itself
+    h = _all_patterns()
+    t = oracle.values_of_16bit(h, F16)
+    e_field = (h >> 10) & 0x1F
+    m_field = (h & 0x3FF).astype(np.int64)
+    finite = e_field < 31
+    want_ups = m_field.copy()
+    sub = (e_field == 0) & (m_field > 0)
+    lead = np.floor(np.log2(np.maximum(m_field, 1))).astype(np.int64)
+    want_ups[sub] = ((m_field[sub] - (1 << lead[sub])) << (10 - lead[sub]))
+    ups = np.zeros(h.size, np.int64)
+    total = np.zeros(h.size, np.float64)
+    lo_e, _ = oracle.cnat_codes(t, np.full(h.size, 1023 << 13, np.uint32))   # never up
+    for r10 in range(1024):
+        r23 = np.full(h.size, r10 << 13, np.uint32)
+        e, _ = oracle.cnat_codes(t, r23)
+        ups += (e != lo_e)
+        total += np.where(finite, oracle.cnat_values(t, r23).astype(np.float64), 0.0)
+    assert np.array_equal(ups[finite], want_ups[finite])
+    assert np.all(ups[~finite] == 0)
+    assert np.array_equal(total / 1024.0, np.where(finite, t.astype(np.float64), 0.0))
+
+
+def test_f16_short_threshold_stream_mapping_and_frequency():
+    rng = np.random.default_rng(12)
+    d = 4099
+    h = rng.integers(0, 1 << 16, d).astype(np.uint16)
+    seed, worker = 0x1234567, 4
+    words = oracle.stream_words(seed, worker, 5, 0, (d + 1) // 2)
+    j = np.arange(d)
+    r10 = (words[j // 2] >> (16 * (j % 2)).astype(np.uint32)) & 0x3FF
+    e_want, s_want = oracle.cnat_codes(oracle.values_of_16bit(h, F16), (r10 << 13).astype(np.uint32))
+    e, s = oracle.nc_compress_f16_r16(h, seed, worker)
+    assert np.array_equal(e, e_want)
+    bits = (s[j // 32] >> (j % 32).astype(np.uint32)) & 1
+    assert np.array_equal(bits.astype(np.uint8), s_want)
+    n = 1 << 20
+    e, _ = oracle.nc_compress_f16_r16(np.full(n, (15 << 10) | 300, np.uint16), 3, 1)   # 1 + 300/1024
+    p = 300 / 1024
+    assert abs((e == 128).mean() - p) < 5 * np.sqrt(p * (1 - p) / n)
+    assert set(np.unique(e)) == {127, 128}
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d", [1, 5, 31, 1024, 4097, 65536, 6 * 1024 + 515, (1 << 20) + 33])
+def test_gpu_f16_short_threshold_matches_oracle(d):
+    import torch
+    import paper_1905_10988_b200 as nc
+    from gpu_util import Guarded, check_nc_planes, dev
+    rng = np.random.default_rng(d + 1)
+    if d == 65536:
+        h = _all_patterns()                       # every pattern: subnormals, inf, NaN
+    else:
+        x = (rng.standard_normal(d) * 10.0 ** rng.uniform(-7, 3, d)).astype(np.float32)
+        h = x.astype(np.float16).view(np.uint16)
+    e = Guarded(nc.nc_exp_bytes(d))
+    s = Guarded(nc.nc_sign_bytes(d))
+    nc.nc_compress_f16_r16(dev(h.view(np.int16)), d, 7, 3, e.buf, s.buf)
+    torch.cuda.synchronize()
+    e_ref, s_ref = oracle.nc_compress_f16_r16(h, 7, 3)
+    check_nc_planes(e, s, d, e_ref, s_ref)
+
+
+@pytest.mark.gpu
+def test_gpu_f16_short_threshold_batch():
+    import torch
+    import paper_1905_10988_b200 as nc
+    from gpu_util import dev
+    rng = np.random.default_rng(6)
+    n, d = 3, 200_003
+    hs = [rng.standard_normal(d).astype(np.float16).view(np.uint16) for _ in range(n)]
+    xd = [dev(h.view(np.int16)) for h in hs]
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    es = [torch.empty(nc.nc_exp_bytes(d), **u8) for _ in range(n)]
+    ss = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
+    nc.nc_compress_f16_r16_batch(xd, d, 1, [5, 6, 7], es, ss, n)
+    torch.cuda.synchronize()
+    for i, h in enumerate(hs):
+        e_ref, s_ref = oracle.nc_compress_f16_r16(h, 1, 5 + i)
+        assert np.array_equal(es[i].cpu().numpy()[:d], e_ref)
+        assert np.array_equal(ss[i].cpu().numpy().view(np.uint32)[:s_ref.size], s_ref)
+    with pytest.raises(nc.NatcompError):
+        nc.nc_compress_f16_r16(xd[0][1:], d - 1, 1, 0, es[0], ss[0])       # misaligned input
