@@ -26,7 +26,8 @@
  *   key = (low32(seed), high32(seed)), counter = (low32(q), high32(q), worker, domain),
  *   q = j / 4; element j of a worker's vector uses output word j mod 4, low 23 bits.
  *   domain 0: C_nat, 1: D_nat rounding, 2: sparsifier selection, 3: low bits of binary64
- *   thresholds, 4: byte-wide draws of nc_compress_bf16_r8.
+ *   thresholds, 4: byte-wide draws of nc_compress_bf16_r8, 5: half-word draws of
+ *   nc_compress_f16_r16.
  * The stream depends on (seed, worker, j) only, so outputs are reproducible and
  * independent of launch geometry.
  *
@@ -333,6 +334,18 @@ nc_status nc_compress_typed_batch(const void* const* xs, int dtype, size_t d, ui
 nc_status nc_compress_bf16_r8(const void* x, size_t d, uint64_t seed, uint32_t worker,
                               uint8_t* exp, uint32_t* sign, cudaStream_t stream);
 nc_status nc_compress_bf16_r8_batch(const void* const* xs, size_t d, uint64_t seed,
+                                    const uint32_t* workers, uint8_t* const* exps,
+                                    uint32_t* const* signs, int n, cudaStream_t stream);
+
+/* binary16 inputs with 10-bit thresholds (Def. 1: a binary16 value has at most 10 mantissa bits,
+ * so its up-probability is a multiple of 1/1024).  Entry j draws the low 10 bits of half-word
+ * (j mod 2) of stream word j / 2 of domain 5 and is rounded up iff draw / 1024 is below its
+ * mantissa fraction (for a subnormal: the fraction above its leading bit): one generator block
+ * serves 8 entries.  Same law as nc_compress_typed with NC_DTYPE_F16, a different draw.
+ * x: d binary16 bit patterns, 32-byte aligned.  Planes, edge cases and errors as for nc_compress. */
+nc_status nc_compress_f16_r16(const void* x, size_t d, uint64_t seed, uint32_t worker,
+                              uint8_t* exp, uint32_t* sign, cudaStream_t stream);
+nc_status nc_compress_f16_r16_batch(const void* const* xs, size_t d, uint64_t seed,
                                     const uint32_t* workers, uint8_t* const* exps,
                                     uint32_t* const* signs, int n, cudaStream_t stream);
 

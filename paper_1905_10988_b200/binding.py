@@ -42,7 +42,7 @@ EXPORTS = (
     "nc_compress_typed_batch", "nc64_compress", "nc64_compress_batch", "nc64_aggregate",
     "nd_sparse_regen_workspace_bytes", "nd_sparse_regen_decode_accumulate",
     "nd_sparse_compact_aggregate", "nc_aggregate_compress_shard", "nc_compress_bf16_r8",
-    "nc_compress_bf16_r8_batch",
+    "nc_compress_bf16_r8_batch", "nc_compress_f16_r16", "nc_compress_f16_r16_batch",
 )
 
 
@@ -165,6 +165,25 @@ def nc_compress_bf16_r8_batch(xs, d, seed, workers, exps, signs, n, stream=None)
     w = (C.c_uint32 * n)(*[int(v) for v in workers])
     _check("nc_compress_bf16_r8_batch",
            _nc_compress_bf16_r8_batch(_ptrs(xs), d, seed, w, _ptrs(exps), _ptrs(signs), n,
+                                      _stream(stream)))
+
+
+_nc_compress_f16_r16 = _sig("nc_compress_f16_r16", C.c_int, _vp, _sz, C.c_uint64, C.c_uint32, _vp,
+                            _vp, _vp)
+_nc_compress_f16_r16_batch = _sig("nc_compress_f16_r16_batch", C.c_int, C.POINTER(_vp), _sz,
+                                  C.c_uint64, C.POINTER(C.c_uint32), C.POINTER(_vp),
+                                  C.POINTER(_vp), C.c_int, _vp)
+
+
+def nc_compress_f16_r16(x, d, seed, worker, exp, sign, stream=None) -> None:
+    _check("nc_compress_f16_r16",
+           _nc_compress_f16_r16(_ptr(x), d, seed, worker, _ptr(exp), _ptr(sign), _stream(stream)))
+
+
+def nc_compress_f16_r16_batch(xs, d, seed, workers, exps, signs, n, stream=None) -> None:
+    w = (C.c_uint32 * n)(*[int(v) for v in workers])
+    _check("nc_compress_f16_r16_batch",
+           _nc_compress_f16_r16_batch(_ptrs(xs), d, seed, w, _ptrs(exps), _ptrs(signs), n,
                                       _stream(stream)))
 
 

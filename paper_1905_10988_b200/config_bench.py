@@ -86,6 +86,10 @@ def run_cnat(config, n, d, make_vector, iters, peak, with_sum=True):
             _report(config, "nc_compress_bf16_r8_batch (bf16 inputs, 7-bit thresholds)", m, b,
                     n * d, n * d * 3.125, peak,
                     {"note": "one generator block per 16 entries: memory-bound"})
+        if code == nc.DTYPE_F16:
+            m, b = _time(lambda: nc.nc_compress_f16_r16_batch(xh, d, 0, workers, es, ss, n), iters)
+            _report(config, "nc_compress_f16_r16_batch (f16 inputs, 10-bit thresholds)", m, b,
+                    n * d, n * d * 3.125, peak, {"note": "one generator block per 8 entries"})
         del xh
     if with_sum:
         m, b = _time(lambda: nc.nc_sum_fp32(xs, n, d, out), iters)

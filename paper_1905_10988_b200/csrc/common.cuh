@@ -72,6 +72,16 @@ __device__ __forceinline__ void st_stream_u32(void* p, uint32_t v) {
     __stcs(reinterpret_cast<unsigned int*>(p), v);
 }
 
+// 4x4 transpose of bytes across each aligned group of 4 lanes: lane i holds bytes b[i][t]
+// (t = 0..3) -> lane t holds bytes b[i][t] (i = 0..3, byte i).
+__device__ __forceinline__ uint32_t transpose_bytes_4x4(uint32_t v, int lane) {
+    uint32_t t = __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+    v = __byte_perm(v, t, (lane & 2) ? 0x3276 : 0x5410);
+    t = __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+    v = __byte_perm(v, t, (lane & 1) ? 0x3715 : 0x6240);
+    return v;
+}
+
 // 8x8 transpose of 4-bit fields across each aligned group of 8 lanes.
 // In: lane i of a group holds nibbles n[i][k], k = 0..7 (nibble k in bits 4k..4k+3).
 // Out: lane k of the group holds nibbles n[i][k], i = 0..7 (nibble i in bits 4i..4i+3).

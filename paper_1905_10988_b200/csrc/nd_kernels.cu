@@ -53,16 +53,6 @@ __device__ __forceinline__ void st_stream_v8(void* p, const V8& r) {
                  : "memory");
 }
 
-// 4x4 transpose of bytes across each aligned group of 4 lanes: lane i holds bytes b[i][t]
-// (t = 0..3) -> lane t holds bytes b[i][t] (i = 0..3, byte i).
-__device__ __forceinline__ uint32_t transpose_bytes_4x4(uint32_t v, int lane) {
-    uint32_t t = __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-    v = __byte_perm(v, t, (lane & 2) ? 0x3276 : 0x5410);
-    t = __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-    v = __byte_perm(v, t, (lane & 1) ? 0x3715 : 0x6240);
-    return v;
-}
-
 // largest b in [0, B-1] with off[b] <= pos (pos < off[B]); skips empty buckets by construction
 __device__ __forceinline__ int find_bucket(const uint64_t* __restrict__ off, int B, uint64_t pos) {
     int lo = 0, hi = B;   // invariant: off[lo] <= pos < off[hi]
