@@ -32,29 +32,42 @@ def e2e_host_steps(nc, hp, steps: int) -> dict:
     gradient vectors host -> device through the C ABI, runs the whole path, and copies the
     three aggregates back to pinned host memory.  Returns ms per step and bytes moved.
 
-    Two streams: the upload and the kernels of step i run on one, the download of its results on
-    the other, so that the download of step i overlaps the upload of step i + 1 (PCIe is full
-    duplex).  The kernels of step i + 1 wait until the download of step i has read the outputs.
-    The timed region runs from the first upload to the end of the last download."""
+    Three streams and two sets of device input buffers: the upload of step i + 1 runs while the
+    kernels of step i work on the other set and while the results of step i (and i - 1) go back
+    (PCIe is full duplex).  An upload waits until the kernels that last read its buffer set are
+    done, the kernels of a step wait for their upload and for the download of the previous
+    results.  The timed region runs from the first upload to the end of the last download."""
     n, d = hp.n, hp.d
     host_x = [torch.empty(d, dtype=torch.float32, pin_memory=True) for _ in range(n)]
     for w in range(n):
         host_x[w].copy_(hp.x[w])
     host_out = [torch.empty(d, dtype=torch.float32, pin_memory=True) for _ in range(3)]
+    sets = [hp.x, [torch.empty_like(t) for t in hp.x]]
     torch.cuda.synchronize()
+    s_up = torch.cuda.Stream()
     s_main = torch.cuda.Stream()
     s_out = torch.cuda.Stream()
-    state = {"downloaded": None}
+    state = {"downloaded": None, "computed": [None, None], "i": 0}
 
     def one_step():
-        with torch.cuda.stream(s_main):
+        b = state["i"] & 1
+        state["i"] += 1
+        with torch.cuda.stream(s_up):
+            if state["computed"][b] is not None:
+                s_up.wait_event(state["computed"][b])       # the set's last readers are done
             for w in range(n):
-                nc.nc_copy_to_device(hp.x[w], host_x[w], 4 * d)
+                nc.nc_copy_to_device(sets[b][w], host_x[w], 4 * d)
+            uploaded = torch.cuda.Event()
+            uploaded.record(s_up)
+        with torch.cuda.stream(s_main):
+            s_main.wait_event(uploaded)
             if state["downloaded"] is not None:
                 s_main.wait_event(state["downloaded"])      # outputs may be overwritten now
+            hp.x = sets[b]
             hp.step()
             computed = torch.cuda.Event()
             computed.record(s_main)
+            state["computed"][b] = computed
         with torch.cuda.stream(s_out):
             s_out.wait_event(computed)
             for dst, src in zip(host_out, (hp.out_nc, hp.out_nd, hp.out_sp)):
@@ -62,15 +75,18 @@ def e2e_host_steps(nc, hp, steps: int) -> dict:
             state["downloaded"] = torch.cuda.Event()
             state["downloaded"].record(s_out)
 
-    one_step()                                   # warm-up
+    one_step()                                   # warm-up (both buffer sets)
+    one_step()
     torch.cuda.synchronize()
     e0 = torch.cuda.Event(enable_timing=True)
     e1 = torch.cuda.Event(enable_timing=True)
-    e0.record(s_main)
+    e0.record(s_up)
     for _ in range(steps):
         one_step()
     e1.record(s_out)
     torch.cuda.synchronize()
+    hp.x = sets[0]
     ms = e0.elapsed_time(e1) / steps
     return {"ms_per_step": ms, "h2d_bytes_per_step": 4 * d * n, "d2h_bytes_per_step": 4 * d * 3,
-            "steps": steps, "overlap": "download of step i overlaps upload of step i+1"}
+            "steps": steps,
+            "overlap": "upload of step i+1 overlaps the kernels and the download of step i"}
