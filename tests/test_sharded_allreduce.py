@@ -249,6 +249,12 @@ def test_cuda_codec_one_nccl_rank(transport):
             out = ar(torch.from_numpy(gradient(0, d)).cuda())
             torch.cuda.synchronize()
             assert same_bits(out.cpu().numpy(), expected(d, 1, master_compress))
+        off = bucket_table(d)
+        ad = DitherAllReduce(d, off, dist, p=0, s=4, seed=SEED, transport=transport,
+                             device="cuda:0")
+        out = ad(torch.from_numpy(gradient(0, d)).cuda())
+        torch.cuda.synchronize()
+        assert same_bits(out.cpu().numpy(), expected_dither(d, 1, off, 0, 4))
     finally:
         dist.destroy_process_group()
 
