@@ -32,6 +32,7 @@ def test_bench_line_has_every_contract_key():
     assert e2e["h2d_bytes_per_step"] == 8 * 4 * 25_557_032
     assert e2e["d2h_bytes_per_step"] == 3 * 4 * 25_557_032
     assert 0 < e2e["value"] < j["value"]                      # host copies are inside its region
+    assert e2e["results_arrived"] is True
     roof = j["roofline"]
     assert roof["bound"] == "hbm" and roof["unit"] == "GB/s"
     assert abs(roof["frac"] - roof["achieved"] / roof["peak"]) < 1e-3
