@@ -469,6 +469,27 @@ def main():
     concurrent = {"ms_per_step": conc_ms, "streams": len(streams), "steps": k_conc,
                   "value": world * units_per_step / (conc_ms * 1e-3) / 1e9, "unit": UNIT}
 
+    # the same single-stream step replayed from a CUDA graph (no launch gaps); reported beside
+    # `value` as well
+    graph_stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(graph_stream):
+        with torch.cuda.graph(graph, stream=graph_stream):
+            hp.step()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    g0 = torch.cuda.Event(enable_timing=True)
+    g1 = torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for _ in range(k_conc):
+        graph.replay()
+    g1.record()
+    torch.cuda.synchronize()
+    graph_ms = timing.max_over_ranks(g0.elapsed_time(g1) / k_conc, dist, device)
+    graph_replay = {"ms_per_step": graph_ms, "steps": k_conc,
+                    "value": world * units_per_step / (graph_ms * 1e-3) / 1e9, "unit": UNIT}
+
     # end to end: host buffers -> device -> whole path -> aggregates back on the host
     e2e = None
     if args.e2e_steps > 0:
@@ -498,6 +519,7 @@ def main():
                        "multi_gpu": "replicas only"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": hp.launches_per_step * args.steps,
             "concurrent_streams": concurrent,
+            "graph_replay": graph_replay,
             "roofline": roofline, "cpu_baseline": cpu, "kernels": kernels,
         }
         print(json.dumps(line))
