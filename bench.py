@@ -471,24 +471,38 @@ def main():
 
     # the same single-stream step replayed from a CUDA graph (no launch gaps); reported beside
     # `value` as well
-    graph_stream = torch.cuda.Stream()
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.stream(graph_stream):
-        with torch.cuda.graph(graph, stream=graph_stream):
-            hp.step()
-    for _ in range(3):
-        graph.replay()
-    torch.cuda.synchronize()
-    g0 = torch.cuda.Event(enable_timing=True)
-    g1 = torch.cuda.Event(enable_timing=True)
-    g0.record()
-    for _ in range(k_conc):
-        graph.replay()
-    g1.record()
-    torch.cuda.synchronize()
-    graph_ms = timing.max_over_ranks(g0.elapsed_time(g1) / k_conc, dist, device)
-    graph_replay = {"ms_per_step": graph_ms, "steps": k_conc,
-                    "value": world * units_per_step / (graph_ms * 1e-3) / 1e9, "unit": UNIT}
+    graph_replay = None
+    try:
+        graph_stream = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(graph_stream):
+            # thread-local capture mode: a CUDA call from another thread of this process (a
+            # communication library's watchdog, the clock sampler) must not break the capture
+            with torch.cuda.graph(graph, stream=graph_stream, capture_error_mode="thread_local"):
+                hp.step()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        g0 = torch.cuda.Event(enable_timing=True)
+        g1 = torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(k_conc):
+            graph.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        graph_ms = g0.elapsed_time(g1) / k_conc
+    except RuntimeError as exc:               # the leg is optional: report why it is missing
+        graph_ms = None
+        graph_error = str(exc).splitlines()[0][:200]
+    if dist is not None:
+        # every rank reaches the reduction, also one whose capture failed
+        worst = timing.max_over_ranks(graph_ms if graph_ms is not None else -1.0, dist, device)
+        graph_ms = None if graph_ms is None else worst
+    if graph_ms is not None and graph_ms > 0:
+        graph_replay = {"ms_per_step": graph_ms, "steps": k_conc,
+                        "value": world * units_per_step / (graph_ms * 1e-3) / 1e9, "unit": UNIT}
+    elif graph_ms is None:
+        graph_replay = {"unavailable": locals().get("graph_error", "capture failed on a rank")}
 
     # end to end: host buffers -> device -> whole path -> aggregates back on the host
     e2e = None
