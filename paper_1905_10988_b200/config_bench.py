@@ -22,7 +22,14 @@ from . import workloads
 HBM_PEAK_FALLBACK = 6650.0
 
 
+REPS = 1     # calls between one pair of events (--reps)
+
+
 def _time(fn, iters, warmup=3):
+    """Median and best device time of one call, in ms.  With --reps > 1 that many calls are queued
+    back to back between two events, so that the host's marshalling of a call overlaps the
+    previous call's kernels (a lone call between two events counts about 10 us of idle GPU as
+    its own)."""
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
@@ -31,10 +38,11 @@ def _time(fn, iters, warmup=3):
         e0 = torch.cuda.Event(enable_timing=True)
         e1 = torch.cuda.Event(enable_timing=True)
         e0.record()
-        fn()
+        for _ in range(REPS):
+            fn()
         e1.record()
         torch.cuda.synchronize()
-        times.append(e0.elapsed_time(e1))
+        times.append(e0.elapsed_time(e1) / REPS)
     return statistics.median(times), min(times)
 
 
@@ -231,11 +239,15 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--peak-gbs", type=float, default=HBM_PEAK_FALLBACK,
                     help="HBM bandwidth the fractions are quoted against")
+    ap.add_argument("--reps", type=int, default=1,
+                    help="calls queued back to back between one pair of events")
     ap.add_argument("--workers", type=int, default=0,
                     help="override the number of simulated workers (smaller cases for profiling)")
     ap.add_argument("--log2-d", type=int, default=0,
                     help="override the vector length of c5 with 2^LOG2_D")
     args = ap.parse_args()
+    global REPS
+    REPS = max(1, args.reps)
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device")
     peak = args.peak_gbs
