@@ -631,24 +631,36 @@ sparse_emit_compact_kernel(const __grid_constant__ SparseBatch batch, const uint
     flush(cnt);
 }
 
-// one warp per 32 listed entries; grid: (ceil(groups / warps per block), n workers)
+// one warp per kPackGroups groups of 32 listed entries (the codes of all its groups are loaded
+// before the ballots); grid: (ceil(groups / (kPackGroups * warps per block)), n workers)
+constexpr int kPackGroups = 8;
+
 __global__ void __launch_bounds__(kBlockThreads)
 sparse_pack_planes_kernel(const __grid_constant__ SparseBatch batch, const uint64_t d,
                           const uint64_t cap, const int s, char* __restrict__ ws_all,
                           const uint64_t ws_stride) {
     const int lane = threadIdx.x & 31;
     const SparseWorkspace ws = sparse_ws_carve(ws_all + (uint64_t)blockIdx.y * ws_stride, d);
-    const uint64_t group = (uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint64_t first =
+        ((uint64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5)) * kPackGroups;
     const uint64_t groups = (cap + 31) / 32;
-    if (group >= groups) return;
+    if (first >= groups) return;
     const uint64_t total = min((uint64_t)*batch.count[blockIdx.y], cap);
-    const uint64_t k = group * 32 + lane;
-    const uint32_t code = (k < total) ? ws.tmp_codes[k] : 0u;
+    uint32_t code[kPackGroups];
+#pragma unroll
+    for (int g = 0; g < kPackGroups; ++g) {
+        const uint64_t k = (first + g) * 32 + lane;
+        code[g] = (k < total) ? ws.tmp_codes[k] : 0u;
+    }
     const int planes = code_value_bits(s) + 1;
-    uint32_t* out = reinterpret_cast<uint32_t*>(batch.codes[blockIdx.y]) + group * planes;
-    for (int b = 0; b < planes; ++b) {
-        const uint32_t wv = __ballot_sync(0xFFFFFFFFu, (code >> b) & 1u);
-        if (lane == 0) out[b] = wv;
+#pragma unroll
+    for (int g = 0; g < kPackGroups; ++g) {
+        if (first + g >= groups) break;
+        uint32_t* out = reinterpret_cast<uint32_t*>(batch.codes[blockIdx.y]) + (first + g) * planes;
+        for (int b = 0; b < planes; ++b) {
+            const uint32_t wv = __ballot_sync(0xFFFFFFFFu, (code[g] >> b) & 1u);
+            if (lane == 0) out[b] = wv;
+        }
     }
 }
 
@@ -693,7 +705,8 @@ void sparse_compact_finish(const SparseBatch& batch, uint64_t d, float scale, in
     sparse_emit_compact_kernel<<<ggrid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, cap,
                                                                     ws, ws_stride);
     const uint64_t groups = (cap + 31) / 32;
-    const dim3 pgrid((unsigned)((groups + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
+    const uint64_t per_block = (uint64_t)kWarpsPerBlock * kPackGroups;
+    const dim3 pgrid((unsigned)((groups + per_block - 1) / per_block), (unsigned)n);
     sparse_pack_planes_kernel<<<pgrid, kBlockThreads, 0, stream>>>(batch, d, cap, s, ws,
                                                                    ws_stride);
 }
