@@ -405,3 +405,20 @@ def test_cuda_codec_dither_emulated_ranks(world, d, p, s):
         want = expected_dither(d, world, off, p, s)
         assert np.allclose(results[0], want, rtol=0, atol=1e-5 * np.abs(want).max() + 1e-30) or \
             np.mean(results[0] != want) < 1e-3
+
+
+@pytest.mark.gpu
+def test_allreduce_bench_runs_with_one_rank():
+    import json
+    import subprocess
+    env = dict(os.environ, RANK="0", WORLD_SIZE="1", LOCAL_RANK="0", MASTER_ADDR="127.0.0.1",
+               MASTER_PORT=str(_free_port()))
+    r = subprocess.run([sys.executable, "-m", "paper_1905_10988_b200.allreduce_bench",
+                        "--log2-d", "20", "--iters", "2"], env=env, cwd=ROOT,
+                       capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert [l["variant"] for l in lines] == ["nccl_allreduce_fp32", "natural_allreduce",
+                                             "natural_allreduce_master_compress",
+                                             "dither_allreduce_p2_s8"]
+    assert all(l["ms"] > 0 and l["n_gpus"] == 1 for l in lines)
