@@ -95,8 +95,8 @@ nc_status nc_compress_batch(const float* const* xs, size_t d, uint64_t seed,
                             const uint32_t* workers, uint8_t* const* exps,
                             uint32_t* const* signs, int n, cudaStream_t stream);
 
-/* The paper's deterministic control variant (experimental set-up appendix: "deterministic
- * rounding to the nearest power of 2", used to expose the cost of sampling): the same 9-bit code,
+/* The paper's deterministic control variant (experimental set-up appendix; there it exposes the
+ * cost of sampling): the same 9-bit code,
  * but every entry goes to the nearer of its two neighbouring powers of two (the midpoint
  * 1.5 * 2^k goes up), with no random numbers.  Biased.  Edge cases as for nc_compress. */
 nc_status nc_compress_nearest(const float* x, size_t d, uint8_t* exp, uint32_t* sign,
@@ -148,12 +148,18 @@ nc_status nc_sum_fp32(const float* const* xs, int n, size_t d, float* out, cudaS
  * workspace: nd_workspace_bytes(d, B) bytes of scratch (contents undefined afterwards).
  * Arithmetic: norm accumulated in binary64 from per-thread binary32 partial sums, rounded once;
  * y = fl32(|x| * fl32(1 / norm)); above 2^(1-s) the up-probability is the mantissa fraction of y
- * (as in C_nat), below it is y * 2^(s-1), both at 2^-23 resolution.  A bucket whose norm is 0,
- * subnormal or not finite gets level code 0 everywhere (its norm is still stored).
- * Given the stored norms the codes are bit-exact w.r.t. Def. 3 in that arithmetic. */
+ * (as in C_nat), below it is y * 2^(s-1), both at 2^-23 resolution.  For a subnormal norm, whose
+ * reciprocal would overflow, |x| and the norm are both multiplied by 2^24 first (exact, y
+ * unchanged).  Given the stored norms the codes are bit-exact w.r.t. Def. 3 in that arithmetic.
+ * Degenerate buckets: norm 0 (x = 0 gives D(x) = 0) and a norm that is inf or NaN (the bucket
+ * holds an inf or a NaN; Def. 3 has no ratio |x| / norm to round then) get level code 0
+ * everywhere, and the norm is stored as it is.  Such a bucket decodes to zeros, so the stored
+ * norm is how a receiver sees it; on the worker side `status` reports it:
+ * status: optional (may be NULL) device uint32, 4-byte aligned; the call adds 1 to it for every
+ * bucket whose norm is inf or NaN.  The caller zeroes it and reads it back when it likes. */
 nc_status nd_compress(const float* x, size_t d, const uint64_t* bucket_off, int B, int p, int s,
                       uint64_t seed, uint32_t worker, float* norms, uint8_t* level,
-                      uint32_t* sign, void* workspace, size_t workspace_bytes,
+                      uint32_t* sign, void* workspace, size_t workspace_bytes, uint32_t* status,
                       cudaStream_t stream);
 
 /* The same for n workers' vectors of equal length d and one shared bucket table, in three launches
@@ -163,7 +169,29 @@ size_t nd_batch_workspace_bytes(size_t d, int num_buckets, int n);
 nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B,
                             int p, int s, uint64_t seed, const uint32_t* workers,
                             float* const* norms, uint8_t* const* levels, uint32_t* const* signs,
-                            int n, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+                            int n, void* workspace, size_t workspace_bytes, uint32_t* status,
+                            cudaStream_t stream);
+
+/* The two halves of nd_compress_batch as calls of their own: the per-bucket norms, and the level
+ * rounding against norms that are given (for example after partial norms of a bucket that is
+ * split over several devices were combined, or norms that were compressed and decoded again).
+ * nd_compress_batch(..) gives exactly what nd_norms_batch(..) followed by nd_round_batch(..)
+ * with the same arguments gives.  Arguments as for nd_compress_batch; `norms` is written by the
+ * first call and read by the second; workspace: nd_batch_workspace_bytes(d, B, n). */
+nc_status nd_norms_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B, int p,
+                         float* const* norms, int n, void* workspace, size_t workspace_bytes,
+                         uint32_t* status, cudaStream_t stream);
+nc_status nd_round_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B, int s,
+                         uint64_t seed, const uint32_t* workers, const float* const* norms,
+                         uint8_t* const* levels, uint32_t* const* signs, int n,
+                         cudaStream_t stream);
+
+/* The same count for norms that are already stored (n workers' norm arrays of B entries each;
+ * host array of n device pointers): *status += number of norms that are inf or NaN.  For the
+ * master before it aggregates received buffers, and for the sparse calls (B = 1, their `norm`
+ * output).  Def. 3 leaves a norm that is not finite undefined; this is how it is made visible. */
+nc_status nd_norm_status(const float* const* norms, int n, int B, uint32_t* status,
+                         cudaStream_t stream);
 
 /* nd_compress for callers that have no device memory to hand over as workspace and may not
  * allocate any.  (The paper has no counterpart; this is a deployment convenience.)  Typical
@@ -187,9 +215,11 @@ nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bu
 size_t nd_static_scratch_bytes(void);
 nc_status nd_compress_static(const float* x, size_t d, const uint64_t* bucket_off, int B, int p,
                              int s, uint64_t seed, uint32_t worker, float* norms, uint8_t* level,
-                             uint32_t* sign, cudaStream_t stream);
+                             uint32_t* sign, uint32_t* status, cudaStream_t stream);
 
-/* Master side, one worker: acc[j] <- acc[j] + sign_j * fl32(norm_b * 2^(c_j - s)); c = 0 adds +-0. */
+/* Master side, one worker: acc[j] <- acc[j] + sign_j * fl32(norm_b * 2^(c_j - s)); c = 0 adds +-0
+ * whatever the norm.  For c > 0 the product is taken as it comes (Def. 3: norm * sign * xi), so
+ * a norm that is inf or NaN gives an entry that is not finite. */
 nc_status nd_decode_accumulate(const float* norms, const uint8_t* level, const uint32_t* sign,
                                size_t d, const uint64_t* bucket_off, int B, int s, float* acc,
                                cudaStream_t stream);
@@ -233,8 +263,8 @@ nc_status nd_sparse_decode_accumulate(const uint32_t* idx, const uint8_t* codes,
 
 /* ---- sparse update without an index list --------------------------------------------------
  * With independent selection the kept set is a function of (seed, worker, keep_threshold), so a
- * receiver that knows them can regenerate it instead of receiving idx ("next" item of the type /
- * mode variants: the wire carries count, norm and the 4-bit codes only, 0.5 byte per kept entry).
+ * receiver that knows them can regenerate it instead of receiving idx: the wire carries count,
+ * norm and the 4-bit codes only, 0.5 byte per kept entry.
  * Applies the output of nd_sparse_compress made with the same d, keep_threshold, seed and worker:
  * the k-th code goes to the k-th kept coordinate in ascending order, k < min(*count, cap);
  * acc[j] <- acc[j] + sign * fl32(norm * 2^(c - s)).  Cost: one pass of the selection generator
@@ -285,10 +315,10 @@ nc_status nd_sparse_compact_aggregate(const uint32_t* const* idxs, const uint32_
                                       cudaStream_t stream);
 
 /* ---- the paper's 8-bit wire format and integer aggregation ----------------------------------
- * Experimental set-up appendix ("1 bit for the sign ... clip the exponents in the range -50~10 ...
- * the remaining one bit is used to represent zeros", "64-bit integers to store the intermediate
- * results") and the "fast aggregation" appendix (values restored as integers with one non-zero
- * bit).  Code byte: bit 7 sign, bit 6 zero flag, bits 0..5 = exponent + 50 of C_nat(x) with the
+ * Experimental set-up appendix: an 8-bit code made of a sign bit, a flag for zero and a 6-bit
+ * exponent clipped to [-50, 10], summed at the aggregator in 64-bit integers; and the "fast
+ * aggregation" appendix (values restored as integers with one non-zero bit).
+ * Code byte: bit 7 sign, bit 6 zero flag, bits 0..5 = exponent + 50 of C_nat(x) with the
  * exponent clipped to [-50, 10] (+-inf and NaN clip to +-2^10).  Planes hold nc_exp_bytes(d) bytes. */
 
 /* Worker side: code[j] <- 8-bit code of C_nat(x_j) with the stream (seed, worker, j). */
@@ -350,7 +380,8 @@ nc_status nc_compress_f16_r16_batch(const void* const* xs, size_t d, uint64_t se
                                     uint32_t* const* signs, int n, cudaStream_t stream);
 
 /* ---- binary64 inputs: 12-bit codes -------------------------------------------------------------
- * Sec. 2: "11 bits for the exponent and 1 for the sign".  C_nat (Def. 1) of a binary64 vector with
+ * Sec. 2 gives the code size for binary64: an 11-bit exponent and a sign bit.  C_nat (Def. 1) of a
+ * binary64 vector with
  * a 52-bit threshold: r52 = (low 23 bits of the stream word (seed, worker, domain 0, j)) << 29 |
  * (stream word (seed, worker, domain 3, j) >> 3); round up iff r52 < the 52-bit mantissa field.
  * Planes: exp_lo[j] = low 8 bits of the rounded 11-bit exponent field (nc_exp_bytes(d) bytes);

@@ -163,9 +163,24 @@ float norm_p(const float* x, uint64_t len, int p) {
 }
 
 bool norm_degenerate(float norm) {
-    // x = 0 gives D(x) = 0 (Def. 3).  A norm that is subnormal or not finite is
-    // treated the same way: every level code is 0, the norm itself is still stored.
-    return !(norm >= 0x1p-126f) || std::isinf(norm);
+    // x = 0 gives D(x) = 0 (Def. 3).  A norm that is not finite has no ratio |x| / norm to
+    // round either: such a bucket gets level code 0 everywhere, and its norm is still stored,
+    // which is how the receiver can tell.  A subnormal norm is an ordinary norm.
+    return !(norm > 0.0f) || std::isinf(norm);
+}
+
+// y = |x| / norm of Def. 3 in the pinned binary32 arithmetic of the "given norm" mode: one
+// reciprocal per bucket, one multiply per entry.  The reciprocal of a subnormal norm would
+// overflow, so below 2^-126 both operands are first multiplied by 2^24; that scaling is exact
+// (norm * 2^24 is a normal number and so is |x| * 2^24 for any |x| <= norm), hence y is the
+// same ratio and E xi(y) = y keeps the operator unbiased for buckets of tiny entries.
+float ratio_given_norm(float ax, float norm) {
+    if (norm < 0x1p-126f) {
+        ax = ax * 0x1p24f;
+        norm = norm * 0x1p24f;
+    }
+    const float rinv = 1.0f / norm;
+    return ax * rinv;
 }
 
 // ------------------------------------------------------- natural dithering
@@ -188,12 +203,13 @@ int nd_level_code(double y, int s, uint32_t r23) {
     return 0;   // not reached for y >= 0
 }
 
-// decoded magnitude of level code c under norm: norm * 2^(c-s) as one binary32
-// multiply by an exact power of two; c = 0 decodes to 0 whatever the norm is, and so does
-// every code under a norm that is not finite (such a bucket was compressed to all-zero codes).
+// Decoded value of level code c under norm (Def. 3: ||x|| * sign * xi with xi = 2^(c-s), and
+// xi = 0 for c = 0): one binary32 multiply by an exact power of two.  c = 0 contributes a zero
+// whatever the norm is; for c > 0 the product is taken as it comes, so a norm that is not
+// finite gives a value that is not finite.
 float nd_decode_value(int c, int s, float norm, uint32_t sign_bit) {
     float mag;
-    if (c == 0 || std::isnan(norm) || std::isinf(norm)) mag = 0.0f;
+    if (c == 0) mag = 0.0f;
     else mag = norm * (float)std::ldexp(1.0, c - s);
     return sign_bit ? -mag : mag;
 }
@@ -372,31 +388,43 @@ void orc_nd_compress(const float* x, uint64_t d, uint64_t j0, const uint64_t* bu
                      int p, int s, uint64_t seed, uint32_t worker, uint32_t domain, int mode,
                      float* norms, uint8_t* level, uint32_t* sign) {
     if (mode == 0) orc_norms(x, bucket_off, B, p, norms);
-    std::memset(level, 0, (size_t)((d + 1) / 2));
-    std::memset(sign, 0, (size_t)((d + 31) / 32) * 4);
-    // bucket starts need not be even or multiples of 32, so buckets are walked serially
+    // Bucket starts need not be even or multiples of 32, so a level byte or a sign word can
+    // belong to two buckets: the codes are first worked out entry by entry (buckets are
+    // independent of each other), then packed.
+    std::vector<uint8_t> code(d), sbit(d);
+#pragma omp parallel for schedule(dynamic, 1)
     for (int b = 0; b < B; ++b) {
         const float norm = norms[b];
         const bool degenerate = norm_degenerate(norm);
-        const float rinv = degenerate ? 0.0f : 1.0f / norm;
         for (uint64_t i = bucket_off[b]; i < bucket_off[b + 1]; ++i) {
             const float t = x[i];
-            const uint32_t sb = std::signbit(t) ? 1u : 0u;
             int c = 0;
             if (!degenerate) {
                 double y;
                 if (mode == 0) {
                     y = std::fabs((double)t) / (double)norm;
                 } else {
-                    const float yf = std::fabs(t) * rinv;
-                    y = (double)yf;
+                    y = (double)ratio_given_norm(std::fabs(t), norm);
                 }
                 const uint32_t r23 = stream_word(seed, worker, domain, j0 + i) & 0x7FFFFFu;
                 c = nd_level_code(y, s, r23);
             }
-            level[i / 2] |= (uint8_t)(c << (4 * (i % 2)));
-            sign[i / 32] |= sb << (i % 32);
+            code[i] = (uint8_t)c;
+            sbit[i] = std::signbit(t) ? 1 : 0;
         }
+    }
+    const int64_t level_bytes = (int64_t)((d + 1) / 2), sign_words = (int64_t)((d + 31) / 32);
+#pragma omp parallel for schedule(static)
+    for (int64_t k = 0; k < level_bytes; ++k) {
+        const uint64_t i = 2 * (uint64_t)k;
+        level[k] = (uint8_t)(code[i] | (i + 1 < d ? code[i + 1] << 4 : 0));
+    }
+#pragma omp parallel for schedule(static)
+    for (int64_t k = 0; k < sign_words; ++k) {
+        uint32_t w = 0;
+        for (uint64_t i = 32 * (uint64_t)k; i < 32 * (uint64_t)k + 32 && i < d; ++i)
+            w |= (uint32_t)sbit[i] << (i % 32);
+        sign[k] = w;
     }
 }
 
@@ -465,7 +493,6 @@ uint64_t orc_sparse_compress(const float* x, uint64_t d, uint64_t keep_threshold
     if (given_norm) norm = *given_norm;      // pins the rounding independently of the summation
     *norm_out = norm;
     const bool degenerate = norm_degenerate(norm);
-    const float rinv = degenerate ? 0.0f : 1.0f / norm;
     // pass 2: level codes of the kept entries, in ascending index order
     uint64_t k = 0;
     const uint64_t stored = count < cap ? count : cap;
@@ -475,7 +502,7 @@ uint64_t orc_sparse_compress(const float* x, uint64_t d, uint64_t keep_threshold
         const float xs = scale * x[j];
         int c = 0;
         if (!degenerate) {
-            const float yf = std::fabs(xs) * rinv;
+            const float yf = ratio_given_norm(std::fabs(xs), norm);
             const uint32_t r23 = stream_word(seed, worker, 1u, j) & 0x7FFFFFu;
             c = nd_level_code((double)yf, s, r23);
         }
@@ -532,12 +559,11 @@ uint64_t orc_sparse_compact_compress(const float* x, uint64_t d, uint64_t keep_t
     const uint64_t groups = (cap + 31) / 32;
     std::memset(planes, 0, (size_t)(groups * (uint64_t)(nb + 1)) * 4);
     if (norm_degenerate(norm)) return 0;            // every level is 0: nothing to list
-    const float rinv = 1.0f / norm;
     uint64_t k = 0;
     for (uint64_t j = 0; j < d; ++j) {
         if ((uint64_t)stream_word(seed, worker, 2u, j) >= keep_threshold) continue;
         const float xs = scale * x[j];
-        const float yf = std::fabs(xs) * rinv;
+        const float yf = ratio_given_norm(std::fabs(xs), norm);
         const uint32_t r23 = stream_word(seed, worker, 1u, j) & 0x7FFFFFu;
         const int c = nd_level_code((double)yf, s, r23);
         if (c == 0) continue;
@@ -678,12 +704,11 @@ uint64_t orc_sparse_exact_compress(const float* x, uint64_t d, uint64_t q, float
     const int nb = bits_for(s);
     std::memset(planes, 0, (size_t)(((cap + 31) / 32) * (uint64_t)(nb + 1)) * 4);
     if (norm_degenerate(norm)) return 0;
-    const float rinv = 1.0f / norm;
     uint64_t k = 0;
     for (uint64_t j = 0; j < d; ++j) {
         if (!mask[j]) continue;
         const float xs = scale * x[j];
-        const float yf = std::fabs(xs) * rinv;
+        const float yf = ratio_given_norm(std::fabs(xs), norm);
         const uint32_t r23 = stream_word(seed, worker, 1u, j) & 0x7FFFFFu;
         const int c = nd_level_code((double)yf, s, r23);
         if (c == 0) continue;

@@ -43,6 +43,7 @@ EXPORTS = (
     "nd_sparse_regen_workspace_bytes", "nd_sparse_regen_decode_accumulate",
     "nd_sparse_compact_aggregate", "nc_aggregate_compress_shard", "nc_compress_bf16_r8",
     "nc_compress_bf16_r8_batch", "nc_compress_f16_r16", "nc_compress_f16_r16_batch",
+    "nd_norm_status", "nd_norms_batch", "nd_round_batch",
 )
 
 
@@ -77,7 +78,7 @@ _nc_aggregate = _sig("nc_aggregate", C.c_int, C.POINTER(_vp), C.POINTER(_vp), C.
                      _vp)
 _nc_sum_fp32 = _sig("nc_sum_fp32", C.c_int, C.POINTER(_vp), C.c_int, _sz, _vp, _vp)
 _nd_compress = _sig("nd_compress", C.c_int, _vp, _sz, _vp, C.c_int, C.c_int, C.c_int, C.c_uint64,
-                    C.c_uint32, _vp, _vp, _vp, _vp, _sz, _vp)
+                    C.c_uint32, _vp, _vp, _vp, _vp, _sz, _vp, _vp)
 _nd_decode_accumulate = _sig("nd_decode_accumulate", C.c_int, _vp, _vp, _vp, _sz, _vp, C.c_int,
                              C.c_int, _vp, _vp)
 _nd_aggregate = _sig("nd_aggregate", C.c_int, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp),
@@ -92,7 +93,8 @@ _nd_sparse_decode_accumulate = _sig("nd_sparse_decode_accumulate", C.c_int, _vp,
 _nd_batch_workspace_bytes = _sig("nd_batch_workspace_bytes", _sz, _sz, C.c_int, C.c_int)
 _nd_compress_batch = _sig("nd_compress_batch", C.c_int, C.POINTER(_vp), _sz, _vp, C.c_int, C.c_int,
                           C.c_int, C.c_uint64, C.POINTER(C.c_uint32), C.POINTER(_vp),
-                          C.POINTER(_vp), C.POINTER(_vp), C.c_int, _vp, _sz, _vp)
+                          C.POINTER(_vp), C.POINTER(_vp), C.c_int, _vp, _sz, _vp, _vp)
+_nd_norm_status = _sig("nd_norm_status", C.c_int, C.POINTER(_vp), C.c_int, C.c_int, _vp, _vp)
 _nd_sparse_batch_workspace_bytes = _sig("nd_sparse_batch_workspace_bytes", _sz, _sz, _sz, C.c_int)
 _nd_sparse_compress_batch = _sig("nd_sparse_compress_batch", C.c_int, C.POINTER(_vp), _sz,
                                  C.c_uint64, C.c_float, C.c_int, C.c_int, C.c_uint64,
@@ -105,12 +107,40 @@ def nd_batch_workspace_bytes(d: int, num_buckets: int, n: int) -> int:
 
 
 def nd_compress_batch(xs, d, bucket_off, B, p, s, seed, workers, norms, levels, signs, n,
-                      workspace, workspace_bytes, stream=None) -> None:
+                      workspace, workspace_bytes, stream=None, status=None) -> None:
+    """status (the C argument before the stream; optional): device uint32 that the call
+    increments once per bucket whose norm is inf or NaN."""
     w = (C.c_uint32 * n)(*[int(v) for v in workers])
     _check("nd_compress_batch", _nd_compress_batch(_ptrs(xs), d, _ptr(bucket_off), B, p, s, seed,
                                                    w, _ptrs(norms), _ptrs(levels), _ptrs(signs),
                                                    n, _ptr(workspace), workspace_bytes,
-                                                   _stream(stream)))
+                                                   _ptr(status), _stream(stream)))
+
+
+_nd_norms_batch = _sig("nd_norms_batch", C.c_int, C.POINTER(_vp), _sz, _vp, C.c_int, C.c_int,
+                       C.POINTER(_vp), C.c_int, _vp, _sz, _vp, _vp)
+_nd_round_batch = _sig("nd_round_batch", C.c_int, C.POINTER(_vp), _sz, _vp, C.c_int, C.c_int,
+                       C.c_uint64, C.POINTER(C.c_uint32), C.POINTER(_vp), C.POINTER(_vp),
+                       C.POINTER(_vp), C.c_int, _vp)
+
+
+def nd_norms_batch(xs, d, bucket_off, B, p, norms, n, workspace, workspace_bytes, stream=None,
+                   status=None) -> None:
+    _check("nd_norms_batch", _nd_norms_batch(_ptrs(xs), d, _ptr(bucket_off), B, p, _ptrs(norms), n,
+                                             _ptr(workspace), workspace_bytes, _ptr(status),
+                                             _stream(stream)))
+
+
+def nd_round_batch(xs, d, bucket_off, B, s, seed, workers, norms, levels, signs, n,
+                   stream=None) -> None:
+    w = (C.c_uint32 * n)(*[int(v) for v in workers])
+    _check("nd_round_batch", _nd_round_batch(_ptrs(xs), d, _ptr(bucket_off), B, s, seed, w,
+                                             _ptrs(norms), _ptrs(levels), _ptrs(signs), n,
+                                             _stream(stream)))
+
+
+def nd_norm_status(norms, n, B, status, stream=None) -> None:
+    _check("nd_norm_status", _nd_norm_status(_ptrs(norms), n, B, _ptr(status), _stream(stream)))
 
 
 def nd_sparse_batch_workspace_bytes(d: int, cap: int, n: int) -> int:
@@ -276,7 +306,7 @@ def nc8_aggregate_compress(codes, n, d, seed, master, out_code, stream=None) -> 
 
 _nd_static_scratch_bytes = _sig("nd_static_scratch_bytes", _sz)
 _nd_compress_static = _sig("nd_compress_static", C.c_int, _vp, _sz, _vp, C.c_int, C.c_int,
-                           C.c_int, C.c_uint64, C.c_uint32, _vp, _vp, _vp, _vp)
+                           C.c_int, C.c_uint64, C.c_uint32, _vp, _vp, _vp, _vp, _vp)
 
 
 def nd_static_scratch_bytes() -> int:
@@ -284,14 +314,14 @@ def nd_static_scratch_bytes() -> int:
 
 
 def nd_compress_static(x, d, bucket_off, B, p, s, seed, worker, norms, level, sign,
-                       stream=None) -> None:
+                       stream=None, status=None) -> None:
     """nd_compress with the library's built-in scratch array instead of a workspace argument:
     for callers that may not allocate device memory.  Raises NatcompError(NC_ERR_TOO_LARGE) when
     nd_workspace_bytes(d, B) exceeds nd_static_scratch_bytes().  Calls on one device share the
     scratch, so they must not overlap on the GPU."""
     _check("nd_compress_static", _nd_compress_static(_ptr(x), d, _ptr(bucket_off), B, p, s, seed,
                                                      worker, _ptr(norms), _ptr(level), _ptr(sign),
-                                                     _stream(stream)))
+                                                     _ptr(status), _stream(stream)))
 
 
 _nc_copy_to_device = _sig("nc_copy_to_device", C.c_int, _vp, _vp, _sz, _vp)
@@ -386,10 +416,10 @@ def nc_sum_fp32(xs, n, d, out, stream=None) -> None:
 
 # ---- D_nat ---------------------------------------------------------------------------
 def nd_compress(x, d, bucket_off, B, p, s, seed, worker, norms, level, sign, workspace,
-                workspace_bytes, stream=None) -> None:
+                workspace_bytes, stream=None, status=None) -> None:
     _check("nd_compress", _nd_compress(_ptr(x), d, _ptr(bucket_off), B, p, s, seed, worker,
                                        _ptr(norms), _ptr(level), _ptr(sign), _ptr(workspace),
-                                       workspace_bytes, _stream(stream)))
+                                       workspace_bytes, _ptr(status), _stream(stream)))
 
 
 def nd_decode_accumulate(norms, level, sign, d, bucket_off, B, s, acc, stream=None) -> None:

@@ -207,7 +207,8 @@ template <int P>
 __global__ void __launch_bounds__(kBlockThreads)
 nd_norm_finalize_kernel(const __grid_constant__ DitherBatch batch,
                         const uint64_t* __restrict__ off, const int B,
-                        const uint64_t* __restrict__ slots_all, const uint64_t slot_stride) {
+                        const uint64_t* __restrict__ slots_all, const uint64_t slot_stride,
+                        uint32_t* __restrict__ status) {
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x;
     const uint64_t* __restrict__ slots = slots_all + (uint64_t)blockIdx.y * slot_stride;
@@ -246,18 +247,24 @@ nd_norm_finalize_kernel(const __grid_constant__ DitherBatch batch,
             result = (float)tot;
         }
         norms[b] = result;
+        // a bucket that holds an inf or a NaN: its codes will all be 0, the caller is told here
+        if (status && !(result <= 3.40282347e38f)) atomicAdd(status, 1u);
     }
 }
 
 struct BucketScale {
-    float rinv;      // fl32(1 / norm), or 0 for a degenerate bucket
+    float pre;       // 1, or 2^24 when the norm is subnormal (its reciprocal would overflow)
+    float rinv;      // fl32(1 / (norm * pre)), or 0 for a degenerate bucket
     uint32_t smax;   // s, or 0 for a degenerate bucket (forces every code to 0)
 };
 
+// Degenerate: norm 0 (x = 0 gives D(x) = 0, Def. 3) or not finite.  A subnormal norm is an
+// ordinary one: entries and norm are scaled by 2^24 first, which is exact and leaves y unchanged.
 __device__ __forceinline__ BucketScale bucket_scale(float norm, int s) {
     BucketScale r;
-    const bool ok = (norm >= 1.17549435e-38f) && (norm <= 3.40282347e38f);
-    r.rinv = ok ? __fdiv_rn(1.0f, norm) : 0.f;
+    const bool ok = (norm > 0.f) && (norm <= 3.40282347e38f);
+    r.pre = norm < 1.17549435e-38f ? 16777216.f : 1.f;
+    r.rinv = ok ? __fdiv_rn(1.0f, __fmul_rn(norm, r.pre)) : 0.f;
     r.smax = ok ? (uint32_t)s : 0u;
     return r;
 }
@@ -265,7 +272,7 @@ __device__ __forceinline__ BucketScale bucket_scale(float norm, int s) {
 // level code of one entry; pow2s = 2^s as a float
 __device__ __forceinline__ uint32_t level_code(uint32_t bits, uint32_t rnd, const BucketScale sc,
                                                float pow2s) {
-    const float y = __fmul_rn(fabsf(__uint_as_float(bits)), sc.rinv);   // |x| is an operand modifier
+    const float y = __fmul_rn(__fmul_rn(fabsf(__uint_as_float(bits)), sc.pre), sc.rinv);
     const float z = __fmul_rn(y, pow2s);
     // below 2 the bottom interval [0, 2^(1-s)] is mapped onto [1, 2): w = 1 + z/2 (> z there);
     // from 2 on 1 + z/2 <= z, so one max selects the right branch
@@ -308,7 +315,9 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
 #pragma unroll
         for (int it = 0; it < 4; ++it) u[it] = ld_stream_v8(x + base + it * 256 + lane * 8);
     }
-    int b = (int)tile_bucket[tile];
+    // the norm pass leaves the bucket of every tile's first entry in the workspace; the rounding
+    // pass on its own looks it up (the loads above are in flight meanwhile)
+    int b = tile_bucket ? (int)tile_bucket[tile] : find_bucket(off, B, base);
 
     // Fast path: the tile lies in one bucket.  z = fl32(fl32(|x| * rinv) * 2^s) is computed as
     // fl32(|x| * (rinv * 2^s)): scaling by 2^s is exact, so the two agree whenever the inner
@@ -319,9 +328,10 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
     // No clamp of the code in this path: the norm was computed from the same entries, so
     // |x| <= norm, |x| * rinv <= 1 + 2^-24 rounds to at most 1 (a tie goes to the even mantissa 0)
     // and z <= 2^s has a zero mantissa at the top exponent, which the random increment cannot carry
-    // out of.  A degenerate bucket (norm 0, subnormal or not finite; all codes 0) takes the
-    // general path, which clamps.
-    if (full && __ldg(off + b + 1) >= base + kTile && rinv_s <= 3.40282347e38f && sc0.smax != 0u) {
+    // out of.  A degenerate bucket (norm 0 or not finite; all codes 0) and one with a subnormal
+    // norm take the general path, which clamps.
+    if (full && __ldg(off + b + 1) >= base + kTile && rinv_s <= 3.40282347e38f && sc0.smax != 0u &&
+        sc0.pre == 1.0f) {
         uint32_t* lv = reinterpret_cast<uint32_t*>(level + (base >> 1));
         const PhiloxTile pt = philox_tile((uint32_t)(base >> 34), worker, kDomainDnat, keys);
         const uint32_t q_lo = (uint32_t)(base >> 2) + (uint32_t)(lane * 2);
@@ -618,15 +628,30 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
         while (j >= bend) { ++b; bend = __ldg(off + b + 1); }
         float a = kFromAcc ? out[j] : 0.f;
         for (int i = 0; i < n; ++i) {
-            float norm = __ldg(planes.norms[i] + b);
-            if (!(fabsf(norm) <= 3.40282347e38f)) norm = 0.f;
+            const float norm = __ldg(planes.norms[i] + b);
             const uint32_t c = (planes.level[i][j >> 1] >> (4 * (j & 1))) & 0xFu;
             const uint32_t sg = (planes.sign[i][j >> 5] >> (j & 31)) & 1u;
             const uint32_t pb = (c ? ((c + 127u - (uint32_t)s) << 23) : 0u) | (sg << 31);
-            a = add_scaled(a, norm, __uint_as_float(pb));
+            // level 0 is the value 0 whatever the norm; any other level is norm * 2^(c-s) as it
+            // comes, so a norm that is not finite shows in the sum
+            a = c ? add_scaled(a, norm, __uint_as_float(pb)) : __fadd_rn(a, __uint_as_float(pb));
         }
         out[j] = a;
     }
+}
+
+struct NormLists {
+    const float* norms[NC_MAX_WORKERS];
+};
+
+// status += number of the n * B norms that are inf or NaN; grid: (ceil(B / threads), n)
+__global__ void __launch_bounds__(kBlockThreads)
+nd_norm_status_kernel(const __grid_constant__ NormLists lists, const int B,
+                      uint32_t* __restrict__ status) {
+    const int b = blockIdx.x * kBlockThreads + threadIdx.x;
+    const bool bad = b < B && !(fabsf(lists.norms[blockIdx.y][b]) <= 3.40282347e38f);
+    const uint32_t votes = __ballot_sync(0xFFFFFFFFu, bad);
+    if ((threadIdx.x & 31) == 0 && votes) atomicAdd(status, (uint32_t)__popc(votes));
 }
 
 inline unsigned nd_tile_blocks(uint64_t d) {
@@ -674,36 +699,42 @@ size_t nd_workspace_bytes(size_t d, int num_buckets) {
     return nd_batch_workspace_bytes(d, num_buckets, 1);
 }
 
-nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B,
-                            int p, int s, uint64_t seed, const uint32_t* workers,
-                            float* const* norms, uint8_t* const* levels, uint32_t* const* signs,
-                            int n, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
-    if (!xs || !bucket_off || !workers || !norms || !levels || !signs || n < 1 ||
-        n > NC_MAX_WORKERS || B < 1 || s < 1 || s > 15)
-        return NC_ERR_INVALID;
-    if (p != 1 && p != 2 && p != NC_P_INF) return NC_ERR_UNSUPPORTED;
-    if (d == 0) return NC_OK;
+// shared argument checks of the dithering compress calls; fills `batch`
+static nc_status nd_check_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B,
+                                const uint32_t* workers, float* const* norms,
+                                uint8_t* const* levels, uint32_t* const* signs, int n,
+                                bool need_planes, DitherBatch* batch) {
+    if (!xs || !bucket_off || !norms || n < 1 || n > NC_MAX_WORKERS || B < 1) return NC_ERR_INVALID;
+    if (need_planes && (!workers || !levels || !signs)) return NC_ERR_INVALID;
     if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
-    if (!workspace) return NC_ERR_INVALID;
-    if (!aligned16(workspace) || ((uintptr_t)bucket_off & 7u)) return NC_ERR_ALIGN;
-    DitherBatch batch;
+    if ((uintptr_t)bucket_off & 7u) return NC_ERR_ALIGN;
     for (int i = 0; i < n; ++i) {
-        if (!xs[i] || !norms[i] || !levels[i] || !signs[i]) return NC_ERR_INVALID;
-        if (!aligned32(xs[i]) || !aligned16(levels[i]) || !aligned16(signs[i]) ||
-            !aligned4(norms[i]))
-            return NC_ERR_ALIGN;
-        batch.x[i] = xs[i];
-        batch.norms[i] = norms[i];
-        batch.level[i] = levels[i];
-        batch.sign[i] = signs[i];
-        batch.worker[i] = workers[i];
+        if (!xs[i] || !norms[i]) return NC_ERR_INVALID;
+        if (!aligned32(xs[i]) || !aligned4(norms[i])) return NC_ERR_ALIGN;
+        batch->x[i] = xs[i];
+        batch->norms[i] = norms[i];
+        batch->level[i] = nullptr;
+        batch->sign[i] = nullptr;
+        batch->worker[i] = 0;
+        if (need_planes) {
+            if (!levels[i] || !signs[i]) return NC_ERR_INVALID;
+            if (!aligned16(levels[i]) || !aligned16(signs[i])) return NC_ERR_ALIGN;
+            batch->level[i] = levels[i];
+            batch->sign[i] = signs[i];
+            batch->worker[i] = workers[i];
+        }
     }
-    if (workspace_bytes < nd_batch_workspace_bytes(d, B, n)) return NC_ERR_WORKSPACE;
+    return NC_OK;
+}
+
+// the two norm launches; returns the tile -> bucket map they leave in the workspace
+static uint32_t* nd_launch_norms(const DitherBatch& batch, uint64_t d, const uint64_t* bucket_off,
+                                 int B, int p, int n, void* workspace, uint32_t* status,
+                                 cudaStream_t stream) {
     const uint64_t tiles = nd_tiles(d);
     const uint64_t slot_stride = round_up16((tiles + (uint64_t)B + 1) * 8) / 8;
     uint64_t* slots = reinterpret_cast<uint64_t*>(workspace);
     uint32_t* tile_bucket = reinterpret_cast<uint32_t*>(slots + (uint64_t)n * slot_stride);
-    const dim3 grid(nd_tile_blocks(d), (unsigned)n);
     const unsigned resident = 2u * (unsigned)device_sm_count();
     const dim3 ngrid(nd_tile_blocks(d) < resident ? nd_tile_blocks(d) : resident, (unsigned)n);
     const dim3 fgrid((unsigned)B, (unsigned)n);
@@ -711,19 +742,74 @@ nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bu
         nd_norm_partials_kernel<1><<<ngrid, kBlockThreads, 0, stream>>>(
             batch, d, bucket_off, B, slots, slot_stride, tile_bucket);
         nd_norm_finalize_kernel<1><<<fgrid, kBlockThreads, 0, stream>>>(batch, bucket_off, B,
-                                                                        slots, slot_stride);
+                                                                        slots, slot_stride, status);
     } else if (p == 2) {
         nd_norm_partials_kernel<2><<<ngrid, kBlockThreads, 0, stream>>>(
             batch, d, bucket_off, B, slots, slot_stride, tile_bucket);
         nd_norm_finalize_kernel<2><<<fgrid, kBlockThreads, 0, stream>>>(batch, bucket_off, B,
-                                                                        slots, slot_stride);
+                                                                        slots, slot_stride, status);
     } else {
         nd_norm_partials_kernel<NC_P_INF><<<ngrid, kBlockThreads, 0, stream>>>(
             batch, d, bucket_off, B, slots, slot_stride, tile_bucket);
         nd_norm_finalize_kernel<NC_P_INF><<<fgrid, kBlockThreads, 0, stream>>>(
-            batch, bucket_off, B, slots, slot_stride);
+            batch, bucket_off, B, slots, slot_stride, status);
     }
+    return tile_bucket;
+}
+
+nc_status nd_norms_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B, int p,
+                         float* const* norms, int n, void* workspace, size_t workspace_bytes,
+                         uint32_t* status, cudaStream_t stream) {
+    if (p != 1 && p != 2 && p != NC_P_INF) return NC_ERR_UNSUPPORTED;
+    DitherBatch batch;
+    const nc_status st = nd_check_batch(xs, d, bucket_off, B, nullptr, norms, nullptr, nullptr, n,
+                                        false, &batch);
+    if (st != NC_OK) return st;
+    if (d == 0) return NC_OK;
+    if (!workspace) return NC_ERR_INVALID;
+    if (!aligned16(workspace) || !aligned4(status)) return NC_ERR_ALIGN;
+    if (workspace_bytes < nd_batch_workspace_bytes(d, B, n)) return NC_ERR_WORKSPACE;
+    nd_launch_norms(batch, d, bucket_off, B, p, n, workspace, status, stream);
+    return launch_status();
+}
+
+nc_status nd_round_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B, int s,
+                         uint64_t seed, const uint32_t* workers, const float* const* norms,
+                         uint8_t* const* levels, uint32_t* const* signs, int n,
+                         cudaStream_t stream) {
+    if (s < 1 || s > 15) return NC_ERR_INVALID;
+    DitherBatch batch;
+    const nc_status st = nd_check_batch(xs, d, bucket_off, B, workers,
+                                        const_cast<float* const*>(norms), levels, signs, n, true,
+                                        &batch);
+    if (st != NC_OK) return st;
+    if (d == 0) return NC_OK;
     const PhiloxKeys keys = make_philox_keys(seed);
+    const dim3 grid(nd_tile_blocks(d), (unsigned)n);
+    nd_round_pack_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, bucket_off, B, s, keys,
+                                                             nullptr);
+    return launch_status();
+}
+
+nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B,
+                            int p, int s, uint64_t seed, const uint32_t* workers,
+                            float* const* norms, uint8_t* const* levels, uint32_t* const* signs,
+                            int n, void* workspace, size_t workspace_bytes, uint32_t* status,
+                            cudaStream_t stream) {
+    if (s < 1 || s > 15) return NC_ERR_INVALID;
+    if (p != 1 && p != 2 && p != NC_P_INF) return NC_ERR_UNSUPPORTED;
+    DitherBatch batch;
+    const nc_status st = nd_check_batch(xs, d, bucket_off, B, workers, norms, levels, signs, n,
+                                        true, &batch);
+    if (st != NC_OK) return st;
+    if (d == 0) return NC_OK;
+    if (!workspace) return NC_ERR_INVALID;
+    if (!aligned16(workspace) || !aligned4(status)) return NC_ERR_ALIGN;
+    if (workspace_bytes < nd_batch_workspace_bytes(d, B, n)) return NC_ERR_WORKSPACE;
+    const uint32_t* tile_bucket =
+        nd_launch_norms(batch, d, bucket_off, B, p, n, workspace, status, stream);
+    const PhiloxKeys keys = make_philox_keys(seed);
+    const dim3 grid(nd_tile_blocks(d), (unsigned)n);
     nd_round_pack_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, bucket_off, B, s, keys,
                                                              tile_bucket);
     return launch_status();
@@ -731,11 +817,11 @@ nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bu
 
 nc_status nd_compress(const float* x, size_t d, const uint64_t* bucket_off, int B, int p, int s,
                       uint64_t seed, uint32_t worker, float* norms, uint8_t* level,
-                      uint32_t* sign, void* workspace, size_t workspace_bytes,
+                      uint32_t* sign, void* workspace, size_t workspace_bytes, uint32_t* status,
                       cudaStream_t stream) {
     if (!x || !norms || !level || !sign) return NC_ERR_INVALID;
     return nd_compress_batch(&x, d, bucket_off, B, p, s, seed, &worker, &norms, &level, &sign, 1,
-                             workspace, workspace_bytes, stream);
+                             workspace, workspace_bytes, status, stream);
 }
 
 static nc_status nd_check_planes(const float* const* norms, const uint8_t* const* levels,
@@ -766,6 +852,22 @@ nc_status nd_aggregate(const float* const* norms, const uint8_t* const* levels,
     const uint64_t big_tiles = nd_aggregate_big_tiles(d);
     nd_aggregate_kernel<false><<<nd_aggregate_blocks(d, big_tiles), kAggregateThreads, 0, stream>>>(
         planes, n, (uint64_t)d, bucket_off, B, s, big_tiles, out);
+    return launch_status();
+}
+
+nc_status nd_norm_status(const float* const* norms, int n, int B, uint32_t* status,
+                         cudaStream_t stream) {
+    if (!norms || !status || n < 1 || n > NC_MAX_WORKERS || B < 0) return NC_ERR_INVALID;
+    if (!aligned4(status)) return NC_ERR_ALIGN;
+    if (B == 0) return NC_OK;
+    NormLists lists;
+    for (int i = 0; i < n; ++i) {
+        if (!norms[i]) return NC_ERR_INVALID;
+        if (!aligned4(norms[i])) return NC_ERR_ALIGN;
+        lists.norms[i] = norms[i];
+    }
+    const dim3 grid((unsigned)((B + kBlockThreads - 1) / kBlockThreads), (unsigned)n);
+    nd_norm_status_kernel<<<grid, kBlockThreads, 0, stream>>>(lists, B, status);
     return launch_status();
 }
 
@@ -822,13 +924,13 @@ size_t nd_static_scratch_bytes(void) { return kStaticScratchBytes; }
 
 nc_status nd_compress_static(const float* x, size_t d, const uint64_t* bucket_off, int B, int p,
                              int s, uint64_t seed, uint32_t worker, float* norms, uint8_t* level,
-                             uint32_t* sign, cudaStream_t stream) {
-    if (B < 0) return NC_ERR_INVALID;
+                             uint32_t* sign, uint32_t* status, cudaStream_t stream) {
+    if (!x || !bucket_off || !norms || !level || !sign || B < 1) return NC_ERR_INVALID;
     if (nd_workspace_bytes(d, B) > kStaticScratchBytes) return NC_ERR_TOO_LARGE;
     void* scratch = static_scratch_address();
     if (!scratch) return NC_ERR_CUDA;
     return nd_compress(x, d, bucket_off, B, p, s, seed, worker, norms, level, sign, scratch,
-                       kStaticScratchBytes, stream);
+                       kStaticScratchBytes, status, stream);
 }
 
 }  // extern "C"

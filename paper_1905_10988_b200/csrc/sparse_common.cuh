@@ -182,14 +182,16 @@ __device__ __forceinline__ void shift_in_drop_bit(uint32_t& drop, uint32_t word,
 }
 
 struct Scale {
-    float rinv;
-    uint32_t smax;
+    float pre;       // 1, or 2^24 when the norm is subnormal (its reciprocal would overflow)
+    float rinv;      // fl32(1 / (norm * pre)), or 0 for a degenerate norm
+    uint32_t smax;   // s, or 0 for a degenerate norm (0 or not finite: every code is 0)
 };
 
 __device__ __forceinline__ Scale make_scale(float norm, int s) {
     Scale r;
-    const bool ok = (norm >= 1.17549435e-38f) && (norm <= 3.40282347e38f);
-    r.rinv = ok ? __fdiv_rn(1.0f, norm) : 0.f;
+    const bool ok = (norm > 0.f) && (norm <= 3.40282347e38f);
+    r.pre = norm < 1.17549435e-38f ? 16777216.f : 1.f;
+    r.rinv = ok ? __fdiv_rn(1.0f, __fmul_rn(norm, r.pre)) : 0.f;
     r.smax = ok ? (uint32_t)s : 0u;
     return r;
 }
@@ -198,7 +200,7 @@ __device__ __forceinline__ Scale make_scale(float norm, int s) {
 __device__ __forceinline__ uint32_t sparse_level_code(uint32_t bits, uint32_t rnd, const Scale sc,
                                                       float pow2s) {
     const float ax = __uint_as_float(bits & 0x7FFFFFFFu);
-    const float y = __fmul_rn(ax, sc.rinv);
+    const float y = __fmul_rn(__fmul_rn(ax, sc.pre), sc.rinv);   // the scaling by pre is exact
     const float z = __fmul_rn(y, pow2s);
     // below 2 the bottom interval [0, 2^(1-s)] is mapped onto [1, 2): w = 1 + z/2 (> z there);
     // from 2 on 1 + z/2 <= z, so one max selects the right branch

@@ -315,13 +315,13 @@ sparse_decode_accumulate_kernel(const uint32_t* __restrict__ idx, const uint8_t*
     const uint64_t total = min((uint64_t)*count, cap);
     if (k >= total) return;
     float nv = *norm;
-    if (!(fabsf(nv) <= 3.40282347e38f)) nv = 0.f;
     const uint32_t j = idx[k];
     if (j >= d) return;
     const uint32_t code = (codes[k >> 1] >> (4 * (k & 1))) & 0xFu;
     const uint32_t c = code & 7u;
     const uint32_t pb = (c ? ((c + 127u - (uint32_t)s) << 23) : 0u) | ((code >> 3) << 31);
-    acc[j] = __fadd_rn(acc[j], __fmul_rn(nv, __uint_as_float(pb)));
+    // level 0 is the value 0 whatever the norm (also one that is not finite)
+    acc[j] = __fadd_rn(acc[j], c ? __fmul_rn(nv, __uint_as_float(pb)) : __uint_as_float(pb));
 }
 
 static void launch_select(const SparseBatch& batch, uint64_t d, uint64_t keep_threshold,
@@ -676,7 +676,6 @@ sparse_compact_decode_accumulate_kernel(const uint32_t* __restrict__ idx,
     const uint64_t total = min((uint64_t)*count, cap);
     if (k >= total) return;
     float nv = *norm;
-    if (!(fabsf(nv) <= 3.40282347e38f)) nv = 0.f;
     const uint32_t j = idx[k];
     if (j >= d) return;
     const int nb = code_value_bits(s);
@@ -868,7 +867,6 @@ sparse_regen_apply_kernel(const uint8_t* __restrict__ codes, const uint32_t* __r
     for (int w = 0; w < warp; ++w) k += s_tile[w];
     const uint64_t total = min((uint64_t)*count, cap);
     float nv = *norm;
-    if (!(fabsf(nv) <= 3.40282347e38f)) nv = 0.f;
     while (word && k < total) {
         const int bit = __ffs(word) - 1;
         word &= word - 1;
@@ -876,7 +874,8 @@ sparse_regen_apply_kernel(const uint8_t* __restrict__ codes, const uint32_t* __r
         const uint32_t code = (codes[k >> 1] >> (4 * (k & 1))) & 0xFu;
         const uint32_t c = code & 7u;
         const uint32_t pb = (c ? ((c + 127u - (uint32_t)s) << 23) : 0u) | ((code >> 3) << 31);
-        acc[j] = __fadd_rn(acc[j], __fmul_rn(nv, __uint_as_float(pb)));
+        // level 0 is the value 0 whatever the norm (also one that is not finite)
+        acc[j] = __fadd_rn(acc[j], c ? __fmul_rn(nv, __uint_as_float(pb)) : __uint_as_float(pb));
         ++k;
     }
 }
@@ -993,7 +992,6 @@ sparse_compact_aggregate_kernel(const __grid_constant__ SparseLists lists, const
             idx = lists.idx[w];
             planes = lists.planes[w];
             nv = *lists.norm[w];
-            if (!(fabsf(nv) <= 3.40282347e38f)) nv = 0.f;
             const uint32_t total = (uint32_t)min((uint64_t)*lists.count[w], cap);
             lo = warp_lower_bound(idx, 0u, total, (uint32_t)r0, lane);
             // ascending distinct indices: at most kAggRange entries fall into the range

@@ -29,6 +29,16 @@ class Guarded:
         return self.buf.cpu().numpy().view(dtype)
 
 
+def assert_same_floats(got, want):
+    """Bit for bit, except that any NaN matches any NaN: IEEE 754 leaves the sign and payload of
+    a generated NaN open, and the host and the device choose differently."""
+    got = np.asarray(got).view(np.float32)
+    want = np.asarray(want).view(np.float32)
+    gn, wn = np.isnan(got), np.isnan(want)
+    assert np.array_equal(gn, wn), "NaN positions differ"
+    assert np.array_equal(got.view(np.uint32)[~gn], want.view(np.uint32)[~wn])
+
+
 def dev(a) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 

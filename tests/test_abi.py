@@ -51,9 +51,21 @@ def test_size_helpers(nc):
     assert nc.status_string(0) == "NC_OK" and nc.status_string(-2) == "NC_ERR_ALIGN"
 
 
+def _scratch_address():
+    """An address for pointer arguments that validation must reject before any launch.  On a
+    box with a GPU it is real device memory (2 MiB, far more than any size used below), so a
+    check that stopped working shows up as a wrong status, not as a fault on the device; without
+    a GPU it is a made-up, well-aligned number that nothing dereferences."""
+    import torch
+    if torch.cuda.is_available():
+        buf = torch.zeros(2 << 20, dtype=torch.uint8, device="cuda")
+        return buf, (buf.data_ptr() + 255) & ~255
+    return None, 1 << 20
+
+
 def test_argument_validation_needs_no_gpu(nc):
     lib = nc.lib
-    A = 1 << 20                                 # a fake, well-aligned "device" address
+    keep_alive, A = _scratch_address()
     u32 = (C.c_uint32 * 1)(0)
     one = (C.c_void_p * 1)(A)
     null = (C.c_void_p * 1)(0)
@@ -83,7 +95,7 @@ def test_argument_validation_needs_no_gpu(nc):
                                   a["B"], a["p"], a["s"], C.c_uint64(a["seed"]), a["worker"],
                                   C.c_void_p(a["norms"]), C.c_void_p(a["level"]),
                                   C.c_void_p(a["sign"]), C.c_void_p(a["ws"]),
-                                  C.c_size_t(a["ws_bytes"]), None))
+                                  C.c_size_t(a["ws_bytes"]), C.c_void_p(a.get("status", 0)), None))
 
     assert nd(p=3) == "NC_ERR_UNSUPPORTED"
     assert nd(s=0) == "NC_ERR_INVALID" and nd(s=16) == "NC_ERR_INVALID"
@@ -91,12 +103,17 @@ def test_argument_validation_needs_no_gpu(nc):
     assert nd(ws_bytes=8) == "NC_ERR_WORKSPACE"
     assert nd(x=A + 16) == "NC_ERR_ALIGN"
     assert nd(d=0) == "NC_OK"
+    assert nd(status=A + 2) == "NC_ERR_ALIGN"
+    assert st(lib.nd_norm_status(one, 1, 4, None, None)) == "NC_ERR_INVALID"
+    assert st(lib.nd_norm_status(null, 1, 4, C.c_void_p(A), None)) == "NC_ERR_INVALID"
+    assert st(lib.nd_norm_status(one, 1, 0, C.c_void_p(A), None)) == "NC_OK"      # B = 0: no launch
     raw = C.CDLL(nc.LIB_PATH)          # a separate handle: the binding's prototypes stay as set
     r = raw.nd_sparse_compress(C.c_void_p(A), C.c_size_t(64), C.c_uint64((1 << 32) + 1),
                                C.c_float(1.0), 0, 4, C.c_uint64(0), 0, C.c_void_p(A),
                                C.c_void_p(A), C.c_void_p(A), C.c_void_p(A), C.c_size_t(64),
                                C.c_void_p(A), C.c_size_t(1 << 20), None)
     assert st(r) == "NC_ERR_INVALID"
+    del keep_alive
 
 
 def test_product_never_imports_the_oracle():

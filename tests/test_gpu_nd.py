@@ -9,7 +9,7 @@ import torch
 import oracle
 import paper_1905_10988_b200 as nc
 from paper_1905_10988_b200 import workloads
-from gpu_util import Guarded, dev, unpack_nibbles
+from gpu_util import Guarded, assert_same_floats, dev, unpack_nibbles
 
 pytestmark = pytest.mark.gpu
 
@@ -34,7 +34,7 @@ def gpu_nd_compress(x_dev, off, p, s, seed, worker):
     return norms, level, sign
 
 
-def check_against_oracle(x, off, p, s, seed, worker, norms, level, sign, *, slack=0):
+def check_against_oracle(x, off, p, s, seed, worker, norms, level, sign):
     d = x.size
     gn = norms.numpy(np.float32)
     lv = level.numpy(np.uint8)
@@ -58,7 +58,7 @@ def check_against_oracle(x, off, p, s, seed, worker, norms, level, sign, *, slac
     # definition mode: few, adjacent differences only
     c0 = unpack_nibbles(l0, d).astype(np.int64)
     diff = cg != c0
-    assert diff.sum() <= CODE_MISMATCH * d + slack
+    assert diff.sum() <= int(CODE_MISMATCH * d)       # at small d: no difference at all
     assert np.all(np.abs(cg - c0)[diff] == 1)
     return gn
 
@@ -72,7 +72,7 @@ def test_compress_ragged_bucket_tables(d, s, p):
     sig = 10.0 ** rng.uniform(-5, -2, len(off) - 1)
     x = (rng.standard_normal(d) * np.repeat(sig, np.diff(off))).astype(np.float32)
     norms, level, sign = gpu_nd_compress(dev(x), off, p, s, seed=d, worker=s)
-    check_against_oracle(x, off, p, s, d, s, norms, level, sign, slack=2)
+    check_against_oracle(x, off, p, s, d, s, norms, level, sign)
 
 
 def test_compress_single_bucket_and_aligned_buckets():
@@ -81,7 +81,7 @@ def test_compress_single_bucket_and_aligned_buckets():
     x = (rng.standard_normal(d) * 2e-3).astype(np.float32)
     for off in ([0, d], list(range(0, d + 1, 4096)), [0, 1024, 1024, 2048, d]):
         norms, level, sign = gpu_nd_compress(dev(x), off, 2, 8, seed=1, worker=0)
-        check_against_oracle(x, off, 2, 8, 1, 0, norms, level, sign, slack=2)
+        check_against_oracle(x, off, 2, 8, 1, 0, norms, level, sign)
 
 
 def test_compress_degenerate_buckets():
@@ -96,13 +96,14 @@ def test_compress_degenerate_buckets():
     x[5100] = np.nan
     for p in (1, 2, 0):
         norms, level, sign = gpu_nd_compress(dev(x), off, p, 8, seed=2, worker=1)
-        gn = check_against_oracle(x, off, p, 8, 2, 1, norms, level, sign, slack=2)
+        gn = check_against_oracle(x, off, p, 8, 2, 1, norms, level, sign)
         c = unpack_nibbles(level.numpy(np.uint8), d)
         assert gn[1] == 0 and gn[2] == 0 and 0 < gn[4] < 2.0 ** -126
         assert np.isinf(gn[5]) and np.isnan(gn[6])
-        for b in (1, 4, 5, 6):
+        for b in (1, 5, 6):
             assert np.all(c[off[b]:off[b + 1]] == 0)
         assert np.any(c[off[3]:off[4]] > 0)
+        assert np.any(c[off[4]:off[5]] > 0)     # a subnormal norm is an ordinary norm
         assert np.any(c[:100] > 0)
 
 
@@ -127,8 +128,11 @@ def test_aggregate_and_decode_accumulate_are_bit_exact(n, d, s):
     norms, levels, signs = _random_planes(rng, n, d, B, s)
     norms[0][0] = 2.0 ** -130                  # subnormal products
     if B > 2:
-        norms[-1][1] = np.inf                  # a non-finite norm decodes as zero
+        norms[-1][1] = np.inf                  # level 0 stays 0, any other level decodes to inf
         norms[0][2] = 0.0
+    if B > 4:
+        norms[n // 2][3] = np.nan              # likewise NaN
+        norms[0][4] = 2.0 ** -140              # a subnormal norm
     off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
     nd_ = [dev(a) for a in norms]
     ld = [dev(a) for a in levels]
@@ -138,7 +142,9 @@ def test_aggregate_and_decode_accumulate_are_bit_exact(n, d, s):
     torch.cuda.synchronize()
     out.check()
     want = oracle.nd_aggregate(norms, [l[:(d + 1) // 2] for l in levels], signs, off, s, d)
-    assert np.array_equal(out.numpy(np.uint32), want.view(np.uint32))
+    assert_same_floats(out.numpy(np.float32), want)
+    if B > 2:
+        assert np.any(np.isinf(want[off[1]:off[2]])) or off[2] - off[1] < 4
     acc = Guarded(4 * d)
     start = rng.standard_normal(d).astype(np.float32)
     acc.buf.copy_(dev(start).view(torch.uint8))
@@ -148,7 +154,48 @@ def test_aggregate_and_decode_accumulate_are_bit_exact(n, d, s):
         oracle.nd_decode_accumulate(norms[i], levels[i][:(d + 1) // 2], signs[i], off, s, ref)
     torch.cuda.synchronize()
     acc.check()
-    assert np.array_equal(acc.numpy(np.uint32), ref.view(np.uint32))
+    assert_same_floats(acc.numpy(np.float32), ref)
+
+
+def test_status_reports_buckets_that_are_not_finite():
+    """A bucket holding an inf or a NaN is compressed to level 0 everywhere; the optional status
+    word of the compress calls, and nd_norm_status on stored norms, count such buckets."""
+    rng = np.random.default_rng(8)
+    d = 9000
+    off = [0, 1000, 1000, 3000, 5000, 7000, d]
+    B = len(off) - 1
+    xs = [(rng.standard_normal(d) * 1e-2).astype(np.float32) for _ in range(3)]
+    xs[0][1500] = np.inf
+    xs[0][5500] = np.nan
+    xs[2][8999] = -np.inf
+    off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
+    status = torch.zeros(2, dtype=torch.int32, device="cuda")
+    n = len(xs)
+    ws_bytes = nc.nd_batch_workspace_bytes(d, B, n)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    norms = [torch.empty(B, dtype=torch.float32, device="cuda") for _ in range(n)]
+    levels = [torch.empty(nc.nd_level_bytes(d), dtype=torch.uint8, device="cuda") for _ in range(n)]
+    signs = [torch.empty(nc.nc_sign_bytes(d), dtype=torch.uint8, device="cuda") for _ in range(n)]
+    for p, expect in ((2, 3), (nc.P_INF, 6), (1, 9)):          # the word accumulates over calls
+        nc.nd_compress_batch([dev(x) for x in xs], d, off_dev, B, p, 8, 0, [0, 1, 2], norms, levels,
+                             signs, n, ws, ws_bytes, status=status[0:1])
+        torch.cuda.synchronize()
+        assert status.cpu().tolist() == [expect, 0]
+    nc.nd_compress(dev(xs[1]), d, off_dev, B, 2, 8, 0, 1, norms[1], levels[1], signs[1], ws,
+                   ws_bytes, status=status[0:1])               # a clean vector adds nothing
+    nc.nd_norm_status(norms, n, B, status[1:2])
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [9, 3]
+    # what the master sees when it aggregates all the same: the three buckets add zeros
+    out = torch.empty(d, dtype=torch.float32, device="cuda")
+    nc.nd_aggregate(norms, levels, signs, n, d, off_dev, B, 8, out)
+    torch.cuda.synchronize()
+    ref = oracle.nd_aggregate([a.cpu().numpy() for a in norms],
+                              [a.cpu().numpy()[:(d + 1) // 2] for a in levels],
+                              [a.cpu().numpy().view(np.uint32)[:(d + 31) // 32] for a in signs],
+                              off, 8, d)
+    assert_same_floats(out.cpu().numpy(), ref)
+    assert np.all(np.isfinite(ref))
 
 
 def test_config3_full_size():
@@ -248,13 +295,25 @@ def test_batch_launch_equals_single_launches():
     torch.cuda.synchronize()
     for g in norms + levels + signs + [ws]:
         g.check()
+    # the two halves as calls of their own give the same bytes (the rounding call finds the
+    # bucket of each tile itself instead of reading the map the norm pass leaves behind)
+    norms2 = [Guarded(4 * B) for _ in range(n)]
+    levels2 = [Guarded(nc.nd_level_bytes(d)) for _ in range(n)]
+    signs2 = [Guarded(nc.nc_sign_bytes(d)) for _ in range(n)]
+    nc.nd_norms_batch(xd, d, off_dev, B, p, [g.buf for g in norms2], n, ws.buf, ws_bytes)
+    ws.buf.fill_(0x5A)                       # the rounding call must not depend on the workspace
+    nc.nd_round_batch(xd, d, off_dev, B, s, 11, workers, [g.buf for g in norms2],
+                      [g.buf for g in levels2], [g.buf for g in signs2], n)
+    torch.cuda.synchronize()
+    for a, b in zip(norms + levels + signs, norms2 + levels2 + signs2):
+        b.check()
+        assert np.array_equal(a.numpy(np.uint8), b.numpy(np.uint8))
     for i in range(n):
         n1, l1, s1 = gpu_nd_compress(xd[i], off, p, s, 11, workers[i])
         assert np.array_equal(norms[i].numpy(np.uint32), n1.numpy(np.uint32))
         assert np.array_equal(levels[i].numpy(np.uint8), l1.numpy(np.uint8))
         assert np.array_equal(signs[i].numpy(np.uint32), s1.numpy(np.uint32))
-        check_against_oracle(xs[i], off, p, s, 11, workers[i], norms[i], levels[i], signs[i],
-                             slack=2)
+        check_against_oracle(xs[i], off, p, s, 11, workers[i], norms[i], levels[i], signs[i])
 
 
 def test_one_element_buckets_and_many_empty_buckets():
@@ -267,13 +326,13 @@ def test_one_element_buckets_and_many_empty_buckets():
     off = list(range(d + 1))
     for p in (2, 0):
         norms, level, sign = gpu_nd_compress(dev(x), off, p, 8, seed=4, worker=2)
-        gn = check_against_oracle(x, off, p, 8, 4, 2, norms, level, sign, slack=2)
+        gn = check_against_oracle(x, off, p, 8, 4, 2, norms, level, sign)
         assert np.array_equal(gn, np.abs(x))            # a one-element bucket: norm = |x|
         c = unpack_nibbles(level.numpy(np.uint8), d)
         assert c[7] == 0 and np.all(c[np.abs(x) >= 2.0 ** -126] == 8)   # y = 1 exactly
     off2 = sorted([0] + list(rng.integers(0, d, 40)) * 3 + [d])
     norms, level, sign = gpu_nd_compress(dev(x), off2, 1, 4, seed=5, worker=0)
-    check_against_oracle(x, off2, 1, 4, 5, 0, norms, level, sign, slack=2)
+    check_against_oracle(x, off2, 1, 4, 5, 0, norms, level, sign)
 
 
 def test_beyond_2_to_32_entries_sampled():

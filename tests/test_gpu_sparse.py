@@ -7,7 +7,7 @@ import torch
 import oracle
 import paper_1905_10988_b200 as nc
 from paper_1905_10988_b200 import workloads
-from gpu_util import Guarded, dev
+from gpu_util import Guarded, assert_same_floats, dev
 
 pytestmark = pytest.mark.gpu
 
@@ -80,6 +80,52 @@ def test_sparse_all_zero_and_nonfinite_inputs():
         codes = got[1].numpy(np.uint8)[:(got[2] + 1) // 2]
         assert got[2] > 0
         assert np.all((codes & 0x77) == 0)        # degenerate norm: every level code is 0
+
+
+def test_sparse_decoders_under_a_norm_that_is_not_finite():
+    """Level 0 decodes to a zero whatever the norm; any other level is norm * 2^(c-s) as it comes
+    (Def. 3), so an infinite or NaN norm shows in the result.  Listed, compact and one-launch
+    aggregate decoders against the oracle."""
+    rng = np.random.default_rng(4)
+    d, s, cnt = 4000, 4, 300
+    idx = np.sort(rng.choice(d, cnt, replace=False)).astype(np.uint32)
+    c4 = (rng.integers(0, s + 1, cnt + 1) | (rng.integers(0, 2, cnt + 1) << 3)).astype(np.uint8)
+    codes = np.zeros(((cnt + 1) // 2 + 15) // 16 * 16, np.uint8)
+    codes[:(cnt + 1) // 2] = (c4[0:cnt + 1:2][:(cnt + 1) // 2] | (c4[1:cnt + 1:2] << 4))[:(cnt + 1) // 2]
+    nb = oracle.code_bits(s) - 1               # value bits; the sign is bit nb
+    c3 = (rng.integers(0, s, cnt) | (rng.integers(0, 2, cnt) << nb)).astype(np.uint32)
+    planes = np.zeros(nc.nd_sparse_plane_bytes(cnt, s) // 4, np.uint32)
+    for k in range(cnt):
+        for b in range(nb + 1):
+            planes[(k // 32) * (nb + 1) + b] |= ((c3[k] >> b) & 1) << (k % 32)
+    for norm in (np.inf, np.nan, 2.0 ** -140):
+        nrm = np.float32(norm)
+        start = rng.standard_normal(d).astype(np.float32)
+        acc = dev(start)
+        nc.nd_sparse_decode_accumulate(dev(idx.view(np.int32)), dev(codes),
+                                       dev(np.int32([cnt])), dev(np.float32([nrm])), s, d, cnt, acc)
+        ref = start.copy()
+        oracle.sparse_decode_accumulate(idx, codes[:(cnt + 1) // 2], cnt, nrm, s, ref)
+        assert_same_floats(acc.cpu().numpy(), ref)
+        acc = dev(start)
+        nc.nd_sparse_compact_decode_accumulate(dev(idx.view(np.int32)), dev(planes.view(np.int32)),
+                                               dev(np.int32([cnt])), dev(np.float32([nrm])), s, d,
+                                               cnt, acc)
+        ref = start.copy()
+        oracle.sparse_compact_decode_accumulate(idx, planes, cnt, nrm, s, ref)
+        assert_same_floats(acc.cpu().numpy(), ref)
+        out = torch.empty(d, dtype=torch.float32, device="cuda")
+        nc.nd_sparse_compact_aggregate([dev(idx.view(np.int32))] * 2, [dev(planes.view(np.int32))] * 2,
+                                       [dev(np.int32([cnt]))] * 2,
+                                       [dev(np.float32([1.5])), dev(np.float32([nrm]))], 2, s, d,
+                                       cnt, out)
+        ref = np.zeros(d, np.float32)
+        oracle.sparse_compact_decode_accumulate(idx, planes, cnt, np.float32(1.5), s, ref)
+        oracle.sparse_compact_decode_accumulate(idx, planes, cnt, nrm, s, ref)
+        torch.cuda.synchronize()
+        assert_same_floats(out.cpu().numpy(), ref)
+        if np.isinf(norm):
+            assert np.isinf(ref).sum() == cnt
 
 
 def test_sparse_decode_accumulate_workers_in_order():

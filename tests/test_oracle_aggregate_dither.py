@@ -267,18 +267,91 @@ def test_dnat_given_norm_mode_matches_definition_mode_closely():
 
 
 def test_dnat_degenerate_norms_give_zero_codes():
-    x = np.float32([1.0, -2.0, 3.0, 0.0, 0.0, 1e-40, -1e-41, np.inf, 1.0, 2.0])
+    x = np.float32([1.0, -2.0, 3.0, 0.0, 0.0, np.nan, -1.0, np.inf, 1.0, 2.0])
     off = [0, 3, 5, 7, 10]
     nrm, level, sign = oracle.nd_compress(x, off, 2, 4, seed=0, worker=0)
     c = np.stack([level & 0xF, level >> 4], 1).ravel()[:10]
-    assert nrm[1] == 0.0 and np.all(c[3:5] == 0)           # x = 0 -> D(x) = 0
-    assert 0 < nrm[2] < 2.0 ** -126 and np.all(c[5:7] == 0)  # subnormal norm
-    assert np.isinf(nrm[3]) and np.all(c[7:10] == 0)       # non-finite norm
+    assert nrm[1] == 0.0 and np.all(c[3:5] == 0)           # x = 0 -> D(x) = 0 (Def. 3)
+    assert np.isnan(nrm[2]) and np.all(c[5:7] == 0)        # NaN norm: no ratio to round
+    assert np.isinf(nrm[3]) and np.all(c[7:10] == 0)       # infinite norm: the same
     assert np.any(c[0:3] > 0)
     dec = np.zeros(10, np.float32)
     oracle.nd_decode_accumulate(nrm, level, sign, off, 4, dec)
+    # level code 0 stands for the value 0 whatever the norm: the compressed bucket adds zeros,
+    # and its stored norm is what tells the receiver that the bucket was not finite
     assert np.all(dec[3:] == 0) and not np.any(np.isnan(dec))
     assert (sign[0] >> 6) & 1 == 1 and (sign[0] >> 5) & 1 == 0   # sign plane keeps sign(x)
+
+
+def test_dnat_decode_under_a_norm_that_is_not_finite():
+    """Def. 3: the decoded entry is norm * sign * 2^(c-s) for c > 0 and 0 for c = 0.  With an
+    infinite norm every non-zero level therefore decodes to an infinity of the entry's sign, with
+    a NaN norm to NaN; level 0 stays a zero.  Expected values written out by hand."""
+    s = 3
+    codes = np.uint8([0, 1, 2, 3, 0, 1, 2, 3])
+    level = (codes[0::2] | (codes[1::2] << 4)).astype(np.uint8)
+    sign = np.uint32([0b10100110])                # entries 1, 2, 5, 7 negative
+    inf = np.float32(np.inf)
+    acc = np.zeros(8, np.float32)
+    oracle.nd_decode_accumulate(np.float32([np.inf]), level, sign, [0, 8], s, acc)
+    want = np.float32([0.0, -inf, -inf, inf, 0.0, -inf, inf, -inf])
+    assert np.array_equal(acc, want)
+    acc = np.full(8, 5.0, np.float32)
+    oracle.nd_decode_accumulate(np.float32([np.nan]), level, sign, [0, 8], s, acc)
+    assert np.array_equal(np.isnan(acc), codes > 0)
+    assert np.all(acc[codes == 0] == 5.0)
+    # two workers, one with an infinite norm: the column sums show it (inf, or inf - inf = NaN)
+    out = oracle.nd_aggregate([np.float32([np.inf]), np.float32([2.0])], [level, level],
+                              [sign, sign], [0, 8], s, 8)
+    assert np.array_equal(out, np.float32([0.0, -inf, -inf, inf, 0.0, -inf, inf, -inf]))
+    out = oracle.nd_aggregate([np.float32([np.inf]), np.float32([np.inf])], [level, level],
+                              [sign, ~sign], [0, 8], s, 8)
+    assert np.array_equal(np.isnan(out), codes > 0) and np.all(out[codes == 0] == 0)
+    # the sparse decoders follow the same rule
+    idx = np.uint32([1, 4, 6])
+    sp = np.uint8([0x0 | (0xB << 4), 0x2])        # codes (sign<<3 | level): 0, 8|3, 2
+    acc = np.zeros(8, np.float32)
+    oracle.sparse_decode_accumulate(idx, sp, 3, np.float32(np.inf), 4, acc)
+    assert np.array_equal(acc, np.float32([0, 0, 0, 0, -inf, 0, inf, 0]))
+
+
+def test_dnat_bucket_with_a_subnormal_norm_is_an_ordinary_bucket():
+    """y = |x| / norm does not change when a bucket is multiplied by a power of two (Def. 3), so
+    neither do the level codes: a bucket of tiny entries, subnormal norm included, must get the
+    codes of the same bucket scaled up by 2^100, in both arithmetic modes, and stays unbiased."""
+    rng = np.random.default_rng(11)
+    big = (rng.standard_normal(4000) * 0.3).astype(np.float32)
+    big = np.ldexp(np.round(np.ldexp(big, 20)), -20).astype(np.float32)   # 21 significant bits
+    tiny = np.ldexp(big, -128).astype(np.float32)                        # exact: multiples of 2^-148
+    assert np.array_equal(np.ldexp(tiny.astype(np.float64), 128), big.astype(np.float64))
+    off = [0, 1000, 4000]
+    for p in (1, 2, oracle.P_INF):
+        nb, lb, sb = oracle.nd_compress(big, off, p, 8, seed=3, worker=2)
+        if p == oracle.P_INF:
+            nt, lt, st = oracle.nd_compress(tiny, off, p, 8, seed=3, worker=2)
+            assert np.all(nt < 2.0 ** -126) and np.all(nt > 0)
+            assert np.array_equal(np.ldexp(nt.astype(np.float64), 128), nb.astype(np.float64))
+            assert np.array_equal(lt, lb) and np.array_equal(st, sb)
+        # given-norm arithmetic (binary32 reciprocal and multiply), norms scaled exactly
+        g_big = oracle.nd_compress(big, off, p, 8, seed=3, worker=2, given_norms=nb)
+        g_norm = np.ldexp(nb.astype(np.float64), -128).astype(np.float32)
+        if np.array_equal(np.ldexp(g_norm.astype(np.float64), 128), nb.astype(np.float64)):
+            g_tiny = oracle.nd_compress(tiny, off, p, 8, seed=3, worker=2, given_norms=g_norm)
+            assert np.array_equal(g_tiny[1], g_big[1]) and np.array_equal(g_tiny[2], g_big[2])
+    # unbiased: the mean decoded value over many seeds approaches x (max-norm, s = 4)
+    x = np.ldexp(np.float32([1.0, -0.75, 0.3125, 0.046875]), -140).astype(np.float32)
+    tot = np.zeros(4, np.float64)
+    reps = 4000
+    for seed in range(reps):
+        nrm, lv, sg = oracle.nd_compress(x, [0, 4], oracle.P_INF, 4, seed=seed, worker=0)
+        acc = np.zeros(4, np.float32)
+        oracle.nd_decode_accumulate(nrm, lv, sg, [0, 4], 4, acc)
+        tot += np.ldexp(acc.astype(np.float64), 140)
+    mean = tot / reps
+    want = np.float64([1.0, -0.75, 0.3125, 0.046875])
+    # standard error of one entry is at most (gap between its levels) / 2 / sqrt(reps)
+    assert np.all(np.abs(mean - want) <= 4 * 0.25 / np.sqrt(reps))
+    assert mean[0] == 1.0
 
 
 def test_dnat_decode_is_norm_times_power_of_two_in_binary32():

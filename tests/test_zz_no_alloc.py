@@ -60,9 +60,20 @@ def test_static_scratch_variant_matches_nd_compress_twice_in_a_row():
 
 
 def test_static_scratch_variant_rejects_sizes_beyond_its_array():
-    d = 200_000_000                             # needs about 2.3 MiB of scratch
-    assert nc.nd_workspace_bytes(d, 161) > nc.nd_static_scratch_bytes()
-    fake = 1 << 20                              # never dereferenced: the call must not launch
+    # A short vector cut into very many (mostly empty) buckets needs more scratch than the array
+    # holds.  Every buffer is real and large enough, so if the size check ever stopped working the
+    # call would run a valid problem and the test would fail on the status, not fault the device.
+    d, B = 1024, 200_000
+    assert nc.nd_workspace_bytes(d, B) > nc.nd_static_scratch_bytes()
+    off = torch.zeros(B + 1, dtype=torch.int64, device="cuda")
+    off[B // 2:] = d // 2
+    off[B] = d
+    x = torch.ones(d, dtype=torch.float32, device="cuda")
+    norms = torch.full((B,), -1.0, dtype=torch.float32, device="cuda")
+    level = torch.zeros(nc.nd_level_bytes(d), dtype=torch.uint8, device="cuda")
+    sign = torch.zeros(nc.nc_sign_bytes(d), dtype=torch.uint8, device="cuda")
     with pytest.raises(nc.NatcompError) as err:
-        nc.nd_compress_static(fake, d, fake, 161, 2, 8, 0, 0, fake, fake, fake)
+        nc.nd_compress_static(x, d, off, B, 2, 8, 0, 0, norms, level, sign)
     assert nc.status_string(err.value.status) == "NC_ERR_TOO_LARGE"
+    torch.cuda.synchronize()
+    assert bool(torch.all(norms == -1.0))       # nothing was launched
