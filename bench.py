@@ -1,25 +1,35 @@
 #!/usr/bin/env python
 """Benchmark of the natural-compression hot path on B200.
 
-One step = one pass of the whole path over one batch of synthetic gradients, on the
-ResNet-50-shaped workload (n = 8 workers, d = 25,557,032 fp32 entries in 161 buckets):
-  C_nat  : nc_compress_batch (8 workers, one launch) + nc_aggregate
-  D_nat  : nd_compress x 8 (p = 2, s = 8, per-bucket norms) + nd_aggregate
-  sparse : nd_sparse_compact_compress_batch (keep 1 %, p = inf, s = 4, 3-bit codes)
-           + nd_sparse_compact_aggregate (all workers, one launch)
-  ref    : nc_sum_fp32 (uncompressed 8-way sum, the reference point)
-The metric is worker-entries taken through the whole path per second (n * d per step).
-Inputs (818 MB) are larger than the 126 MB L2, so no flush is needed between steps.
+Headline workload (c4, the largest configuration that fits one GPU): n = 16 workers, each an
+fp32 gradient of d = 335,141,888 entries (Student-t(3) * 1e-4).  One step = one pass of the path
+over that batch:
+    nc_compress_batch   C_nat of the 16 vectors, one launch          (worker side)
+    nc_aggregate        fixed-order fp32 sum of the 16 packed buffers (master side)
+    nc_sum_fp32         the uncompressed 16-way sum of the same buffers (reference point)
+`value` = n * d worker-entries per step / step time.  Inputs are 21.45 GB, far larger than the
+126 MB L2, so nothing is flushed between steps.
+
+The other four configurations run as legs of the same invocation (rank 0, N = 1) and are
+reported per call under `kernels`:
+    c1  d = 2^20, n = 4             nc_compress_batch, nc_aggregate (launch-bound, L2-resident)
+    c2  ResNet-50 shape, n = 8      nc_compress_batch, nc_aggregate, nc_sum_fp32
+    c3  same buffers, D_nat^{2,8}   nd_norms_batch, nd_round_batch, nd_compress_batch, nd_aggregate
+    c5  d = 2^28, n = 8, keep 1 %   nd_sparse_compact_compress_batch, nd_sparse_compact_aggregate
+Every leg is timed for at least --leg-seconds with an event after every call, while the SM clock
+is sampled; each call is reported against the measured copy bandwidth and the nominal 8 TB/s.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
-With N > 1 (under torchrun) every rank runs an independent replica of the same workload
+With N > 1 (under torchrun) every rank runs an independent replica of the headline workload
 ("replicas only": the path has no exchange step on one node) and the value is the sum.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
 """
 import argparse
+import importlib.util
 import json
 import os
+import statistics
 import sys
 import threading
 import time
@@ -31,19 +41,24 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-N_WORKERS = 8
+METRIC = "compress + decode-accumulate throughput (worker-entries through the whole path)"
+UNIT = "Gelem/s"
+NOMINAL_HBM_GBPS = 8000.0
+C4_N, C4_D = 16, 335_141_888
 P_DITHER, S_DITHER = 2, 8
 S_SPARSE = 4
 SPARSE_CAP_FRACTION = 0.0125
-METRIC = "hot-path throughput (C_nat + D_nat + sparse compress / decode-accumulate)"
-UNIT = "Gelem/s"
+CPU_SAMPLE_D = 1 << 22            # entries per worker of the oracle's bounded sample
 
-# Per-launch DRAM traffic of the dominant kernel (nc_compress_kernel, 8-worker batch launch):
-# dram__bytes_read.sum + dram__bytes_write.sum of the 2-worker capture summarised in
-# profiles/nc_compress_c2_2workers.md (204.48 MB + 31.59 MB), scaled by 4 to the 8-worker launch
-# (traffic is proportional to the number of workers).  The write part is below the 28.75 MB per
-# worker that the kernel stores because some output is still dirty in L2 when the kernel ends.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * (204_482_816 + 31_589_376)
+
+def load_workloads():
+    """The seeded input generators, loaded by file path: they hold none of the method's
+    arithmetic, and the reference arm must be able to use them without the CUDA library."""
+    spec = importlib.util.spec_from_file_location(
+        "_natcomp_workloads", os.path.join(ROOT, "paper_1905_10988_b200", "workloads.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod
 
 
 def measured_hbm_peak():
@@ -55,8 +70,19 @@ def measured_hbm_peak():
         return 6650.0, "fallback"
 
 
+def ncu_traffic_per_entry(kernel):
+    """DRAM bytes (read + written) per worker-entry that an ncu capture of `kernel` showed, from
+    the table kept beside the profile summaries; None when the table has no such row."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")) as f:
+            row = json.load(f)["kernels"][kernel]
+        return float(row["dram_bytes_per_entry"]), row.get("capture")
+    except Exception:
+        return None, None
+
+
 class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML (read-only) while a timed region runs."""
 
     def __init__(self, index, period=0.02):
         super().__init__(daemon=True)
@@ -105,7 +131,8 @@ class ClockSampler(threading.Thread):
         self.join(timeout=2)
         med = int(np.median(self.samples)) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "samples": len(self.samples),
+                "sm_mhz_min": min(self.samples) if self.samples else None}
 
 
 def physical_gpu_index(local_rank):
@@ -118,193 +145,322 @@ def physical_gpu_index(local_rank):
     return local_rank
 
 
-DOMINANT_MARKS = ("start", "nc_compress")
+# ---------------------------------------------------------------------------------------------
+# headline workload
 
 
-class HotPath:
-    """Device buffers for one replica of the workload and the sequence of C-ABI calls of a step."""
+class HeadlineC4:
+    """Device buffers of one replica of workload c4 and the C-ABI calls of a step."""
 
-    GROUPS = ("nc_compress", "nc_aggregate", "nd_compress", "nd_aggregate", "sparse_compress",
-              "sparse_accumulate", "sum_fp32")
+    GROUPS = ("nc_compress", "nc_aggregate", "sum_fp32")
+    KERNEL_OF = {"nc_compress": "nc_compress_kernel", "nc_aggregate": "nc_aggregate_kernel",
+                 "sum_fp32": "nc_sum_fp32_kernel"}
+    LAUNCHES_PER_STEP = 3
 
-    def __init__(self, nc, rank, device, n_workers=N_WORKERS, only=None):
-        from paper_1905_10988_b200 import workloads
-        self.nc = nc
-        self.n = n_workers
-        self.only = only
-        sizes = workloads.resnet50_tensor_sizes()
-        off = workloads.offsets_from_sizes(sizes)
-        self.d, self.B = off[-1], len(sizes)
-        n, d, B = self.n, self.d, self.B
-        u8 = dict(dtype=torch.uint8, device=device)
-        f32 = dict(dtype=torch.float32, device=device)
+    def __init__(self, nc, workloads, rank, device, n=C4_N, d=C4_D):
         from paper_1905_10988_b200 import timing
+        self.nc, self.n, self.d = nc, n, d
+        u8 = dict(dtype=torch.uint8, device=device)
         self.workers = timing.replica_worker_ids(rank, n)
-        self.x = [workloads.config2_vector(w, device, sizes) for w in self.workers]
-        self.off = torch.tensor(off, dtype=torch.int64, device=device)
+        self.x = [workloads.config4_vector(w, d, device) for w in self.workers]
         self.exp = [torch.empty(nc.nc_exp_bytes(d), **u8) for _ in range(n)]
         self.sign = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
-        self.out_nc = torch.empty(d, **f32)
-        self.norms = [torch.empty(B, **f32) for _ in range(n)]
-        self.level = [torch.empty(nc.nd_level_bytes(d), **u8) for _ in range(n)]
-        self.sign_nd = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
-        self.ws_bytes = nc.nd_batch_workspace_bytes(d, B, n)
-        self.ws = torch.empty(self.ws_bytes, **u8)
-        self.out_nd = torch.empty(d, **f32)
-        self.cap = int(d * SPARSE_CAP_FRACTION)
-        self.idx = [torch.empty(self.cap, dtype=torch.int32, device=device) for _ in range(n)]
-        self.codes = [torch.empty(nc.nd_sparse_plane_bytes(self.cap, S_SPARSE), **u8)
-                      for _ in range(n)]
-        self.count = [torch.zeros(1, dtype=torch.int32, device=device) for _ in range(n)]
-        self.snorm = [torch.zeros(1, **f32) for _ in range(n)]
-        self.sws_bytes = nc.nd_sparse_batch_workspace_bytes(d, self.cap, n)
-        self.sws = torch.empty(self.sws_bytes, **u8)
-        self.out_sp = torch.empty(d, **f32)
-        self.out_sum = torch.empty(d, **f32)
-        # nc_compress_batch 1, nc_aggregate 1, nd_compress_batch 3, nd_aggregate 1,
-        # nd_sparse_compact_compress_batch 6, nd_sparse_compact_aggregate 1, nc_sum_fp32 1
-        self.launches_per_step = 1 + 1 + 3 + 1 + 6 + 1 + 1
+        self.out_nc = torch.empty(d, dtype=torch.float32, device=device)
+        self.out_sum = torch.empty(d, dtype=torch.float32, device=device)
+        self.outputs = (self.out_nc, self.out_sum)
         self.seed = 0
 
-    def step(self, marks=None, mark_names=None):
-        nc, n, d, B = self.nc, self.n, self.d, self.B
-        from paper_1905_10988_b200 import workloads
+    def step(self, marks=None):
+        nc, n, d = self.nc, self.n, self.d
 
         def mark(name):
-            if marks is not None and (mark_names is None or name in mark_names):
+            if marks is not None:
                 ev = torch.cuda.Event(enable_timing=True)
                 ev.record()
                 marks.append((name, ev))
 
-        def want(name):
-            return self.only is None or self.only == name
-
         mark("start")
-        if want("nc_compress"):
-            nc.nc_compress_batch(self.x, d, self.seed, self.workers, self.exp, self.sign, n)
+        nc.nc_compress_batch(self.x, d, self.seed, self.workers, self.exp, self.sign, n)
         mark("nc_compress")
-        if want("nc_aggregate"):
-            nc.nc_aggregate(self.exp, self.sign, n, d, self.out_nc)
+        nc.nc_aggregate(self.exp, self.sign, n, d, self.out_nc)
         mark("nc_aggregate")
-        if want("nd_compress"):
-            nc.nd_compress_batch(self.x, d, self.off, B, P_DITHER, S_DITHER, self.seed,
-                                 self.workers, self.norms, self.level, self.sign_nd, n, self.ws,
-                                 self.ws_bytes)
-        mark("nd_compress")
-        if want("nd_aggregate"):
-            nc.nd_aggregate(self.norms, self.level, self.sign_nd, n, d, self.off, B, S_DITHER,
-                            self.out_nd)
-        mark("nd_aggregate")
-        if want("sparse_compress"):
-            nc.nd_sparse_compact_compress_batch(self.x, d, workloads.KEEP_1PCT_THRESHOLD,
-                                                workloads.KEEP_1PCT_SCALE, nc.P_INF, S_SPARSE,
-                                                self.seed, self.workers, self.idx, self.codes,
-                                                self.count, self.snorm, self.cap, n, self.sws,
-                                                self.sws_bytes)
-        mark("sparse_compress")
-        if want("sparse_accumulate"):
-            nc.nd_sparse_compact_aggregate(self.idx, self.codes, self.count, self.snorm, n,
-                                           S_SPARSE, d, self.cap, self.out_sp)
-        mark("sparse_accumulate")
-        if want("sum_fp32"):
-            nc.nc_sum_fp32(self.x, n, d, self.out_sum)
+        nc.nc_sum_fp32(self.x, n, d, self.out_sum)
         mark("sum_fp32")
 
-    STREAM_GROUPS = (("nc_compress", "nc_aggregate"), ("nd_compress", "nd_aggregate"),
-                     ("sparse_compress", "sparse_accumulate"), ("sum_fp32",))
-
-    def step_on_streams(self, streams):
-        """The same step with its four independent call chains on four streams (fork from the
-        current stream, join back into it): the HBM-bound and the integer-bound kernels of
-        different chains overlap at their tails."""
-        main = torch.cuda.current_stream()
-        fork = torch.cuda.Event()
-        fork.record(main)
-        keep = self.only
-        for stream, chain in zip(streams, self.STREAM_GROUPS):
-            stream.wait_event(fork)
-            with torch.cuda.stream(stream):
-                for g in chain:
-                    self.only = g
-                    self.step()
-            done = torch.cuda.Event()
-            done.record(stream)
-            main.wait_event(done)
-        self.only = keep
-
     def algorithmic_bytes(self):
-        """Compulsory HBM bytes per call group (per step)."""
         n, d = self.n, self.d
-        kept = 0.01 * d
-        return {
-            "nc_compress": n * d * (4 + 1.125),
-            "nc_aggregate": d * (1.125 * n + 4),
-            "nd_compress": n * d * (4 + 4 + 0.625),        # x is read by the norm and rounding passes
-            "nd_aggregate": d * (0.625 * n + 4),
-            # kept entries are read as 32-byte sectors in three passes (norm, filter, emit);
-            # about half of them survive the level-0 filter and are listed (4 B index + 3 bits)
-            "sparse_compress": n * kept * (3 * 32 + 0.5 * 4.375),
-            # dense output written once; the listed entries (about half of the kept) read once
-            "sparse_accumulate": 4 * d + n * kept * 0.5 * 4.375,
-            "sum_fp32": d * (4 * n + 4),
-        }
+        return {"nc_compress": n * d * (4 + 1.125), "nc_aggregate": d * (1.125 * n + 4),
+                "sum_fp32": d * (4 * n + 4)}
+
+    def units(self):
+        return {"nc_compress": self.n * self.d, "nc_aggregate": self.d, "sum_fp32": self.d}
 
 
-def cpu_baseline_sample(steps=1):
-    """Times the CPU oracle, as it stands, on a bounded sample of the same workload: the first
-    tensors of the ResNet-50 layout (about 1.6 M entries) for all 8 workers, whole path."""
-    import oracle
-    from paper_1905_10988_b200 import workloads
-    sizes_all = workloads.resnet50_tensor_sizes()
-    sizes, tot = [], 0
-    for s in sizes_all:
-        if tot + s > 1_700_000:
-            break
-        sizes.append(s)
-        tot += s
+# ---------------------------------------------------------------------------------------------
+# legs: the other configurations, one call after the other with an event after each
+
+
+def time_sequence(calls, min_seconds, gpu_index, max_iters=20000):
+    """Runs the sequence of (name, fn) repeatedly for at least `min_seconds` of device time, an
+    event after every call, the SM clock sampled meanwhile.  Returns per call the list of
+    device times in ms, and the clock record."""
+    for _ in range(3):
+        for _, fn in calls:
+            fn()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _, fn in calls:
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    one = max(e0.elapsed_time(e1), 1e-3)
+    iters = int(min(max_iters, max(20, min_seconds * 1e3 / one + 1)))
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
+    rows = []
+    done = 0
+    while done < iters:                       # in batches, so that events do not pile up
+        batch = min(200, iters - done)
+        evs = []
+        for _ in range(batch):
+            row = [torch.cuda.Event(enable_timing=True)]
+            row[0].record()
+            for _, fn in calls:
+                fn()
+                ev = torch.cuda.Event(enable_timing=True)
+                ev.record()
+                row.append(ev)
+            evs.append(row)
+        torch.cuda.synchronize()
+        for row in evs:
+            rows.append([a.elapsed_time(b) for a, b in zip(row[:-1], row[1:])])
+        done += batch
+    clocks = sampler.stop()
+    per_call = {name: [r[i] for r in rows] for i, (name, _) in enumerate(calls)}
+    return per_call, clocks, iters
+
+
+def summarize_call(times_ms, nbytes, units, unit_name, peak, clocks, extra=None):
+    mean = sum(times_ms) / len(times_ms)
+    med = statistics.median(times_ms)
+    out = {"ms": round(mean, 5), "ms_median": round(med, 5), "ms_best": round(min(times_ms), 5)}
+    if nbytes:
+        gbps = nbytes / mean / 1e6
+        out.update({"algorithmic_GBps": round(gbps, 1),
+                    "frac_of_measured_peak": round(gbps / peak, 4),
+                    "frac_of_nominal_8TBps": round(gbps / NOMINAL_HBM_GBPS, 4)})
+    if units:
+        out[unit_name] = round(units / mean / 1e6, 1)
+    if clocks.get("sm_mhz"):
+        # time x clock: comparable across runs that settled at different SM clocks
+        out["ms_x_sm_mhz"] = round(mean * clocks["sm_mhz"], 2)
+    if extra:
+        out.update(extra)
+    return out
+
+
+def leg_c1(nc, workloads, device, peak, seconds, gpu_index):
+    n, d = 4, 1 << 20
+    u8 = dict(dtype=torch.uint8, device=device)
+    # two buffer sets used in turn; all of it (21 MB) stays L2-resident either way
+    sets = []
+    for k in range(2):
+        xs = [workloads.config1_vector(w, d, device) for w in range(n)]
+        es = [torch.empty(nc.nc_exp_bytes(d), **u8) for _ in range(n)]
+        ss = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
+        sets.append((xs, es, ss, torch.empty(d, dtype=torch.float32, device=device)))
+    state = {"k": 0}
+    workers = list(range(n))
+
+    def compress():
+        state["k"] ^= 1
+        xs, es, ss, _ = sets[state["k"]]
+        nc.nc_compress_batch(xs, d, 0, workers, es, ss, n)
+
+    def aggregate():
+        _, es, ss, out = sets[state["k"]]
+        nc.nc_aggregate(es, ss, n, d, out)
+
+    t, clocks, iters = time_sequence([("nc_compress_batch", compress), ("nc_aggregate", aggregate)],
+                                     min(seconds, 0.3), gpu_index)
+    note = {"note": "launch-bound and L2-resident (21 MB): the time is what counts, not the fraction"}
+    return {
+        "workload": "c1: d=2^20, n=4, N(0,1e-3^2) + 1% zeros + 0.1% powers of two",
+        "iterations": iters, "clocks": clocks,
+        "nc_compress_batch": summarize_call(t["nc_compress_batch"], n * d * 5.125, n * d,
+                                            "Gelem_per_s", peak, clocks, note),
+        "nc_aggregate": summarize_call(t["nc_aggregate"], d * (1.125 * n + 4), d, "Gelem_per_s",
+                                       peak, clocks, note),
+    }
+
+
+def leg_c2_c3(nc, workloads, device, peak, seconds, gpu_index):
+    n = 8
+    sizes = workloads.resnet50_tensor_sizes()
     off = workloads.offsets_from_sizes(sizes)
-    d, n = off[-1], N_WORKERS
-    xs = [workloads.config2_vector(w, "cpu", sizes).numpy() for w in range(n)]
-    times = []
-    for _ in range(steps):
+    d, B = off[-1], len(sizes)
+    u8 = dict(dtype=torch.uint8, device=device)
+    f32 = dict(dtype=torch.float32, device=device)
+    xs = [workloads.config2_vector(w, device, sizes) for w in range(n)]
+    workers = list(range(n))
+    es = [torch.empty(nc.nc_exp_bytes(d), **u8) for _ in range(n)]
+    ss = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
+    out = torch.empty(d, **f32)
+    out2 = torch.empty(d, **f32)
+    t, clocks, iters = time_sequence([
+        ("nc_compress_batch", lambda: nc.nc_compress_batch(xs, d, 0, workers, es, ss, n)),
+        ("nc_aggregate", lambda: nc.nc_aggregate(es, ss, n, d, out)),
+        ("nc_sum_fp32", lambda: nc.nc_sum_fp32(xs, n, d, out2)),
+    ], seconds, gpu_index)
+    c2 = {
+        "workload": "c2: ResNet-50-shaped gradients, d=25,557,032 in 161 tensors, n=8",
+        "iterations": iters, "clocks": clocks,
+        "nc_compress_batch": summarize_call(t["nc_compress_batch"], n * d * 5.125, n * d,
+                                            "Gelem_per_s", peak, clocks),
+        "nc_aggregate": summarize_call(t["nc_aggregate"], d * (1.125 * n + 4), d, "Gelem_per_s",
+                                       peak, clocks),
+        "nc_sum_fp32": summarize_call(t["nc_sum_fp32"], d * (4 * n + 4), d, "Gelem_per_s", peak,
+                                      clocks),
+    }
+    del es, ss
+    # c3: D_nat^{2,8} on the same buffers; the norm pass and the rounding pass also on their own
+    offd = torch.tensor(off, dtype=torch.int64, device=device)
+    norms = [torch.empty(B, **f32) for _ in range(n)]
+    levels = [torch.empty(nc.nd_level_bytes(d), **u8) for _ in range(n)]
+    signs = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
+    wsb = nc.nd_batch_workspace_bytes(d, B, n)
+    ws = torch.empty(wsb, **u8)
+    t, clocks, iters = time_sequence([
+        ("nd_norms_batch", lambda: nc.nd_norms_batch(xs, d, offd, B, P_DITHER, norms, n, ws, wsb)),
+        ("nd_round_batch", lambda: nc.nd_round_batch(xs, d, offd, B, S_DITHER, 0, workers, norms,
+                                                     levels, signs, n)),
+        ("nd_compress_batch", lambda: nc.nd_compress_batch(xs, d, offd, B, P_DITHER, S_DITHER, 0,
+                                                           workers, norms, levels, signs, n, ws,
+                                                           wsb)),
+        ("nd_aggregate", lambda: nc.nd_aggregate(norms, levels, signs, n, d, offd, B, S_DITHER,
+                                                 out)),
+    ], seconds, gpu_index)
+    two_reads = {"bytes_counted": "x once (4 + 0.625 B per entry); the call reads x twice from "
+                                  "HBM where a bucket does not stay on chip"}
+    c3 = {
+        "workload": "c3: D_nat^{2,8} on the c2 buffers (161 buckets), n=8",
+        "iterations": iters, "clocks": clocks,
+        "nd_norms_batch": summarize_call(t["nd_norms_batch"], n * d * 4.0, n * d, "Gelem_per_s",
+                                         peak, clocks),
+        "nd_round_batch": summarize_call(t["nd_round_batch"], n * d * 4.625, n * d, "Gelem_per_s",
+                                         peak, clocks),
+        "nd_compress_batch": summarize_call(t["nd_compress_batch"], n * d * 4.625, n * d,
+                                            "Gelem_per_s", peak, clocks, two_reads),
+        "nd_aggregate": summarize_call(t["nd_aggregate"], d * (0.625 * n + 4), d, "Gelem_per_s",
+                                       peak, clocks),
+    }
+    return c2, c3
+
+
+def leg_c5(nc, workloads, device, peak, seconds, gpu_index, sm_count):
+    n, d = 8, 1 << 28
+    u8 = dict(dtype=torch.uint8, device=device)
+    xs = [workloads.config5_vector(w, d, device) for w in range(n)]
+    workers = list(range(n))
+    cap = int(d * SPARSE_CAP_FRACTION)
+    idx = [torch.empty(cap, dtype=torch.int32, device=device) for _ in range(n)]
+    planes = [torch.empty(nc.nd_sparse_plane_bytes(cap, S_SPARSE), **u8) for _ in range(n)]
+    count = [torch.zeros(1, dtype=torch.int32, device=device) for _ in range(n)]
+    norm = [torch.zeros(1, dtype=torch.float32, device=device) for _ in range(n)]
+    wsb = nc.nd_sparse_batch_workspace_bytes(d, cap, n)
+    ws = torch.empty(wsb, **u8)
+    out = torch.empty(d, dtype=torch.float32, device=device)
+    t, clocks, iters = time_sequence([
+        ("nd_sparse_compact_compress_batch", lambda: nc.nd_sparse_compact_compress_batch(
+            xs, d, workloads.KEEP_1PCT_THRESHOLD, workloads.KEEP_1PCT_SCALE, nc.P_INF, S_SPARSE, 0,
+            workers, idx, planes, count, norm, cap, n, ws, wsb)),
+        ("nd_sparse_compact_aggregate", lambda: nc.nd_sparse_compact_aggregate(
+            idx, planes, count, norm, n, S_SPARSE, d, cap, out)),
+    ], seconds, gpu_index)
+    listed = int(sum(int(c.cpu().numpy().view(np.uint32)[0]) for c in count))
+    kept = 0.01 * d * n
+    mhz = clocks.get("sm_mhz") or 1965
+    # the selection draws one generator block (18 wide multiplies) per 4 coordinates; a
+    # sub-partition issues one wide multiply per 4 cycles
+    ceiling = sm_count * 4 * 32 * mhz * 1e6 / 4 / 4.5 / 1e9
+    comp = summarize_call(t["nd_sparse_compact_compress_batch"],
+                          kept * 32 + listed * 4.375, n * d, "Gcoord_per_s", peak, clocks,
+                          {"bound": "alu", "generator_ceiling_Gcoord_per_s": round(ceiling, 1)})
+    comp["frac_of_generator_ceiling"] = round(comp["Gcoord_per_s"] / ceiling, 4)
+    return {
+        "workload": "c5: d=2^28, n=8, N(0,1), keep 1% then D_nat^{inf,4}, index list + 3-bit codes",
+        "iterations": iters, "clocks": clocks, "listed_entries": listed,
+        "nd_sparse_compact_compress_batch": comp,
+        "nd_sparse_compact_aggregate": summarize_call(
+            t["nd_sparse_compact_aggregate"], 4.0 * d + listed * 4.375, d, "Gelem_per_s", peak,
+            clocks),
+    }
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle legs
+
+
+def cpu_sample_inputs(workloads, d=CPU_SAMPLE_D, n=C4_N):
+    return [workloads.config4_vector(w, d, "cpu").numpy() for w in range(n)]
+
+
+def cpu_oracle_step(oracle, xs):
+    """The headline step on the oracle, as it stands."""
+    d = xs[0].size
+    packed = [oracle.nc_compress(x, 0, w) for w, x in enumerate(xs)]
+    oracle.nc_aggregate([p[0] for p in packed], [p[1] for p in packed], d)
+    oracle.sum_fp32(xs)
+
+
+def cpu_baseline(workloads):
+    import oracle
+    xs = cpu_sample_inputs(workloads)
+    units = len(xs) * xs[0].size
+    all_cores = oracle.max_threads()
+    cpu_oracle_step(oracle, [x[:4096] for x in xs])          # first call builds / loads
+    res = {}
+    for label, threads in (("one_thread", 1), ("all_cores", all_cores)):
+        oracle.set_threads(threads)
         t0 = time.perf_counter()
-        packed = [oracle.nc_compress(xs[w], 0, w) for w in range(n)]
-        oracle.nc_aggregate([p[0] for p in packed], [p[1] for p in packed], d)
-        dn = [oracle.nd_compress(xs[w], off, P_DITHER, S_DITHER, 0, w) for w in range(n)]
-        oracle.nd_aggregate([q[0] for q in dn], [q[1] for q in dn], [q[2] for q in dn], off,
-                            S_DITHER, d)
-        acc = np.zeros(d, np.float32)
-        for w in range(n):
-            idx, planes, count, nrm = oracle.sparse_compact_compress(
-                xs[w], workloads.KEEP_1PCT_THRESHOLD, workloads.KEEP_1PCT_SCALE, oracle.P_INF,
-                S_SPARSE, 0, w)
-            oracle.sparse_compact_decode_accumulate(idx, planes, count, nrm, S_SPARSE, acc)
-        oracle.sum_fp32(xs)
-        times.append(time.perf_counter() - t0)
-    sample = ("first %d tensors of the ResNet-50 layout (%d entries) x %d workers, whole path; "
-              "C_nat and the sums use OpenMP over entries, D_nat and sparse legs are serial"
-              % (len(sizes), d, n))
-    return n * d, times, oracle.max_threads(), sample
+        cpu_oracle_step(oracle, xs)
+        res[label] = {"value": units / (time.perf_counter() - t0) / 1e9, "cores": threads}
+    oracle.set_threads(all_cores)
+    sample = ("the headline step (C_nat of 16 workers, 16-way aggregate, 16-way fp32 sum) on the "
+              "first %d entries' worth of each worker's c4 vector (%d worker-entries), OpenMP "
+              "over entries" % (xs[0].size, units))
+    return {"value": res["all_cores"]["value"], "unit": UNIT, "cores": all_cores, "kind": "oracle",
+            "sample": sample, "one_thread": res["one_thread"]["value"]}
 
 
 def run_reference(args, rank):
     if rank != 0:
         return
-    units, times, cores, sample = cpu_baseline_sample(steps=1)      # untimed warm-up of the build
-    all_t = []
-    for _ in range(max(1, args.warmup) - 1):
-        cpu_baseline_sample(steps=1)
+    import oracle
+    workloads = load_workloads()
+    xs = cpu_sample_inputs(workloads)
+    units = len(xs) * xs[0].size
+    cores = oracle.max_threads()
+    cpu_oracle_step(oracle, [x[:4096] for x in xs])
+    for _ in range(min(args.warmup, 3)):
+        cpu_oracle_step(oracle, [x[:1 << 18] for x in xs])
+    times = []
     for _ in range(args.steps):
-        _, t, _, _ = cpu_baseline_sample(steps=1)
-        all_t.extend(t)
-    total = sum(all_t)
-    value = units * len(all_t) / total / 1e9
+        t0 = time.perf_counter()
+        cpu_oracle_step(oracle, xs)
+        times.append(time.perf_counter() - t0)
+    total = sum(times)
+    value = units * len(times) / total / 1e9
+    sample = ("every step = the headline step on the first %d entries of each of the 16 c4 "
+              "vectors (%d worker-entries), all host cores" % (xs[0].size, units))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(all_t),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32+f32",
         "data": "synthetic",
-        "config": {"workload": "c2: ResNet-50-shaped gradients, n=8 workers (bounded sample)"},
+        "config": {"workload": "c4: n=16 workers, d=335,141,888 fp32 entries each (bounded sample)"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -313,18 +469,92 @@ def run_reference(args, rank):
     print(json.dumps(line))
 
 
+# ---------------------------------------------------------------------------------------------
+
+
+PROFILE_CASES = ("nc_compress", "nc_aggregate", "sum_fp32", "nd_norms", "nd_round", "nd_compress",
+                 "nd_aggregate", "sparse_compress", "sparse_aggregate")
+
+
+def run_profile_case(nc, workloads, args, device):
+    """Profiling aid: one call alone on a small case (the ResNet-50 shape with --workers workers,
+    larger than L2 from 2 workers on), timed with events; the command ncu captures."""
+    n = args.workers
+    sizes = workloads.resnet50_tensor_sizes()
+    off = workloads.offsets_from_sizes(sizes)
+    d, B = off[-1], len(sizes)
+    u8 = dict(dtype=torch.uint8, device=device)
+    f32 = dict(dtype=torch.float32, device=device)
+    xs = [workloads.config2_vector(w, device, sizes) for w in range(n)]
+    workers = list(range(n))
+    es = [torch.empty(nc.nc_exp_bytes(d), **u8) for _ in range(n)]
+    ss = [torch.empty(nc.nc_sign_bytes(d), **u8) for _ in range(n)]
+    out = torch.empty(d, **f32)
+    offd = torch.tensor(off, dtype=torch.int64, device=device)
+    norms = [torch.empty(B, **f32) for _ in range(n)]
+    levels = [torch.empty(nc.nd_level_bytes(d), **u8) for _ in range(n)]
+    wsb = nc.nd_batch_workspace_bytes(d, B, n)
+    ws = torch.empty(wsb, **u8)
+    cap = int(d * SPARSE_CAP_FRACTION)
+    idx = [torch.empty(cap, dtype=torch.int32, device=device) for _ in range(n)]
+    planes = [torch.empty(nc.nd_sparse_plane_bytes(cap, S_SPARSE), **u8) for _ in range(n)]
+    count = [torch.zeros(1, dtype=torch.int32, device=device) for _ in range(n)]
+    norm = [torch.zeros(1, **f32) for _ in range(n)]
+    swsb = nc.nd_sparse_batch_workspace_bytes(d, cap, n)
+    sws = torch.empty(swsb, **u8)
+    kept = 0.01 * d * n
+    cases = {
+        "nc_compress": (lambda: nc.nc_compress_batch(xs, d, 0, workers, es, ss, n), n * d * 5.125),
+        "nc_aggregate": (lambda: nc.nc_aggregate(es, ss, n, d, out), d * (1.125 * n + 4)),
+        "sum_fp32": (lambda: nc.nc_sum_fp32(xs, n, d, out), d * (4 * n + 4)),
+        "nd_norms": (lambda: nc.nd_norms_batch(xs, d, offd, B, P_DITHER, norms, n, ws, wsb),
+                     n * d * 4.0),
+        "nd_round": (lambda: nc.nd_round_batch(xs, d, offd, B, S_DITHER, 0, workers, norms, levels,
+                                               ss, n), n * d * 4.625),
+        "nd_compress": (lambda: nc.nd_compress_batch(xs, d, offd, B, P_DITHER, S_DITHER, 0, workers,
+                                                     norms, levels, ss, n, ws, wsb), n * d * 4.625),
+        "nd_aggregate": (lambda: nc.nd_aggregate(norms, levels, ss, n, d, offd, B, S_DITHER, out),
+                         d * (0.625 * n + 4)),
+        "sparse_compress": (lambda: nc.nd_sparse_compact_compress_batch(
+            xs, d, workloads.KEEP_1PCT_THRESHOLD, workloads.KEEP_1PCT_SCALE, nc.P_INF, S_SPARSE, 0,
+            workers, idx, planes, count, norm, cap, n, sws, swsb), kept * 34.2),
+        "sparse_aggregate": (lambda: nc.nd_sparse_compact_aggregate(
+            idx, planes, count, norm, n, S_SPARSE, d, cap, out), 4.0 * d + kept * 2.2),
+    }
+    # what the master-side calls read must exist first
+    for first in ("nc_compress", "nd_compress", "sparse_compress"):
+        cases[first][0]()
+    fn, nbytes = cases[args.profile]
+    for _ in range(args.warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    print(json.dumps({"profile": args.profile, "workers": n, "d": d, "ms": ms,
+                      "algorithmic_GBps": nbytes / ms / 1e6}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--e2e-steps", type=int, default=6)
-    ap.add_argument("--only", default=None, choices=list(HotPath.GROUPS),
-                    help="profiling aid: time one call group alone")
-    ap.add_argument("--workers", type=int, default=N_WORKERS,
-                    help="number of simulated workers with --only")
+    ap.add_argument("--no-legs", action="store_true", help="skip the c1, c2, c3 and c5 legs")
+    ap.add_argument("--leg-seconds", type=float, default=0.6,
+                    help="device time spent on each leg (the SM clock is sampled every 20 ms)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--profile", default=None, choices=list(PROFILE_CASES),
+                    help="profiling aid: time one call alone on the ResNet-50 shape")
+    ap.add_argument("--workers", type=int, default=2,
+                    help="number of simulated workers with --profile")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -339,42 +569,39 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     import paper_1905_10988_b200 as nc
-    from paper_1905_10988_b200 import timing
+    from paper_1905_10988_b200 import timing, workloads
 
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
+    gpu_index = physical_gpu_index(local_rank)
+    sm_count = torch.cuda.get_device_properties(device).multi_processor_count
     dist = None
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
 
-    if args.only:
-        # profiling aid: one call group alone, on a smaller case (still larger than L2)
-        hp = HotPath(nc, rank, device, n_workers=args.workers)
-        hp.step()                               # produces the planes the master-side calls read
-        hp.only = args.only
-        for _ in range(args.warmup):
-            hp.step()
-        torch.cuda.synchronize()
-        e0 = torch.cuda.Event(enable_timing=True)
-        e1 = torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(args.steps):
-            hp.step()
-        e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / args.steps
-        gb = hp.algorithmic_bytes()[args.only]
-        print(json.dumps({"only": args.only, "workers": hp.n, "d": hp.d, "ms": ms,
-                          "algorithmic_GBps": gb / ms / 1e6}))
+    if args.profile:
+        run_profile_case(nc, workloads, args, device)
         return
 
-    hp = HotPath(nc, rank, device)
+    peak, peak_kind = measured_hbm_peak()
+
+    # ---- legs first (their buffers are freed before the headline buffers are made)
+    legs = {}
+    if rank == 0 and world == 1 and not args.no_legs:
+        legs["c1"] = leg_c1(nc, workloads, device, peak, args.leg_seconds, gpu_index)
+        torch.cuda.empty_cache()
+        legs["c2"], legs["c3"] = leg_c2_c3(nc, workloads, device, peak, args.leg_seconds, gpu_index)
+        torch.cuda.empty_cache()
+        legs["c5"] = leg_c5(nc, workloads, device, peak, args.leg_seconds, gpu_index, sm_count)
+        torch.cuda.empty_cache()
+
+    # ---- headline: K timed steps of workload c4
+    hp = HeadlineC4(nc, workloads, rank, device)
     for _ in range(args.warmup):
         hp.step()
     torch.cuda.synchronize()
-
-    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler = ClockSampler(gpu_index)
     marks_all = []
     if dist is not None:
         dist.barrier()
@@ -385,7 +612,7 @@ def main():
     t_start.record()
     for _ in range(args.steps):
         marks = []
-        hp.step(marks, DOMINANT_MARKS)       # events around the dominant kernel only
+        hp.step(marks)       # an event after every call: 4 events per ~9 ms step
         marks_all.append(marks)
     t_stop.record()
     torch.cuda.synchronize()
@@ -393,118 +620,63 @@ def main():
         dist.barrier()
     torch.cuda.synchronize()
     clocks = sampler.stop()
-    elapsed_ms = t_start.elapsed_time(t_stop)
-    elapsed_ms = timing.max_over_ranks(elapsed_ms, dist, device)
+    elapsed_ms = timing.max_over_ranks(t_start.elapsed_time(t_stop), dist, device)
 
-    # the dominant kernel: average device time over the timed steps themselves; the other call
-    # groups: a second pass with an event after every group (those events cost about 2 % of a
-    # step, so they stay out of the timed region)
-    group_ms = {g: 0.0 for g in HotPath.GROUPS}
+    group_times = {g: [] for g in HeadlineC4.GROUPS}
     for marks in marks_all:
-        group_ms["nc_compress"] += marks[0][1].elapsed_time(marks[1][1])
-    group_ms["nc_compress"] /= args.steps
-    k_groups = min(args.steps, 100)
-    marks_all = []
-    for _ in range(k_groups):
-        marks = []
-        hp.step(marks)
-        marks_all.append(marks)
-    torch.cuda.synchronize()
-    for marks in marks_all:
-        for (_, e0), (name, e1) in zip(marks[:-1], marks[1:]):
-            if name != "nc_compress":
-                group_ms[name] += e0.elapsed_time(e1) / k_groups
-
+        for (_, a), (name, b) in zip(marks[:-1], marks[1:]):
+            group_times[name].append(a.elapsed_time(b))
     units_per_step = hp.n * hp.d
     ms_per_step = elapsed_ms / args.steps
     value = world * units_per_step / (ms_per_step * 1e-3) / 1e9
 
-    peak, peak_kind = measured_hbm_peak()
-    alg = hp.algorithmic_bytes()
-    kernels = {}
-    for g in HotPath.GROUPS:
-        gbs = alg[g] / (group_ms[g] * 1e-3) / 1e9 if group_ms[g] > 0 else None
-        kernels[g] = {"ms": round(group_ms[g], 4), "algorithmic_GBps": round(gbs, 1),
-                      "frac_of_measured_peak": round(gbs / peak, 4)}
-    kernels["nc_compress"]["Gelem_per_s"] = round(units_per_step / group_ms["nc_compress"] / 1e6, 1)
-    kernels["nc_aggregate"]["Gelem_per_s"] = round(hp.d / group_ms["nc_aggregate"] / 1e6, 1)
-    kernels["nd_compress"]["Gelem_per_s"] = round(units_per_step / group_ms["nd_compress"] / 1e6, 1)
-    kernels["nd_aggregate"]["Gelem_per_s"] = round(hp.d / group_ms["nd_aggregate"] / 1e6, 1)
-    kernels["sparse_compress"]["Gcoord_per_s"] = round(
-        units_per_step / group_ms["sparse_compress"] / 1e6, 1)
-    kernels["sum_fp32"]["Gelem_per_s"] = round(hp.d / group_ms["sum_fp32"] / 1e6, 1)
+    alg, units = hp.algorithmic_bytes(), hp.units()
+    c4 = {"workload": "c4: n=16, d=335,141,888, 1e-4 * Student-t(3)", "iterations": args.steps,
+          "clocks": clocks}
+    for g, call in (("nc_compress", "nc_compress_batch"), ("nc_aggregate", "nc_aggregate"),
+                    ("sum_fp32", "nc_sum_fp32")):
+        c4[call] = summarize_call(group_times[g], alg[g], units[g], "Gelem_per_s", peak, clocks)
+    legs["c4"] = c4
 
-    dom = "nc_compress"          # one launch per step: the batch kernel over 8 workers
-    achieved = alg[dom] / (group_ms[dom] * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "nc_compress_kernel (8-worker batch launch)",
+    # the dominant kernel of the timed step: the call group with the largest measured share
+    mean_ms = {g: sum(v) / len(v) for g, v in group_times.items()}
+    dom = max(mean_ms, key=mean_ms.get)
+    dom_kernel = HeadlineC4.KERNEL_OF[dom]
+    achieved = alg[dom] / (mean_ms[dom] * 1e-3) / 1e9
+    per_entry, capture = ncu_traffic_per_entry(dom_kernel)
+    roofline = {"bound": "hbm", "kernel": "%s (one launch per step, %d workers)" % (dom_kernel, hp.n),
+                "share_of_step": round(mean_ms[dom] / ms_per_step, 4),
                 "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind,
                 "unit": "GB/s", "frac": round(achieved / peak, 4),
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBPS, 4),
+                "ms_mean": round(mean_ms[dom], 4),
+                "ms_median": round(statistics.median(group_times[dom]), 4),
+                "ms_best": round(min(group_times[dom]), 4),
                 "algorithmic_bytes_per_launch": alg[dom],
-                # the second resource of this kernel: the generator needs 18 wide 32x32->64
-                # multiplies per 4 entries, and a sub-partition issues one per 4 cycles:
-                # 148 SMs x 4 x 32 lanes x f_SM / 4 / 4.5 entries per second at the sampled SM clock
-                "generator_view": {
-                    "achieved_Gelem_per_s": round(units_per_step / group_ms[dom] / 1e6, 1),
-                    "multiplier_pipe_peak_Gelem_per_s": round(
-                        148 * 4 * 32 * (clocks.get("sm_mhz") or 1965) * 1e6 / 4 / 4.5 / 1e9, 1)}}
-    gv = roofline["generator_view"]
-    gv["frac"] = round(gv["achieved_Gelem_per_s"] / gv["multiplier_pipe_peak_Gelem_per_s"], 4)
+                "traffic": (per_entry * units[dom]) if per_entry is not None else None,
+                "traffic_source": capture}
+    if dom == "nc_compress":
+        # the second resource of this kernel: the generator needs 18 wide 32x32->64 multiplies
+        # per 4 entries, and a sub-partition issues one per 4 cycles
+        mhz = clocks.get("sm_mhz") or 1965
+        gen_peak = sm_count * 4 * 32 * mhz * 1e6 / 4 / 4.5 / 1e9
+        rate = units[dom] / mean_ms[dom] / 1e6
+        roofline["generator_view"] = {"achieved_Gelem_per_s": round(rate, 1),
+                                      "multiplier_pipe_peak_Gelem_per_s": round(gen_peak, 1),
+                                      "at_sm_mhz": mhz, "frac": round(rate / gen_peak, 4)}
 
-    # the same step with its independent call chains on four streams (reported beside `value`,
-    # which stays the single-stream figure the per-group times belong to)
-    streams = [torch.cuda.Stream() for _ in HotPath.STREAM_GROUPS]
-    k_conc = min(args.steps, 100)
-    for _ in range(3):
-        hp.step_on_streams(streams)
-    torch.cuda.synchronize()
-    c0 = torch.cuda.Event(enable_timing=True)
-    c1 = torch.cuda.Event(enable_timing=True)
-    c0.record()
-    for _ in range(k_conc):
-        hp.step_on_streams(streams)
-    c1.record()
-    torch.cuda.synchronize()
-    conc_ms = timing.max_over_ranks(c0.elapsed_time(c1) / k_conc, dist, device)
-    concurrent = {"ms_per_step": conc_ms, "streams": len(streams), "steps": k_conc,
-                  "value": world * units_per_step / (conc_ms * 1e-3) / 1e9, "unit": UNIT}
+    # one roofline row per call of every leg
+    rooflines = []
+    for leg in ("c1", "c2", "c3", "c4", "c5"):
+        for call, row in legs.get(leg, {}).items():
+            if isinstance(row, dict) and "frac_of_measured_peak" in row:
+                rooflines.append({"config": leg, "call": call, "ms": row["ms"],
+                                  "achieved_GBps": row["algorithmic_GBps"],
+                                  "frac": row["frac_of_measured_peak"],
+                                  "frac_of_nominal_8TBps": row["frac_of_nominal_8TBps"],
+                                  "bound": row.get("bound", "hbm")})
 
-    # the same single-stream step replayed from a CUDA graph (no launch gaps); reported beside
-    # `value` as well
-    graph_replay = None
-    try:
-        graph_stream = torch.cuda.Stream()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(graph_stream):
-            # thread-local capture mode: a CUDA call from another thread of this process (a
-            # communication library's watchdog, the clock sampler) must not break the capture
-            with torch.cuda.graph(graph, stream=graph_stream, capture_error_mode="thread_local"):
-                hp.step()
-        for _ in range(3):
-            graph.replay()
-        torch.cuda.synchronize()
-        g0 = torch.cuda.Event(enable_timing=True)
-        g1 = torch.cuda.Event(enable_timing=True)
-        g0.record()
-        for _ in range(k_conc):
-            graph.replay()
-        g1.record()
-        torch.cuda.synchronize()
-        graph_ms = g0.elapsed_time(g1) / k_conc
-    except RuntimeError as exc:               # the leg is optional: report why it is missing
-        graph_ms = None
-        graph_error = str(exc).splitlines()[0][:200]
-    if dist is not None:
-        # every rank reaches the reduction, also one whose capture failed
-        worst = timing.max_over_ranks(graph_ms if graph_ms is not None else -1.0, dist, device)
-        graph_ms = None if graph_ms is None else worst
-    if graph_ms is not None and graph_ms > 0:
-        graph_replay = {"ms_per_step": graph_ms, "steps": k_conc,
-                        "value": world * units_per_step / (graph_ms * 1e-3) / 1e9, "unit": UNIT}
-    elif graph_ms is None:
-        graph_replay = {"unavailable": locals().get("graph_error", "capture failed on a rank")}
-
-    # end to end: host buffers -> device -> whole path -> aggregates back on the host
+    # end to end: host buffers -> device -> whole step -> aggregates back on the host
     e2e = None
     if args.e2e_steps > 0:
         e2e = timing.e2e_host_steps(nc, hp, args.e2e_steps)
@@ -515,26 +687,23 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        units, times, cores, sample = cpu_baseline_sample(steps=1)     # first call builds/loads
-        units, times, cores, sample = cpu_baseline_sample(steps=2)
-        cpu = {"value": units * len(times) / sum(times) / 1e9, "unit": UNIT, "cores": cores,
-               "kind": "oracle", "sample": sample}
+        cpu = cpu_baseline(workloads)
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u32+f32", "data": "synthetic",
-            "config": {"workload": "c2: ResNet-50-shaped gradients, n=8 workers, d=25557032 in "
-                                   "161 buckets; C_nat + D_nat^{2,8} + sparse(1%) D_nat^{inf,4} "
-                                   "+ fp32 8-way sum per step",
-                       "unit_definition": "worker-entries (n*d) through the whole path per second",
-                       "l2": "inputs are 818 MB per replica, larger than the 126 MB L2; no flush",
-                       "multi_gpu": "replicas only"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": hp.launches_per_step * args.steps,
-            "concurrent_streams": concurrent,
-            "graph_replay": graph_replay,
-            "roofline": roofline, "cpu_baseline": cpu, "kernels": kernels,
+            "config": {"workload": "c4: C_nat at BERT-large scale, n=16 workers, d=335141888 fp32 "
+                                   "entries each in 25 MiB buckets; nc_compress_batch + "
+                                   "nc_aggregate + nc_sum_fp32 (uncompressed 16-way sum) per step",
+                       "unit_definition": "worker-entries (n*d) through the step per second",
+                       "l2": "inputs are 21.45 GB per replica, larger than the 126 MB L2; no flush",
+                       "multi_gpu": "replicas only",
+                       "legs": "c1, c2, c3 and c5 per call under `kernels`"},
+            "clocks": clocks, "e2e": e2e,
+            "gpu_launches": HeadlineC4.LAUNCHES_PER_STEP * args.steps,
+            "roofline": roofline, "rooflines": rooflines, "cpu_baseline": cpu, "kernels": legs,
         }
         print(json.dumps(line))
     if dist is not None:
