@@ -541,16 +541,28 @@ uint64_t orc_sparse_compact_compress(const float* x, uint64_t d, uint64_t keep_t
                                      float scale, int p, int s, uint64_t seed, uint32_t worker,
                                      uint32_t* idx, uint32_t* planes, uint64_t cap,
                                      float* norm_out) {
+    // pass 1: the norm of the kept, scaled entries.  Sums are taken in index order; the maximum
+    // does not depend on the order, so that case may be split over threads.
     double acc = 0.0;
     bool saw_nan = false;
-    for (uint64_t j = 0; j < d; ++j) {
-        if ((uint64_t)stream_word(seed, worker, 2u, j) >= keep_threshold) continue;
-        const float xs = scale * x[j];
-        const double a = std::fabs((double)xs);
-        if (std::isnan(a)) saw_nan = true;
-        if (p == 1) acc += a;
-        else if (p == 2) acc += a * a;
-        else if (a > acc) acc = a;
+    if (p == 0) {
+#pragma omp parallel for schedule(static) reduction(max : acc) reduction(|| : saw_nan)
+        for (int64_t j = 0; j < (int64_t)d; ++j) {
+            if ((uint64_t)stream_word(seed, worker, 2u, (uint64_t)j) >= keep_threshold) continue;
+            const float xs = scale * x[j];
+            const double a = std::fabs((double)xs);
+            if (std::isnan(a)) saw_nan = true;
+            else if (a > acc) acc = a;
+        }
+    } else {
+        for (uint64_t j = 0; j < d; ++j) {
+            if ((uint64_t)stream_word(seed, worker, 2u, j) >= keep_threshold) continue;
+            const float xs = scale * x[j];
+            const double a = std::fabs((double)xs);
+            if (std::isnan(a)) saw_nan = true;
+            if (p == 1) acc += a;
+            else acc += a * a;
+        }
     }
     if (p == 2) acc = std::sqrt(acc);
     const float norm = saw_nan ? std::numeric_limits<float>::quiet_NaN() : (float)acc;
@@ -559,16 +571,25 @@ uint64_t orc_sparse_compact_compress(const float* x, uint64_t d, uint64_t keep_t
     const uint64_t groups = (cap + 31) / 32;
     std::memset(planes, 0, (size_t)(groups * (uint64_t)(nb + 1)) * 4);
     if (norm_degenerate(norm)) return 0;            // every level is 0: nothing to list
-    uint64_t k = 0;
-    for (uint64_t j = 0; j < d; ++j) {
-        if ((uint64_t)stream_word(seed, worker, 2u, j) >= keep_threshold) continue;
+    // pass 2: per coordinate, 0 = not listed, else code + 1 (coordinates are independent);
+    // then the list is written in ascending index order
+    std::vector<uint8_t> entry(d);
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < (int64_t)d; ++j) {
+        entry[j] = 0;
+        if ((uint64_t)stream_word(seed, worker, 2u, (uint64_t)j) >= keep_threshold) continue;
         const float xs = scale * x[j];
         const float yf = ratio_given_norm(std::fabs(xs), norm);
-        const uint32_t r23 = stream_word(seed, worker, 1u, j) & 0x7FFFFFu;
+        const uint32_t r23 = stream_word(seed, worker, 1u, (uint64_t)j) & 0x7FFFFFu;
         const int c = nd_level_code((double)yf, s, r23);
         if (c == 0) continue;
+        entry[j] = (uint8_t)((((std::signbit(xs) ? 1u : 0u) << nb) | (uint32_t)(c - 1)) + 1u);
+    }
+    uint64_t k = 0;
+    for (uint64_t j = 0; j < d; ++j) {
+        if (!entry[j]) continue;
         if (k < cap) {
-            const uint32_t code = ((std::signbit(xs) ? 1u : 0u) << nb) | (uint32_t)(c - 1);
+            const uint32_t code = (uint32_t)entry[j] - 1u;
             idx[k] = (uint32_t)j;
             for (int b = 0; b <= nb; ++b)
                 planes[(k / 32) * (uint64_t)(nb + 1) + (uint64_t)b] |= ((code >> b) & 1u) << (k % 32);

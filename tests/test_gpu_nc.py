@@ -52,6 +52,34 @@ def test_compress_random_bit_patterns():
     check_nc_planes(e, s, d, e_ref, s_ref)
 
 
+def test_compress_all_2_to_32_bit_patterns():
+    """Every binary32 bit pattern once, as one vector of 2^32 entries (element j holds the pattern
+    j xor 2^31), in two sweeps with different streams: closes every sign / exponent / mantissa
+    corner of the field rule (Sec. 2), of the kernel's unguarded fast path and of the edge
+    policy.  Compared with the oracle chunk by chunk."""
+    d = 1 << 32
+    free, _ = torch.cuda.mem_get_info()
+    if free < 30 * (1 << 30):
+        pytest.skip("needs ~22 GB of free device memory")
+    x = torch.arange(-(1 << 31), 1 << 31, dtype=torch.int32, device="cuda").view(torch.float32)
+    e = torch.empty(nc.nc_exp_bytes(d), dtype=torch.uint8, device="cuda")
+    s = torch.empty(nc.nc_sign_bytes(d), dtype=torch.uint8, device="cuda")
+    chunk = 1 << 27
+    for seed, worker in ((0, 0), ((1 << 63) + 5, 0xFFFFFFFF)):
+        e.fill_(0xEE)
+        s.fill_(0xEE)
+        nc.nc_compress(x, d, seed, worker, e, s)
+        torch.cuda.synchronize()
+        for j0 in range(0, d, chunk):
+            xs = x[j0:j0 + chunk].cpu().numpy()
+            e_ref, s_ref = oracle.nc_compress(xs, seed, worker, j0=j0)
+            assert np.array_equal(e[j0:j0 + chunk].cpu().numpy(), e_ref), (seed, j0)
+            got = s[j0 // 8:(j0 + chunk) // 8].cpu().numpy().view(np.uint32)
+            assert np.array_equal(got, s_ref), (seed, j0)
+    del x, e, s
+    torch.cuda.empty_cache()
+
+
 def _aggregate_gpu(exps, signs, d):
     out = Guarded(4 * d)
     nc.nc_aggregate(exps, signs, len(exps), d, out.buf)

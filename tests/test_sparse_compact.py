@@ -181,6 +181,44 @@ def test_config5_full_size_compact_one_worker():
 
 
 @pytest.mark.gpu
+def test_config5_full_size_all_workers_batch_and_aggregate():
+    # config 5 at its own shape in the calls the benchmark times: d = 2^28, n = 8, one batch
+    # compress call and the one-launch aggregate; every list and the whole dense sum compared
+    import torch
+    import paper_1905_10988_b200 as nc
+    n, d, s = 8, 1 << 28, 4
+    free, _ = torch.cuda.mem_get_info()
+    if free < 16 * (1 << 30):
+        pytest.skip("needs ~12 GB of free device memory")
+    cap = int(d * 0.0125)
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    xd = [workloads.config5_vector(w, d, "cuda") for w in range(n)]
+    idx = [torch.empty(cap, dtype=torch.int32, device="cuda") for _ in range(n)]
+    planes = [torch.empty(nc.nd_sparse_plane_bytes(cap, s), **u8) for _ in range(n)]
+    count = [torch.zeros(1, dtype=torch.int32, device="cuda") for _ in range(n)]
+    norm = [torch.zeros(1, dtype=torch.float32, device="cuda") for _ in range(n)]
+    ws_bytes = nc.nd_sparse_batch_workspace_bytes(d, cap, n)
+    ws = torch.empty(ws_bytes, **u8)
+    nc.nd_sparse_compact_compress_batch(xd, d, THR, SCALE, nc.P_INF, s, 0, list(range(n)), idx,
+                                        planes, count, norm, cap, n, ws, ws_bytes)
+    out = torch.empty(d, dtype=torch.float32, device="cuda")
+    nc.nd_sparse_compact_aggregate(idx, planes, count, norm, n, s, d, cap, out)
+    torch.cuda.synchronize()
+    ref = np.zeros(d, np.float32)
+    for w in range(n):
+        i_ref, p_ref, c_ref, n_ref = oracle.sparse_compact_compress(xd[w].cpu().numpy(), THR, SCALE,
+                                                                    oracle.P_INF, s, 0, w, cap=cap)
+        cnt = int(count[w].cpu().numpy().view(np.uint32)[0])
+        assert cnt == c_ref <= cap and float(norm[w].cpu()[0]) == float(n_ref)
+        assert np.array_equal(idx[w][:cnt].cpu().numpy().view(np.uint32), i_ref)
+        assert np.array_equal(planes[w].cpu().numpy().view(np.uint32)[:p_ref.size], p_ref)
+        oracle.sparse_compact_decode_accumulate(i_ref, p_ref, c_ref, n_ref, s, ref)
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+    del xd, out
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.gpu
 @pytest.mark.parametrize("n,d,thr,scale,cap_frac", [(1, 5, 1 << 32, 1.0, 1.0),
                                                     (3, 8192, 1 << 30, 4.0, 1.0),
                                                     (4, 300_000, THR * 8, 12.5, 1.0),
