@@ -64,7 +64,7 @@ class NaturalAllReduce:
     """
 
     def __init__(self, d: int, dist, group=None, *, seed: int = 0, transport: str = "collective",
-                 master_compress: bool = False, device=None, codec=None):
+                 master_compress: bool = False, device=None, codec=None, symm_mem=None):
         if transport not in ("collective", "peer"):
             raise ValueError("transport must be 'collective' or 'peer'")
         if codec is None:
@@ -83,7 +83,8 @@ class NaturalAllReduce:
         dev = self.device
         self._symm = None
         if transport == "peer":
-            import torch.distributed._symmetric_memory as symm_mem
+            if symm_mem is None:      # `symm_mem`: what provides empty() and rendezvous()
+                import torch.distributed._symmetric_memory as symm_mem
             # one allocation for both planes: exponents, then sign bytes
             self._send = symm_mem.empty(P + P // 8, dtype=torch.uint8, device=dev)
             self._send.zero_()
@@ -187,7 +188,8 @@ class DitherAllReduce:
     with the same norm."""
 
     def __init__(self, d: int, bucket_off, dist, group=None, *, p: int = 2, s: int = 8,
-                 seed: int = 0, transport: str = "collective", device=None, codec=None):
+                 seed: int = 0, transport: str = "collective", device=None, codec=None,
+                 symm_mem=None):
         if transport not in ("collective", "peer"):
             raise ValueError("transport must be 'collective' or 'peer'")
         bucket_off = [int(v) for v in bucket_off]
@@ -210,7 +212,8 @@ class DitherAllReduce:
         nbytes = P // 2 + P // 8                      # level nibbles, then sign bytes
         self._symm = None
         if transport == "peer":
-            import torch.distributed._symmetric_memory as symm_mem
+            if symm_mem is None:
+                import torch.distributed._symmetric_memory as symm_mem
             self._send = symm_mem.empty(nbytes, dtype=torch.uint8, device=dev)
             self._send.zero_()
             self._symm = symm_mem.rendezvous(self._send, group if group is not None

@@ -176,6 +176,7 @@ class ThreadFabric:
         self.local = threading.local()
         self.barrier = threading.Barrier(world)
         self.slots = [None] * world
+        self.group = type("group", (), {"WORLD": None})     # what dist.group.WORLD stands for
 
     def get_rank(self, group=None):
         return self.local.rank
@@ -233,6 +234,84 @@ def test_cuda_codec_four_emulated_ranks(world, d, master_compress):
     want = expected(d, world, master_compress)
     for r in range(world):
         assert same_bits(results[r], want), "rank %d" % r
+
+
+class ThreadSymmetricMemory:
+    """Stands in for symmetric memory among the host threads of ThreadFabric: every rank's
+    buffer is an ordinary tensor on the one device, get_buffer(i) hands out rank i's, and the
+    barrier is the host barrier (all ranks enqueue on one stream, so what was enqueued before
+    the barrier runs before what is enqueued after it).  The aggregate kernel then reads the
+    other ranks' planes in place, exactly as it reads peer-mapped memory."""
+
+    def __init__(self, fabric):
+        self.fabric = fabric
+        self.buffers = {}
+
+    def empty(self, *shape, dtype, device):
+        return torch.empty(*shape, dtype=dtype, device=device)
+
+    def rendezvous(self, tensor, group=None):
+        owner = self
+        rank = self.fabric.local.rank
+        self.buffers.setdefault(tensor.numel(), [None] * self.fabric.world)[rank] = tensor
+        self.fabric.barrier.wait()
+
+        class Handle:
+            def barrier(self, channel=0):
+                owner.fabric.barrier.wait()
+
+            def get_buffer(self, i, shape, dtype):
+                n = 1
+                for v in shape:
+                    n *= v
+                return owner.buffers[tensor.numel()][i][:n].view(dtype)
+
+        return Handle()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("world,d", [(4, 300_000), (3, 5 * 1024 + 1)])
+def test_cuda_codec_peer_transport_emulated_ranks(world, d):
+    """The "peer" transport with more than one rank: plane slicing, the order of the two barriers
+    and the in-place reads of the other ranks' buffers, for C_nat (with and without the master's
+    compression) and for D_nat.  Results must equal the single-master result bit for bit."""
+    off = bucket_table(d)
+    fabric = ThreadFabric(world)
+    symm = ThreadSymmetricMemory(fabric)
+    results, errors = [None] * world, []
+
+    def run(rank):
+        try:
+            fabric.local.rank = rank
+            torch.cuda.set_device(0)
+            g = torch.from_numpy(gradient(rank, d)).cuda()
+            outs = []
+            for master_compress in (False, True):
+                ar = NaturalAllReduce(d, fabric, seed=SEED, transport="peer",
+                                      master_compress=master_compress, symm_mem=symm)
+                ar(g)
+                outs.append(ar(g).cpu().numpy())         # the second call reuses every buffer
+            ad = DitherAllReduce(d, off, fabric, p=0, s=4, seed=SEED, transport="peer",
+                                 symm_mem=symm)
+            ad(g)
+            outs.append(ad(g).cpu().numpy())
+            torch.cuda.synchronize()
+            results[rank] = outs
+        except Exception as e:
+            errors.append(e)
+            fabric.barrier.abort()
+
+    threads = [threading.Thread(target=run, args=(r,)) for r in range(world)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=300)
+    assert not errors, errors
+    want = [expected(d, world, False), expected(d, world, True),
+            expected_dither(d, world, off, 0, 4)]
+    for r in range(world):
+        for got, ref in zip(results[r], want):
+            assert same_bits(got, ref), "rank %d" % r
 
 
 @pytest.mark.gpu
