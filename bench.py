@@ -286,9 +286,33 @@ def leg_c1(nc, workloads, device, peak, seconds, gpu_index):
     t, clocks, iters = time_sequence([("nc_compress_batch", compress), ("nc_aggregate", aggregate)],
                                      min(seconds, 0.3), gpu_index)
     note = {"note": "launch-bound and L2-resident (21 MB): the time is what counts, not the fraction"}
+    # the same two calls replayed from a CUDA graph: what is left when the host's marshalling and
+    # launch latency are out of the way
+    graph = None
+    try:
+        gs = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(gs):
+            with torch.cuda.graph(g, stream=gs, capture_error_mode="thread_local"):
+                compress()
+                aggregate()
+        for _ in range(10):
+            g.replay()
+        torch.cuda.synchronize()
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        reps = 2000
+        a.record()
+        for _ in range(reps):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        graph = {"ms_per_compress_plus_aggregate": round(a.elapsed_time(b) / reps, 5), "replays": reps}
+    except RuntimeError as exc:               # optional: report why it is missing
+        graph = {"unavailable": str(exc).splitlines()[0][:160]}
     return {
         "workload": "c1: d=2^20, n=4, N(0,1e-3^2) + 1% zeros + 0.1% powers of two",
-        "iterations": iters, "clocks": clocks,
+        "iterations": iters, "clocks": clocks, "graph_replay": graph,
         "nc_compress_batch": summarize_call(t["nc_compress_batch"], n * d * 5.125, n * d,
                                             "Gelem_per_s", peak, clocks, note),
         "nc_aggregate": summarize_call(t["nc_aggregate"], d * (1.125 * n + 4), d, "Gelem_per_s",
