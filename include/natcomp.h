@@ -177,7 +177,10 @@ nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bu
  * split over several devices were combined, or norms that were compressed and decoded again).
  * nd_compress_batch(..) gives exactly what nd_norms_batch(..) followed by nd_round_batch(..)
  * with the same arguments gives.  Arguments as for nd_compress_batch; `norms` is written by the
- * first call and read by the second; workspace: nd_batch_workspace_bytes(d, B, n). */
+ * first call and read by the second; workspace: nd_batch_workspace_bytes(d, B, n).
+ * Against norms that are not the entries' own, a ratio |x| / norm above 1 (or NaN: a NaN entry
+ * under a finite norm) takes the top level s; a norm that is 0, negative, inf or NaN gives level 0
+ * for its whole bucket. */
 nc_status nd_norms_batch(const float* const* xs, size_t d, const uint64_t* bucket_off, int B, int p,
                          float* const* norms, int n, void* workspace, size_t workspace_bytes,
                          uint32_t* status, cudaStream_t stream);

@@ -190,6 +190,10 @@ float ratio_given_norm(float ax, float norm) {
 // The draw: "up" iff r23 < floor(probability * 2^23).
 int nd_level_code(double y, int s, uint32_t r23) {
     if (y >= 1.0) return s;                       // y = l_0 (or a rounding excess)
+    // xi is defined on [0, 1] (Def. 3).  A ratio outside it can only come from a norm that is not
+    // the norm of these entries (norms given by the caller): y > 1 takes the top level above, and
+    // so does a ratio that is not a number (a NaN entry against a finite norm).
+    if (std::isnan(y)) return s;
     for (int u = 0; u < s; ++u) {
         const double upper = std::ldexp(1.0, -u);
         const double lower = (u + 1 == s) ? 0.0 : std::ldexp(1.0, -(u + 1));

@@ -292,7 +292,9 @@ __device__ __forceinline__ uint32_t level_code_scaled(uint32_t bits, uint32_t rn
     return min(t >> 23, smax);
 }
 
-// grid: ceil(tiles / warps per block)
+// grid: ceil(tiles / warps per block).  kClamp: the norms are the caller's, not necessarily those
+// of the entries, so |x| / norm may exceed 1 (or be NaN) and the level code is clamped to s.
+template <bool kClamp>
 __global__ void __launch_bounds__(kBlockThreads, 4)
 nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d,
                      const uint64_t* __restrict__ off, const int B, const int s,
@@ -325,7 +327,7 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
     // level code 0.  If rinv * 2^s overflows (norm below 2^(s-126)) the general path is used.
     const BucketScale sc0 = bucket_scale(norms[b], s);
     const float rinv_s = __fmul_rn(sc0.rinv, pow2s);
-    // No clamp of the code in this path: the norm was computed from the same entries, so
+    // No clamp of the code in this path unless kClamp: the norm was computed from the same entries, so
     // |x| <= norm, |x| * rinv <= 1 + 2^-24 rounds to at most 1 (a tie goes to the even mantissa 0)
     // and z <= 2^s has a zero mantissa at the top exponent, which the random increment cannot carry
     // out of.  A degenerate bucket (norm 0 or not finite; all codes 0) and one with a subnormal
@@ -355,7 +357,8 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
             uint32_t nib = 0;
 #pragma unroll
             for (int c = 7; c >= 0; --c) {
-                const float z = __fmul_rn(fabsf(__uint_as_float(u[it].v[c])), rinv_s);
+                float z = __fmul_rn(fabsf(__uint_as_float(u[it].v[c])), rinv_s);
+                if (kClamp) z = fminf(z, pow2s);      // y >= 1 (and a NaN ratio): the top level
                 const float w = fmaxf(z, __fmaf_rz(z, 0.5f, 1.0f));       // see level_code_scaled
                 const uint32_t e = (__float_as_uint(w) + (~rnd[c] & 0x7FFFFFu)) >> 23;
                 nib = nib * 16u + e;
@@ -786,8 +789,8 @@ nc_status nd_round_batch(const float* const* xs, size_t d, const uint64_t* bucke
     if (d == 0) return NC_OK;
     const PhiloxKeys keys = make_philox_keys(seed);
     const dim3 grid(nd_tile_blocks(d), (unsigned)n);
-    nd_round_pack_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, bucket_off, B, s, keys,
-                                                             nullptr);
+    nd_round_pack_kernel<true><<<grid, kBlockThreads, 0, stream>>>(batch, d, bucket_off, B, s, keys,
+                                                                   nullptr);
     return launch_status();
 }
 
@@ -810,8 +813,8 @@ nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bu
         nd_launch_norms(batch, d, bucket_off, B, p, n, workspace, status, stream);
     const PhiloxKeys keys = make_philox_keys(seed);
     const dim3 grid(nd_tile_blocks(d), (unsigned)n);
-    nd_round_pack_kernel<<<grid, kBlockThreads, 0, stream>>>(batch, d, bucket_off, B, s, keys,
-                                                             tile_bucket);
+    nd_round_pack_kernel<false><<<grid, kBlockThreads, 0, stream>>>(batch, d, bucket_off, B, s,
+                                                                    keys, tile_bucket);
     return launch_status();
 }
 

@@ -308,6 +308,42 @@ def test_batch_launch_equals_single_launches():
         check_against_oracle(xs[i], off, p, s, 11, workers[i], norms[i], levels[i], signs[i])
 
 
+def test_round_batch_against_norms_that_are_not_the_entries_own():
+    """nd_round_batch rounds against whatever norms the caller gives (norms that were compressed
+    and decoded again, combined partial norms).  Ratios above 1 and NaN ratios take the top
+    level, degenerate norms give level 0; codes equal the given-norm oracle's bit for bit."""
+    rng = np.random.default_rng(77)
+    n, d, s = 3, 70001 + 2048, 8
+    off = workloads.small_bucket_table(d, seed=12)
+    B = len(off) - 1
+    off_dev = dev(np.asarray(off, np.uint64).view(np.int64))
+    xs = [(rng.standard_normal(d) * 1e-2).astype(np.float32) for _ in range(n)]
+    xs[1][rng.choice(d, 50, replace=False)] = np.nan
+    xs[2][rng.choice(d, 50, replace=False)] = np.inf
+    workers = [4, 9, 2]
+    given = []
+    for i, x in enumerate(xs):
+        own = oracle.norms(np.nan_to_num(x, nan=0.0, posinf=0.0), off, 2)
+        g = own * (2.0 ** rng.integers(-6, 3, B)).astype(np.float32)   # far too small .. too large
+        g[rng.choice(B, max(B // 10, 1), replace=False)] = [0.0, np.inf, np.nan][i]
+        g[rng.choice(B, 2, replace=False)] = [-1.0, 1e-42]              # negative; subnormal
+        given.append(g.astype(np.float32))
+    norms = [dev(g) for g in given]
+    levels = [Guarded(nc.nd_level_bytes(d)) for _ in range(n)]
+    signs = [Guarded(nc.nc_sign_bytes(d)) for _ in range(n)]
+    nc.nd_round_batch([dev(x) for x in xs], d, off_dev, B, s, 5, workers, norms,
+                      [g.buf for g in levels], [g.buf for g in signs], n)
+    torch.cuda.synchronize()
+    for i in range(n):
+        levels[i].check()
+        signs[i].check()
+        _, l_ref, s_ref = oracle.nd_compress(xs[i], off, 2, s, 5, workers[i], given_norms=given[i])
+        assert np.array_equal(levels[i].numpy(np.uint8)[:(d + 1) // 2], l_ref), i
+        assert np.array_equal(signs[i].numpy(np.uint32)[:(d + 31) // 32], s_ref), i
+        c = unpack_nibbles(l_ref, d)
+        assert np.any(c == s) and np.all(c <= s)
+
+
 def test_one_element_buckets_and_many_empty_buckets():
     # every tile takes the multi-bucket path: B = d one-element buckets, then a table that is
     # mostly empty buckets

@@ -315,6 +315,23 @@ def test_dnat_decode_under_a_norm_that_is_not_finite():
     assert np.array_equal(acc, np.float32([0, 0, 0, 0, -inf, 0, inf, 0]))
 
 
+def test_dnat_ratios_outside_the_unit_interval_take_the_top_level():
+    """xi(y) is defined for y in [0, 1] (Def. 3).  With norms given by the caller a ratio can
+    exceed 1 or be NaN (a NaN entry against a finite norm); both are read as the top level s,
+    whatever the draw.  Values written out by hand."""
+    r = np.uint32([0, 1, (1 << 23) - 1, 12345])
+    for s in (1, 4, 8, 15):
+        for y in (1.0, 1.5, 1e30, np.inf, np.nan):
+            assert np.array_equal(oracle.nd_level_codes(np.full(4, y), r, s), np.full(4, s))
+    x = np.float32([0.5, -3.0, np.nan, 0.25, 8.0, -0.125, 0.0, 1.0])
+    nrm, level, sign = oracle.nd_compress(x, [0, 8], 2, 3, seed=1, worker=0,
+                                          given_norms=np.float32([1.0]))
+    c = np.stack([level & 0xF, level >> 4], 1).ravel()[:8]
+    assert c[1] == 3 and c[2] == 3 and c[4] == 3 and c[7] == 3 and c[6] == 0
+    assert c[0] in (2, 3) and c[3] in (1, 2) and c[5] in (0, 1)
+    assert sign[0] == 0b00100010 | (int(np.signbit(x[2])) << 2)
+
+
 def test_dnat_bucket_with_a_subnormal_norm_is_an_ordinary_bucket():
     """y = |x| / norm does not change when a bucket is multiplied by a power of two (Def. 3), so
     neither do the level codes: a bucket of tiny entries, subnormal norm included, must get the
