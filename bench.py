@@ -703,7 +703,8 @@ def main():
     # end to end: host buffers -> device -> whole step -> aggregates back on the host
     e2e = None
     if args.e2e_steps > 0:
-        e2e = timing.e2e_host_steps(nc, hp, args.e2e_steps)
+        # several ranks share one host's memory: four distinct pinned vectors per rank then
+        e2e = timing.e2e_host_steps(nc, hp, args.e2e_steps, 0 if world == 1 else 4)
         e2e_ms = timing.max_over_ranks(e2e["ms_per_step"], dist, device)
         e2e["value"] = world * units_per_step / (e2e_ms * 1e-3) / 1e9
         e2e["ms_per_step"] = e2e_ms

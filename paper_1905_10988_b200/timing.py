@@ -27,11 +27,13 @@ def replica_worker_ids(rank: int, n_workers: int):
     return [rank * n_workers + w for w in range(n_workers)]
 
 
-def e2e_host_steps(nc, hp, steps: int) -> dict:
+def e2e_host_steps(nc, hp, steps: int, max_pinned_buffers: int = 0) -> dict:
     """Runs `steps` steps with the inputs in pinned host memory: every step copies the n
     gradient vectors host -> device through the C ABI, runs the whole step, and copies the
     step's results (`hp.outputs`) back to pinned host memory.  Returns ms per step and bytes moved.
     `hp` provides n, d, x (list of n device vectors), outputs (device vectors) and step().
+    max_pinned_buffers > 0 limits the distinct pinned input buffers (they are then uploaded in
+    turn: same bytes per step, less host memory; for several ranks sharing one host).
 
     Three streams and two sets of device input buffers: the upload of step i + 1 runs while the
     kernels of step i work on the other set and while the results of step i (and i - 1) go back
@@ -41,7 +43,7 @@ def e2e_host_steps(nc, hp, steps: int) -> dict:
     n, d = hp.n, hp.d
     host_x = []
     try:
-        for w in range(n):
+        for w in range(n if max_pinned_buffers <= 0 else min(n, max_pinned_buffers)):
             host_x.append(torch.empty(d, dtype=torch.float32, pin_memory=True))
     except RuntimeError:
         # the host cannot pin n vectors: keep what it could, at least two, and upload them in turn
