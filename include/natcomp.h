@@ -434,6 +434,23 @@ nc_status nc_topk_compress(const float* x, size_t d, uint64_t K, uint64_t seed, 
 nc_status nc_topk_decode_accumulate(const uint32_t* idx, const uint8_t* exp, const uint32_t* sign,
                                     size_t count, size_t d, float* acc, cudaStream_t stream);
 
+/* ---- debug build (no counterpart in the paper) ------------------------------------------------
+ * `python paper_1905_10988_b200/build.py --bounds` builds libnatcomp_bounds.so with -DNC_BOUNDS:
+ * the same entry points, but every global store of the C_nat and D_nat kernels (nc_compress*,
+ * nc_aggregate*, nc_decode_accumulate, nc_sum_fp32, nd_compress*, nd_norms_batch, nd_round_batch,
+ * nd_aggregate, nd_decode_accumulate) first checks its address against the ranges the call may
+ * write (its outputs and workspace, sized by the *_bytes helpers).  A store outside them is
+ * skipped and counted; the kernel runs on and nothing traps.  Calls must not overlap on the GPU in
+ * that build (the range table is shared), and it is several times slower.
+ * nc_debug_bounds_status: synchronises the device, then *violations = skipped stores since the
+ * last reset, *first_address = address of the first one (0 if none); reset != 0 clears the count.
+ * nc_debug_bounds_selftest: aims one store 64 bytes past a 16-byte range at the start of
+ * `scratch` (device memory, >= 128 bytes, 16-byte aligned), which the check must skip and count:
+ * shows that the mechanism is alive without any invalid access.
+ * In the regular library both return NC_ERR_UNSUPPORTED. */
+nc_status nc_debug_bounds_status(uint64_t* violations, uint64_t* first_address, int reset);
+nc_status nc_debug_bounds_selftest(void* scratch, cudaStream_t stream);
+
 /* ---- host-buffer plumbing (no counterpart in the paper, where workers and master exchange
  * these buffers over a network) ------------------------------------------------------------- */
 

@@ -43,7 +43,8 @@ EXPORTS = (
     "nd_sparse_regen_workspace_bytes", "nd_sparse_regen_decode_accumulate",
     "nd_sparse_compact_aggregate", "nc_aggregate_compress_shard", "nc_compress_bf16_r8",
     "nc_compress_bf16_r8_batch", "nc_compress_f16_r16", "nc_compress_f16_r16_batch",
-    "nd_norm_status", "nd_norms_batch", "nd_round_batch",
+    "nd_norm_status", "nd_norms_batch", "nd_round_batch", "nc_debug_bounds_status",
+    "nc_debug_bounds_selftest",
 )
 
 
@@ -322,6 +323,23 @@ def nd_compress_static(x, d, bucket_off, B, p, s, seed, worker, norms, level, si
     _check("nd_compress_static", _nd_compress_static(_ptr(x), d, _ptr(bucket_off), B, p, s, seed,
                                                      worker, _ptr(norms), _ptr(level), _ptr(sign),
                                                      _ptr(status), _stream(stream)))
+
+
+_nc_debug_bounds_status = _sig("nc_debug_bounds_status", C.c_int, C.POINTER(C.c_uint64),
+                               C.POINTER(C.c_uint64), C.c_int)
+_nc_debug_bounds_selftest = _sig("nc_debug_bounds_selftest", C.c_int, _vp, _vp)
+
+
+def nc_debug_bounds_status(reset: bool = False):
+    """(violations, first_address) of the debug build; the regular library raises
+    NatcompError(NC_ERR_UNSUPPORTED)."""
+    v, a = C.c_uint64(0), C.c_uint64(0)
+    _check("nc_debug_bounds_status", _nc_debug_bounds_status(C.byref(v), C.byref(a), int(reset)))
+    return int(v.value), int(a.value)
+
+
+def nc_debug_bounds_selftest(scratch, stream=None) -> None:
+    _check("nc_debug_bounds_selftest", _nc_debug_bounds_selftest(_ptr(scratch), _stream(stream)))
 
 
 _nc_copy_to_device = _sig("nc_copy_to_device", C.c_int, _vp, _vp, _sz, _vp)

@@ -57,6 +57,89 @@ inline nc_status launch_status() {
     return cudaPeekAtLastError() == cudaSuccess ? NC_OK : NC_ERR_CUDA;
 }
 
+// ---- debug build (-DNC_BOUNDS) --------------------------------------------------------------
+// Every global store of the C_nat and D_nat kernels first checks its address against the table of
+// output ranges that the entry point filled in for this call (outputs and workspace, as sized by
+// the *_bytes helpers).  A store outside every range is skipped and recorded in a device status
+// block that nc_debug_bounds_status reads: the kernel goes on, nothing traps.  The table and the
+// record exist once per translation unit; calls of one unit must not overlap on the GPU in this
+// build.  Without NC_BOUNDS all of this compiles to nothing.
+struct BoundsRecord {
+    unsigned long long violations;     // stores that were skipped
+    unsigned long long first_address;  // address of the first one
+    unsigned int first_bytes, first_block, first_thread, pad;
+};
+
+#ifdef NC_BOUNDS
+constexpr int kBoundsRanges = 4 * NC_MAX_WORKERS + 8;
+struct BoundsTable {
+    unsigned long long lo[kBoundsRanges];
+    unsigned long long hi[kBoundsRanges];
+    int count;
+};
+static __device__ BoundsTable g_bounds_table;
+static __device__ BoundsRecord g_bounds_record;
+
+static __device__ __noinline__ bool nc_store_ok(const void* p, unsigned bytes) {
+    const unsigned long long a = (unsigned long long)p;
+    const int n = g_bounds_table.count;
+    if (n == 0) return true;           // a unit whose entry points fill in no table checks nothing
+    for (int i = 0; i < n; ++i)
+        if (a >= g_bounds_table.lo[i] && a + bytes <= g_bounds_table.hi[i]) return true;
+    if (atomicAdd(&g_bounds_record.violations, 1ull) == 0ull) {
+        g_bounds_record.first_address = a;
+        g_bounds_record.first_bytes = bytes;
+        g_bounds_record.first_block = blockIdx.x;
+        g_bounds_record.first_thread = threadIdx.x;
+    }
+    return false;
+}
+#define NC_STORE_OK(p, bytes) nc_store_ok((p), (bytes))
+
+typedef cudaError_t (*BoundsFetch)(BoundsRecord* out, bool reset);
+void nc_bounds_register(BoundsFetch fetch);          // api_misc.cu keeps the list of units
+
+static cudaError_t bounds_fetch_this_unit(BoundsRecord* out, bool reset) {
+    cudaError_t e = cudaMemcpyFromSymbol(out, g_bounds_record, sizeof(BoundsRecord));
+    if (e == cudaSuccess && reset) {
+        const BoundsRecord zero = {};
+        e = cudaMemcpyToSymbol(g_bounds_record, &zero, sizeof(BoundsRecord));
+    }
+    return e;
+}
+static struct BoundsRegistrar {
+    BoundsRegistrar() { nc_bounds_register(&bounds_fetch_this_unit); }
+} g_bounds_registrar;
+
+// Host side: the ranges a call may write, sent to the device in stream order before its launches.
+struct BoundsScope {
+    BoundsTable t;
+    BoundsScope() { t.count = 0; }
+    void add(const void* p, size_t bytes) {
+        if (!p || !bytes || t.count >= kBoundsRanges) return;
+        t.lo[t.count] = (unsigned long long)(uintptr_t)p;
+        t.hi[t.count] = t.lo[t.count] + bytes;
+        ++t.count;
+    }
+    void commit(cudaStream_t stream) {
+        cudaMemcpyToSymbolAsync(g_bounds_table, &t, sizeof(BoundsTable), 0, cudaMemcpyHostToDevice,
+                                stream);
+    }
+};
+#else
+#define NC_STORE_OK(p, bytes) true
+struct BoundsScope {
+    void add(const void*, size_t) {}
+    void commit(cudaStream_t) {}
+};
+#endif
+
+// a plain store through the same check
+#define NC_STORE(ptr, value)                                        \
+    do {                                                            \
+        if (NC_STORE_OK((ptr), (unsigned)sizeof(*(ptr)))) *(ptr) = (value); \
+    } while (0)
+
 // ---- streaming loads / stores: every plane is touched once, keep it out of L1 and
 // mark it evict-first in L2.
 __device__ __forceinline__ uint4 ld_stream_u4(const void* p) {
@@ -66,10 +149,13 @@ __device__ __forceinline__ uint32_t ld_stream_u32(const void* p) {
     return __ldcs(reinterpret_cast<const unsigned int*>(p));
 }
 __device__ __forceinline__ void st_stream_u4(void* p, uint4 v) {
-    __stcs(reinterpret_cast<uint4*>(p), v);
+    if (NC_STORE_OK(p, 16u)) __stcs(reinterpret_cast<uint4*>(p), v);
 }
 __device__ __forceinline__ void st_stream_u32(void* p, uint32_t v) {
-    __stcs(reinterpret_cast<unsigned int*>(p), v);
+    if (NC_STORE_OK(p, 4u)) __stcs(reinterpret_cast<unsigned int*>(p), v);
+}
+__device__ __forceinline__ void st_stream_f4(void* p, float4 v) {
+    if (NC_STORE_OK(p, 16u)) __stcs(reinterpret_cast<float4*>(p), v);
 }
 
 // 4x4 transpose of bytes across each aligned group of 4 lanes: lane i holds bytes b[i][t]

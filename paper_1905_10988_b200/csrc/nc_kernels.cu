@@ -134,11 +134,11 @@ __device__ __forceinline__ void cnat_ragged_tile(LoadBits load_bits, const uint6
             }
             e = cnat_exp_byte(bits, r);
         }
-        if (j < exp_end) exp[j] = (uint8_t)e;
+        if (j < exp_end) NC_STORE(exp + j, (uint8_t)e);
         const uint32_t word = __ballot_sync(0xFFFFFFFFu, (bits >> 31) != 0);
-        if (lane == 0 && (j0 >> 5) < sign_words) sign[j0 >> 5] = word;
+        if (lane == 0 && (j0 >> 5) < sign_words) NC_STORE(sign + (j0 >> 5), word);
     }
-    if (lane < (int)(sign_words_padded - sign_words)) sign[sign_words + lane] = 0;
+    if (lane < (int)(sign_words_padded - sign_words)) NC_STORE(sign + sign_words + lane, 0u);
 }
 
 // grid: (ceil(tiles / warps per block), n workers).  kDet: round to the nearest power of two
@@ -359,11 +359,11 @@ nc_aggregate_kernel(const __grid_constant__ PackedPlanes planes, const int n, co
         }
         aggregate_full_tile(planes, n, base, acc, lane);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) __stcs(ov + k * 32 + lane, acc[k]);
+        for (int k = 0; k < 8; ++k) st_stream_f4(ov + k * 32 + lane, acc[k]);
         return;
     }
     for (uint64_t j = base + lane; j < d; j += 32)      // ragged last tile: scalar
-        out[j] = aggregate_element(planes, n, j, kFromAcc ? out[j] : 0.f);
+        NC_STORE(out + j, aggregate_element(planes, n, j, kFromAcc ? out[j] : 0.f));
 }
 
 // Master side with compression of the aggregate (Algorithm 1: g = C_M(sum_i Delta_i) with
@@ -423,13 +423,13 @@ nc_sum_fp32_kernel(const __grid_constant__ DensePlanes planes, const int n, cons
         }
         float4* ov = reinterpret_cast<float4*>(out + base);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) __stcs(ov + k * 32 + lane, acc[k]);
+        for (int k = 0; k < 8; ++k) st_stream_f4(ov + k * 32 + lane, acc[k]);
         return;
     }
     for (uint64_t j = base + lane; j < d; j += 32) {
         float a = 0.f;
         for (int i = 0; i < n; ++i) a += planes.x[i][j];
-        out[j] = a;
+        NC_STORE(out + j, a);
     }
 }
 
@@ -453,6 +453,7 @@ static nc_status compress_batch_impl(const float* const* xs, size_t d, uint64_t 
     if (d == 0) return NC_OK;
     if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
     CompressBatch batch;
+    BoundsScope scope;
     for (int i = 0; i < n; ++i) {
         if (!xs[i] || !exps[i] || !signs[i]) return NC_ERR_INVALID;
         if (!aligned32(xs[i]) || !aligned16(exps[i]) || !aligned16(signs[i])) return NC_ERR_ALIGN;
@@ -460,7 +461,10 @@ static nc_status compress_batch_impl(const float* const* xs, size_t d, uint64_t 
         batch.exp[i] = exps[i];
         batch.sign[i] = signs[i];
         batch.worker[i] = workers ? workers[i] : 0u;
+        scope.add(exps[i], nc_exp_bytes(d));
+        scope.add(signs[i], nc_sign_bytes(d));
     }
+    scope.commit(stream);
     const PhiloxKeys keys = make_philox_keys(seed);
     dim3 grid(tile_blocks(d), (unsigned)n);
     if (deterministic)
@@ -502,6 +506,7 @@ nc_status nc_compress_typed_batch(const void* const* xs, int dtype, size_t d, ui
     if (d == 0) return NC_OK;
     if (d > ((uint64_t)1 << 40)) return NC_ERR_INVALID;
     Compress16Batch batch;
+    BoundsScope scope;
     for (int i = 0; i < n; ++i) {
         if (!xs[i] || !exps[i] || !signs[i]) return NC_ERR_INVALID;
         if (!aligned16(xs[i]) || !aligned16(exps[i]) || !aligned16(signs[i])) return NC_ERR_ALIGN;
@@ -509,7 +514,10 @@ nc_status nc_compress_typed_batch(const void* const* xs, int dtype, size_t d, ui
         batch.exp[i] = exps[i];
         batch.sign[i] = signs[i];
         batch.worker[i] = workers[i];
+        scope.add(exps[i], nc_exp_bytes(d));
+        scope.add(signs[i], nc_sign_bytes(d));
     }
+    scope.commit(stream);
     const PhiloxKeys keys = make_philox_keys(seed);
     dim3 grid(tile_blocks(d), (unsigned)n);
     if (dtype == NC_DTYPE_BF16)
@@ -539,6 +547,9 @@ nc_status nc_aggregate(const uint8_t* const* exps, const uint32_t* const* signs,
         planes.exp[i] = exps[i];
         planes.sign[i] = signs[i];
     }
+    BoundsScope scope;
+    scope.add(out, 4 * (size_t)d);
+    scope.commit(stream);
     nc_aggregate_kernel<false><<<tile_blocks(d), kBlockThreads, 0, stream>>>(planes, n,
                                                                              (uint64_t)d, out);
     return launch_status();
@@ -565,6 +576,10 @@ nc_status nc_aggregate_compress_shard(const uint8_t* const* exps, const uint32_t
         planes.sign[i] = reinterpret_cast<const uint32_t*>((uintptr_t)signs[i] - sign_back);
     }
     const PhiloxKeys keys = make_philox_keys(seed);
+    BoundsScope scope;
+    scope.add(out_exp, nc_exp_bytes(d));
+    scope.add(out_sign, nc_sign_bytes(d));
+    scope.commit(stream);
     nc_aggregate_compress_kernel<<<tile_blocks(d), kBlockThreads, 0, stream>>>(
         planes, n, first_index, first_index + (uint64_t)d, master, keys,
         reinterpret_cast<uint8_t*>((uintptr_t)out_exp - exp_back),
@@ -588,6 +603,9 @@ nc_status nc_decode_accumulate(const uint8_t* exp, const uint32_t* sign, size_t 
     PackedPlanes planes;
     planes.exp[0] = exp;
     planes.sign[0] = sign;
+    BoundsScope scope;
+    scope.add(acc, 4 * (size_t)d);
+    scope.commit(stream);
     nc_aggregate_kernel<true><<<tile_blocks(d), kBlockThreads, 0, stream>>>(planes, 1,
                                                                             (uint64_t)d, acc);
     return launch_status();
@@ -604,6 +622,9 @@ nc_status nc_sum_fp32(const float* const* xs, int n, size_t d, float* out, cudaS
         if (!aligned32(xs[i])) return NC_ERR_ALIGN;
         planes.x[i] = xs[i];
     }
+    BoundsScope scope;
+    scope.add(out, 4 * (size_t)d);
+    scope.commit(stream);
     nc_sum_fp32_kernel<<<tile_blocks(d), kBlockThreads, 0, stream>>>(planes, n, (uint64_t)d, out);
     return launch_status();
 }

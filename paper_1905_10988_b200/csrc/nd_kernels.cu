@@ -47,6 +47,7 @@ __device__ __forceinline__ V8 ld_stream_v8(const void* p) {
 }
 
 __device__ __forceinline__ void st_stream_v8(void* p, const V8& r) {
+    if (!NC_STORE_OK(p, 32u)) return;
     asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(r.v[0]),
                  "r"(r.v[1]), "r"(r.v[2]), "r"(r.v[3]), "r"(r.v[4]), "r"(r.v[5]), "r"(r.v[6]),
                  "r"(r.v[7])
@@ -128,7 +129,7 @@ __device__ __forceinline__ void norm_tile(const float* __restrict__ x, uint64_t*
     const uint64_t base = tile * kTile;
     const uint64_t end = full ? base + kTile : d;
     int b = find_bucket(off, B, base);
-    if (lane == 0) tile_bucket[tile] = (uint32_t)b;
+    if (lane == 0) NC_STORE(tile_bucket + tile, (uint32_t)b);
 
     NormAcc<P> acc;
     if (full && __ldg(off + b + 1) >= end) {
@@ -139,7 +140,7 @@ __device__ __forceinline__ void norm_tile(const float* __restrict__ x, uint64_t*
             for (int c = 0; c < 8; ++c) acc.add(u[it].v[c], c & 3);
         }
         const uint64_t r = acc.reduce();
-        if (lane == 0) slots[tile + (uint64_t)b] = r;
+        if (lane == 0) NC_STORE(slots + tile + (uint64_t)b, r);
         return;
     }
     // the tile spans several buckets or is ragged: one segment at a time, lane-strided
@@ -154,7 +155,7 @@ __device__ __forceinline__ void norm_tile(const float* __restrict__ x, uint64_t*
             if (++cnt == 8) { acc.flush(); cnt = 0; }
         }
         const uint64_t r = acc.reduce();
-        if (lane == 0) slots[tile + (uint64_t)b] = r;
+        if (lane == 0) NC_STORE(slots + tile + (uint64_t)b, r);
         pos = seg_end;
         if (pos < end) {
             ++b;
@@ -217,7 +218,7 @@ nd_norm_finalize_kernel(const __grid_constant__ DitherBatch batch,
     __shared__ uint32_t s_max[kWarpsPerBlock];
     const uint64_t lo = off[b], hi = off[b + 1];
     if (hi <= lo) {                      // empty bucket (uniform over the block)
-        if (threadIdx.x == 0) norms[b] = 0.f;
+        if (threadIdx.x == 0) NC_STORE(norms + b, 0.f);
         return;
     }
     const uint64_t t_first = lo / kTile, t_last = (hi - 1) / kTile;
@@ -246,7 +247,7 @@ nd_norm_finalize_kernel(const __grid_constant__ DitherBatch batch,
             if (P == 2) tot = sqrt(tot);
             result = (float)tot;
         }
-        norms[b] = result;
+        NC_STORE(norms + b, result);
         // a bucket that holds an inf or a NaN: its codes will all be 0, the caller is told here
         if (status && !(result <= 3.40282347e38f)) atomicAdd(status, 1u);
     }
@@ -398,11 +399,11 @@ nd_round_pack_kernel(const __grid_constant__ DitherBatch batch, const uint64_t d
             code = level_code(bits, r, sc, pow2s);
         }
         const uint32_t next = __shfl_down_sync(0xFFFFFFFFu, code, 1);
-        if ((lane & 1) == 0 && j < lvl_end) level[j >> 1] = (uint8_t)(code | (next << 4));
+        if ((lane & 1) == 0 && j < lvl_end) NC_STORE(level + (j >> 1), (uint8_t)(code | (next << 4)));
         const uint32_t word = __ballot_sync(0xFFFFFFFFu, (bits >> 31) != 0);
-        if (lane == 0 && (j0 >> 5) < sign_words) sign[j0 >> 5] = word;
+        if (lane == 0 && (j0 >> 5) < sign_words) NC_STORE(sign + (j0 >> 5), word);
     }
-    if (!full && lane < (int)(sign_words_padded - sign_words)) sign[sign_words + lane] = 0;
+    if (!full && lane < (int)(sign_words_padded - sign_words)) NC_STORE(sign + sign_words + lane, 0u);
 }
 
 // ---- master side ------------------------------------------------------------------------
@@ -639,7 +640,7 @@ nd_aggregate_kernel(const __grid_constant__ DitherPlanes planes, const int n, co
             // comes, so a norm that is not finite shows in the sum
             a = c ? add_scaled(a, norm, __uint_as_float(pb)) : __fadd_rn(a, __uint_as_float(pb));
         }
-        out[j] = a;
+        NC_STORE(out + j, a);
     }
 }
 
@@ -730,6 +731,19 @@ static nc_status nd_check_batch(const float* const* xs, size_t d, const uint64_t
     return NC_OK;
 }
 
+// debug build: what a dithering compress call may write
+static void nd_scope_batch(BoundsScope& scope, const DitherBatch& batch, uint64_t d, int B, int n,
+                           bool norms, bool planes, void* workspace) {
+    for (int i = 0; i < n; ++i) {
+        if (norms) scope.add(batch.norms[i], 4 * (size_t)B);
+        if (planes) {
+            scope.add(batch.level[i], nd_level_bytes(d));
+            scope.add(batch.sign[i], nc_sign_bytes(d));
+        }
+    }
+    if (workspace) scope.add(workspace, nd_batch_workspace_bytes(d, B, n));
+}
+
 // the two norm launches; returns the tile -> bucket map they leave in the workspace
 static uint32_t* nd_launch_norms(const DitherBatch& batch, uint64_t d, const uint64_t* bucket_off,
                                  int B, int p, int n, void* workspace, uint32_t* status,
@@ -772,6 +786,9 @@ nc_status nd_norms_batch(const float* const* xs, size_t d, const uint64_t* bucke
     if (!workspace) return NC_ERR_INVALID;
     if (!aligned16(workspace) || !aligned4(status)) return NC_ERR_ALIGN;
     if (workspace_bytes < nd_batch_workspace_bytes(d, B, n)) return NC_ERR_WORKSPACE;
+    BoundsScope scope;
+    nd_scope_batch(scope, batch, d, B, n, true, false, workspace);
+    scope.commit(stream);
     nd_launch_norms(batch, d, bucket_off, B, p, n, workspace, status, stream);
     return launch_status();
 }
@@ -789,6 +806,9 @@ nc_status nd_round_batch(const float* const* xs, size_t d, const uint64_t* bucke
     if (d == 0) return NC_OK;
     const PhiloxKeys keys = make_philox_keys(seed);
     const dim3 grid(nd_tile_blocks(d), (unsigned)n);
+    BoundsScope scope;
+    nd_scope_batch(scope, batch, d, B, n, false, true, nullptr);
+    scope.commit(stream);
     nd_round_pack_kernel<true><<<grid, kBlockThreads, 0, stream>>>(batch, d, bucket_off, B, s, keys,
                                                                    nullptr);
     return launch_status();
@@ -809,6 +829,9 @@ nc_status nd_compress_batch(const float* const* xs, size_t d, const uint64_t* bu
     if (!workspace) return NC_ERR_INVALID;
     if (!aligned16(workspace) || !aligned4(status)) return NC_ERR_ALIGN;
     if (workspace_bytes < nd_batch_workspace_bytes(d, B, n)) return NC_ERR_WORKSPACE;
+    BoundsScope scope;
+    nd_scope_batch(scope, batch, d, B, n, true, true, workspace);
+    scope.commit(stream);
     const uint32_t* tile_bucket =
         nd_launch_norms(batch, d, bucket_off, B, p, n, workspace, status, stream);
     const PhiloxKeys keys = make_philox_keys(seed);
@@ -853,6 +876,9 @@ nc_status nd_aggregate(const float* const* norms, const uint8_t* const* levels,
     const nc_status st = nd_check_planes(norms, levels, signs, n, &planes);
     if (st != NC_OK) return st;
     const uint64_t big_tiles = nd_aggregate_big_tiles(d);
+    BoundsScope scope;
+    scope.add(out, 4 * (size_t)d);
+    scope.commit(stream);
     nd_aggregate_kernel<false><<<nd_aggregate_blocks(d, big_tiles), kAggregateThreads, 0, stream>>>(
         planes, n, (uint64_t)d, bucket_off, B, s, big_tiles, out);
     return launch_status();
@@ -886,6 +912,9 @@ nc_status nd_decode_accumulate(const float* norms, const uint8_t* level, const u
     const nc_status st = nd_check_planes(&norms, &level, &sign, 1, &planes);
     if (st != NC_OK) return st;
     const uint64_t big_tiles = nd_aggregate_big_tiles(d);
+    BoundsScope scope;
+    scope.add(acc, 4 * (size_t)d);
+    scope.commit(stream);
     nd_aggregate_kernel<true><<<nd_aggregate_blocks(d, big_tiles), kAggregateThreads, 0, stream>>>(
         planes, 1, (uint64_t)d, bucket_off, B, s, big_tiles, acc);
     return launch_status();
