@@ -23,6 +23,7 @@ struct SparseWorkspace {
     uint32_t* bitmask;      // tiles * 32 words
     uint32_t* block_count;   // one per block of 8 tiles (the exclusive offset after the scan)
     uint64_t* block_partial; // one per block of 8 tiles
+    uint8_t* stage;          // 64 bytes per group of 8 tiles: see kStageEntries
     uint8_t* tmp_codes;     // cap bytes
 };
 
@@ -30,7 +31,8 @@ __host__ __device__ inline uint64_t sparse_tiles(uint64_t d) { return (d + kTile
 
 inline size_t sparse_ws_bytes(uint64_t d, uint64_t cap) {
     const uint64_t t = sparse_tiles(d);
-    return round_up16(t * 128) + round_up16(t * 4) + round_up16(t * 8) + round_up16(cap);
+    return round_up16(t * 128) + round_up16(t * 4) + round_up16(t * 8) +
+           round_up16(((t + 7) / 8) * 64) + round_up16(cap);
 }
 
 __host__ __device__ inline SparseWorkspace sparse_ws_carve(void* ws, uint64_t d) {
@@ -40,6 +42,7 @@ __host__ __device__ inline SparseWorkspace sparse_ws_carve(void* ws, uint64_t d)
     w.bitmask = reinterpret_cast<uint32_t*>(p);      p += round_up16(t * 128);
     w.block_count = reinterpret_cast<uint32_t*>(p);   p += round_up16(t * 4);
     w.block_partial = reinterpret_cast<uint64_t*>(p); p += round_up16(t * 8);
+    w.stage = reinterpret_cast<uint8_t*>(p);          p += round_up16(((t + 7) / 8) * 64);
     w.tmp_codes = reinterpret_cast<uint8_t*>(p);
     return w;
 }
@@ -84,6 +87,14 @@ __device__ __forceinline__ uint32_t warp_list_positions(uint32_t word, int lane,
 // counts): at 1 % density a single tile has about ten kept entries, so the sparse passes give a
 // warp a whole group and work on the listed entries with all lanes busy.
 constexpr uint32_t kGroupListCap = 2048;      // >= kTile: one tile always fits into an empty list
+
+// The level filter of the compact form leaves the codes of a group's surviving entries in the
+// workspace, so that the emit pass needs neither the gather from x nor the generator again:
+// 64 bytes per group = up to 126 four-bit codes in ascending position order (code r in bits
+// 4 (r mod 2).. of byte r / 2) and, in byte 63, 1 if the codes are there.  A group with more
+// surviving entries, or more than 128 kept ones, is not staged and is emitted the long way.
+constexpr uint32_t kStageEntries = 126;
+constexpr uint32_t kStageBytes = 64;
 
 // appends the positions (inside the group, tile w) of the set bits of `word` (lane l = word l of
 // the tile) to list[at ..]; returns how many

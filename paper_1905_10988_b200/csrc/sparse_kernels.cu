@@ -501,13 +501,43 @@ sparse_round_filter_kernel(const __grid_constant__ SparseBatch batch, const uint
     const float pow2s = __uint_as_float((uint32_t)(127 + s) << 23);
     __syncwarp();
 
-    auto round_one = [&](uint32_t p, float xv) {
+    const int nb = code_value_bits(s);
+    // codes of the surviving entries by rank: staging only happens for a group of at most 128
+    // kept entries, whose list leaves the upper half of the warp's list area free (one more
+    // kilobyte of shared memory per block would cost a resident block)
+    uint8_t* code_of_rank = reinterpret_cast<uint8_t*>(list + kGroupListCap / 2);
+    uint32_t staged = 0;                                 // survivors whose codes are in s_code
+    bool stageable = true;                               // false once a flush took the long way
+
+    // level code of one kept entry (no side effect, so that the generator chains of several
+    // entries interleave)
+    auto level_of = [&](uint32_t p, float xv, uint32_t& sign_bit) -> uint32_t {
         const float xs = __fmul_rn(scale, xv);
+        sign_bit = __float_as_uint(xs) >> 31;
         const uint32_t r = stream_word_at(gbase + p, worker, kDomainDnat, keys);
-        if (sparse_level_code(__float_as_uint(xs), r, sc, pow2s) == 0u)
-            atomicAnd(&mask[p >> 5], ~(1u << (p & 31)));
+        return sparse_level_code(__float_as_uint(xs), r, sc, pow2s);
     };
-    auto flush = [&](uint32_t cnt) {
+    // clears the mask bit of a level-0 entry; returns the 4-bit code (sign << nb) | (level - 1)
+    // of a surviving entry, 0xFF otherwise
+    auto settle = [&](uint32_t p, uint32_t level, uint32_t sign_bit) -> uint32_t {
+        if (level == 0u) {
+            atomicAnd(&mask[p >> 5], ~(1u << (p & 31)));
+            return 0xFFu;
+        }
+        return (sign_bit << nb) | (level - 1u);
+    };
+    // a list that filled up before the group ended (dense selections only): no staging
+    auto flush_part = [&](uint32_t cnt) {
+        __syncwarp();
+        for (uint32_t t = lane; t < cnt; t += 32) {
+            const uint32_t p = list[t];
+            uint32_t sg;
+            const uint32_t level = level_of(p, x[gbase + p], sg);
+            settle(p, level, sg);
+        }
+        __syncwarp();
+    };
+    auto flush = [&](uint32_t cnt, bool whole_group) {
         __syncwarp();
         if (cnt <= 4u * 32u) {
             // the usual case: all gathers of the group are issued before any is used
@@ -519,35 +549,75 @@ sparse_round_filter_kernel(const __grid_constant__ SparseBatch batch, const uint
                 pp[e] = (t < cnt) ? (uint32_t)list[t] : 0xFFFFFFFFu;
                 xv[e] = (t < cnt) ? x[gbase + pp[e]] : 0.f;
             }
+            // the four roundings first (independent generator chains), then the side effects
+            uint32_t level[4], sgn[4], code[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) level[e] = level_of(pp[e] & 0x1FFFu, xv[e], sgn[e]);
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-                if (pp[e] != 0xFFFFFFFFu) round_one(pp[e], xv[e]);
+                code[e] = (pp[e] != 0xFFFFFFFFu) ? settle(pp[e], level[e], sgn[e]) : 0xFFu;
+            uint32_t rank0 = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                // list order is ascending position, so the rank among the survivors is the
+                // number of survivors at smaller list positions
+                const uint32_t alive = __ballot_sync(0xFFFFFFFFu, code[e] != 0xFFu);
+                if (whole_group && code[e] != 0xFFu) {
+                    const uint32_t rank = rank0 + __popc(alive & ((1u << lane) - 1u));
+                    if (rank < 128u) code_of_rank[rank] = (uint8_t)code[e];
+                }
+                rank0 += __popc(alive);
+            }
+            if (whole_group) staged = rank0;
+            else stageable = false;
         } else {
+            stageable = false;
             for (uint32_t t = lane; t < cnt; t += 32) {
                 const uint32_t p = list[t];
-                round_one(p, x[gbase + p]);
+                uint32_t sg;
+                const uint32_t level = level_of(p, x[gbase + p], sg);
+                settle(p, level, sg);
             }
         }
         __syncwarp();
     };
     uint32_t cnt = 0;
+    bool flushed_before = false;
 #pragma unroll
     for (int w = 0; w < kWarpsPerBlock; ++w) {
         const uint32_t tile_cnt = warp_sum_u(__popc(word[w]));
         if (cnt + tile_cnt > kGroupListCap) {
-            flush(cnt);
+            flush_part(cnt);
+            flushed_before = true;
             cnt = 0;
         }
         group_list_append(word[w], lane, w, list, cnt);
         cnt += tile_cnt;
     }
-    flush(cnt);
+    flush(cnt, !flushed_before);
     uint32_t total = 0;
 #pragma unroll
     for (int w = 0; w < kWarpsPerBlock; ++w) {
         const uint32_t kept = mask[w * 32 + lane];
         if (tile0 + w < tiles) ws.bitmask[(tile0 + w) * 32 + lane] = kept;
         total += __popc(kept);
+    }
+    // the staged codes of the group: 16 lanes write one word of eight codes each; byte 63 says
+    // whether they are there
+    {
+        const bool ok = stageable && !flushed_before && staged <= kStageEntries;
+        if (lane < 16) {
+            uint32_t wv = 0;
+            if (ok) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t r = (uint32_t)(lane * 8 + c);
+                    if (r < staged) wv |= (uint32_t)(code_of_rank[r] & 0xFu) << (4 * c);
+                }
+                if (lane == 15) wv = (wv & 0x00FFFFFFu) | (1u << 24);
+            }
+            reinterpret_cast<uint32_t*>(ws.stage + grp * kStageBytes)[lane] = wv;
+        }
     }
     total = warp_sum_u(total);
     if (lane == 0) ws.block_count[grp] = total;
@@ -617,6 +687,34 @@ sparse_emit_compact_kernel(const __grid_constant__ SparseBatch batch, const uint
         __syncwarp();
         k0 += cnt;
     };
+    // The usual case: the level filter left the codes of this group's entries in the workspace,
+    // so the entries are written from the mask and those codes alone (no gather from x, no
+    // generator).  Lane l holds staged codes 8 l .. 8 l + 7 (lanes 0..15).
+    const uint32_t stage_word =
+        lane < 16 ? reinterpret_cast<const uint32_t*>(ws.stage + grp * kStageBytes)[lane] : 0u;
+    const bool is_staged = (__shfl_sync(0xFFFFFFFFu, stage_word, 15) >> 24) == 1u;
+    if (is_staged) {
+        uint32_t cnt = 0;
+#pragma unroll
+        for (int w = 0; w < kWarpsPerBlock; ++w) {
+            const uint32_t tile_cnt = warp_sum_u(__popc(word[w]));
+            group_list_append(word[w], lane, w, list, cnt);     // at most 126 entries in all
+            cnt += tile_cnt;
+        }
+        __syncwarp();
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const uint32_t t = (uint32_t)(e * 32 + lane);
+            // code t sits in bits 4 (t mod 8).. of the word of lane t / 8
+            const uint32_t wv = __shfl_sync(0xFFFFFFFFu, stage_word, (int)(t >> 3) & 15);
+            const uint64_t k = k0 + t;
+            if (t < cnt && k < cap) {
+                idx[k] = (uint32_t)(gbase + list[t]);
+                ws.tmp_codes[k] = (uint8_t)((wv >> (4 * (t & 7u))) & 0xFu);
+            }
+        }
+        return;
+    }
     uint32_t cnt = 0;
 #pragma unroll
     for (int w = 0; w < kWarpsPerBlock; ++w) {
@@ -691,12 +789,27 @@ sparse_compact_decode_accumulate_kernel(const uint32_t* __restrict__ idx,
 
 namespace natcomp {
 
+// The level filter is bound by its random 32-byte gathers and by shared-memory traffic, and it runs
+// faster with four resident blocks per SM and a large L1 than with five and a small one (the
+// driver sizes the shared-memory carve-out for the highest occupancy otherwise: 24 instead of
+// 92 KB of L1, 426 -> 640 us on 8 x 2^28 coordinates).  Asked for once per device: a carve-out
+// of 164 KB, which holds four blocks.
+static void filter_prefers_large_l1() {
+    static bool done[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || done[dev]) return;
+    cudaFuncSetAttribute(sparse_round_filter_kernel,
+                         cudaFuncAttributePreferredSharedMemoryCarveout, 71);
+    done[dev] = true;
+}
+
 void sparse_compact_finish(const SparseBatch& batch, uint64_t d, float scale, int p, int s,
                            const PhiloxKeys& keys, uint64_t cap, char* ws, uint64_t ws_stride,
                            int n, cudaStream_t stream) {
     const uint64_t tile_groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
     const dim3 ggrid((unsigned)((tile_groups + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
     launch_scan(batch, d, p, ws, ws_stride, n, stream);          // norm (and the kept count)
+    filter_prefers_large_l1();
     sparse_round_filter_kernel<<<ggrid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, ws,
                                                                     ws_stride);
     // second scan: offsets and count of the surviving entries (the norm partials are unchanged)
