@@ -118,7 +118,7 @@ sparse_select_group_kernel(const __grid_constant__ SparseBatch batch, const uint
     // counter groups of elements 32l .. 32l+31, so its 32 bits are word l of the tile mask.
     // phase 2: the kept positions of the whole group are listed and gathered together.
     uint32_t cnt = 0, kept = 0;
-#pragma unroll 1
+#pragma unroll
     for (int w = 0; w < kWarpsPerBlock; ++w) {
         const uint64_t tile = tile0 + w;
         const uint64_t base = tile * kTile;
@@ -581,20 +581,27 @@ sparse_round_filter_kernel(const __grid_constant__ SparseBatch batch, const uint
         }
         __syncwarp();
     };
-    uint32_t cnt = 0;
+    static_assert(kWarpsPerBlock == 8, "a group is 8 tiles");
     bool flushed_before = false;
+    uint32_t tile_cnt[kWarpsPerBlock];
+    const uint32_t group_cnt = group_list_build(word, lane, list, tile_cnt);
+    if (group_cnt <= kGroupListCap) {
+        flush(group_cnt, true);                  // the whole group in one list
+    } else {
+        // a dense selection: tile by tile, flushing whenever the next tile would not fit
+        uint32_t cnt = 0;
 #pragma unroll
-    for (int w = 0; w < kWarpsPerBlock; ++w) {
-        const uint32_t tile_cnt = warp_sum_u(__popc(word[w]));
-        if (cnt + tile_cnt > kGroupListCap) {
-            flush_part(cnt);
-            flushed_before = true;
-            cnt = 0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) {
+            if (cnt + tile_cnt[w] > kGroupListCap) {
+                flush_part(cnt);
+                cnt = 0;
+            }
+            group_list_append(word[w], lane, w, list, cnt);
+            cnt += tile_cnt[w];
         }
-        group_list_append(word[w], lane, w, list, cnt);
-        cnt += tile_cnt;
+        flush_part(cnt);
+        flushed_before = true;
     }
-    flush(cnt, !flushed_before);
     uint32_t total = 0;
 #pragma unroll
     for (int w = 0; w < kWarpsPerBlock; ++w) {
@@ -693,14 +700,10 @@ sparse_emit_compact_kernel(const __grid_constant__ SparseBatch batch, const uint
     const uint32_t stage_word =
         lane < 16 ? reinterpret_cast<const uint32_t*>(ws.stage + grp * kStageBytes)[lane] : 0u;
     const bool is_staged = (__shfl_sync(0xFFFFFFFFu, stage_word, 15) >> 24) == 1u;
+    uint32_t tile_cnt[kWarpsPerBlock];
+    const uint32_t group_cnt = group_list_build(word, lane, list, tile_cnt);
     if (is_staged) {
-        uint32_t cnt = 0;
-#pragma unroll
-        for (int w = 0; w < kWarpsPerBlock; ++w) {
-            const uint32_t tile_cnt = warp_sum_u(__popc(word[w]));
-            group_list_append(word[w], lane, w, list, cnt);     // at most 126 entries in all
-            cnt += tile_cnt;
-        }
+        const uint32_t cnt = group_cnt;                         // at most 126 entries
         __syncwarp();
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -715,16 +718,19 @@ sparse_emit_compact_kernel(const __grid_constant__ SparseBatch batch, const uint
         }
         return;
     }
+    if (group_cnt <= kGroupListCap) {
+        flush(group_cnt);                        // the whole group is listed already
+        return;
+    }
     uint32_t cnt = 0;
 #pragma unroll
     for (int w = 0; w < kWarpsPerBlock; ++w) {
-        const uint32_t tile_cnt = warp_sum_u(__popc(word[w]));
-        if (cnt + tile_cnt > kGroupListCap) {
+        if (cnt + tile_cnt[w] > kGroupListCap) {
             flush(cnt);
             cnt = 0;
         }
         group_list_append(word[w], lane, w, list, cnt);
-        cnt += tile_cnt;
+        cnt += tile_cnt[w];
     }
     flush(cnt);
 }
