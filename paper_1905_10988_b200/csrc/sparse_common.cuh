@@ -86,7 +86,11 @@ __device__ __forceinline__ uint32_t warp_list_positions(uint32_t word, int lane,
 // Lists of kept positions for a group of 8 tiles (8192 coordinates, the unit of the per-block
 // counts): at 1 % density a single tile has about ten kept entries, so the sparse passes give a
 // warp a whole group and work on the listed entries with all lanes busy.
-constexpr uint32_t kGroupListCap = 2048;      // >= kTile: one tile always fits into an empty list
+// >= kTile: one tile always fits into an empty list.  Not larger either: the level filter is bound
+// by its gathers and its shared-memory traffic and is sensitive to how the driver splits L1 and
+// shared memory (with 4 KB lists and one more kilobyte per block it got five resident blocks, a
+// 228 KB carve-out and 24 KB of L1, and took 640 instead of 430 us on 8 x 2^28 coordinates).
+constexpr uint32_t kGroupListCap = 1024;
 
 // The level filter of the compact form leaves the codes of a group's surviving entries in the
 // workspace, so that the emit pass needs neither the gather from x nor the generator again:

@@ -795,27 +795,12 @@ sparse_compact_decode_accumulate_kernel(const uint32_t* __restrict__ idx,
 
 namespace natcomp {
 
-// The level filter is bound by its random 32-byte gathers and by shared-memory traffic, and it runs
-// faster with four resident blocks per SM and a large L1 than with five and a small one (the
-// driver sizes the shared-memory carve-out for the highest occupancy otherwise: 24 instead of
-// 92 KB of L1, 426 -> 640 us on 8 x 2^28 coordinates).  Asked for once per device: a carve-out
-// of 164 KB, which holds four blocks.
-static void filter_prefers_large_l1() {
-    static bool done[64] = {false};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || done[dev]) return;
-    cudaFuncSetAttribute(sparse_round_filter_kernel,
-                         cudaFuncAttributePreferredSharedMemoryCarveout, 71);
-    done[dev] = true;
-}
-
 void sparse_compact_finish(const SparseBatch& batch, uint64_t d, float scale, int p, int s,
                            const PhiloxKeys& keys, uint64_t cap, char* ws, uint64_t ws_stride,
                            int n, cudaStream_t stream) {
     const uint64_t tile_groups = (sparse_tiles(d) + kWarpsPerBlock - 1) / kWarpsPerBlock;
     const dim3 ggrid((unsigned)((tile_groups + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)n);
     launch_scan(batch, d, p, ws, ws_stride, n, stream);          // norm (and the kept count)
-    filter_prefers_large_l1();
     sparse_round_filter_kernel<<<ggrid, kBlockThreads, 0, stream>>>(batch, d, scale, s, keys, ws,
                                                                     ws_stride);
     // second scan: offsets and count of the surviving entries (the norm partials are unchanged)
